@@ -1,0 +1,155 @@
+"""ctypes front end of the CPU oracle (``tuna_oracle.c``).
+
+TEST INFRASTRUCTURE ONLY: imported by the tests, by the smoke check and by the
+benchmark's CPU-baseline leg.  The CUDA library and its Python binding never
+import this package.  The C file is compiled with gcc on first use.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+import threading
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "tuna_oracle.c")
+_OUT_DIR = os.path.join(_HERE, "_build")
+_LIB = os.path.join(_OUT_DIR, "libtuna_oracle.so")
+_lock = threading.Lock()
+_lib = None
+
+RS_COLS = 6
+RS_LEVEL, RS_X, RS_Z, RS_UNITS, RS_BYTES_SENT, RS_BYTES_RECV = range(6)
+TR_COLS = 8
+TR_ROUND, TR_KIND, TR_PARTNER, TR_OFFSET, TR_ORIGIN, TR_DEST, TR_BYTES, TR_PLACE = range(8)
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle into a shared object beside its source."""
+    os.makedirs(_OUT_DIR, exist_ok=True)
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + ".tmp.%d" % os.getpid()
+        subprocess.check_call(["gcc", "-O2", "-std=c11", "-Wall", "-Wextra", "-shared", "-fPIC",
+                               "-o", tmp, _SRC])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+_I64P = ctypes.POINTER(ctypes.c_int64)
+_U8P = ctypes.POINTER(ctypes.c_uint8)
+_IP = ctypes.POINTER(ctypes.c_int)
+
+
+def _load():
+    global _lib
+    with _lock:
+        if _lib is None:
+            lib = ctypes.CDLL(build())
+            lib.oracle_num_digits.argtypes = [ctypes.c_int, ctypes.c_int]
+            lib.oracle_round_list.argtypes = [ctypes.c_int, ctypes.c_int, _IP, _IP, ctypes.c_int]
+            lib.oracle_tmap.argtypes = [ctypes.c_int] * 3
+            lib.oracle_bruteforce.argtypes = [ctypes.c_int, ctypes.c_int] + [_I64P] * 5 + [_U8P, _U8P]
+            lib.oracle_tuna_flat.argtypes = (
+                [ctypes.c_int] * 3 + [_I64P] * 5 + [_U8P, _U8P, _I64P, ctypes.c_int, _IP, _IP,
+                                                    ctypes.c_int, _I64P, ctypes.c_int64, _I64P])
+            lib.oracle_tuna_hier.argtypes = (
+                [ctypes.c_int] * 5 + [_I64P] * 5 + [_U8P, _U8P, ctypes.c_int64, _U8P, _I64P,
+                                                    ctypes.c_int, _IP])
+            _lib = lib
+    return _lib
+
+
+def _i64(a):
+    a = np.ascontiguousarray(a, dtype=np.int64)
+    return a, a.ctypes.data_as(_I64P)
+
+
+def _u8(a):
+    assert a.dtype == np.uint8 and a.flags["C_CONTIGUOUS"]
+    return a.ctypes.data_as(_U8P)
+
+
+def num_digits(P: int, r: int) -> int:
+    return _load().oracle_num_digits(P, r)
+
+
+def round_list(P: int, r: int):
+    """The rounds [(x, z), ...] of a flat exchange in execution order."""
+    lib = _load()
+    K = lib.oracle_round_list(P, r, None, None, 0)
+    xs = (ctypes.c_int * max(K, 1))()
+    zs = (ctypes.c_int * max(K, 1))()
+    lib.oracle_round_list(P, r, xs, zs, K)
+    return [(xs[i], zs[i]) for i in range(K)]
+
+
+def tmap(P: int, r: int, o: int) -> int:
+    return _load().oracle_tmap(P, r, o)
+
+
+def _check(rc, what):
+    if rc != 0:
+        raise RuntimeError(f"{what} failed with oracle status {rc}")
+
+
+def bruteforce(wl, send: np.ndarray, recv: np.ndarray) -> np.ndarray:
+    """The exchange by its definition; writes into and returns ``recv``."""
+    c, cp = _i64(wl.sendcounts)
+    sd, sdp = _i64(wl.sdispls)
+    rd, rdp = _i64(wl.rdispls)
+    sb, sbp = _i64(wl.sendbase)
+    rb, rbp = _i64(wl.recvbase)
+    _check(_load().oracle_bruteforce(wl.P, wl.elem_size, cp, sdp, rdp, sbp, rbp, _u8(send),
+                                     _u8(recv)), "oracle_bruteforce")
+    return recv
+
+
+def tuna_flat(wl, r: int, send: np.ndarray, recv: np.ndarray, trace_rank: int = -1):
+    """Algorithm 1.  Returns (recv, rounds[K, RS_COLS], B, trace or None)."""
+    lib = _load()
+    c, cp = _i64(wl.sendcounts)
+    sd, sdp = _i64(wl.sdispls)
+    rd, rdp = _i64(wl.rdispls)
+    sb, sbp = _i64(wl.sendbase)
+    rb, rbp = _i64(wl.recvbase)
+    K = lib.oracle_round_list(wl.P, r, None, None, 0)
+    rounds = np.zeros((max(K, 1), RS_COLS), dtype=np.int64)
+    Kc, Bc = ctypes.c_int(0), ctypes.c_int(0)
+    trace = None
+    tp, tcap, trows = None, 0, ctypes.c_int64(0)
+    if trace_rank >= 0:
+        tcap = 2 * wl.P * max(K, 1)
+        trace = np.zeros((tcap, TR_COLS), dtype=np.int64)
+        tp = trace.ctypes.data_as(_I64P)
+    _check(lib.oracle_tuna_flat(wl.P, r, wl.elem_size, cp, sdp, rdp, sbp, rbp, _u8(send),
+                                _u8(recv), rounds.ctypes.data_as(_I64P), K, ctypes.byref(Kc),
+                                ctypes.byref(Bc), trace_rank, tp, tcap, ctypes.byref(trows)),
+           "oracle_tuna_flat")
+    assert Kc.value == K
+    if trace is not None:
+        assert trows.value <= tcap
+        trace = trace[:trows.value]
+    return recv, rounds[:K], Bc.value, trace
+
+
+def tuna_hier(wl, Q: int, N: int, rl: int, rg: int, send: np.ndarray, recv: np.ndarray,
+              want_after_local: bool = False):
+    """Hierarchical exchange.  Returns (recv, rounds, (K_local, K_global), recv_after_local)."""
+    lib = _load()
+    assert Q * N == wl.P
+    c, cp = _i64(wl.sendcounts)
+    sd, sdp = _i64(wl.sdispls)
+    rd, rdp = _i64(wl.rdispls)
+    sb, sbp = _i64(wl.sendbase)
+    rb, rbp = _i64(wl.recvbase)
+    K = lib.oracle_round_list(Q, rl, None, None, 0) + lib.oracle_round_list(N, rg, None, None, 0)
+    rounds = np.zeros((max(K, 1), RS_COLS), dtype=np.int64)
+    Ks = (ctypes.c_int * 2)()
+    after = np.empty_like(recv) if want_after_local else None
+    _check(lib.oracle_tuna_hier(Q, N, rl, rg, wl.elem_size, cp, sdp, rdp, sbp, rbp, _u8(send),
+                                _u8(recv), recv.nbytes, _u8(after) if after is not None else None,
+                                rounds.ctypes.data_as(_I64P), K, Ks), "oracle_tuna_hier")
+    assert Ks[0] + Ks[1] == K
+    return recv, rounds[:K], (Ks[0], Ks[1]), after
