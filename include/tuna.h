@@ -1,0 +1,210 @@
+/*
+ * tuna.h - C ABI of the TuNA (tunable-radix non-uniform all-to-all) library for
+ * one NVIDIA B200.
+ *
+ * All P logical ranks live inside one GPU: the "send buffers" of the P ranks are
+ * regions of a single device buffer, likewise the "receive buffers".  The exchange
+ * has exactly the semantics of MPI_Alltoallv (the paper's Sec. VI-B and Conclusion
+ * state that the algorithms keep its signature and meaning): block j of rank i's
+ * send region arrives as block i of rank j's receive region; bytes of the receive
+ * buffer that no block covers are left untouched.
+ *
+ * Conventions for every function
+ *   - returns TUNA_OK (0) or a negative tuna_status; never aborts; a validation
+ *     failure touches no GPU state.
+ *   - "host" pointers are ordinary CPU memory, "device" pointers are CUDA device
+ *     memory of the current device.  The library copies every host array it is
+ *     given before returning; the caller may free them at once.
+ *   - counts and displacements are 64-bit and in ELEMENTS of elem_size bytes.
+ *     Matrices are row-major P x P: sendcounts[s*P + d], sdispls[s*P + d]
+ *     (relative to rank s's send region), rdispls[d*P + s] (relative to rank d's
+ *     receive region).  sendbase[p] / recvbase[p] give the element offset of rank
+ *     p's region inside the one send / receive buffer.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *     Work is enqueued on it; unless stated otherwise nothing synchronises.
+ *   - the caller owns send buffer, receive buffer and workspace; the plan owns
+ *     only its descriptor tables, freed by tuna_plan_destroy.
+ */
+#ifndef TUNA_H
+#define TUNA_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct tuna_plan tuna_plan_t;
+
+typedef enum tuna_status {
+  TUNA_OK = 0,
+  TUNA_ERR_INVALID_ARG = -1,    /* null pointer, P < 1, elem_size < 1, negative count or offset */
+  TUNA_ERR_BAD_RADIX = -2,      /* radix outside [2, max(2, ranks of its level)] */
+  TUNA_ERR_BAD_HIERARCHY = -3,  /* l * g != P */
+  TUNA_ERR_COUNT_MISMATCH = -4, /* counts/displacements differ from the plan's, or recv != send^T */
+  TUNA_ERR_OVERLAP = -5,        /* send and receive ranges alias (no in-place exchange) */
+  TUNA_ERR_WORKSPACE = -6,      /* workspace missing, misaligned or too small */
+  TUNA_ERR_CUDA = -7,           /* a CUDA runtime call failed; see tuna_plan_cuda_error */
+  TUNA_ERR_NOMEM = -8,          /* host or device allocation of the plan's tables failed */
+  TUNA_ERR_RANGE = -9           /* index (round, phase, ...) out of range, or size above a stated limit */
+} tuna_status;
+
+/* flags for tuna_plan_create */
+#define TUNA_FLAG_DIRECT_TO_R 0u    /* default: a block's last hop writes straight into the receive buffer */
+#define TUNA_FLAG_CLASSIC_ROTATE 1u /* last hops land in the workspace; one final rotation pass reorders them */
+
+/* schedules for the host-buffer entry point */
+#define TUNA_SCHEDULE_TUNA 0
+#define TUNA_SCHEDULE_DIRECT 1
+
+/*
+ * tuna_plan_create - build the schedule and every displacement for one count matrix.
+ *
+ * Defines: Sec. III-A (radix-r rounds: round (x, z) moves the blocks whose x-th
+ * base-r digit of the offset (dst - src) mod P equals z to the rank at distance
+ * +z*r^x), Sec. III-B (per-round metadata: the sizes of the blocks a rank holds,
+ * obtained here by applying the same rank shift to the size table), Sec. III-C
+ * (placement of intermediate blocks; here exact offsets from segmented exclusive
+ * prefix sums over the sizes instead of max-size slots), Sec. IV (hierarchical
+ * variant: ranks p = n*l + q; local rounds of radix `radix` on the local offset
+ * inside every group of l consecutive ranks, for all g destination groups at
+ * once; then global rounds of radix `radix_global` on the group offset between
+ * ranks with equal local id; radix_global == g is the paper's coalesced exchange).
+ *
+ *   out           host; receives the plan.
+ *   P             number of ranks, >= 1.
+ *   radix         flat radix (g == 1) or local radix, in [2, max(2, l)].
+ *   radix_global  global radix in [2, max(2, g)]; ignored when g == 1.
+ *   l, g          ranks per group and number of groups, l*g == P; g == 1 is flat TuNA.
+ *   elem_size     bytes per element, >= 1.
+ *   flags         TUNA_FLAG_*.
+ *   sendcounts    host, P*P.
+ *   sdispls, rdispls, sendbase, recvbase
+ *                 host, P*P / P*P / P / P; any of them may be NULL, meaning blocks
+ *                 packed back to back in ascending index order (sdispls, rdispls)
+ *                 and regions packed in rank order (sendbase, recvbase); these
+ *                 defaults are computed on the device by the same scan kernel.
+ *   stream        the plan kernels run on it; the call synchronises it once to read
+ *                 back the phase totals that size the workspace.
+ */
+int tuna_plan_create(tuna_plan_t **out, int P, int radix, int radix_global, int l, int g,
+                     int elem_size, unsigned flags, const int64_t *sendcounts,
+                     const int64_t *sdispls, const int64_t *rdispls, const int64_t *sendbase,
+                     const int64_t *recvbase, void *stream);
+
+/*
+ * tuna_plan_update_counts - same plan shape, new counts (e.g. routing that changes
+ * every step): re-runs the metadata exchange and the prefix sums on the device.
+ * Arguments as in tuna_plan_create.  Synchronises `stream` once.  The required
+ * workspace size may change; query it again.
+ */
+int tuna_plan_update_counts(tuna_plan_t *plan, const int64_t *sendcounts, const int64_t *sdispls,
+                            const int64_t *rdispls, const int64_t *sendbase,
+                            const int64_t *recvbase, void *stream);
+
+/* Frees the plan's device tables and the plan.  NULL is accepted. */
+int tuna_plan_destroy(tuna_plan_t *plan);
+
+/*
+ * Workspace (the paper's temporary buffer T, Sec. III-C, sized exactly).
+ * tuna_plan_workspace_bytes: bytes needed by tuna_alltoallv on device buffers.
+ * tuna_plan_host_staging_bytes: extra bytes needed by tuna_alltoallv_host for
+ * device copies of the send and receive buffers.
+ * tuna_plan_set_workspace: device pointer, 256-byte aligned, caller-owned, must
+ * stay valid while the plan uses it; `bytes` is checked by each exchange call.
+ */
+int tuna_plan_workspace_bytes(const tuna_plan_t *plan, size_t *bytes);
+int tuna_plan_host_staging_bytes(const tuna_plan_t *plan, size_t *bytes);
+int tuna_plan_set_workspace(tuna_plan_t *plan, void *dev_ptr, size_t bytes);
+
+/* Extents the plan's layout implies, in bytes: the send buffer is read inside
+ * [0, send_bytes), the receive buffer written inside [0, recv_bytes). */
+int tuna_plan_extents(const tuna_plan_t *plan, size_t *send_bytes, size_t *recv_bytes,
+                      size_t *payload_bytes);
+
+/*
+ * tuna_alltoallv - run the plan's TuNA schedule (Algorithm 1, or Sec. IV /
+ * Algorithm 3 when g > 1): one fused pack-move-unpack launch per digit phase
+ * (all rounds z of one digit position x touch disjoint blocks), then one
+ * rotation launch (self blocks; in TUNA_FLAG_CLASSIC_ROTATE mode every block).
+ *
+ *   sendbuf, recvbuf   device; must not overlap.
+ *   sendcounts, sdispls, recvcounts, rdispls
+ *                      host, P*P each, or NULL.  Non-NULL arrays are only checked
+ *                      against the plan (TUNA_ERR_COUNT_MISMATCH); the plan's own
+ *                      copies drive the kernels.  recvcounts[d*P+s] must equal
+ *                      sendcounts[s*P+d].
+ * Asynchronous on `stream`; re-runnable; two calls on one plan must not overlap
+ * in time (they share the workspace).
+ */
+int tuna_alltoallv(tuna_plan_t *plan, const void *sendbuf, const int64_t *sendcounts,
+                   const int64_t *sdispls, void *recvbuf, const int64_t *recvcounts,
+                   const int64_t *rdispls, void *stream);
+
+/*
+ * tuna_direct_alltoallv - the linear spread-out exchange (Sec. II-d; the r = P end
+ * of Sec. III-C) as ONE launch: every (src, dst) block is read once and written
+ * once.  Needs no workspace.  Arguments as tuna_alltoallv.
+ */
+int tuna_direct_alltoallv(tuna_plan_t *plan, const void *sendbuf, const int64_t *sendcounts,
+                          const int64_t *sdispls, void *recvbuf, const int64_t *recvcounts,
+                          const int64_t *rdispls, void *stream);
+
+/*
+ * tuna_alltoallv_host - the same exchange on HOST buffers: copies
+ * [0, send_bytes) of host_send to the device, runs the chosen schedule
+ * (TUNA_SCHEDULE_*), copies [0, recv_bytes) back into host_recv, all on `stream`,
+ * and returns without synchronising (pinned host memory makes the copies
+ * asynchronous).  The workspace must hold workspace_bytes + host_staging_bytes.
+ * Receive-buffer bytes that no block covers are overwritten with unspecified
+ * values by the copy back.
+ */
+int tuna_alltoallv_host(tuna_plan_t *plan, const void *host_send, void *host_recv, int schedule,
+                        void *stream);
+
+/*
+ * Schedule introspection (host values, filled at plan time).
+ * Rounds are the paper's (x, z) pairs in execution order (Sec. III-A); `level` is 0
+ * for flat/local rounds and 1 for global rounds; `units` counts blocks sent by all
+ * ranks (level 0) or super-blocks of l blocks (level 1); `bytes` is the round's
+ * message volume summed over ranks.  Phases are the digit positions, one kernel
+ * launch each: `entries` descriptor rows, `bytes` moved, `stream_bytes` the
+ * 16-byte-padded length of the phase's destination stream.
+ */
+int tuna_plan_num_rounds(const tuna_plan_t *plan, int *K);
+int tuna_plan_round_info(const tuna_plan_t *plan, int k, int *level, int *x, int *z,
+                         int64_t *units, int64_t *bytes);
+int tuna_plan_num_phases(const tuna_plan_t *plan, int *n);
+int tuna_plan_phase_info(const tuna_plan_t *plan, int phase, int *level, int *x, int64_t *entries,
+                         int64_t *bytes, int64_t *stream_bytes);
+
+/*
+ * tuna_plan_phase_tables - copy one phase's descriptor table to the host (debug /
+ * test hook; synchronises the device).  phase in [0, num_phases) selects a digit
+ * phase, -1 the rotation list, -2 the direct list.  Each output (host, `cap` rows,
+ * may be NULL) receives, per descriptor in receive-side order (rank, then slot):
+ * the block length in bytes, the position in the phase's padded stream (the
+ * exclusive prefix sum that also partitions the work), and source / destination
+ * as (buffer id << 56 | byte offset), buffer ids 0 = send, 1 = receive, 2 = workspace.
+ * *rows receives the number of descriptors.
+ */
+int tuna_plan_phase_tables(const tuna_plan_t *plan, int phase, int64_t cap, int64_t *len,
+                           int64_t *pos, int64_t *src, int64_t *dst, int64_t *rows);
+
+/* Kernels launched by the last exchange call on this plan (host counter). */
+int tuna_plan_last_launches(const tuna_plan_t *plan, int *launches);
+
+/* The cudaError_t of the most recent failing runtime call (0 if none). */
+int tuna_plan_cuda_error(const tuna_plan_t *plan);
+
+/* Static string for a status code. */
+const char *tuna_strerror(int status);
+
+/* Library version, major*100 + minor. */
+int tuna_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TUNA_H */

@@ -53,7 +53,10 @@ def _load():
             lib.oracle_bruteforce.argtypes = [ctypes.c_int, ctypes.c_int] + [_I64P] * 5 + [_U8P, _U8P]
             lib.oracle_tuna_flat.argtypes = (
                 [ctypes.c_int] * 3 + [_I64P] * 5 + [_U8P, _U8P, _I64P, ctypes.c_int, _IP, _IP,
-                                                    ctypes.c_int, _I64P, ctypes.c_int64, _I64P])
+                                                    ctypes.c_int, _I64P, ctypes.c_int64, _I64P,
+                                                    _I64P])
+            lib.oracle_segmented_exclusive_scan.argtypes = [_I64P, ctypes.c_int64, ctypes.c_int64,
+                                                            ctypes.c_int64, _I64P, _I64P]
             lib.oracle_tuna_hier.argtypes = (
                 [ctypes.c_int] * 5 + [_I64P] * 5 + [_U8P, _U8P, ctypes.c_int64, _U8P, _I64P,
                                                     ctypes.c_int, _IP])
@@ -106,8 +109,23 @@ def bruteforce(wl, send: np.ndarray, recv: np.ndarray) -> np.ndarray:
     return recv
 
 
-def tuna_flat(wl, r: int, send: np.ndarray, recv: np.ndarray, trace_rank: int = -1):
-    """Algorithm 1.  Returns (recv, rounds[K, RS_COLS], B, trace or None)."""
+def segmented_exclusive_scan(val: np.ndarray, align: int = 1):
+    """Per-row exclusive running sums of a 2-D int64 array; returns (scan, row totals)."""
+    v, vp = _i64(val)
+    nseg, seglen = v.shape
+    out = np.zeros_like(v)
+    tot = np.zeros(nseg, dtype=np.int64)
+    _check(_load().oracle_segmented_exclusive_scan(vp, nseg, seglen, align,
+                                                   out.ctypes.data_as(_I64P),
+                                                   tot.ctypes.data_as(_I64P)),
+           "oracle_segmented_exclusive_scan")
+    return out, tot
+
+
+def tuna_flat(wl, r: int, send: np.ndarray, recv: np.ndarray, trace_rank: int = -1,
+              want_sizes: bool = False):
+    """Algorithm 1.  Returns (recv, rounds[K, RS_COLS], B, trace or None); with
+    ``want_sizes`` a fifth item: the size tables [w, P, P] after every digit phase."""
     lib = _load()
     c, cp = _i64(wl.sendcounts)
     sd, sdp = _i64(wl.sdispls)
@@ -123,14 +141,20 @@ def tuna_flat(wl, r: int, send: np.ndarray, recv: np.ndarray, trace_rank: int = 
         tcap = 2 * wl.P * max(K, 1)
         trace = np.zeros((tcap, TR_COLS), dtype=np.int64)
         tp = trace.ctypes.data_as(_I64P)
+    sizes, szp = None, None
+    if want_sizes:
+        sizes = np.zeros((max(lib.oracle_num_digits(wl.P, r), 1), wl.P, wl.P), dtype=np.int64)
+        szp = sizes.ctypes.data_as(_I64P)
     _check(lib.oracle_tuna_flat(wl.P, r, wl.elem_size, cp, sdp, rdp, sbp, rbp, _u8(send),
                                 _u8(recv), rounds.ctypes.data_as(_I64P), K, ctypes.byref(Kc),
-                                ctypes.byref(Bc), trace_rank, tp, tcap, ctypes.byref(trows)),
+                                ctypes.byref(Bc), trace_rank, tp, tcap, ctypes.byref(trows), szp),
            "oracle_tuna_flat")
     assert Kc.value == K
     if trace is not None:
         assert trows.value <= tcap
         trace = trace[:trows.value]
+    if want_sizes:
+        return recv, rounds[:K], Bc.value, trace, sizes[:lib.oracle_num_digits(wl.P, r)]
     return recv, rounds[:K], Bc.value, trace
 
 

@@ -149,6 +149,27 @@ int oracle_bruteforce(int P, int elem, const int64_t *counts, const int64_t *sdi
   return ORACLE_OK;
 }
 
+/* Segmented exclusive prefix sum, the textbook running sum: nseg segments of
+   seglen values; each value is first rounded up to a multiple of `align`
+   (align = 1: no rounding).  out[s][i] = sum of the rounded values before i in
+   segment s; totals[s] (may be NULL) = the segment's sum.  These sums are what
+   turns a rank's list of block sizes into displacements (Sec. III-B/C). */
+int oracle_segmented_exclusive_scan(const int64_t *val, int64_t nseg, int64_t seglen,
+                                    int64_t align, int64_t *out, int64_t *totals) {
+  if (nseg < 0 || seglen < 0 || align < 1) return ORACLE_EARG;
+  for (int64_t s = 0; s < nseg; s++) {
+    int64_t run = 0;
+    for (int64_t i = 0; i < seglen; i++) {
+      int64_t v = val[s * seglen + i];
+      v = (v + align - 1) / align * align;
+      out[s * seglen + i] = run;
+      run += v;
+    }
+    if (totals) totals[s] = run;
+  }
+  return ORACLE_OK;
+}
+
 /* ---- small helpers shared by the two schedules ---- */
 
 typedef struct {
@@ -203,12 +224,15 @@ static void trace_row(int64_t *trace, int64_t cap, int64_t *rows, int64_t round,
  * Algorithm 1.  `rounds` (may be NULL) receives K rows of RS_COLS values;
  * `trace` (may be NULL) receives what rank `trace_rank` sent and received.
  * `tslots_out` (may be NULL) receives B, the number of T slots per rank.
+ * `sz_phases` (may be NULL, w*P*P values) receives, after all rounds of digit
+ * position x, the metadata every rank holds: sz_phases[x][p][o] = bytes of the
+ * block rank p holds for offset o (Sec. III-B: sizes travel ahead of the data).
  */
 int oracle_tuna_flat(int P, int r, int elem, const int64_t *counts, const int64_t *sdispls,
                      const int64_t *rdispls, const int64_t *sendbase, const int64_t *recvbase,
                      const uint8_t *send, uint8_t *recv, int64_t *rounds, int rounds_cap,
                      int *K_out, int *tslots_out, int trace_rank, int64_t *trace,
-                     int64_t trace_cap, int64_t *trace_rows) {
+                     int64_t trace_cap, int64_t *trace_rows, int64_t *sz_phases) {
   if (P < 1 || r < 2 || elem < 1) return ORACLE_EARG;
   int rc = ORACLE_OK;
   int w = oracle_num_digits(P, r);
@@ -337,6 +361,7 @@ int oracle_tuna_flat(int P, int r, int elem, const int64_t *counts, const int64_
       }
       k++;
     }
+    if (sz_phases) memcpy(sz_phases + (int64_t)x * P * P, sz, sizeof(int64_t) * (size_t)P * P);
   }
   if (k != K) rc = ORACLE_ESCHED;
 

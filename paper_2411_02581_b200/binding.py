@@ -1,0 +1,252 @@
+"""Thin ctypes binding over the C ABI declared in ``include/tuna.h``.
+
+Only argument marshalling happens here: every step of the exchange runs in the
+CUDA library.  There is no CPU fallback; if the shared library is missing the
+import of :func:`lib` raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import numpy as np
+
+from . import build as _build
+
+_I64P = ctypes.POINTER(ctypes.c_int64)
+_INTP = ctypes.POINTER(ctypes.c_int)
+_SZP = ctypes.POINTER(ctypes.c_size_t)
+_VP = ctypes.c_void_p
+
+FLAG_DIRECT_TO_R = 0
+FLAG_CLASSIC_ROTATE = 1
+SCHEDULE_TUNA = 0
+SCHEDULE_DIRECT = 1
+
+STATUS = {
+    0: "TUNA_OK", -1: "TUNA_ERR_INVALID_ARG", -2: "TUNA_ERR_BAD_RADIX",
+    -3: "TUNA_ERR_BAD_HIERARCHY", -4: "TUNA_ERR_COUNT_MISMATCH", -5: "TUNA_ERR_OVERLAP",
+    -6: "TUNA_ERR_WORKSPACE", -7: "TUNA_ERR_CUDA", -8: "TUNA_ERR_NOMEM", -9: "TUNA_ERR_RANGE",
+}
+
+# name -> (restype, argtypes); must list every symbol include/tuna.h declares
+SIGNATURES = {
+    "tuna_plan_create": (ctypes.c_int, [ctypes.POINTER(_VP)] + [ctypes.c_int] * 6 + [ctypes.c_uint]
+                         + [_I64P] * 5 + [_VP]),
+    "tuna_plan_update_counts": (ctypes.c_int, [_VP] + [_I64P] * 5 + [_VP]),
+    "tuna_plan_destroy": (ctypes.c_int, [_VP]),
+    "tuna_plan_workspace_bytes": (ctypes.c_int, [_VP, _SZP]),
+    "tuna_plan_host_staging_bytes": (ctypes.c_int, [_VP, _SZP]),
+    "tuna_plan_set_workspace": (ctypes.c_int, [_VP, _VP, ctypes.c_size_t]),
+    "tuna_plan_extents": (ctypes.c_int, [_VP, _SZP, _SZP, _SZP]),
+    "tuna_alltoallv": (ctypes.c_int, [_VP, _VP, _I64P, _I64P, _VP, _I64P, _I64P, _VP]),
+    "tuna_direct_alltoallv": (ctypes.c_int, [_VP, _VP, _I64P, _I64P, _VP, _I64P, _I64P, _VP]),
+    "tuna_alltoallv_host": (ctypes.c_int, [_VP, _VP, _VP, ctypes.c_int, _VP]),
+    "tuna_plan_num_rounds": (ctypes.c_int, [_VP, _INTP]),
+    "tuna_plan_round_info": (ctypes.c_int, [_VP, ctypes.c_int, _INTP, _INTP, _INTP, _I64P, _I64P]),
+    "tuna_plan_num_phases": (ctypes.c_int, [_VP, _INTP]),
+    "tuna_plan_phase_info": (ctypes.c_int, [_VP, ctypes.c_int, _INTP, _INTP, _I64P, _I64P, _I64P]),
+    "tuna_plan_phase_tables": (ctypes.c_int, [_VP, ctypes.c_int, ctypes.c_int64] + [_I64P] * 5),
+    "tuna_plan_last_launches": (ctypes.c_int, [_VP, _INTP]),
+    "tuna_plan_cuda_error": (ctypes.c_int, [_VP]),
+    "tuna_strerror": (ctypes.c_char_p, [ctypes.c_int]),
+    "tuna_version": (ctypes.c_int, []),
+}
+
+_lib = None
+
+
+class TunaError(RuntimeError):
+    def __init__(self, status: int, what: str, cuda: int = 0):
+        self.status = status
+        self.cuda_error = cuda
+        super().__init__(f"{what}: {STATUS.get(status, status)}"
+                         + (f" (cudaError {cuda})" if cuda else ""))
+
+
+def lib() -> ctypes.CDLL:
+    """Load the CUDA library (built in-tree); raise if it does not exist."""
+    global _lib
+    if _lib is None:
+        path = _build.LIB_PATH
+        if not os.path.exists(path):
+            raise RuntimeError(
+                f"{path} is missing: build it with `python -m paper_2411_02581_b200.build` "
+                "(there is no CPU fallback)")
+        l = ctypes.CDLL(path)
+        for name, (res, args) in SIGNATURES.items():
+            fn = getattr(l, name)
+            fn.restype = res
+            fn.argtypes = args
+        _lib = l
+    return _lib
+
+
+def _h(a):
+    """Host int64 array (or None) -> (keepalive, pointer)."""
+    if a is None:
+        return None, None
+    a = np.ascontiguousarray(a, dtype=np.int64)
+    return a, a.ctypes.data_as(_I64P)
+
+
+def _ptr(t):
+    """Device/host pointer of a torch tensor, numpy array or int."""
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    if isinstance(t, np.ndarray):
+        return t.ctypes.data
+    return t.data_ptr()
+
+
+def _stream(stream):
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream
+    if isinstance(stream, int):
+        return stream
+    return stream.cuda_stream
+
+
+class Plan:
+    """Owner of a ``tuna_plan_t``; methods carry the C function names."""
+
+    def __init__(self, P, radix, l=None, g=1, radix_global=2, elem_size=1, flags=0,
+                 sendcounts=None, sdispls=None, rdispls=None, sendbase=None, recvbase=None,
+                 stream=None):
+        self._h = _VP()
+        self._ws = None
+        l = P if l is None else l
+        keep = [_h(x) for x in (sendcounts, sdispls, rdispls, sendbase, recvbase)]
+        rc = lib().tuna_plan_create(ctypes.byref(self._h), P, radix, radix_global, l, g, elem_size,
+                                    flags, *[k[1] for k in keep], _stream(stream))
+        if rc != 0:
+            self._h = _VP()
+            raise TunaError(rc, "tuna_plan_create")
+        self.P, self.elem_size = P, elem_size
+
+    def _check(self, rc, what):
+        if rc != 0:
+            raise TunaError(rc, what, lib().tuna_plan_cuda_error(self._h))
+
+    def destroy(self):
+        if self._h:
+            lib().tuna_plan_destroy(self._h)
+            self._h = _VP()
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+    def update_counts(self, sendcounts, sdispls=None, rdispls=None, sendbase=None, recvbase=None,
+                      stream=None):
+        keep = [_h(x) for x in (sendcounts, sdispls, rdispls, sendbase, recvbase)]
+        self._check(lib().tuna_plan_update_counts(self._h, *[k[1] for k in keep], _stream(stream)),
+                    "tuna_plan_update_counts")
+
+    def workspace_bytes(self) -> int:
+        n = ctypes.c_size_t()
+        self._check(lib().tuna_plan_workspace_bytes(self._h, ctypes.byref(n)), "tuna_plan_workspace_bytes")
+        return n.value
+
+    def host_staging_bytes(self) -> int:
+        n = ctypes.c_size_t()
+        self._check(lib().tuna_plan_host_staging_bytes(self._h, ctypes.byref(n)),
+                    "tuna_plan_host_staging_bytes")
+        return n.value
+
+    def set_workspace(self, tensor, nbytes=None):
+        """``tensor``: a torch uint8 CUDA tensor (kept alive by the plan) or None."""
+        self._ws = tensor
+        nb = 0 if tensor is None else (tensor.numel() * tensor.element_size() if nbytes is None else nbytes)
+        self._check(lib().tuna_plan_set_workspace(self._h, _ptr(tensor), nb), "tuna_plan_set_workspace")
+
+    def alloc_workspace(self, host_staging=False, device="cuda"):
+        """Allocate the workspace through torch (256-byte aligned) and attach it."""
+        import torch
+        need = self.workspace_bytes()
+        need = (need + 255) // 256 * 256 + (self.host_staging_bytes() if host_staging else 0)
+        ws = torch.empty(max(need, 256), dtype=torch.uint8, device=device)
+        self.set_workspace(ws)
+        return ws
+
+    def extents(self):
+        a, b, c = ctypes.c_size_t(), ctypes.c_size_t(), ctypes.c_size_t()
+        self._check(lib().tuna_plan_extents(self._h, ctypes.byref(a), ctypes.byref(b), ctypes.byref(c)),
+                    "tuna_plan_extents")
+        return a.value, b.value, c.value
+
+    def alltoallv(self, sendbuf, recvbuf, sendcounts=None, sdispls=None, recvcounts=None,
+                  rdispls=None, stream=None):
+        keep = [_h(x) for x in (sendcounts, sdispls, recvcounts, rdispls)]
+        self._check(lib().tuna_alltoallv(self._h, _ptr(sendbuf), keep[0][1], keep[1][1],
+                                         _ptr(recvbuf), keep[2][1], keep[3][1], _stream(stream)),
+                    "tuna_alltoallv")
+
+    def direct_alltoallv(self, sendbuf, recvbuf, sendcounts=None, sdispls=None, recvcounts=None,
+                         rdispls=None, stream=None):
+        keep = [_h(x) for x in (sendcounts, sdispls, recvcounts, rdispls)]
+        self._check(lib().tuna_direct_alltoallv(self._h, _ptr(sendbuf), keep[0][1], keep[1][1],
+                                                _ptr(recvbuf), keep[2][1], keep[3][1],
+                                                _stream(stream)), "tuna_direct_alltoallv")
+
+    def alltoallv_host(self, host_send, host_recv, schedule=SCHEDULE_TUNA, stream=None):
+        self._check(lib().tuna_alltoallv_host(self._h, _ptr(host_send), _ptr(host_recv), schedule,
+                                              _stream(stream)), "tuna_alltoallv_host")
+
+    def num_rounds(self) -> int:
+        k = ctypes.c_int()
+        self._check(lib().tuna_plan_num_rounds(self._h, ctypes.byref(k)), "tuna_plan_num_rounds")
+        return k.value
+
+    def round_info(self, k):
+        lv, x, z = ctypes.c_int(), ctypes.c_int(), ctypes.c_int()
+        u, b = ctypes.c_int64(), ctypes.c_int64()
+        self._check(lib().tuna_plan_round_info(self._h, k, ctypes.byref(lv), ctypes.byref(x),
+                                               ctypes.byref(z), ctypes.byref(u), ctypes.byref(b)),
+                    "tuna_plan_round_info")
+        return dict(level=lv.value, x=x.value, z=z.value, units=u.value, bytes=b.value)
+
+    def rounds(self):
+        return [self.round_info(k) for k in range(self.num_rounds())]
+
+    def num_phases(self) -> int:
+        n = ctypes.c_int()
+        self._check(lib().tuna_plan_num_phases(self._h, ctypes.byref(n)), "tuna_plan_num_phases")
+        return n.value
+
+    def phase_info(self, phase):
+        lv, x = ctypes.c_int(), ctypes.c_int()
+        e, b, s = ctypes.c_int64(), ctypes.c_int64(), ctypes.c_int64()
+        self._check(lib().tuna_plan_phase_info(self._h, phase, ctypes.byref(lv), ctypes.byref(x),
+                                               ctypes.byref(e), ctypes.byref(b), ctypes.byref(s)),
+                    "tuna_plan_phase_info")
+        return dict(level=lv.value, x=x.value, entries=e.value, bytes=b.value, stream_bytes=s.value)
+
+    def phase_tables(self, phase):
+        n = self.phase_info(phase)["entries"]
+        arrs = [np.zeros(max(n, 1), dtype=np.int64) for _ in range(4)]
+        rows = ctypes.c_int64()
+        self._check(lib().tuna_plan_phase_tables(self._h, phase, n,
+                                                 *[a.ctypes.data_as(_I64P) for a in arrs],
+                                                 ctypes.byref(rows)), "tuna_plan_phase_tables")
+        assert rows.value == n
+        return dict(len=arrs[0][:n], pos=arrs[1][:n], src=arrs[2][:n], dst=arrs[3][:n])
+
+    def last_launches(self) -> int:
+        n = ctypes.c_int()
+        self._check(lib().tuna_plan_last_launches(self._h, ctypes.byref(n)), "tuna_plan_last_launches")
+        return n.value
+
+
+def plan_for(wl, radix, l=None, g=1, radix_global=2, flags=0, explicit_layout=True, stream=None) -> Plan:
+    """A plan for a :class:`workloads.Workload`."""
+    kw = dict(sendcounts=wl.sendcounts)
+    if explicit_layout:
+        kw.update(sdispls=wl.sdispls, rdispls=wl.rdispls, sendbase=wl.sendbase, recvbase=wl.recvbase)
+    return Plan(wl.P, radix, l=l, g=g, radix_global=radix_global, elem_size=wl.elem_size,
+                flags=flags, stream=stream, **kw)

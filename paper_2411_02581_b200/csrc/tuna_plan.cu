@@ -1,0 +1,1003 @@
+// Plan construction (count-metadata exchange + segmented prefix sums) and the
+// C-ABI entry points.
+//
+// Device-side picture.  Rank p = n*Q + q (Q = l ranks per group, N = g groups;
+// flat TuNA is N = 1).  Every rank names its P blocks by slot sigma = io*Q + jo,
+// the block for rank (n+io mod N, q+jo mod Q): this is the paper's index-only
+// rotation (Algorithm 1, the array I), no data moves.  A digit phase (level, x)
+// with radix r moves every slot whose digit x of jo (level 0) or io (level 1) is
+// z != 0 to the rank at distance +z*r^x on that level (Sec. III-A, Sec. IV).
+// Two dense P x P tables follow the blocks through the phases:
+//     sz[p][sigma]   size of the block rank p holds in that slot    (Sec. III-B:
+//                    the per-round metadata message is the same rank shift
+//                    applied to this table)
+//     loc[p][sigma]  where its bytes are (send buffer or a workspace offset)
+// and every phase emits a compact descriptor list in receive-side order whose
+// destination offsets are exclusive prefix sums of the 16-byte-padded sizes
+// (Sec. III-C's temporary buffer, sized exactly instead of by the maximum block).
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <algorithm>
+#include <new>
+
+#include "tuna_internal.h"
+
+namespace {
+
+// ------------------------------------------------------------------ device helpers
+
+__device__ __forceinline__ int64_t pad16(int64_t v) { return (v + (TUNA_ALIGN - 1)) & ~(int64_t)(TUNA_ALIGN - 1); }
+
+// Compact index of offset v among the offsets whose digit (v / stride) % radix is
+// non-zero, ascending.  Only called for such v.
+__device__ __forceinline__ int64_t compact_of(int64_t v, int64_t stride, int radix) {
+  const int64_t hi = v / (stride * radix);
+  const int64_t rem = v - hi * stride * radix;  // z*stride + lo
+  return hi * (radix - 1) * stride + (rem - stride);
+}
+
+struct PhaseDev {
+  int level, radix, count;
+  int64_t stride, moving, per_rank;
+};
+
+// Initial tables (before any phase): every block is in its owner's send region.
+// Also fills the direct list (receive-side order (d, s)) and the self entries of
+// the rotation list.
+__global__ void tuna_init_tables_kernel(TunaTopo t, const int64_t *__restrict__ counts,
+                                        const int64_t *__restrict__ sdispls,
+                                        const int64_t *__restrict__ rdispls,
+                                        const int64_t *__restrict__ sendbase,
+                                        const int64_t *__restrict__ recvbase, int64_t *sz,
+                                        int64_t *loc, int64_t *dir_len, int64_t *dir_src,
+                                        int64_t *dir_dst, int64_t *rot_len, int64_t *rot_src,
+                                        int64_t *rot_dst, int rot_dense) {
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int64_t PP = (int64_t)t.P * t.P;
+  if (idx >= PP) return;
+  const int p = (int)(idx / t.P), sigma = (int)(idx % t.P);
+  const int n = p / t.Q, q = p % t.Q, io = sigma / t.Q, jo = sigma % t.Q;
+  const int dest = ((n + io) % t.N) * t.Q + (q + jo) % t.Q;
+  const int64_t bytes = counts[(int64_t)p * t.P + dest] * t.elem;
+  const int64_t sloc = TUNA_LOC(TUNA_BUF_SEND, (sendbase[p] + sdispls[(int64_t)p * t.P + dest]) * t.elem);
+  sz[idx] = bytes;
+  loc[idx] = sloc;
+  // direct list entry (d = p as receiver, s = sigma as source index)
+  {
+    const int d = p, s = sigma;
+    dir_len[idx] = counts[(int64_t)s * t.P + d] * t.elem;
+    dir_src[idx] = TUNA_LOC(TUNA_BUF_SEND, (sendbase[s] + sdispls[(int64_t)s * t.P + d]) * t.elem);
+    dir_dst[idx] = TUNA_LOC(TUNA_BUF_RECV, (recvbase[d] + rdispls[(int64_t)d * t.P + s]) * t.elem);
+  }
+  if (sigma == 0) {
+    const int64_t r = rot_dense ? idx : p;
+    rot_len[r] = bytes;
+    rot_src[r] = sloc;
+    rot_dst[r] = TUNA_LOC(TUNA_BUF_RECV, (recvbase[p] + rdispls[(int64_t)p * t.P + p]) * t.elem);
+  }
+}
+
+// Count-metadata exchange of one digit phase: the receiver (p', sigma) of every
+// moving slot learns the size of the block its partner holds, and where the
+// partner keeps it.  Non-moving slots keep their size.  Also accumulates the
+// per-round byte totals (round z = the slots whose digit equals z).
+__global__ void tuna_meta_exchange_kernel(TunaTopo t, PhaseDev ph, const int64_t *__restrict__ sz_cur,
+                                          const int64_t *__restrict__ loc_cur, int64_t *sz_next,
+                                          int64_t *len, int64_t *src,
+                                          unsigned long long *round_bytes) {
+  extern __shared__ unsigned long long s_hist[];
+  const bool use_smem = ph.radix <= 4096;
+  if (use_smem) {
+    for (int i = threadIdx.x; i < ph.radix; i += blockDim.x) s_hist[i] = 0;
+    __syncthreads();
+  }
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int64_t PP = (int64_t)t.P * t.P;
+  if (idx < PP) {
+    const int p = (int)(idx / t.P), sigma = (int)(idx % t.P);
+    const int n = p / t.Q, q = p % t.Q, io = sigma / t.Q, jo = sigma % t.Q;
+    const int v = ph.level == 0 ? jo : io;
+    const int dig = (int)((v / ph.stride) % ph.radix);
+    if (dig == 0) {
+      sz_next[idx] = sz_cur[idx];
+    } else {
+      const int64_t dist = dig * ph.stride;
+      int sender;
+      int64_t e;
+      if (ph.level == 0) {
+        sender = n * t.Q + (int)(((q - dist) % t.Q + t.Q) % t.Q);
+        e = (int64_t)p * ph.per_rank + (int64_t)io * ph.moving + compact_of(jo, ph.stride, ph.radix);
+      } else {
+        sender = (int)(((n - dist) % t.N + t.N) % t.N) * t.Q + q;
+        e = (int64_t)p * ph.per_rank + compact_of(io, ph.stride, ph.radix) * t.Q + jo;
+      }
+      const int64_t bytes = sz_cur[(int64_t)sender * t.P + sigma];
+      sz_next[idx] = bytes;
+      len[e] = bytes;
+      src[e] = loc_cur[(int64_t)sender * t.P + sigma];
+      if (bytes > 0) {
+        if (use_smem)
+          atomicAdd(&s_hist[dig], (unsigned long long)bytes);
+        else
+          atomicAdd(&round_bytes[dig], (unsigned long long)bytes);
+      }
+    }
+  }
+  if (use_smem) {
+    __syncthreads();
+    for (int i = threadIdx.x; i < ph.radix; i += blockDim.x)
+      if (s_hist[i]) atomicAdd(&round_bytes[i], s_hist[i]);
+  }
+}
+
+// Segmented exclusive prefix sum, one warp per segment, warp-shuffle scan over
+// 32-wide tiles with a running carry.  PAD rounds every value up to 16 first.
+// seg_total[s] receives the segment's (padded) sum, seg_raw[s] (optional) the
+// unpadded sum.
+template <bool PAD>
+__global__ void tuna_segscan_kernel(const int64_t *__restrict__ val, int64_t *out,
+                                    int64_t *seg_total, int64_t *seg_raw, int64_t seglen,
+                                    int64_t nseg) {
+  const int64_t w = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (w >= nseg) return;
+  int64_t carry = 0, raw = 0;
+  const int64_t *v = val + w * seglen;
+  int64_t *o = out + w * seglen;
+  for (int64_t base = 0; base < seglen; base += 32) {
+    const int64_t i = base + lane;
+    int64_t x = i < seglen ? v[i] : 0;
+    raw += x;
+    if (PAD) x = pad16(x);
+    int64_t incl = x;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const int64_t y = __shfl_up_sync(0xffffffffu, incl, d);
+      if (lane >= d) incl += y;
+    }
+    if (i < seglen) o[i] = carry + incl - x;
+    carry += __shfl_sync(0xffffffffu, incl, 31);
+  }
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) raw += __shfl_xor_sync(0xffffffffu, raw, d);
+  if (lane == 0) {
+    seg_total[w] = carry;
+    if (seg_raw) seg_raw[w] = raw;
+  }
+}
+
+// Exclusive scan of the nseg segment totals (one CTA), giving every segment's
+// base in the list's stream.  scal[0] = stream bytes, scal[1] = bytes moved.
+// If wbase is given, wbase[1] = wbase[0] + (stream bytes rounded up to 256),
+// or wbase[0] when the phase keeps nothing in the workspace.
+__global__ void tuna_segbase_kernel(const int64_t *__restrict__ seg_total,
+                                    const int64_t *__restrict__ seg_raw, int64_t *seg_base,
+                                    int64_t nseg, int64_t *scal, int64_t *wbase, int uses_work) {
+  __shared__ int64_t s_warp[32];
+  __shared__ int64_t s_carry;
+  __shared__ int64_t s_raw[32];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+  if (threadIdx.x == 0) s_carry = 0;
+  int64_t raw = 0;
+  __syncthreads();
+  for (int64_t base = 0; base < nseg; base += blockDim.x) {
+    const int64_t i = base + threadIdx.x;
+    const int64_t x = i < nseg ? seg_total[i] : 0;
+    if (seg_raw && i < nseg) raw += seg_raw[i];
+    int64_t incl = x;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const int64_t y = __shfl_up_sync(0xffffffffu, incl, d);
+      if (lane >= d) incl += y;
+    }
+    if (lane == 31) s_warp[warp] = incl;
+    __syncthreads();
+    int64_t woff = 0;
+    for (int k = 0; k < warp; k++) woff += s_warp[k];
+    const int64_t carry = s_carry;
+    if (i < nseg) seg_base[i] = carry + woff + incl - x;
+    __syncthreads();
+    if (threadIdx.x == blockDim.x - 1) s_carry = carry + woff + incl;
+    __syncthreads();
+  }
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) raw += __shfl_xor_sync(0xffffffffu, raw, d);
+  if (lane == 0) s_raw[warp] = raw;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int64_t r = 0;
+    for (int k = 0; k < nw; k++) r += s_raw[k];
+    scal[0] = s_carry;
+    scal[1] = r;
+    if (wbase) wbase[1] = wbase[0] + (uses_work ? ((s_carry + 255) & ~(int64_t)255) : 0);
+  }
+}
+
+// pos[e] += base of its segment (turns per-rank scans into one stream position).
+__global__ void tuna_add_base_kernel(int64_t *pos, const int64_t *__restrict__ seg_base,
+                                     int64_t seglen, int64_t n) {
+  const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (e < n) pos[e] += seg_base[e / seglen];
+}
+
+// Second half of a digit phase, after the prefix sums: destination of every
+// moving block, and the location table for the next phase.  A block whose
+// remaining digits are all zero has arrived: its destination is its place in
+// the receive buffer (direct-to-R) or, in classic mode, still the workspace,
+// with a rotation descriptor recorded for the final reorder.
+__global__ void tuna_place_kernel(TunaTopo t, PhaseDev ph, const int64_t *__restrict__ loc_cur,
+                                  int64_t *loc_next, int64_t *pos,
+                                  const int64_t *__restrict__ seg_base,
+                                  const int64_t *__restrict__ len, int64_t *dst,
+                                  const int64_t *__restrict__ wbase,
+                                  const int64_t *__restrict__ rdispls,
+                                  const int64_t *__restrict__ recvbase, int classic,
+                                  int64_t *rot_len, int64_t *rot_src, int64_t *rot_dst) {
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int64_t PP = (int64_t)t.P * t.P;
+  if (idx >= PP) return;
+  const int p = (int)(idx / t.P), sigma = (int)(idx % t.P);
+  const int n = p / t.Q, q = p % t.Q, io = sigma / t.Q, jo = sigma % t.Q;
+  const int v = ph.level == 0 ? jo : io;
+  const int dig = (int)((v / ph.stride) % ph.radix);
+  if (dig == 0) {
+    loc_next[idx] = loc_cur[idx];
+    return;
+  }
+  int64_t e;
+  bool fin;
+  if (ph.level == 0) {
+    e = (int64_t)p * ph.per_rank + (int64_t)io * ph.moving + compact_of(jo, ph.stride, ph.radix);
+    fin = (io == 0) && (jo / (ph.stride * ph.radix) == 0);
+  } else {
+    e = (int64_t)p * ph.per_rank + compact_of(io, ph.stride, ph.radix) * t.Q + jo;
+    fin = io / (ph.stride * ph.radix) == 0;
+  }
+  const int64_t w = pos[e] + seg_base[p];
+  pos[e] = w;
+  const int64_t wloc = TUNA_LOC(TUNA_BUF_WORK, wbase[0] + w);
+  int64_t d = wloc;
+  if (fin) {
+    const int origin = ((n - io + t.N) % t.N) * t.Q + (q - jo + t.Q) % t.Q;
+    const int64_t rloc =
+        TUNA_LOC(TUNA_BUF_RECV, (recvbase[p] + rdispls[(int64_t)p * t.P + origin]) * t.elem);
+    if (classic) {
+      rot_len[idx] = len[e];
+      rot_src[idx] = wloc;
+      rot_dst[idx] = rloc;
+    } else {
+      d = rloc;
+    }
+  }
+  dst[e] = d;
+  loc_next[idx] = d;
+}
+
+// First descriptor of every chunk: the last e with pos[e] <= c * chunk.
+__global__ void tuna_chunk_index_kernel(const int64_t *__restrict__ pos, int64_t n, int64_t chunk,
+                                        int64_t nchunks, int32_t *first) {
+  const int64_t c = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= nchunks) return;
+  const int64_t target = c * chunk;
+  int64_t lo = 0, hi = n;  // first index with pos > target
+  while (lo < hi) {
+    const int64_t mid = (lo + hi) >> 1;
+    if (pos[mid] <= target)
+      lo = mid + 1;
+    else
+      hi = mid;
+  }
+  first[c] = (int32_t)(lo > 0 ? lo - 1 : 0);
+}
+
+__global__ void tuna_transpose_kernel(const int64_t *__restrict__ in, int64_t *out, int P) {
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= (int64_t)P * P) return;
+  const int r = (int)(idx / P), c = (int)(idx % P);
+  out[idx] = in[(int64_t)c * P + r];
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------ the plan object
+
+struct tuna_plan {
+  TunaTopo topo{};
+  int radix_l = 2, radix_g = 2;
+  unsigned flags = 0;
+  bool classic = false;
+  int cuda_err = 0;
+  int last_launches = 0;
+
+  std::vector<TunaPhase> phases;
+  std::vector<TunaList> lists;  // one per phase
+  TunaList rot, dir;
+
+  struct Round {
+    int level, x, z, phase;
+    int64_t units, bytes;
+  };
+  std::vector<Round> rounds;
+
+  // host copies for validation
+  std::vector<int64_t> h_counts, h_sdispls, h_rdispls;
+  bool have_sdispls = false, have_rdispls = false;
+  int64_t send_extent = 0, recv_extent = 0, payload = 0;  // bytes
+
+  // device tables
+  int64_t *d_counts = nullptr, *d_sdispls = nullptr, *d_rdispls = nullptr;
+  int64_t *d_sendbase = nullptr, *d_recvbase = nullptr;
+  int64_t *d_sz[2] = {nullptr, nullptr}, *d_loc[2] = {nullptr, nullptr};
+  int64_t *d_seg_total = nullptr, *d_seg_raw = nullptr, *d_seg_base = nullptr;
+  int64_t *d_tmp = nullptr;      // P*P scratch (transpose)
+  int64_t *d_scal = nullptr;     // per list: stream bytes, bytes moved
+  int64_t *d_wbase = nullptr;    // phases + 1 workspace offsets
+  unsigned long long *d_round_bytes = nullptr;
+  int64_t stats_n = 0;
+
+  int64_t workspace_need = 0;
+  char *workspace = nullptr;
+  size_t workspace_bytes = 0;
+};
+
+namespace {
+
+#define TUNA_CUDA(plan, call)                     \
+  do {                                            \
+    cudaError_t e_ = (call);                      \
+    if (e_ != cudaSuccess) {                      \
+      (plan)->cuda_err = (int)e_;                 \
+      return TUNA_ERR_CUDA;                       \
+    }                                             \
+  } while (0)
+
+int64_t ipow64(int64_t r, int x) {
+  int64_t v = 1;
+  while (x-- > 0) v *= r;
+  return v;
+}
+
+int num_digits(int count, int r) {
+  int w = 0;
+  int64_t pw = 1;
+  while (pw < count) {
+    pw *= r;
+    w++;
+  }
+  return w;
+}
+
+int64_t count_digit(int count, int r, int x, int z) {  // offsets < count with digit x == z
+  int64_t c = 0, stride = ipow64(r, x);
+  for (int v = 0; v < count; v++) c += ((v / stride) % r) == z;
+  return c;
+}
+
+template <class T>
+cudaError_t dev_alloc(T **p, int64_t n) {
+  return cudaMalloc((void **)p, (size_t)std::max<int64_t>(n, 1) * sizeof(T));
+}
+
+void free_list(TunaList &l) {
+  cudaFree(l.len);
+  cudaFree(l.pos);
+  cudaFree(l.src);
+  cudaFree(l.dst);
+  cudaFree(l.chunk_first);
+  l = TunaList();
+}
+
+int alloc_list(tuna_plan *pl, TunaList &l, int64_t n) {
+  l.n = n;
+  TUNA_CUDA(pl, dev_alloc(&l.len, n));
+  TUNA_CUDA(pl, dev_alloc(&l.pos, n));
+  TUNA_CUDA(pl, dev_alloc(&l.src, n));
+  TUNA_CUDA(pl, dev_alloc(&l.dst, n));
+  return TUNA_OK;
+}
+
+int64_t env_i64(const char *name, int64_t dflt) {
+  const char *s = getenv(name);
+  if (!s || !*s) return dflt;
+  return strtoll(s, nullptr, 10);
+}
+
+// Bytes of destination stream per CTA: enough chunks to fill the machine several
+// times over, but no smaller than a few KiB (descriptor overhead) and no larger
+// than 128 KiB (tail effect).
+int64_t pick_chunk(int64_t total) {
+  const int64_t forced = env_i64("TUNA_CHUNK_BYTES", 0);
+  if (forced >= 1024) return (forced + 15) & ~(int64_t)15;
+  int64_t c = 8192;
+  while (c < 65536 && total / c > 148 * 32) c <<= 1;
+  return c;
+}
+
+int build_chunks(tuna_plan *pl, TunaList &l, cudaStream_t st) {
+  l.chunk = pick_chunk(l.total);
+  l.nchunks = l.total > 0 ? (l.total + l.chunk - 1) / l.chunk : 0;
+  if (l.nchunks > l.chunk_cap) {
+    cudaFree(l.chunk_first);
+    l.chunk_first = nullptr;
+    l.chunk_cap = 0;
+    TUNA_CUDA(pl, dev_alloc(&l.chunk_first, l.nchunks));
+    l.chunk_cap = l.nchunks;
+  }
+  if (l.nchunks > 0) {
+    const int th = 128;
+    tuna_chunk_index_kernel<<<(unsigned)((l.nchunks + th - 1) / th), th, 0, st>>>(
+        l.pos, l.n, l.chunk, l.nchunks, l.chunk_first);
+    TUNA_CUDA(pl, cudaGetLastError());
+  }
+  return TUNA_OK;
+}
+
+// scan of one list: per-rank warp scans, segment bases, (optionally) add bases
+int scan_list(tuna_plan *pl, TunaList &l, int64_t seglen, int64_t nseg, int list_id,
+              int64_t *wbase_slot, int uses_work, bool add_base, cudaStream_t st) {
+  if (nseg > 0 && seglen > 0) {
+    const int th = 256;
+    const int64_t blocks = (nseg * 32 + th - 1) / th;
+    tuna_segscan_kernel<true><<<(unsigned)blocks, th, 0, st>>>(l.len, l.pos, pl->d_seg_total,
+                                                                pl->d_seg_raw, seglen, nseg);
+    TUNA_CUDA(pl, cudaGetLastError());
+  }
+  tuna_segbase_kernel<<<1, 1024, 0, st>>>(pl->d_seg_total, pl->d_seg_raw, pl->d_seg_base,
+                                          (nseg > 0 && seglen > 0) ? nseg : 0,
+                                          pl->d_scal + 2 * list_id, wbase_slot, uses_work);
+  TUNA_CUDA(pl, cudaGetLastError());
+  if (add_base && l.n > 0) {
+    const int th = 256;
+    tuna_add_base_kernel<<<(unsigned)((l.n + th - 1) / th), th, 0, st>>>(l.pos, pl->d_seg_base,
+                                                                          seglen, l.n);
+    TUNA_CUDA(pl, cudaGetLastError());
+  }
+  return TUNA_OK;
+}
+
+int validate_layout(int P, const int64_t *counts, const int64_t *sdispls, const int64_t *rdispls,
+                    const int64_t *sendbase, const int64_t *recvbase) {
+  if (!counts) return TUNA_ERR_INVALID_ARG;
+  const int64_t PP = (int64_t)P * P;
+  for (int64_t i = 0; i < PP; i++) {
+    if (counts[i] < 0) return TUNA_ERR_INVALID_ARG;
+    if (sdispls && sdispls[i] < 0) return TUNA_ERR_INVALID_ARG;
+    if (rdispls && rdispls[i] < 0) return TUNA_ERR_INVALID_ARG;
+  }
+  for (int p = 0; p < P; p++) {
+    if (sendbase && sendbase[p] < 0) return TUNA_ERR_INVALID_ARG;
+    if (recvbase && recvbase[p] < 0) return TUNA_ERR_INVALID_ARG;
+  }
+  return TUNA_OK;
+}
+
+// Uploads the layout, runs every plan kernel, reads the totals back.
+int build_tables(tuna_plan *pl, const int64_t *counts, const int64_t *sdispls,
+                 const int64_t *rdispls, const int64_t *sendbase, const int64_t *recvbase,
+                 cudaStream_t st) {
+  const TunaTopo &t = pl->topo;
+  const int P = t.P;
+  const int64_t PP = (int64_t)P * P;
+  int rc = validate_layout(P, counts, sdispls, rdispls, sendbase, recvbase);
+  if (rc) return rc;
+
+  // host bookkeeping: copies for later validation, region sizes, extents
+  pl->h_counts.assign(counts, counts + PP);
+  pl->have_sdispls = sdispls != nullptr;
+  pl->have_rdispls = rdispls != nullptr;
+  if (sdispls) pl->h_sdispls.assign(sdispls, sdispls + PP); else pl->h_sdispls.clear();
+  if (rdispls) pl->h_rdispls.assign(rdispls, rdispls + PP); else pl->h_rdispls.clear();
+  std::vector<int64_t> sreg(P, 0), rreg(P, 0), sb(P), rb(P);
+  int64_t payload = 0;
+  for (int s = 0; s < P; s++)
+    for (int d = 0; d < P; d++) {
+      const int64_t c = counts[(int64_t)s * P + d];
+      payload += c;
+      if (sdispls) sreg[s] = std::max(sreg[s], sdispls[(int64_t)s * P + d] + c); else sreg[s] += c;
+      if (rdispls) rreg[d] = std::max(rreg[d], rdispls[(int64_t)d * P + s] + c); else rreg[d] += c;
+    }
+  int64_t se = 0, re = 0, acc_s = 0, acc_r = 0;
+  for (int p = 0; p < P; p++) {
+    sb[p] = sendbase ? sendbase[p] : acc_s;
+    rb[p] = recvbase ? recvbase[p] : acc_r;
+    acc_s += sreg[p];
+    acc_r += rreg[p];
+    se = std::max(se, sb[p] + sreg[p]);
+    re = std::max(re, rb[p] + rreg[p]);
+  }
+  pl->payload = payload * t.elem;
+  pl->send_extent = se * t.elem;
+  pl->recv_extent = re * t.elem;
+
+  TUNA_CUDA(pl, cudaMemcpyAsync(pl->d_counts, counts, PP * 8, cudaMemcpyHostToDevice, st));
+  TUNA_CUDA(pl, cudaMemcpyAsync(pl->d_sendbase, sb.data(), P * 8, cudaMemcpyHostToDevice, st));
+  TUNA_CUDA(pl, cudaMemcpyAsync(pl->d_recvbase, rb.data(), P * 8, cudaMemcpyHostToDevice, st));
+  // sb/rb are pageable stack-owned vectors: the copies above are staged by the
+  // runtime before returning, so they may go out of scope.
+  const int th = 256;
+  const unsigned gPP = (unsigned)((PP + th - 1) / th);
+  const unsigned gseg = (unsigned)(((int64_t)P * 32 + th - 1) / th);
+  if (sdispls) {
+    TUNA_CUDA(pl, cudaMemcpyAsync(pl->d_sdispls, sdispls, PP * 8, cudaMemcpyHostToDevice, st));
+  } else {  // packed: exclusive scan of every rank's row of counts
+    tuna_segscan_kernel<false><<<gseg, th, 0, st>>>(pl->d_counts, pl->d_sdispls, pl->d_seg_total,
+                                                     nullptr, P, P);
+    TUNA_CUDA(pl, cudaGetLastError());
+  }
+  if (rdispls) {
+    TUNA_CUDA(pl, cudaMemcpyAsync(pl->d_rdispls, rdispls, PP * 8, cudaMemcpyHostToDevice, st));
+  } else {  // packed: scan of the receive counts = rows of the transposed matrix
+    tuna_transpose_kernel<<<gPP, th, 0, st>>>(pl->d_counts, pl->d_tmp, P);
+    TUNA_CUDA(pl, cudaGetLastError());
+    tuna_segscan_kernel<false><<<gseg, th, 0, st>>>(pl->d_tmp, pl->d_rdispls, pl->d_seg_total,
+                                                     nullptr, P, P);
+    TUNA_CUDA(pl, cudaGetLastError());
+  }
+
+  const int nph = (int)pl->phases.size();
+  TUNA_CUDA(pl, cudaMemsetAsync(pl->d_round_bytes, 0, (size_t)std::max<int64_t>(pl->stats_n, 1) * 8, st));
+  TUNA_CUDA(pl, cudaMemsetAsync(pl->d_wbase, 0, (size_t)(nph + 1) * 8, st));
+  if (pl->classic) {
+    TUNA_CUDA(pl, cudaMemsetAsync(pl->rot.len, 0, (size_t)PP * 8, st));
+    TUNA_CUDA(pl, cudaMemsetAsync(pl->rot.src, 0, (size_t)PP * 8, st));
+    TUNA_CUDA(pl, cudaMemsetAsync(pl->rot.dst, 0, (size_t)PP * 8, st));
+  }
+  tuna_init_tables_kernel<<<gPP, th, 0, st>>>(t, pl->d_counts, pl->d_sdispls, pl->d_rdispls,
+                                              pl->d_sendbase, pl->d_recvbase, pl->d_sz[0],
+                                              pl->d_loc[0], pl->dir.len, pl->dir.src, pl->dir.dst,
+                                              pl->rot.len, pl->rot.src, pl->rot.dst,
+                                              pl->classic ? 1 : 0);
+  TUNA_CUDA(pl, cudaGetLastError());
+
+  int cur = 0;
+  for (int f = 0; f < nph; f++) {
+    const TunaPhase &ph = pl->phases[f];
+    TunaList &l = pl->lists[f];
+    PhaseDev pd{ph.level, ph.radix, ph.count, ph.stride, ph.moving, ph.per_rank};
+    const size_t smem = ph.radix <= 4096 ? (size_t)ph.radix * 8 : 0;
+    tuna_meta_exchange_kernel<<<gPP, th, smem, st>>>(t, pd, pl->d_sz[cur], pl->d_loc[cur],
+                                                     pl->d_sz[cur ^ 1], l.len, l.src,
+                                                     pl->d_round_bytes + ph.stats_off);
+    TUNA_CUDA(pl, cudaGetLastError());
+    // in direct-to-R mode the last phase delivers everything: it keeps nothing
+    const int uses_work = (pl->classic || f + 1 < nph) ? 1 : 0;
+    rc = scan_list(pl, l, ph.per_rank, P, f, pl->d_wbase + f, uses_work, false, st);
+    if (rc) return rc;
+    tuna_place_kernel<<<gPP, th, 0, st>>>(t, pd, pl->d_loc[cur], pl->d_loc[cur ^ 1], l.pos,
+                                          pl->d_seg_base, l.len, l.dst, pl->d_wbase + f,
+                                          pl->d_rdispls, pl->d_recvbase, pl->classic ? 1 : 0,
+                                          pl->rot.len, pl->rot.src, pl->rot.dst);
+    TUNA_CUDA(pl, cudaGetLastError());
+    cur ^= 1;
+  }
+  // work partitions of the rotation and direct lists
+  rc = scan_list(pl, pl->rot, pl->classic ? P : 1, P, nph, nullptr, 0, true, st);
+  if (rc) return rc;
+  rc = scan_list(pl, pl->dir, P, P, nph + 1, nullptr, 0, true, st);
+  if (rc) return rc;
+
+  // one read-back: stream totals, workspace offsets, per-round bytes
+  std::vector<int64_t> scal(2 * (nph + 2)), wbase(nph + 1);
+  std::vector<unsigned long long> rbytes(std::max<int64_t>(pl->stats_n, 1));
+  TUNA_CUDA(pl, cudaMemcpyAsync(scal.data(), pl->d_scal, scal.size() * 8, cudaMemcpyDeviceToHost, st));
+  TUNA_CUDA(pl, cudaMemcpyAsync(wbase.data(), pl->d_wbase, wbase.size() * 8, cudaMemcpyDeviceToHost, st));
+  TUNA_CUDA(pl, cudaMemcpyAsync(rbytes.data(), pl->d_round_bytes, rbytes.size() * 8,
+                                cudaMemcpyDeviceToHost, st));
+  TUNA_CUDA(pl, cudaStreamSynchronize(st));
+  for (int f = 0; f < nph; f++) {
+    pl->lists[f].total = scal[2 * f];
+    pl->lists[f].bytes = scal[2 * f + 1];
+  }
+  pl->rot.total = scal[2 * nph];
+  pl->rot.bytes = scal[2 * nph + 1];
+  pl->dir.total = scal[2 * (nph + 1)];
+  pl->dir.bytes = scal[2 * (nph + 1) + 1];
+  pl->workspace_need = wbase[nph];
+  for (auto &r : pl->rounds) r.bytes = (int64_t)rbytes[pl->phases[r.phase].stats_off + r.z];
+
+  for (int f = 0; f < nph; f++) {
+    rc = build_chunks(pl, pl->lists[f], st);
+    if (rc) return rc;
+  }
+  rc = build_chunks(pl, pl->rot, st);
+  if (rc) return rc;
+  rc = build_chunks(pl, pl->dir, st);
+  if (rc) return rc;
+  TUNA_CUDA(pl, cudaStreamSynchronize(st));
+  return TUNA_OK;
+}
+
+void add_level(tuna_plan *pl, int level, int count, int radix, int other) {
+  const int w = num_digits(count, radix);
+  for (int x = 0; x < w; x++) {
+    TunaPhase ph{};
+    ph.level = level;
+    ph.x = x;
+    ph.radix = radix;
+    ph.count = count;
+    ph.stride = ipow64(radix, x);
+    ph.moving = count - count_digit(count, radix, x, 0);
+    ph.per_rank = ph.moving * other;
+    ph.stats_off = pl->stats_n;
+    pl->stats_n += radix;
+    const int phase = (int)pl->phases.size();
+    pl->phases.push_back(ph);
+    for (int z = 1; z < radix; z++) {
+      if ((int64_t)z * ph.stride >= count) continue;
+      tuna_plan::Round r{};
+      r.level = level;
+      r.x = x;
+      r.z = z;
+      r.phase = phase;
+      // level 0 counts blocks, level 1 super-blocks (Q blocks each)
+      r.units = (int64_t)pl->topo.P * count_digit(count, radix, x, z) * (level == 0 ? other : 1);
+      pl->rounds.push_back(r);
+    }
+  }
+}
+
+int check_call_args(const tuna_plan *pl, const int64_t *sendcounts, const int64_t *sdispls,
+                    const int64_t *recvcounts, const int64_t *rdispls) {
+  const int P = pl->topo.P;
+  const int64_t PP = (int64_t)P * P;
+  if (sendcounts && memcmp(sendcounts, pl->h_counts.data(), PP * 8) != 0) return TUNA_ERR_COUNT_MISMATCH;
+  if (recvcounts)
+    for (int d = 0; d < P; d++)
+      for (int s = 0; s < P; s++)
+        if (recvcounts[(int64_t)d * P + s] != pl->h_counts[(int64_t)s * P + d])
+          return TUNA_ERR_COUNT_MISMATCH;
+  if (sdispls) {
+    if (pl->have_sdispls) {
+      if (memcmp(sdispls, pl->h_sdispls.data(), PP * 8) != 0) return TUNA_ERR_COUNT_MISMATCH;
+    } else {
+      for (int s = 0; s < P; s++) {
+        int64_t acc = 0;
+        for (int d = 0; d < P; d++) {
+          if (sdispls[(int64_t)s * P + d] != acc) return TUNA_ERR_COUNT_MISMATCH;
+          acc += pl->h_counts[(int64_t)s * P + d];
+        }
+      }
+    }
+  }
+  if (rdispls) {
+    if (pl->have_rdispls) {
+      if (memcmp(rdispls, pl->h_rdispls.data(), PP * 8) != 0) return TUNA_ERR_COUNT_MISMATCH;
+    } else {
+      for (int d = 0; d < P; d++) {
+        int64_t acc = 0;
+        for (int s = 0; s < P; s++) {
+          if (rdispls[(int64_t)d * P + s] != acc) return TUNA_ERR_COUNT_MISMATCH;
+          acc += pl->h_counts[(int64_t)s * P + d];
+        }
+      }
+    }
+  }
+  return TUNA_OK;
+}
+
+bool ranges_overlap(const void *a, size_t na, const void *b, size_t nb) {
+  const uintptr_t a0 = (uintptr_t)a, b0 = (uintptr_t)b;
+  return na > 0 && nb > 0 && a0 < b0 + nb && b0 < a0 + na;
+}
+
+TunaMoveArgs move_args(const TunaList &l, const void *send, void *recv, char *work) {
+  TunaMoveArgs a{};
+  a.len = l.len;
+  a.pos = l.pos;
+  a.src = l.src;
+  a.dst = l.dst;
+  a.chunk_first = l.chunk_first;
+  a.n = l.n;
+  a.total = l.total;
+  a.chunk = l.chunk;
+  a.nchunks = l.nchunks;
+  a.base[TUNA_BUF_SEND] = (char *)const_cast<void *>(send);
+  a.base[TUNA_BUF_RECV] = (char *)recv;
+  a.base[TUNA_BUF_WORK] = work;
+  return a;
+}
+
+int run_tuna(tuna_plan *pl, const void *send, void *recv, cudaStream_t st) {
+  if (pl->workspace_need > 0 &&
+      (!pl->workspace || pl->workspace_bytes < (size_t)pl->workspace_need))
+    return TUNA_ERR_WORKSPACE;
+  int launches = 0;
+  for (size_t f = 0; f < pl->lists.size(); f++) {
+    const TunaList &l = pl->lists[f];
+    if (l.nchunks == 0) continue;
+    TUNA_CUDA(pl, tuna_launch_move(TUNA_MOVE_ROUND, move_args(l, send, recv, pl->workspace), st));
+    launches++;
+  }
+  if (pl->rot.nchunks > 0) {
+    TUNA_CUDA(pl, tuna_launch_move(TUNA_MOVE_ROTATE, move_args(pl->rot, send, recv, pl->workspace), st));
+    launches++;
+  }
+  pl->last_launches = launches;
+  return TUNA_OK;
+}
+
+int run_direct(tuna_plan *pl, const void *send, void *recv, cudaStream_t st) {
+  int launches = 0;
+  if (pl->dir.nchunks > 0) {
+    TUNA_CUDA(pl, tuna_launch_move(TUNA_MOVE_DIRECT, move_args(pl->dir, send, recv, nullptr), st));
+    launches++;
+  }
+  pl->last_launches = launches;
+  return TUNA_OK;
+}
+
+int64_t align256(int64_t v) { return (v + 255) & ~(int64_t)255; }
+
+}  // namespace
+
+// ------------------------------------------------------------------ C ABI
+
+extern "C" {
+
+int tuna_version(void) { return 100; }
+
+const char *tuna_strerror(int status) {
+  switch (status) {
+    case TUNA_OK: return "success";
+    case TUNA_ERR_INVALID_ARG: return "invalid argument";
+    case TUNA_ERR_BAD_RADIX: return "radix out of range";
+    case TUNA_ERR_BAD_HIERARCHY: return "l * g != P";
+    case TUNA_ERR_COUNT_MISMATCH: return "counts or displacements do not match the plan";
+    case TUNA_ERR_OVERLAP: return "send and receive buffers overlap";
+    case TUNA_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case TUNA_ERR_CUDA: return "CUDA runtime error";
+    case TUNA_ERR_NOMEM: return "out of memory";
+    case TUNA_ERR_RANGE: return "index or size out of range";
+    default: return "unknown status";
+  }
+}
+
+int tuna_plan_destroy(tuna_plan_t *pl) {
+  if (!pl) return TUNA_OK;
+  for (auto &l : pl->lists) free_list(l);
+  free_list(pl->rot);
+  free_list(pl->dir);
+  cudaFree(pl->d_counts);
+  cudaFree(pl->d_sdispls);
+  cudaFree(pl->d_rdispls);
+  cudaFree(pl->d_sendbase);
+  cudaFree(pl->d_recvbase);
+  for (int i = 0; i < 2; i++) {
+    cudaFree(pl->d_sz[i]);
+    cudaFree(pl->d_loc[i]);
+  }
+  cudaFree(pl->d_seg_total);
+  cudaFree(pl->d_seg_raw);
+  cudaFree(pl->d_seg_base);
+  cudaFree(pl->d_tmp);
+  cudaFree(pl->d_scal);
+  cudaFree(pl->d_wbase);
+  cudaFree(pl->d_round_bytes);
+  delete pl;
+  return TUNA_OK;
+}
+
+int tuna_plan_create(tuna_plan_t **out, int P, int radix, int radix_global, int l, int g,
+                     int elem_size, unsigned flags, const int64_t *sendcounts,
+                     const int64_t *sdispls, const int64_t *rdispls, const int64_t *sendbase,
+                     const int64_t *recvbase, void *stream) {
+  if (!out) return TUNA_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (P < 1 || P > 32768 || elem_size < 1 || !sendcounts || l < 1 || g < 1) return TUNA_ERR_INVALID_ARG;
+  if ((int64_t)l * g != P) return TUNA_ERR_BAD_HIERARCHY;
+  if (radix < 2 || radix > std::max(2, l)) return TUNA_ERR_BAD_RADIX;
+  if (g > 1 && (radix_global < 2 || radix_global > std::max(2, g))) return TUNA_ERR_BAD_RADIX;
+  int rc = validate_layout(P, sendcounts, sdispls, rdispls, sendbase, recvbase);
+  if (rc) return rc;
+
+  tuna_plan *pl = new (std::nothrow) tuna_plan();
+  if (!pl) return TUNA_ERR_NOMEM;
+  pl->topo = TunaTopo{P, l, g, elem_size};
+  pl->radix_l = radix;
+  pl->radix_g = g > 1 ? radix_global : 2;
+  pl->flags = flags;
+  pl->classic = (flags & TUNA_FLAG_CLASSIC_ROTATE) != 0;
+  add_level(pl, 0, l, radix, g);
+  if (g > 1) add_level(pl, 1, g, pl->radix_g, l);
+
+  const int64_t PP = (int64_t)P * P;
+  const int nph = (int)pl->phases.size();
+  cudaStream_t st = (cudaStream_t)stream;
+  auto fail = [&](int code) {
+    tuna_plan_destroy(pl);
+    return code;
+  };
+#define TUNA_TRY(call)                                  \
+  do {                                                  \
+    cudaError_t e_ = (call);                            \
+    if (e_ != cudaSuccess) {                            \
+      int code_ = e_ == cudaErrorMemoryAllocation ? TUNA_ERR_NOMEM : TUNA_ERR_CUDA; \
+      (void)cudaGetLastError();                         \
+      return fail(code_);                               \
+    }                                                   \
+  } while (0)
+  TUNA_TRY(dev_alloc(&pl->d_counts, PP));
+  TUNA_TRY(dev_alloc(&pl->d_sdispls, PP));
+  TUNA_TRY(dev_alloc(&pl->d_rdispls, PP));
+  TUNA_TRY(dev_alloc(&pl->d_sendbase, P));
+  TUNA_TRY(dev_alloc(&pl->d_recvbase, P));
+  for (int i = 0; i < 2; i++) {
+    TUNA_TRY(dev_alloc(&pl->d_sz[i], PP));
+    TUNA_TRY(dev_alloc(&pl->d_loc[i], PP));
+  }
+  TUNA_TRY(dev_alloc(&pl->d_seg_total, P));
+  TUNA_TRY(dev_alloc(&pl->d_seg_raw, P));
+  TUNA_TRY(dev_alloc(&pl->d_seg_base, P));
+  TUNA_TRY(dev_alloc(&pl->d_tmp, PP));
+  TUNA_TRY(dev_alloc(&pl->d_scal, 2 * (nph + 2)));
+  TUNA_TRY(dev_alloc(&pl->d_wbase, nph + 1));
+  TUNA_TRY(dev_alloc(&pl->d_round_bytes, pl->stats_n));
+  pl->lists.resize(nph);
+  for (int f = 0; f < nph; f++) {
+    rc = alloc_list(pl, pl->lists[f], (int64_t)P * pl->phases[f].per_rank);
+    if (rc) return fail(pl->cuda_err == (int)cudaErrorMemoryAllocation ? TUNA_ERR_NOMEM : rc);
+  }
+  rc = alloc_list(pl, pl->rot, pl->classic ? PP : P);
+  if (rc) return fail(rc);
+  rc = alloc_list(pl, pl->dir, PP);
+  if (rc) return fail(rc);
+#undef TUNA_TRY
+  rc = build_tables(pl, sendcounts, sdispls, rdispls, sendbase, recvbase, st);
+  if (rc) return fail(rc);
+  *out = pl;
+  return TUNA_OK;
+}
+
+int tuna_plan_update_counts(tuna_plan_t *pl, const int64_t *sendcounts, const int64_t *sdispls,
+                            const int64_t *rdispls, const int64_t *sendbase,
+                            const int64_t *recvbase, void *stream) {
+  if (!pl || !sendcounts) return TUNA_ERR_INVALID_ARG;
+  return build_tables(pl, sendcounts, sdispls, rdispls, sendbase, recvbase, (cudaStream_t)stream);
+}
+
+int tuna_plan_workspace_bytes(const tuna_plan_t *pl, size_t *bytes) {
+  if (!pl || !bytes) return TUNA_ERR_INVALID_ARG;
+  *bytes = (size_t)pl->workspace_need;
+  return TUNA_OK;
+}
+
+int tuna_plan_host_staging_bytes(const tuna_plan_t *pl, size_t *bytes) {
+  if (!pl || !bytes) return TUNA_ERR_INVALID_ARG;
+  *bytes = (size_t)(align256(pl->send_extent) + align256(pl->recv_extent) + 256);
+  return TUNA_OK;
+}
+
+int tuna_plan_set_workspace(tuna_plan_t *pl, void *dev_ptr, size_t bytes) {
+  if (!pl) return TUNA_ERR_INVALID_ARG;
+  if (dev_ptr && ((uintptr_t)dev_ptr & 255)) return TUNA_ERR_WORKSPACE;
+  pl->workspace = (char *)dev_ptr;
+  pl->workspace_bytes = dev_ptr ? bytes : 0;
+  return TUNA_OK;
+}
+
+int tuna_plan_extents(const tuna_plan_t *pl, size_t *send_bytes, size_t *recv_bytes,
+                      size_t *payload_bytes) {
+  if (!pl) return TUNA_ERR_INVALID_ARG;
+  if (send_bytes) *send_bytes = (size_t)pl->send_extent;
+  if (recv_bytes) *recv_bytes = (size_t)pl->recv_extent;
+  if (payload_bytes) *payload_bytes = (size_t)pl->payload;
+  return TUNA_OK;
+}
+
+int tuna_alltoallv(tuna_plan_t *pl, const void *sendbuf, const int64_t *sendcounts,
+                   const int64_t *sdispls, void *recvbuf, const int64_t *recvcounts,
+                   const int64_t *rdispls, void *stream) {
+  if (!pl) return TUNA_ERR_INVALID_ARG;
+  if ((!sendbuf && pl->send_extent > 0) || (!recvbuf && pl->recv_extent > 0)) return TUNA_ERR_INVALID_ARG;
+  int rc = check_call_args(pl, sendcounts, sdispls, recvcounts, rdispls);
+  if (rc) return rc;
+  if (ranges_overlap(sendbuf, (size_t)pl->send_extent, recvbuf, (size_t)pl->recv_extent))
+    return TUNA_ERR_OVERLAP;
+  return run_tuna(pl, sendbuf, recvbuf, (cudaStream_t)stream);
+}
+
+int tuna_direct_alltoallv(tuna_plan_t *pl, const void *sendbuf, const int64_t *sendcounts,
+                          const int64_t *sdispls, void *recvbuf, const int64_t *recvcounts,
+                          const int64_t *rdispls, void *stream) {
+  if (!pl) return TUNA_ERR_INVALID_ARG;
+  if ((!sendbuf && pl->send_extent > 0) || (!recvbuf && pl->recv_extent > 0)) return TUNA_ERR_INVALID_ARG;
+  int rc = check_call_args(pl, sendcounts, sdispls, recvcounts, rdispls);
+  if (rc) return rc;
+  if (ranges_overlap(sendbuf, (size_t)pl->send_extent, recvbuf, (size_t)pl->recv_extent))
+    return TUNA_ERR_OVERLAP;
+  return run_direct(pl, sendbuf, recvbuf, (cudaStream_t)stream);
+}
+
+int tuna_alltoallv_host(tuna_plan_t *pl, const void *host_send, void *host_recv, int schedule,
+                        void *stream) {
+  if (!pl) return TUNA_ERR_INVALID_ARG;
+  if ((!host_send && pl->send_extent > 0) || (!host_recv && pl->recv_extent > 0)) return TUNA_ERR_INVALID_ARG;
+  if (schedule != TUNA_SCHEDULE_TUNA && schedule != TUNA_SCHEDULE_DIRECT) return TUNA_ERR_INVALID_ARG;
+  const int64_t w = align256(pl->workspace_need);
+  const int64_t need = w + align256(pl->send_extent) + align256(pl->recv_extent) + 256;
+  if (!pl->workspace || pl->workspace_bytes < (size_t)need) return TUNA_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  char *d_send = pl->workspace + w;
+  char *d_recv = d_send + align256(pl->send_extent);
+  if (pl->send_extent > 0)
+    TUNA_CUDA(pl, cudaMemcpyAsync(d_send, host_send, (size_t)pl->send_extent, cudaMemcpyHostToDevice, st));
+  int rc = schedule == TUNA_SCHEDULE_TUNA ? run_tuna(pl, d_send, d_recv, st)
+                                          : run_direct(pl, d_send, d_recv, st);
+  if (rc) return rc;
+  if (pl->recv_extent > 0)
+    TUNA_CUDA(pl, cudaMemcpyAsync(host_recv, d_recv, (size_t)pl->recv_extent, cudaMemcpyDeviceToHost, st));
+  return TUNA_OK;
+}
+
+int tuna_plan_num_rounds(const tuna_plan_t *pl, int *K) {
+  if (!pl || !K) return TUNA_ERR_INVALID_ARG;
+  *K = (int)pl->rounds.size();
+  return TUNA_OK;
+}
+
+int tuna_plan_round_info(const tuna_plan_t *pl, int k, int *level, int *x, int *z, int64_t *units,
+                         int64_t *bytes) {
+  if (!pl) return TUNA_ERR_INVALID_ARG;
+  if (k < 0 || k >= (int)pl->rounds.size()) return TUNA_ERR_RANGE;
+  const auto &r = pl->rounds[k];
+  if (level) *level = r.level;
+  if (x) *x = r.x;
+  if (z) *z = r.z;
+  if (units) *units = r.units;
+  if (bytes) *bytes = r.bytes;
+  return TUNA_OK;
+}
+
+int tuna_plan_num_phases(const tuna_plan_t *pl, int *n) {
+  if (!pl || !n) return TUNA_ERR_INVALID_ARG;
+  *n = (int)pl->phases.size();
+  return TUNA_OK;
+}
+
+int tuna_plan_phase_info(const tuna_plan_t *pl, int phase, int *level, int *x, int64_t *entries,
+                         int64_t *bytes, int64_t *stream_bytes) {
+  if (!pl) return TUNA_ERR_INVALID_ARG;
+  const TunaList *l;
+  if (phase == -1) l = &pl->rot;
+  else if (phase == -2) l = &pl->dir;
+  else if (phase >= 0 && phase < (int)pl->phases.size()) l = &pl->lists[phase];
+  else return TUNA_ERR_RANGE;
+  if (level) *level = phase >= 0 ? pl->phases[phase].level : -1;
+  if (x) *x = phase >= 0 ? pl->phases[phase].x : -1;
+  if (entries) *entries = l->n;
+  if (bytes) *bytes = l->bytes;
+  if (stream_bytes) *stream_bytes = l->total;
+  return TUNA_OK;
+}
+
+int tuna_plan_phase_tables(const tuna_plan_t *pl, int phase, int64_t cap, int64_t *len,
+                           int64_t *pos, int64_t *src, int64_t *dst, int64_t *rows) {
+  if (!pl) return TUNA_ERR_INVALID_ARG;
+  const TunaList *l;
+  if (phase == -1) l = &pl->rot;
+  else if (phase == -2) l = &pl->dir;
+  else if (phase >= 0 && phase < (int)pl->phases.size()) l = &pl->lists[phase];
+  else return TUNA_ERR_RANGE;
+  if (rows) *rows = l->n;
+  const int64_t n = std::min(cap, l->n);
+  if (n <= 0) return TUNA_OK;
+  tuna_plan *m = const_cast<tuna_plan *>(pl);
+  TUNA_CUDA(m, cudaDeviceSynchronize());
+  if (len) TUNA_CUDA(m, cudaMemcpy(len, l->len, n * 8, cudaMemcpyDeviceToHost));
+  if (pos) TUNA_CUDA(m, cudaMemcpy(pos, l->pos, n * 8, cudaMemcpyDeviceToHost));
+  if (src) TUNA_CUDA(m, cudaMemcpy(src, l->src, n * 8, cudaMemcpyDeviceToHost));
+  if (dst) TUNA_CUDA(m, cudaMemcpy(dst, l->dst, n * 8, cudaMemcpyDeviceToHost));
+  return TUNA_OK;
+}
+
+int tuna_plan_last_launches(const tuna_plan_t *pl, int *launches) {
+  if (!pl || !launches) return TUNA_ERR_INVALID_ARG;
+  *launches = pl->last_launches;
+  return TUNA_OK;
+}
+
+int tuna_plan_cuda_error(const tuna_plan_t *pl) { return pl ? pl->cuda_err : 0; }
+
+}  // extern "C"

@@ -1,0 +1,328 @@
+"""CUDA path vs CPU oracle, bit-exact, through the C ABI.  Needs a GPU."""
+import itertools
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2411_02581_b200 import binding as B
+from paper_2411_02581_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+CANARY = 0xA5
+
+
+def oracle_flat(wl, r, want_sizes=False):
+    send = wl.make_send().numpy()
+    recv = wl.make_recv(fill=CANARY).numpy().copy()
+    return oracle.tuna_flat(wl, r, send, recv, want_sizes=want_sizes)
+
+
+def oracle_hier(wl, Q, N, rl, rg):
+    send = wl.make_send().numpy()
+    recv = wl.make_recv(fill=CANARY).numpy().copy()
+    return oracle.tuna_hier(wl, Q, N, rl, rg, send, recv)
+
+
+def oracle_brute(wl):
+    send = wl.make_send().numpy()
+    recv = wl.make_recv(fill=CANARY).numpy().copy()
+    return oracle.bruteforce(wl, send, recv)
+
+
+def gpu_run(wl, radix, l=None, g=1, rg=2, flags=0, direct=False, explicit=True, pass_args=True,
+            misalign=0):
+    """Run the exchange on the GPU; returns (recv bytes as numpy, plan).
+    ``misalign`` shifts both device buffers by that many bytes off 256-byte alignment."""
+    send0 = wl.make_send("cuda")
+    recv0 = wl.make_recv("cuda", fill=CANARY)
+    if misalign:
+        sbuf = torch.empty(send0.numel() + 64, dtype=torch.uint8, device="cuda")
+        rbuf = torch.full((recv0.numel() + 64,), CANARY, dtype=torch.uint8, device="cuda")
+        send = sbuf[misalign:misalign + send0.numel()]
+        send.copy_(send0)
+        recv = rbuf[misalign:misalign + recv0.numel()]
+    else:
+        send, recv = send0, recv0
+    plan = B.plan_for(wl, radix, l=l, g=g, radix_global=rg, flags=flags, explicit_layout=explicit)
+    plan.alloc_workspace()
+    args = {}
+    if pass_args and explicit:
+        args = dict(sendcounts=wl.sendcounts, sdispls=wl.sdispls, recvcounts=wl.recvcounts,
+                    rdispls=wl.rdispls)
+    if direct:
+        plan.direct_alltoallv(send, recv, **args)
+    else:
+        plan.alltoallv(send, recv, **args)
+    torch.cuda.synchronize()
+    if misalign:
+        assert bool((rbuf[:misalign] == CANARY).all()) and bool((rbuf[misalign + recv0.numel():] == CANARY).all())
+    return recv.cpu().numpy(), plan
+
+
+def check_rounds(plan, rounds):
+    got = plan.rounds()
+    assert len(got) == len(rounds)
+    for g, row in zip(got, rounds):
+        assert (g["level"], g["x"], g["z"]) == tuple(int(v) for v in row[:3])
+        assert g["units"] == row[oracle.RS_UNITS]
+        assert g["bytes"] == row[oracle.RS_BYTES_SENT] == row[oracle.RS_BYTES_RECV]
+
+
+FLAT = [(P, r) for P in (1, 2, 3, 5, 8, 9, 16, 17) for r in sorted({2, 3, max(2, P // 2), max(2, P)})
+        if r <= max(2, P)]
+FLAT += [(33, 2), (33, 6), (64, 4), (100, 10), (130, 2), (130, 130)]
+
+
+@pytest.mark.parametrize("P,r", FLAT)
+@pytest.mark.parametrize("flags", [B.FLAG_DIRECT_TO_R, B.FLAG_CLASSIC_ROTATE])
+def test_flat_small(P, r, flags):
+    """Unaligned byte counts, gaps with canaries, every radix class, both placements."""
+    wl = W.make_random(P, 300, elem_size=1, seed=1000 + P, zero_frac=0.25, gaps=True)
+    ref, rounds, _, _ = oracle_flat(wl, r)
+    got, plan = gpu_run(wl, r, flags=flags)
+    assert np.array_equal(got, ref)
+    check_rounds(plan, rounds)
+    got_d, _ = gpu_run(wl, r, direct=True)
+    assert np.array_equal(got_d, ref)
+
+
+@pytest.mark.parametrize("elem", [1, 2, 3, 4, 8, 16, 48])
+@pytest.mark.parametrize("misalign", [0, 1, 4, 7])
+def test_element_sizes_and_buffer_alignment(elem, misalign):
+    wl = W.make_random(12, 700, elem_size=elem, seed=elem, zero_frac=0.1, gaps=True)
+    ref = oracle_brute(wl)
+    for r in (2, 4, 12):
+        got, _ = gpu_run(wl, r, misalign=misalign)
+        assert np.array_equal(got, ref)
+    got, _ = gpu_run(wl, 3, flags=B.FLAG_CLASSIC_ROTATE, misalign=misalign)
+    assert np.array_equal(got, ref)
+    got, _ = gpu_run(wl, 2, direct=True, misalign=misalign)
+    assert np.array_equal(got, ref)
+
+
+def test_large_blocks_span_many_chunks():
+    """Blocks far larger than one CTA's chunk, plus a ragged tail."""
+    wl = W.make_random(6, 3_000_000, elem_size=1, seed=77, zero_frac=0.2)
+    ref, rounds, _, _ = oracle_flat(wl, 2)
+    for flags in (0, B.FLAG_CLASSIC_ROTATE):
+        got, plan = gpu_run(wl, 2, flags=flags)
+        assert np.array_equal(got, ref)
+    check_rounds(plan, rounds)
+    got, _ = gpu_run(wl, 6, direct=True)
+    assert np.array_equal(got, ref)
+
+
+HIER = [(Q, N, rl, rg) for Q, N in [(1, 4), (4, 1), (2, 2), (3, 4), (5, 3), (4, 4), (8, 4), (6, 5)]
+        for rl in sorted({2, max(2, Q)}) for rg in sorted({2, 3, max(2, N)})
+        if rl <= max(2, Q) and rg <= max(2, N)]
+
+
+@pytest.mark.parametrize("Q,N,rl,rg", HIER)
+def test_hier_small(Q, N, rl, rg):
+    P = Q * N
+    wl = W.make_random(P, 200, elem_size=2, seed=31 * P + rl + rg, zero_frac=0.2, gaps=True)
+    ref, rounds, _, _ = oracle_hier(wl, Q, N, rl, rg)
+    for flags in (0, B.FLAG_CLASSIC_ROTATE):
+        got, plan = gpu_run(wl, rl, l=Q, g=N, rg=rg, flags=flags)
+        assert np.array_equal(got, ref)
+        check_rounds(plan, rounds)
+
+
+@pytest.mark.parametrize("P,r", [(8, 2), (9, 3), (16, 4), (20, 5), (64, 8)])
+def test_metadata_and_prefix_sums(P, r):
+    """Descriptor tables of every digit phase: sizes equal the oracle's
+    message-passed metadata, positions equal its running sums."""
+    wl = W.make_random(P, 500, elem_size=3, seed=P + r, zero_frac=0.3)
+    _, _, _, _, sizes = oracle_flat(wl, r, want_sizes=True)
+    plan = B.plan_for(wl, r)
+    assert plan.num_phases() == sizes.shape[0]
+    work_off = 0
+    for x in range(plan.num_phases()):
+        t = plan.phase_tables(x)
+        moving = [o for o in range(P) if (o // r ** x) % r != 0]
+        exp_len = sizes[x][:, moving]                        # receive-side order (rank, offset)
+        assert np.array_equal(t["len"].reshape(P, len(moving)), exp_len)
+        scan, tot = oracle.segmented_exclusive_scan(exp_len, 16)
+        base, _ = oracle.segmented_exclusive_scan(tot.reshape(1, P), 1)
+        exp_pos = scan + base.reshape(P, 1)
+        assert np.array_equal(t["pos"].reshape(P, len(moving)), exp_pos)
+        info = plan.phase_info(x)
+        assert info["bytes"] == exp_len.sum() and info["stream_bytes"] == tot.sum()
+        # destinations: final blocks in the receive buffer, the rest at their stream position
+        dst = t["dst"].reshape(P, len(moving))
+        for p in range(P):
+            for j, o in enumerate(moving):
+                if o < r ** (x + 1):
+                    s = (p - o) % P
+                    want = (1 << 56) | int(wl.recvbase[p] + wl.rdispls[p, s]) * wl.elem_size
+                else:
+                    want = (2 << 56) | (work_off + int(exp_pos[p, j]))
+                assert dst[p, j] == want
+        if x + 1 < plan.num_phases():
+            work_off += (int(tot.sum()) + 255) // 256 * 256
+    assert plan.workspace_bytes() == work_off
+
+
+def test_packed_layout_defaults_match_explicit():
+    """NULL displacement arrays mean 'packed'; the device-side scans must give
+    the same layout the generator computed on the host."""
+    wl = W.make_random(19, 90, elem_size=4, seed=8, zero_frac=0.2)
+    ref = oracle_brute(wl)
+    got, plan = gpu_run(wl, 3, explicit=False)
+    assert np.array_equal(got, ref)
+    assert plan.extents() == (wl.send_bytes, wl.recv_bytes, wl.payload_bytes_total)
+    d = plan.phase_tables(-2)
+    assert np.array_equal(d["len"].reshape(19, 19), wl.sendcounts.T * 4)
+    exp_dst = (wl.recvbase[:, None] + wl.rdispls) * 4 + (1 << 56)
+    assert np.array_equal(d["dst"].reshape(19, 19), exp_dst)
+
+
+def test_call_time_validation():
+    wl = W.make_random(6, 50, seed=4)
+    send = wl.make_send("cuda")
+    recv = wl.make_recv("cuda")
+    plan = B.plan_for(wl, 2)
+    with pytest.raises(B.TunaError, match="WORKSPACE"):
+        plan.alltoallv(send, recv)
+    plan.alloc_workspace()
+    bad = wl.sendcounts.copy()
+    bad[0, 1] += 1
+    with pytest.raises(B.TunaError, match="COUNT_MISMATCH"):
+        plan.alltoallv(send, recv, sendcounts=bad)
+    with pytest.raises(B.TunaError, match="COUNT_MISMATCH"):
+        plan.alltoallv(send, recv, recvcounts=wl.sendcounts + np.eye(6, dtype=np.int64))
+    with pytest.raises(B.TunaError, match="COUNT_MISMATCH"):
+        plan.alltoallv(send, recv, rdispls=wl.rdispls + 1)
+    both = torch.zeros(wl.send_bytes + wl.recv_bytes, dtype=torch.uint8, device="cuda")
+    with pytest.raises(B.TunaError, match="OVERLAP"):
+        plan.alltoallv(both, both[8:])
+    before = recv.clone()
+    torch.cuda.synchronize()
+    assert torch.equal(recv, before)            # failed calls wrote nothing
+    plan.alltoallv(send, recv, wl.sendcounts, wl.sdispls, wl.recvcounts, wl.rdispls)
+    torch.cuda.synchronize()
+    assert np.array_equal(recv.cpu().numpy(), oracle_brute(wl))
+
+
+def test_update_counts_and_rerun():
+    wl1 = W.make_random(10, 400, seed=21, zero_frac=0.1)
+    wl2 = W.make_random(10, 900, seed=22, zero_frac=0.4)
+    plan = B.plan_for(wl1, 3)
+    plan.alloc_workspace()
+    for wl in (wl1, wl2, wl1):
+        plan.update_counts(wl.sendcounts, wl.sdispls, wl.rdispls, wl.sendbase, wl.recvbase)
+        plan.alloc_workspace()
+        send, recv = wl.make_send("cuda"), wl.make_recv("cuda", fill=CANARY)
+        for _ in range(2):                       # re-runnable with the same plan
+            recv.fill_(CANARY)
+            plan.alltoallv(send, recv)
+            torch.cuda.synchronize()
+            ref, rounds, _, _ = oracle_flat(wl, 3)
+            assert np.array_equal(recv.cpu().numpy(), ref)
+        check_rounds(plan, rounds)
+
+
+def test_host_buffer_entry_point():
+    wl = W.make_random(9, 5000, seed=5, zero_frac=0.2)
+    ref = oracle_brute(wl)
+    plan = B.plan_for(wl, 3)
+    plan.alloc_workspace(host_staging=True)
+    hs = wl.make_send().pin_memory()
+    for schedule in (B.SCHEDULE_TUNA, B.SCHEDULE_DIRECT):
+        hr = torch.zeros(wl.recv_bytes, dtype=torch.uint8).pin_memory()
+        plan.alltoallv_host(hs, hr, schedule)
+        torch.cuda.synchronize()
+        assert np.array_equal(hr.numpy(), ref)
+    small = B.plan_for(wl, 3)
+    small.alloc_workspace(host_staging=False)
+    with pytest.raises(B.TunaError, match="WORKSPACE"):
+        small.alltoallv_host(hs, hr, B.SCHEDULE_TUNA)
+
+
+def test_degenerate_inputs():
+    for P in (1, 2, 7):
+        z = W._finish("zeros", P, 4, 1, np.zeros((P, P), dtype=np.int64))
+        got, plan = gpu_run(z, 2)
+        assert got.size == 0 and plan.last_launches() == 0
+        one = np.zeros((P, P), dtype=np.int64)
+        one[P - 1, 0] = 123457
+        wl = W._finish("one", P, 1, 1, one)
+        got, _ = gpu_run(wl, 2)
+        assert np.array_equal(got, oracle_brute(wl))
+        rc = W.make_random(P, 60, seed=9).sendcounts.copy()
+        rc[0, :] = 0
+        rc[:, P - 1] = 0
+        wl = W._finish("rc", P, 1, 1, rc)
+        for r in (2, max(2, P)):
+            got, _ = gpu_run(wl, r)
+            assert np.array_equal(got, oracle_brute(wl))
+
+
+# ---------------------------------------------------------------- the five workloads
+
+def test_c1_full():
+    wl = W.make_c1()
+    ref, rounds, _, _ = oracle_flat(wl, 2)
+    got, plan = gpu_run(wl, 2)
+    assert np.array_equal(got, ref)
+    check_rounds(plan, rounds)
+    v = got.view(np.int32)
+    for d in range(wl.P):                       # the payload names its own home
+        lo, hi = int(wl.recvbase[d]), int(wl.recvbase[d] + wl.recvcounts[d].sum())
+        assert np.all(((v[lo:hi] >> 10) & 1023) == d)
+
+
+@pytest.mark.parametrize("r", [2, 4, 8, 16, 64])
+def test_c2_full(r):
+    wl = W.make_c2()
+    ref, rounds, _, _ = oracle_flat(wl, r)
+    for flags in (0, B.FLAG_CLASSIC_ROTATE):
+        got, plan = gpu_run(wl, r, flags=flags)
+        assert np.array_equal(got, ref)
+    check_rounds(plan, rounds)
+    got, _ = gpu_run(wl, r, direct=True)
+    assert np.array_equal(got, ref)
+
+
+@pytest.mark.parametrize("rl,rg", list(itertools.product((2, 4, 16), (2, 4, 16))))
+def test_c3_full(rl, rg):
+    wl = W.make_c3()
+    ref, rounds, _, _ = oracle_hier(wl, 16, 16, rl, rg)
+    got, plan = gpu_run(wl, rl, l=16, g=16, rg=rg)
+    assert np.array_equal(got, ref)
+    check_rounds(plan, rounds)
+
+
+def test_c4_scaled_down():
+    """The token-dispatch shape with fewer tokens and a narrower hidden size, so
+    that the oracle finishes in seconds; blocks still span many chunks."""
+    wl = W.make_c4(P=64, tokens=256, hidden=512)
+    for r in (2, 8, 64):
+        ref, rounds, _, _ = oracle_flat(wl, r)
+        got, plan = gpu_run(wl, r)
+        assert np.array_equal(got, ref)
+        check_rounds(plan, rounds)
+    got, _ = gpu_run(wl, 2, direct=True)
+    assert np.array_equal(got, ref)
+
+
+@pytest.mark.parametrize("r", [2, 8, 32, 2048])
+def test_c5_full_flat(r):
+    wl = W.make_c5()
+    ref, rounds, _, _ = oracle_flat(wl, r)
+    got, plan = gpu_run(wl, r, pass_args=False)
+    assert np.array_equal(got, ref)
+    check_rounds(plan, rounds)
+
+
+def test_c5_full_hier_and_direct():
+    wl = W.make_c5()
+    ref, rounds, _, _ = oracle_hier(wl, 32, 64, 32, 64)
+    got, plan = gpu_run(wl, 32, l=32, g=64, rg=64, pass_args=False)
+    assert np.array_equal(got, ref)
+    check_rounds(plan, rounds)
+    got, _ = gpu_run(wl, 2, direct=True, pass_args=False)
+    assert np.array_equal(got, ref)

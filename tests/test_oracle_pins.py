@@ -373,3 +373,34 @@ def test_workload_shapes_small():
         assert np.array_equal(recv, brute(c5))
     recv, _, _, _ = run_hier(c5, 8, 8, 8, 8)
     assert np.array_equal(recv, brute(c5))
+
+
+# ---------------------------------------------------------------- metadata and prefix sums
+
+@pytest.mark.parametrize("P,r", [(8, 2), (9, 3), (16, 4), (13, 2), (20, 5), (12, 12)])
+def test_size_tables_follow_the_blocks(P, r):
+    """After the rounds of digit x, the block a rank holds for offset o has come
+    from the rank (o mod r^(x+1)) places below it; its size is the owner's count."""
+    wl = W.make_random(P, 40, elem_size=2, seed=P * r)
+    send = wl.make_send().numpy()
+    recv = wl.make_recv().numpy().copy()
+    _, _, _, _, sizes = oracle.tuna_flat(wl, r, send, recv, want_sizes=True)
+    C = wl.sendcounts * wl.elem_size
+    for x in range(sizes.shape[0]):
+        for p in range(P):
+            for o in range(P):
+                s = (p - o % r ** (x + 1)) % P
+                assert sizes[x, p, o] == C[s, (s + o) % P]
+
+
+def test_segmented_scan_against_numpy():
+    rng = np.random.default_rng(5)
+    for nseg, seglen, align in [(1, 1, 1), (3, 7, 1), (5, 33, 16), (64, 64, 16), (2, 100, 4)]:
+        v = rng.integers(0, 1000, size=(nseg, seglen)).astype(np.int64)
+        v[rng.random(v.shape) < 0.3] = 0
+        scan, tot = oracle.segmented_exclusive_scan(v, align)
+        pv = (v + align - 1) // align * align
+        assert np.array_equal(scan, np.cumsum(pv, axis=1) - pv)
+        assert np.array_equal(tot, pv.sum(axis=1))
+        assert np.all(scan[:, 0] == 0)
+        assert np.array_equal(scan[:, -1] + pv[:, -1], tot)      # last displacement + size = total
