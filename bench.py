@@ -1,0 +1,453 @@
+#!/usr/bin/env python
+"""Benchmark of the TuNA hot path on one B200 (or N independent replicas).
+
+A step is one pass of the whole path over one batch: the device-side re-plan
+for the batch's counts (count-metadata exchange + segmented prefix sums), then
+the exchange itself (one fused pack-move-unpack launch per digit phase and the
+rotation launch).  The headline workload is the mixture-of-experts token
+dispatch shape (P = 64 ranks, 8192 tokens per rank routed top-2, 8 KiB rows,
+8 GiB of payload) at the radix named by --radix; the other schedules (radix
+sweep, hierarchical, the single-pass direct exchange) are timed the same way
+and reported under "sweep".
+
+Prints ONE JSON line (rank 0).
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "alltoallv_payload_throughput"
+UNIT = "GB/s"
+
+# DRAM traffic of the dominant kernel from an ncu capture
+# (dram__bytes_read.sum + dram__bytes_write.sum per launch) divided by the payload
+# bytes that launch moved, keyed by the SHA-256 of the kernel source the capture
+# was taken with.  A changed source makes the figure stale: it is then reported
+# as null.
+NCU_TRAFFIC_PER_PAYLOAD_BYTE: dict[str, float] = {}
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c4", choices=["c1", "c2", "c3", "c4", "c4_skew", "c5"])
+    ap.add_argument("--radix", type=int, default=0, help="headline radix (0: the workload's largest)")
+    ap.add_argument("--no-sweep", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep-steps", type=int, default=10)
+    return ap.parse_args()
+
+
+def make_workload(name):
+    from paper_2411_02581_b200 import workloads as W
+    if name == "c4_skew":
+        return W.make_c4(skew=True)
+    return W.FULL[name]()
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and slowdown reasons through NVML while the timed region runs."""
+    REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown",
+               0x40: "hw_thermal_slowdown", 0x80: "hw_power_brake_slowdown",
+               0x2: "applications_clocks_setting"}
+
+    def __init__(self, device_index):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        self._h = None
+        try:
+            import pynvml
+            import torch
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            uuid = getattr(torch.cuda.get_device_properties(device_index), "uuid", None)
+            h = None
+            if uuid is not None:
+                try:
+                    h = pynvml.nvmlDeviceGetHandleByUUID(("GPU-" + str(uuid)).encode())
+                except Exception:
+                    h = None
+            if h is None:
+                vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+                idx = device_index
+                if vis:
+                    try:
+                        idx = int(vis.split(",")[device_index])
+                    except Exception:
+                        pass
+                h = pynvml.nvmlDeviceGetHandleByIndex(idx)
+            self._h = h
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self._h = None
+
+    def _loop(self):
+        nv = self._nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM))
+                get = getattr(nv, "nvmlDeviceGetCurrentClocksEventReasons", None) or \
+                    nv.nvmlDeviceGetCurrentClocksThrottleReasons
+                bits = get(self._h)
+                for b, name in self.REASONS.items():
+                    if bits & b:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(0.01)
+
+    def __enter__(self):
+        if self._h is not None:
+            self._thread = threading.Thread(target=self._loop, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._thread:
+            self._thread.join()
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": ["nvml unavailable"]}
+        return {"sm_mhz": statistics.median(self.samples), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def kernel_source_sha():
+    h = hashlib.sha256()
+    with open(os.path.join(ROOT, "paper_2411_02581_b200", "csrc", "tuna_move.cu"), "rb") as f:
+        h.update(f.read())
+    return h.hexdigest()
+
+
+# ----------------------------------------------------------------------------- reference arm
+
+def oracle_sample_workload(name, budget_s):
+    """A scaled-down instance of the workload that the oracle moves in about budget_s."""
+    from paper_2411_02581_b200 import workloads as W
+    if name.startswith("c4"):
+        rate = 0.8e9  # bytes/s the plain oracle sustains on large blocks, order of magnitude
+        tokens = 64
+        while tokens < 2048 and (2 * tokens) * 64 * 2 * 8192 <= budget_s * rate:
+            tokens *= 2
+        wl = W.make_c4(tokens=tokens, skew=name.endswith("skew"))
+        return wl, f"{name} shape with {tokens} of 8192 tokens per rank ({wl.payload_bytes_total / 2**30:.2f} GiB)"
+    wl = make_workload(name)
+    return wl, f"{name} at full size ({wl.payload_bytes_total / 2**20:.1f} MiB)"
+
+
+def default_radix(wl, radix):
+    if radix:
+        return radix
+    return max(wl.radices) if wl.radices else 0
+
+
+def run_oracle_once(wl, radix, send, recv):
+    import oracle
+    t0 = time.perf_counter()
+    if wl.hier and not wl.radices:
+        l, g = wl.hier
+        rl, rg = wl.hier_radices[-1]
+        oracle.tuna_hier(wl, l, g, rl, rg, send, recv)
+    else:
+        oracle.tuna_flat(wl, radix, send, recv)
+    return time.perf_counter() - t0
+
+
+def reference_arm(args):
+    """Times the CPU oracle, as it stands, on the host cores (rank 0 only)."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    import numpy as np
+    budget = max(0.5, min(10.0, 150.0 / max(1, args.steps + args.warmup)))
+    wl, sample = oracle_sample_workload(args.workload, budget)
+    radix = default_radix(wl, args.radix)
+    send = wl.make_send().numpy()
+    recv = np.empty(max(wl.recv_bytes, 1), dtype=np.uint8)[:wl.recv_bytes]
+    for _ in range(args.warmup):
+        run_oracle_once(wl, radix, send, recv)
+    t = [run_oracle_once(wl, radix, send, recv) for _ in range(args.steps)]
+    total = sum(t)
+    value = wl.payload_bytes_total * args.steps / total / 1e9
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u8",
+        "data": "synthetic",
+        "config": {"workload": f"{wl.name} P={wl.P} flat radix {radix}", "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ----------------------------------------------------------------------------- our arm
+
+def time_schedule(plan, wl, send, recv, steps, warmup, direct=False, replan=True):
+    """Median-free timing of `steps` back-to-back steps with CUDA events; returns ms per step."""
+    import torch
+    run = plan.direct_alltoallv if direct else plan.alltoallv
+    layout = (wl.sendcounts, wl.sdispls, wl.rdispls, wl.sendbase, wl.recvbase)
+
+    def step():
+        if replan:
+            plan.update_counts(*layout)
+        run(send, recv)
+
+    for _ in range(warmup):
+        step()
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(steps):
+        step()
+    b.record()
+    torch.cuda.synchronize()
+    return a.elapsed_time(b) / steps
+
+
+def verify_samples(wl, recv, n=4096):
+    """Sampled parity at full size: a received byte must equal the generator's byte
+    at the position the exchange's definition says it came from."""
+    import numpy as np
+    import torch
+    from paper_2411_02581_b200 import workloads as W
+    if wl.payload_kind != "bytes" or wl.payload_bytes_total == 0:
+        return None
+    rng = np.random.default_rng(12345)
+    C = wl.sendcounts
+    nz = np.argwhere(C > 0)
+    pick = nz[rng.integers(0, len(nz), size=n)]
+    s, d = pick[:, 0], pick[:, 1]
+    k = (rng.random(n) * (C[s, d] * wl.elem_size)).astype(np.int64)
+    src = (wl.sendbase[s] + wl.sdispls[s, d]) * wl.elem_size + k
+    dst = (wl.recvbase[d] + wl.rdispls[d, s]) * wl.elem_size + k
+    want = W.payload_byte_at(wl.seed, torch.from_numpy(src))
+    got = recv[torch.from_numpy(dst).to(recv.device)].cpu()
+    return bool(torch.equal(want, got))
+
+
+def ours_arm(args):
+    import numpy as np
+    import torch
+    from paper_2411_02581_b200 import binding as B
+    from paper_2411_02581_b200 import build as build_mod
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if rank == 0:
+        build_mod.build()
+    if dist:
+        dist.barrier()
+    B.lib()
+
+    wl = make_workload(args.workload)
+    radix = default_radix(wl, args.radix)
+    hier_headline = not wl.radices and wl.hier
+    dev = torch.device("cuda", local)
+    send = wl.make_send(dev)
+    recv = wl.make_recv(dev)
+    payload = wl.payload_bytes_total
+
+    def make_plan(r, l=None, g=1, rg=2, flags=0):
+        return B.plan_for(wl, r, l=l, g=g, radix_global=rg, flags=flags)
+
+    if hier_headline:
+        l, g = wl.hier
+        rl, rg = wl.hier_radices[-1]
+        plan = make_plan(rl, l=l, g=g, rg=rg)
+        sched = f"hierarchical l={l} g={g} radix {rl}/{rg}"
+    else:
+        plan = make_plan(radix)
+        sched = f"flat radix {radix}"
+    plan.alloc_workspace(host_staging=not args.no_e2e, device=dev)
+    layout = (wl.sendcounts, wl.sdispls, wl.rdispls, wl.sendbase, wl.recvbase)
+
+    def step():
+        plan.update_counts(*layout)
+        plan.alltoallv(send, recv)
+
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    ok = verify_samples(wl, recv)
+    plan.enable_timing(True)
+    plan.get_timing(reset=True)
+    launches0 = plan.launch_count()
+    if dist:
+        dist.barrier()
+    torch.cuda.synchronize()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local) as clocks:
+        ev0.record()
+        for _ in range(args.steps):
+            step()
+        ev1.record()
+        torch.cuda.synchronize()
+    if dist:
+        dist.barrier()
+    elapsed_ms = ev0.elapsed_time(ev1)
+    launches = plan.launch_count() - launches0
+    timing = plan.get_timing(reset=True)
+    plan.enable_timing(False)
+    if dist:
+        t = torch.tensor([elapsed_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        elapsed_ms = float(t.item())
+    ms_per_step = elapsed_ms / args.steps
+    value = world * payload / (ms_per_step * 1e-3) / 1e9
+
+    # roofline of the dominant kernel: the fused round kernel
+    peak, peak_kind = measured_peaks()
+    rk = timing["round_local"]
+    rk_ms = rk["ms"] + timing["round_global"]["ms"]
+    rk_launches = rk["launches"] + timing["round_global"]["launches"]
+    rk_bytes = rk["bytes"] + timing["round_global"]["bytes"]
+    achieved = 2.0 * rk_bytes / (rk_ms * 1e-3) / 1e9 if rk_ms > 0 else 0.0
+    per_byte = NCU_TRAFFIC_PER_PAYLOAD_BYTE.get(kernel_source_sha())
+    roofline = {
+        "bound": "hbm", "kernel": "tuna_round_kernel", "achieved": achieved, "peak": peak,
+        "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,
+        "traffic": (per_byte * rk_bytes / rk_launches) if per_byte and rk_launches else None,
+        "algorithmic_bytes_per_launch": 2.0 * rk_bytes / rk_launches if rk_launches else 0,
+        "avg_launch_ms": rk_ms / rk_launches if rk_launches else None,
+        "launches": rk_launches,
+        "plan_ms_per_step": timing["plan"]["ms"] / args.steps,
+        "rotate_ms_per_step": timing["rotate"]["ms"] / args.steps,
+    }
+
+    # end to end through the host-buffer entry point (pinned host memory)
+    e2e = None
+    if not args.no_e2e:
+        hs = torch.empty(max(wl.send_bytes, 1), dtype=torch.uint8, pin_memory=True)[:wl.send_bytes]
+        hr = torch.empty(max(wl.recv_bytes, 1), dtype=torch.uint8, pin_memory=True)[:wl.recv_bytes]
+        hs.copy_(send)
+        e_steps = max(2, min(args.steps, 5))
+
+        def estep():
+            plan.update_counts(*layout)
+            plan.alltoallv_host(hs, hr, B.SCHEDULE_TUNA)
+            torch.cuda.synchronize()
+
+        estep()
+        if dist:
+            dist.barrier()
+        t0 = time.perf_counter()
+        for _ in range(e_steps):
+            estep()
+        e_ms = (time.perf_counter() - t0) * 1e3 / e_steps
+        if dist:
+            t = torch.tensor([e_ms], dtype=torch.float64, device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e_ms = float(t.item())
+        e2e = {"value": world * payload / (e_ms * 1e-3) / 1e9, "unit": UNIT,
+               "h2d_bytes_per_step": wl.send_bytes + 8 * (3 * wl.P * wl.P + 2 * wl.P),
+               "d2h_bytes_per_step": wl.recv_bytes, "ms_per_step": e_ms, "steps": e_steps}
+        del hs, hr
+
+    # the other schedules of the workload, timed the same way (exchange + re-plan)
+    sweep = []
+    if not args.no_sweep and rank == 0:
+        def entry(name, p, direct=False):
+            p.alloc_workspace(device=dev)
+            ms = time_schedule(p, wl, send, recv, args.sweep_steps, 3, direct=direct)
+            ms_x = time_schedule(p, wl, send, recv, args.sweep_steps, 1, direct=direct, replan=False)
+            hops = sum(r["bytes"] for r in p.rounds()) / max(payload, 1)
+            sweep.append({"schedule": name, "ms_per_step": ms, "payload_GBps": payload / ms / 1e6,
+                          "exchange_only_ms": ms_x, "rounds": p.num_rounds(),
+                          "phases": p.num_phases(), "mean_hops": 0.0 if direct else hops,
+                          "effective_hbm_GBps": 2 * payload * (1 if direct else hops) / ms_x / 1e6
+                          if not direct else 2 * payload / ms_x / 1e6,
+                          "workspace_bytes": 0 if direct else p.workspace_bytes()})
+            p.set_workspace(None)
+            p.destroy()
+            torch.cuda.empty_cache()
+
+        plan.set_workspace(None)
+        torch.cuda.empty_cache()
+        entry("direct", make_plan(2), direct=True)
+        for r in wl.radices:
+            entry(f"flat r={r}", make_plan(r))
+        if wl.radices:
+            entry(f"flat r={wl.radices[0]} classic-rotate", make_plan(wl.radices[0], flags=B.FLAG_CLASSIC_ROTATE))
+        if wl.hier:
+            l, g = wl.hier
+            for rl, rg in wl.hier_radices:
+                entry(f"hier {l}x{g} r={rl}/{rg}", make_plan(rl, l=l, g=g, rg=rg))
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle  # noqa: F401  (the CPU-baseline leg is the one place bench.py runs the oracle)
+        wls, sample = oracle_sample_workload(args.workload, 8.0)
+        hs = wls.make_send().numpy()
+        hr = np.empty(max(wls.recv_bytes, 1), dtype=np.uint8)[:wls.recv_bytes]
+        r = default_radix(wls, args.radix)
+        times = [run_oracle_once(wls, r, hs, hr) for _ in range(3)]
+        cpu = {"value": wls.payload_bytes_total / statistics.median(times) / 1e9, "unit": UNIT,
+               "cores": 1, "kind": "oracle", "sample": sample + ", median of 3 runs",
+               "host_cores_available": os.cpu_count()}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+            "config": {"workload": f"{wl.name} P={wl.P} {sched}, payload {payload} bytes, "
+                                   f"elem {wl.elem_size} B, re-plan every step",
+                       "l2": "inputs larger than L2" if payload > 256e6 else
+                             "inputs fit in L2 (latency-bound case)",
+                       "replicas": "one independent exchange per GPU" if world > 1 else "single GPU"},
+            "gpu_launches": int(launches), "parity_samples_ok": ok,
+            "clocks": clocks.summary(), "e2e": e2e, "roofline": roofline,
+            "cpu_baseline": cpu, "sweep": sweep,
+        }
+        print(json.dumps(line), flush=True)
+    if dist:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        reference_arm(args)
+    else:
+        ours_arm(args)
+
+
+if __name__ == "__main__":
+    main()

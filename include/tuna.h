@@ -192,8 +192,33 @@ int tuna_plan_phase_info(const tuna_plan_t *plan, int phase, int *level, int *x,
 int tuna_plan_phase_tables(const tuna_plan_t *plan, int phase, int64_t cap, int64_t *len,
                            int64_t *pos, int64_t *src, int64_t *dst, int64_t *rows);
 
-/* Kernels launched by the last exchange call on this plan (host counter). */
+/* Kernels launched by the last exchange call on this plan (host counter), and by
+ * every call on this plan since its creation, plan kernels included. */
 int tuna_plan_last_launches(const tuna_plan_t *plan, int *launches);
+int tuna_plan_launch_count(const tuna_plan_t *plan, int64_t *launches);
+
+/*
+ * Per-kernel timing with the paper's cost components (Sec. V-B lists prepare,
+ * metadata, data, replace, rearrange and inter-node cost).  With timing enabled
+ * every launch is bracketed by CUDA events on the caller's stream:
+ *   TUNA_TIMER_PLAN          metadata exchange + prefix sums (prepare + metadata)
+ *   TUNA_TIMER_ROUND_LOCAL   flat / local digit phases (data; "replace" is fused away)
+ *   TUNA_TIMER_ROUND_GLOBAL  global digit phases (inter-group cost)
+ *   TUNA_TIMER_ROTATE        final rotation (rearrange)
+ *   TUNA_TIMER_DIRECT        the single-pass direct exchange
+ * tuna_plan_get_timing waits for the recorded events and returns, per kind
+ * (arrays of TUNA_TIMER_KINDS, any may be NULL), accumulated milliseconds,
+ * launches and payload bytes moved; `reset` non-zero clears the accumulators.
+ */
+#define TUNA_TIMER_PLAN 0
+#define TUNA_TIMER_ROUND_LOCAL 1
+#define TUNA_TIMER_ROUND_GLOBAL 2
+#define TUNA_TIMER_ROTATE 3
+#define TUNA_TIMER_DIRECT 4
+#define TUNA_TIMER_KINDS 5
+int tuna_plan_enable_timing(tuna_plan_t *plan, int on);
+int tuna_plan_get_timing(tuna_plan_t *plan, int reset, double *ms, int64_t *launches,
+                         int64_t *bytes);
 
 /* The cudaError_t of the most recent failing runtime call (0 if none). */
 int tuna_plan_cuda_error(const tuna_plan_t *plan);

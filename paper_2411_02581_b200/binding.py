@@ -23,6 +23,9 @@ FLAG_CLASSIC_ROTATE = 1
 SCHEDULE_TUNA = 0
 SCHEDULE_DIRECT = 1
 
+TIMER_NAMES = ("plan", "round_local", "round_global", "rotate", "direct")
+TIMER_KINDS = len(TIMER_NAMES)
+
 STATUS = {
     0: "TUNA_OK", -1: "TUNA_ERR_INVALID_ARG", -2: "TUNA_ERR_BAD_RADIX",
     -3: "TUNA_ERR_BAD_HIERARCHY", -4: "TUNA_ERR_COUNT_MISMATCH", -5: "TUNA_ERR_OVERLAP",
@@ -48,6 +51,9 @@ SIGNATURES = {
     "tuna_plan_phase_info": (ctypes.c_int, [_VP, ctypes.c_int, _INTP, _INTP, _I64P, _I64P, _I64P]),
     "tuna_plan_phase_tables": (ctypes.c_int, [_VP, ctypes.c_int, ctypes.c_int64] + [_I64P] * 5),
     "tuna_plan_last_launches": (ctypes.c_int, [_VP, _INTP]),
+    "tuna_plan_launch_count": (ctypes.c_int, [_VP, _I64P]),
+    "tuna_plan_enable_timing": (ctypes.c_int, [_VP, ctypes.c_int]),
+    "tuna_plan_get_timing": (ctypes.c_int, [_VP, ctypes.c_int, ctypes.POINTER(ctypes.c_double), _I64P, _I64P]),
     "tuna_plan_cuda_error": (ctypes.c_int, [_VP]),
     "tuna_strerror": (ctypes.c_char_p, [ctypes.c_int]),
     "tuna_version": (ctypes.c_int, []),
@@ -241,6 +247,23 @@ class Plan:
         n = ctypes.c_int()
         self._check(lib().tuna_plan_last_launches(self._h, ctypes.byref(n)), "tuna_plan_last_launches")
         return n.value
+
+
+    def launch_count(self) -> int:
+        n = ctypes.c_int64()
+        self._check(lib().tuna_plan_launch_count(self._h, ctypes.byref(n)), "tuna_plan_launch_count")
+        return n.value
+
+    def enable_timing(self, on=True):
+        self._check(lib().tuna_plan_enable_timing(self._h, int(bool(on))), "tuna_plan_enable_timing")
+
+    def get_timing(self, reset=True):
+        """{kind: dict(ms, launches, bytes)} accumulated since the last reset."""
+        ms = (ctypes.c_double * TIMER_KINDS)()
+        ln = (ctypes.c_int64 * TIMER_KINDS)()
+        by = (ctypes.c_int64 * TIMER_KINDS)()
+        self._check(lib().tuna_plan_get_timing(self._h, int(bool(reset)), ms, ln, by), "tuna_plan_get_timing")
+        return {name: dict(ms=ms[i], launches=ln[i], bytes=by[i]) for i, name in enumerate(TIMER_NAMES)}
 
 
 def plan_for(wl, radix, l=None, g=1, radix_global=2, flags=0, explicit_layout=True, stream=None) -> Plan:

@@ -340,6 +340,21 @@ struct tuna_plan {
   int64_t workspace_need = 0;
   char *workspace = nullptr;
   size_t workspace_bytes = 0;
+
+  int64_t launch_count = 0;  // kernels launched by this plan since creation
+
+  // optional per-launch timing (CUDA events on the caller's stream)
+  bool timing = false;
+  struct Stamp {
+    int kind;
+    int64_t bytes;
+    cudaEvent_t a, b;
+  };
+  std::vector<Stamp> stamps;
+  std::vector<cudaEvent_t> event_pool;
+  double t_ms[TUNA_TIMER_KINDS] = {0, 0, 0, 0, 0};
+  int64_t t_launches[TUNA_TIMER_KINDS] = {0, 0, 0, 0, 0};
+  int64_t t_bytes[TUNA_TIMER_KINDS] = {0, 0, 0, 0, 0};
 };
 
 namespace {
@@ -352,6 +367,51 @@ namespace {
       return TUNA_ERR_CUDA;                       \
     }                                             \
   } while (0)
+
+// after a kernel launch: count it and check the launch status
+#define TUNA_LAUNCHED(plan)                       \
+  do {                                            \
+    (plan)->launch_count++;                       \
+    TUNA_CUDA(plan, cudaGetLastError());          \
+  } while (0)
+
+cudaEvent_t take_event(tuna_plan *pl) {
+  cudaEvent_t e = nullptr;
+  if (!pl->event_pool.empty()) {
+    e = pl->event_pool.back();
+    pl->event_pool.pop_back();
+  } else if (cudaEventCreate(&e) != cudaSuccess) {
+    e = nullptr;
+  }
+  return e;
+}
+
+// Brackets one launch (or the plan kernels) with events when timing is on.
+struct Timed {
+  tuna_plan *pl;
+  cudaStream_t st;
+  tuna_plan::Stamp s{};
+  bool on;
+  Timed(tuna_plan *p, int kind, int64_t bytes, cudaStream_t stream) : pl(p), st(stream), on(p->timing) {
+    if (!on) return;
+    s.kind = kind;
+    s.bytes = bytes;
+    s.a = take_event(pl);
+    s.b = take_event(pl);
+    if (!s.a || !s.b) {
+      on = false;
+      return;
+    }
+    cudaEventRecord(s.a, st);
+  }
+  void stop() {
+    if (!on) return;
+    on = false;
+    cudaEventRecord(s.b, st);
+    pl->stamps.push_back(s);
+  }
+  ~Timed() { stop(); }
+};
 
 int64_t ipow64(int64_t r, int x) {
   int64_t v = 1;
@@ -429,7 +489,7 @@ int build_chunks(tuna_plan *pl, TunaList &l, cudaStream_t st) {
     const int th = 128;
     tuna_chunk_index_kernel<<<(unsigned)((l.nchunks + th - 1) / th), th, 0, st>>>(
         l.pos, l.n, l.chunk, l.nchunks, l.chunk_first);
-    TUNA_CUDA(pl, cudaGetLastError());
+    TUNA_LAUNCHED(pl);
   }
   return TUNA_OK;
 }
@@ -442,17 +502,17 @@ int scan_list(tuna_plan *pl, TunaList &l, int64_t seglen, int64_t nseg, int list
     const int64_t blocks = (nseg * 32 + th - 1) / th;
     tuna_segscan_kernel<true><<<(unsigned)blocks, th, 0, st>>>(l.len, l.pos, pl->d_seg_total,
                                                                 pl->d_seg_raw, seglen, nseg);
-    TUNA_CUDA(pl, cudaGetLastError());
+    TUNA_LAUNCHED(pl);
   }
   tuna_segbase_kernel<<<1, 1024, 0, st>>>(pl->d_seg_total, pl->d_seg_raw, pl->d_seg_base,
                                           (nseg > 0 && seglen > 0) ? nseg : 0,
                                           pl->d_scal + 2 * list_id, wbase_slot, uses_work);
-  TUNA_CUDA(pl, cudaGetLastError());
+  TUNA_LAUNCHED(pl);
   if (add_base && l.n > 0) {
     const int th = 256;
     tuna_add_base_kernel<<<(unsigned)((l.n + th - 1) / th), th, 0, st>>>(l.pos, pl->d_seg_base,
                                                                           seglen, l.n);
-    TUNA_CUDA(pl, cudaGetLastError());
+    TUNA_LAUNCHED(pl);
   }
   return TUNA_OK;
 }
@@ -511,6 +571,7 @@ int build_tables(tuna_plan *pl, const int64_t *counts, const int64_t *sdispls,
   pl->send_extent = se * t.elem;
   pl->recv_extent = re * t.elem;
 
+  Timed plan_timer(pl, TUNA_TIMER_PLAN, 0, st);
   TUNA_CUDA(pl, cudaMemcpyAsync(pl->d_counts, counts, PP * 8, cudaMemcpyHostToDevice, st));
   TUNA_CUDA(pl, cudaMemcpyAsync(pl->d_sendbase, sb.data(), P * 8, cudaMemcpyHostToDevice, st));
   TUNA_CUDA(pl, cudaMemcpyAsync(pl->d_recvbase, rb.data(), P * 8, cudaMemcpyHostToDevice, st));
@@ -524,16 +585,16 @@ int build_tables(tuna_plan *pl, const int64_t *counts, const int64_t *sdispls,
   } else {  // packed: exclusive scan of every rank's row of counts
     tuna_segscan_kernel<false><<<gseg, th, 0, st>>>(pl->d_counts, pl->d_sdispls, pl->d_seg_total,
                                                      nullptr, P, P);
-    TUNA_CUDA(pl, cudaGetLastError());
+    TUNA_LAUNCHED(pl);
   }
   if (rdispls) {
     TUNA_CUDA(pl, cudaMemcpyAsync(pl->d_rdispls, rdispls, PP * 8, cudaMemcpyHostToDevice, st));
   } else {  // packed: scan of the receive counts = rows of the transposed matrix
     tuna_transpose_kernel<<<gPP, th, 0, st>>>(pl->d_counts, pl->d_tmp, P);
-    TUNA_CUDA(pl, cudaGetLastError());
+    TUNA_LAUNCHED(pl);
     tuna_segscan_kernel<false><<<gseg, th, 0, st>>>(pl->d_tmp, pl->d_rdispls, pl->d_seg_total,
                                                      nullptr, P, P);
-    TUNA_CUDA(pl, cudaGetLastError());
+    TUNA_LAUNCHED(pl);
   }
 
   const int nph = (int)pl->phases.size();
@@ -549,7 +610,7 @@ int build_tables(tuna_plan *pl, const int64_t *counts, const int64_t *sdispls,
                                               pl->d_loc[0], pl->dir.len, pl->dir.src, pl->dir.dst,
                                               pl->rot.len, pl->rot.src, pl->rot.dst,
                                               pl->classic ? 1 : 0);
-  TUNA_CUDA(pl, cudaGetLastError());
+  TUNA_LAUNCHED(pl);
 
   int cur = 0;
   for (int f = 0; f < nph; f++) {
@@ -560,7 +621,7 @@ int build_tables(tuna_plan *pl, const int64_t *counts, const int64_t *sdispls,
     tuna_meta_exchange_kernel<<<gPP, th, smem, st>>>(t, pd, pl->d_sz[cur], pl->d_loc[cur],
                                                      pl->d_sz[cur ^ 1], l.len, l.src,
                                                      pl->d_round_bytes + ph.stats_off);
-    TUNA_CUDA(pl, cudaGetLastError());
+    TUNA_LAUNCHED(pl);
     // in direct-to-R mode the last phase delivers everything: it keeps nothing
     const int uses_work = (pl->classic || f + 1 < nph) ? 1 : 0;
     rc = scan_list(pl, l, ph.per_rank, P, f, pl->d_wbase + f, uses_work, false, st);
@@ -569,7 +630,7 @@ int build_tables(tuna_plan *pl, const int64_t *counts, const int64_t *sdispls,
                                           pl->d_seg_base, l.len, l.dst, pl->d_wbase + f,
                                           pl->d_rdispls, pl->d_recvbase, pl->classic ? 1 : 0,
                                           pl->rot.len, pl->rot.src, pl->rot.dst);
-    TUNA_CUDA(pl, cudaGetLastError());
+    TUNA_LAUNCHED(pl);
     cur ^= 1;
   }
   // work partitions of the rotation and direct lists
@@ -578,6 +639,7 @@ int build_tables(tuna_plan *pl, const int64_t *counts, const int64_t *sdispls,
   rc = scan_list(pl, pl->dir, P, P, nph + 1, nullptr, 0, true, st);
   if (rc) return rc;
 
+  plan_timer.stop();  // the chunk tables below are timed separately, after the read-back
   // one read-back: stream totals, workspace offsets, per-round bytes
   std::vector<int64_t> scal(2 * (nph + 2)), wbase(nph + 1);
   std::vector<unsigned long long> rbytes(std::max<int64_t>(pl->stats_n, 1));
@@ -597,6 +659,7 @@ int build_tables(tuna_plan *pl, const int64_t *counts, const int64_t *sdispls,
   pl->workspace_need = wbase[nph];
   for (auto &r : pl->rounds) r.bytes = (int64_t)rbytes[pl->phases[r.phase].stats_off + r.z];
 
+  Timed chunk_timer(pl, TUNA_TIMER_PLAN, 0, st);
   for (int f = 0; f < nph; f++) {
     rc = build_chunks(pl, pl->lists[f], st);
     if (rc) return rc;
@@ -707,24 +770,32 @@ int run_tuna(tuna_plan *pl, const void *send, void *recv, cudaStream_t st) {
   for (size_t f = 0; f < pl->lists.size(); f++) {
     const TunaList &l = pl->lists[f];
     if (l.nchunks == 0) continue;
-    TUNA_CUDA(pl, tuna_launch_move(TUNA_MOVE_ROUND, move_args(l, send, recv, pl->workspace), st));
+    {
+      Timed tm(pl, pl->phases[f].level == 0 ? TUNA_TIMER_ROUND_LOCAL : TUNA_TIMER_ROUND_GLOBAL,
+               l.bytes, st);
+      TUNA_CUDA(pl, tuna_launch_move(TUNA_MOVE_ROUND, move_args(l, send, recv, pl->workspace), st));
+    }
     launches++;
   }
   if (pl->rot.nchunks > 0) {
+    Timed tm(pl, TUNA_TIMER_ROTATE, pl->rot.bytes, st);
     TUNA_CUDA(pl, tuna_launch_move(TUNA_MOVE_ROTATE, move_args(pl->rot, send, recv, pl->workspace), st));
     launches++;
   }
   pl->last_launches = launches;
+  pl->launch_count += launches;
   return TUNA_OK;
 }
 
 int run_direct(tuna_plan *pl, const void *send, void *recv, cudaStream_t st) {
   int launches = 0;
   if (pl->dir.nchunks > 0) {
+    Timed tm(pl, TUNA_TIMER_DIRECT, pl->dir.bytes, st);
     TUNA_CUDA(pl, tuna_launch_move(TUNA_MOVE_DIRECT, move_args(pl->dir, send, recv, nullptr), st));
     launches++;
   }
   pl->last_launches = launches;
+  pl->launch_count += launches;
   return TUNA_OK;
 }
 
@@ -775,6 +846,11 @@ int tuna_plan_destroy(tuna_plan_t *pl) {
   cudaFree(pl->d_scal);
   cudaFree(pl->d_wbase);
   cudaFree(pl->d_round_bytes);
+  for (auto &s : pl->stamps) {
+    cudaEventDestroy(s.a);
+    cudaEventDestroy(s.b);
+  }
+  for (auto e : pl->event_pool) cudaEventDestroy(e);
   delete pl;
   return TUNA_OK;
 }
@@ -995,6 +1071,44 @@ int tuna_plan_phase_tables(const tuna_plan_t *pl, int phase, int64_t cap, int64_
 int tuna_plan_last_launches(const tuna_plan_t *pl, int *launches) {
   if (!pl || !launches) return TUNA_ERR_INVALID_ARG;
   *launches = pl->last_launches;
+  return TUNA_OK;
+}
+
+int tuna_plan_launch_count(const tuna_plan_t *pl, int64_t *launches) {
+  if (!pl || !launches) return TUNA_ERR_INVALID_ARG;
+  *launches = pl->launch_count;
+  return TUNA_OK;
+}
+
+int tuna_plan_enable_timing(tuna_plan_t *pl, int on) {
+  if (!pl) return TUNA_ERR_INVALID_ARG;
+  pl->timing = on != 0;
+  return TUNA_OK;
+}
+
+int tuna_plan_get_timing(tuna_plan_t *pl, int reset, double *ms, int64_t *launches, int64_t *bytes) {
+  if (!pl) return TUNA_ERR_INVALID_ARG;
+  for (auto &s : pl->stamps) {
+    TUNA_CUDA(pl, cudaEventSynchronize(s.b));
+    float t = 0.f;
+    TUNA_CUDA(pl, cudaEventElapsedTime(&t, s.a, s.b));
+    pl->t_ms[s.kind] += t;
+    pl->t_launches[s.kind] += 1;
+    pl->t_bytes[s.kind] += s.bytes;
+    pl->event_pool.push_back(s.a);
+    pl->event_pool.push_back(s.b);
+  }
+  pl->stamps.clear();
+  for (int k = 0; k < TUNA_TIMER_KINDS; k++) {
+    if (ms) ms[k] = pl->t_ms[k];
+    if (launches) launches[k] = pl->t_launches[k];
+    if (bytes) bytes[k] = pl->t_bytes[k];
+    if (reset) {
+      pl->t_ms[k] = 0;
+      pl->t_launches[k] = 0;
+      pl->t_bytes[k] = 0;
+    }
+  }
   return TUNA_OK;
 }
 
