@@ -41,7 +41,7 @@ NCU_TRAFFIC_PER_PAYLOAD_BYTE: dict[str, float] = {}
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c4", choices=["c1", "c2", "c3", "c4", "c4_skew", "c5"])
@@ -50,13 +50,16 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sweep-steps", type=int, default=10)
+    ap.add_argument("--tokens", type=int, default=0,
+                    help="c4 only: tokens per rank (default 8192); smaller values give the "
+                         "reduced case used for profiler captures")
     return ap.parse_args()
 
 
-def make_workload(name):
+def make_workload(name, tokens=0):
     from paper_2411_02581_b200 import workloads as W
-    if name == "c4_skew":
-        return W.make_c4(skew=True)
+    if name.startswith("c4"):
+        return W.make_c4(skew=name.endswith("skew"), **({"tokens": tokens} if tokens else {}))
     return W.FULL[name]()
 
 
@@ -275,7 +278,7 @@ def ours_arm(args):
         dist.barrier()
     B.lib()
 
-    wl = make_workload(args.workload)
+    wl = make_workload(args.workload, args.tokens)
     radix = default_radix(wl, args.radix)
     hier_headline = not wl.radices and wl.hier
     dev = torch.device("cuda", local)
@@ -386,12 +389,17 @@ def ours_arm(args):
             p.alloc_workspace(device=dev)
             ms = time_schedule(p, wl, send, recv, args.sweep_steps, 3, direct=direct)
             ms_x = time_schedule(p, wl, send, recv, args.sweep_steps, 1, direct=direct, replan=False)
-            hops = sum(r["bytes"] for r in p.rounds()) / max(payload, 1)
+            # bytes every launch of the exchange moves: each hop of each block, the self
+            # blocks (rotation launch) and, in classic mode, every block once more
+            if direct:
+                moved = payload
+            else:
+                moved = sum(r["bytes"] for r in p.rounds()) + p.phase_info(-1)["bytes"]
             sweep.append({"schedule": name, "ms_per_step": ms, "payload_GBps": payload / ms / 1e6,
-                          "exchange_only_ms": ms_x, "rounds": p.num_rounds(),
-                          "phases": p.num_phases(), "mean_hops": 0.0 if direct else hops,
-                          "effective_hbm_GBps": 2 * payload * (1 if direct else hops) / ms_x / 1e6
-                          if not direct else 2 * payload / ms_x / 1e6,
+                          "exchange_only_ms": ms_x, "rounds": 1 if direct else p.num_rounds(),
+                          "launches": p.last_launches(),
+                          "moved_over_payload": moved / max(payload, 1),
+                          "effective_hbm_GBps": 2 * moved / ms_x / 1e6,
                           "workspace_bytes": 0 if direct else p.workspace_bytes()})
             p.set_workspace(None)
             p.destroy()
