@@ -59,6 +59,7 @@ struct TunaMoveArgs {
   const int32_t *chunk_first;
   int64_t n, total, chunk, nchunks;
   char *base[3];
+  int64_t extent[3];  // bytes of each buffer that may be accessed, from its base
 };
 
 enum TunaMoveKind { TUNA_MOVE_ROUND = 0, TUNA_MOVE_ROTATE = 1, TUNA_MOVE_DIRECT = 2 };

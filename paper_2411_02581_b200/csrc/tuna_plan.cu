@@ -469,7 +469,7 @@ int64_t env_i64(const char *name, int64_t dflt) {
 // than 128 KiB (tail effect).
 int64_t pick_chunk(int64_t total) {
   const int64_t forced = env_i64("TUNA_CHUNK_BYTES", 0);
-  if (forced >= 1024) return (forced + 15) & ~(int64_t)15;
+  if (forced >= 1024) return std::min<int64_t>((forced + 15) & ~(int64_t)15, (int64_t)1 << 24);
   int64_t c = 8192;
   while (c < 65536 && total / c > 148 * 32) c <<= 1;
   return c;
@@ -745,7 +745,8 @@ bool ranges_overlap(const void *a, size_t na, const void *b, size_t nb) {
   return na > 0 && nb > 0 && a0 < b0 + nb && b0 < a0 + na;
 }
 
-TunaMoveArgs move_args(const TunaList &l, const void *send, void *recv, char *work) {
+TunaMoveArgs move_args(const tuna_plan *pl, const TunaList &l, const void *send, void *recv,
+                       char *work) {
   TunaMoveArgs a{};
   a.len = l.len;
   a.pos = l.pos;
@@ -759,6 +760,9 @@ TunaMoveArgs move_args(const TunaList &l, const void *send, void *recv, char *wo
   a.base[TUNA_BUF_SEND] = (char *)const_cast<void *>(send);
   a.base[TUNA_BUF_RECV] = (char *)recv;
   a.base[TUNA_BUF_WORK] = work;
+  a.extent[TUNA_BUF_SEND] = pl->send_extent;
+  a.extent[TUNA_BUF_RECV] = pl->recv_extent;
+  a.extent[TUNA_BUF_WORK] = work ? pl->workspace_need : 0;
   return a;
 }
 
@@ -773,13 +777,13 @@ int run_tuna(tuna_plan *pl, const void *send, void *recv, cudaStream_t st) {
     {
       Timed tm(pl, pl->phases[f].level == 0 ? TUNA_TIMER_ROUND_LOCAL : TUNA_TIMER_ROUND_GLOBAL,
                l.bytes, st);
-      TUNA_CUDA(pl, tuna_launch_move(TUNA_MOVE_ROUND, move_args(l, send, recv, pl->workspace), st));
+      TUNA_CUDA(pl, tuna_launch_move(TUNA_MOVE_ROUND, move_args(pl, l, send, recv, pl->workspace), st));
     }
     launches++;
   }
   if (pl->rot.nchunks > 0) {
     Timed tm(pl, TUNA_TIMER_ROTATE, pl->rot.bytes, st);
-    TUNA_CUDA(pl, tuna_launch_move(TUNA_MOVE_ROTATE, move_args(pl->rot, send, recv, pl->workspace), st));
+    TUNA_CUDA(pl, tuna_launch_move(TUNA_MOVE_ROTATE, move_args(pl, pl->rot, send, recv, pl->workspace), st));
     launches++;
   }
   pl->last_launches = launches;
@@ -791,7 +795,7 @@ int run_direct(tuna_plan *pl, const void *send, void *recv, cudaStream_t st) {
   int launches = 0;
   if (pl->dir.nchunks > 0) {
     Timed tm(pl, TUNA_TIMER_DIRECT, pl->dir.bytes, st);
-    TUNA_CUDA(pl, tuna_launch_move(TUNA_MOVE_DIRECT, move_args(pl->dir, send, recv, nullptr), st));
+    TUNA_CUDA(pl, tuna_launch_move(TUNA_MOVE_DIRECT, move_args(pl, pl->dir, send, recv, nullptr), st));
     launches++;
   }
   pl->last_launches = launches;
