@@ -125,9 +125,10 @@ int tuna_plan_extents(const tuna_plan_t *plan, size_t *send_bytes, size_t *recv_
 
 /*
  * tuna_alltoallv - run the plan's TuNA schedule (Algorithm 1, or Sec. IV /
- * Algorithm 3 when g > 1): one fused pack-move-unpack launch per digit phase
- * (all rounds z of one digit position x touch disjoint blocks), then one
- * rotation launch (self blocks; in TUNA_FLAG_CLASSIC_ROTATE mode every block).
+ * Algorithm 3 when g > 1): per digit phase one fused pack-move-unpack launch for
+ * the blocks that travel on and one for the blocks that have arrived (all rounds
+ * z of one digit position x touch disjoint blocks, so they share a launch), then
+ * one rotation launch (self blocks; in TUNA_FLAG_CLASSIC_ROTATE mode every block).
  *
  *   sendbuf, recvbuf   device; must not overlap.
  *   sendcounts, sdispls, recvcounts, rdispls
@@ -168,28 +169,35 @@ int tuna_alltoallv_host(tuna_plan_t *plan, const void *host_send, void *host_rec
  * Rounds are the paper's (x, z) pairs in execution order (Sec. III-A); `level` is 0
  * for flat/local rounds and 1 for global rounds; `units` counts blocks sent by all
  * ranks (level 0) or super-blocks of l blocks (level 1); `bytes` is the round's
- * message volume summed over ranks.  Phases are the digit positions, one kernel
- * launch each: `entries` descriptor rows, `bytes` moved, `stream_bytes` the
- * 16-byte-padded length of the phase's destination stream.
+ * message volume summed over ranks.  Phases are the digit positions.  Every phase
+ * has two descriptor lists, selected by `part`: TUNA_PART_KEEP, the blocks that
+ * travel on in a later phase and land in the workspace, and TUNA_PART_DELIVER, the
+ * blocks that have arrived and land in the receive buffer (empty in
+ * TUNA_FLAG_CLASSIC_ROTATE mode); each non-empty list is one kernel launch.
+ * phase -1 selects the rotation list and -2 the direct list (`part` ignored).
+ * `entries` descriptor rows, `bytes` moved, `stream_bytes` the padded length of the
+ * list's stream (for a KEEP list: the size of its workspace region).
  */
+#define TUNA_PART_KEEP 0
+#define TUNA_PART_DELIVER 1
 int tuna_plan_num_rounds(const tuna_plan_t *plan, int *K);
 int tuna_plan_round_info(const tuna_plan_t *plan, int k, int *level, int *x, int *z,
                          int64_t *units, int64_t *bytes);
 int tuna_plan_num_phases(const tuna_plan_t *plan, int *n);
-int tuna_plan_phase_info(const tuna_plan_t *plan, int phase, int *level, int *x, int64_t *entries,
-                         int64_t *bytes, int64_t *stream_bytes);
+int tuna_plan_phase_info(const tuna_plan_t *plan, int phase, int part, int *level, int *x,
+                         int64_t *entries, int64_t *bytes, int64_t *stream_bytes);
 
 /*
- * tuna_plan_phase_tables - copy one phase's descriptor table to the host (debug /
- * test hook; synchronises the device).  phase in [0, num_phases) selects a digit
- * phase, -1 the rotation list, -2 the direct list.  Each output (host, `cap` rows,
- * may be NULL) receives, per descriptor in receive-side order (rank, then slot):
- * the block length in bytes, the position in the phase's padded stream (the
- * exclusive prefix sum that also partitions the work), and source / destination
- * as (buffer id << 56 | byte offset), buffer ids 0 = send, 1 = receive, 2 = workspace.
- * *rows receives the number of descriptors.
+ * tuna_plan_phase_tables - copy one descriptor list to the host (debug / test hook;
+ * synchronises the device).  Each output (host, `cap` rows, may be NULL) receives,
+ * per descriptor in receive-side order (rank, then slot): the block length in
+ * bytes; its position in the list's stream (the segmented exclusive prefix sum
+ * that also partitions the work: lengths rounded up to 16 bytes, plus 16 spare
+ * bytes per non-empty block in DELIVER, rotation and direct lists); source and
+ * destination as (buffer id << 56 | byte offset), buffer ids 0 = send,
+ * 1 = receive, 2 = workspace.  *rows receives the number of descriptors.
  */
-int tuna_plan_phase_tables(const tuna_plan_t *plan, int phase, int64_t cap, int64_t *len,
+int tuna_plan_phase_tables(const tuna_plan_t *plan, int phase, int part, int64_t cap, int64_t *len,
                            int64_t *pos, int64_t *src, int64_t *dst, int64_t *rows);
 
 /* Kernels launched by the last exchange call on this plan (host counter), and by

@@ -20,6 +20,8 @@ _VP = ctypes.c_void_p
 
 FLAG_DIRECT_TO_R = 0
 FLAG_CLASSIC_ROTATE = 1
+PART_KEEP = 0
+PART_DELIVER = 1
 SCHEDULE_TUNA = 0
 SCHEDULE_DIRECT = 1
 
@@ -48,8 +50,8 @@ SIGNATURES = {
     "tuna_plan_num_rounds": (ctypes.c_int, [_VP, _INTP]),
     "tuna_plan_round_info": (ctypes.c_int, [_VP, ctypes.c_int, _INTP, _INTP, _INTP, _I64P, _I64P]),
     "tuna_plan_num_phases": (ctypes.c_int, [_VP, _INTP]),
-    "tuna_plan_phase_info": (ctypes.c_int, [_VP, ctypes.c_int, _INTP, _INTP, _I64P, _I64P, _I64P]),
-    "tuna_plan_phase_tables": (ctypes.c_int, [_VP, ctypes.c_int, ctypes.c_int64] + [_I64P] * 5),
+    "tuna_plan_phase_info": (ctypes.c_int, [_VP, ctypes.c_int, ctypes.c_int, _INTP, _INTP, _I64P, _I64P, _I64P]),
+    "tuna_plan_phase_tables": (ctypes.c_int, [_VP, ctypes.c_int, ctypes.c_int, ctypes.c_int64] + [_I64P] * 5),
     "tuna_plan_last_launches": (ctypes.c_int, [_VP, _INTP]),
     "tuna_plan_launch_count": (ctypes.c_int, [_VP, _I64P]),
     "tuna_plan_enable_timing": (ctypes.c_int, [_VP, ctypes.c_int]),
@@ -225,19 +227,19 @@ class Plan:
         self._check(lib().tuna_plan_num_phases(self._h, ctypes.byref(n)), "tuna_plan_num_phases")
         return n.value
 
-    def phase_info(self, phase):
+    def phase_info(self, phase, part=PART_KEEP):
         lv, x = ctypes.c_int(), ctypes.c_int()
         e, b, s = ctypes.c_int64(), ctypes.c_int64(), ctypes.c_int64()
-        self._check(lib().tuna_plan_phase_info(self._h, phase, ctypes.byref(lv), ctypes.byref(x),
+        self._check(lib().tuna_plan_phase_info(self._h, phase, part, ctypes.byref(lv), ctypes.byref(x),
                                                ctypes.byref(e), ctypes.byref(b), ctypes.byref(s)),
                     "tuna_plan_phase_info")
         return dict(level=lv.value, x=x.value, entries=e.value, bytes=b.value, stream_bytes=s.value)
 
-    def phase_tables(self, phase):
-        n = self.phase_info(phase)["entries"]
+    def phase_tables(self, phase, part=PART_KEEP):
+        n = self.phase_info(phase, part)["entries"]
         arrs = [np.zeros(max(n, 1), dtype=np.int64) for _ in range(4)]
         rows = ctypes.c_int64()
-        self._check(lib().tuna_plan_phase_tables(self._h, phase, n,
+        self._check(lib().tuna_plan_phase_tables(self._h, phase, part, n,
                                                  *[a.ctypes.data_as(_I64P) for a in arrs],
                                                  ctypes.byref(rows)), "tuna_plan_phase_tables")
         assert rows.value == n

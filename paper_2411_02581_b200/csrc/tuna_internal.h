@@ -35,20 +35,30 @@ struct TunaPhase {
   int count;       // Q or N: number of offsets at this level
   int64_t stride;  // radix^x
   int64_t moving;  // offsets below count whose digit x is non-zero
-  int64_t per_rank;  // descriptors per receiving rank
+  int64_t per_rank;  // blocks a rank receives in this phase
+  int64_t finals;    // the first `finals` of them (in slot order) have arrived and are delivered
   int64_t stats_off; // first of `radix` counters in the stats array
 };
 
+// How a list's stream positions are spaced.
+//   KEEP:    pos = exclusive prefix sum of the lengths rounded up to 16.  The stream
+//            is the destination itself (a region of the workspace).
+//   DELIVER: 16 further bytes per non-empty block, so that a block can sit in a
+//            staging buffer at its destination's alignment whatever that is; the
+//            stream only partitions the work.
+enum TunaListKind { TUNA_LIST_KEEP = 0, TUNA_LIST_DELIVER = 1 };
+
 // A list of copy descriptors in receive-side order with its work partition.
 struct TunaList {
+  int kind = TUNA_LIST_KEEP;
   int64_t n = 0;          // descriptors
   int64_t *len = nullptr; // bytes
-  int64_t *pos = nullptr; // exclusive prefix sum of 16-byte-padded lengths
+  int64_t *pos = nullptr; // n + 1 stream positions (pos[n] = total)
   int64_t *src = nullptr; // location
-  int64_t *dst = nullptr; // location
+  int64_t *dst = nullptr; // location (DELIVER lists only)
   int32_t *chunk_first = nullptr;
   int64_t chunk_cap = 0;  // allocated entries of chunk_first
-  int64_t total = 0;      // padded stream bytes (host copy)
+  int64_t total = 0;      // stream bytes (host copy)
   int64_t bytes = 0;      // bytes moved (host copy)
   int64_t chunk = 0;      // bytes of stream per CTA
   int64_t nchunks = 0;
@@ -60,11 +70,17 @@ struct TunaMoveArgs {
   int64_t n, total, chunk, nchunks;
   char *base[3];
   int64_t extent[3];  // bytes of each buffer that may be accessed, from its base
+  int64_t keep_base;  // KEEP lists: workspace offset of stream position 0
 };
 
-enum TunaMoveKind { TUNA_MOVE_ROUND = 0, TUNA_MOVE_ROTATE = 1, TUNA_MOVE_DIRECT = 2 };
+enum TunaMoveKernel {
+  TUNA_K_ROUND = 0,    // KEEP list of a digit phase: blocks that travel on
+  TUNA_K_DELIVER = 1,  // DELIVER list of a digit phase: blocks that have arrived
+  TUNA_K_ROTATE = 2,   // final rotation / self blocks
+  TUNA_K_DIRECT = 3    // single-pass direct exchange
+};
 
-// Launches the fused pack-move-unpack kernel over one list (tuna_move.cu).
-cudaError_t tuna_launch_move(int kind, const TunaMoveArgs &a, cudaStream_t stream);
+// Launches one mover kernel over one list (tuna_move.cu).
+cudaError_t tuna_launch_move(int kernel, const TunaMoveArgs &a, cudaStream_t stream);
 
 #endif

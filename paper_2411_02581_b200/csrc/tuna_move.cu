@@ -1,45 +1,51 @@
 // Fused pack-move-unpack kernels.
 //
-// One launch executes every copy descriptor of one list: a digit phase of the
+// One launch executes every copy descriptor of one list.  A digit phase of the
 // radix-r schedule (all rounds z of one digit position x: the blocks whose x-th
-// offset digit equals z leave the rank that holds them and land, already in
-// their slot order, in the buffer of the rank at distance +z*r^x; Sec. III-A/B of
-// the paper), the final rotation into the MPI_Alltoallv receive layout, or the
-// single-pass direct exchange (Sec. II-d).  "Pack" is the gather from the
-// source rank's buffer, "move" the rank shift, "unpack" the placement at the
-// destination offset; with all ranks in one memory the three are one copy, so
-// each payload byte is read once and written once per hop.
+// offset digit equals z leave the rank that holds them for the rank at distance
+// +z*r^x; Sec. III-A/B of the paper) has two lists: the blocks that travel on
+// afterwards (KEEP: they land, in slot order, in that phase's region of the
+// workspace) and the blocks that have arrived (DELIVER: they land in the
+// receive buffer at their MPI_Alltoallv displacement).  The final rotation and
+// the single-pass direct exchange (Sec. II-d) are DELIVER lists too.  "Pack" is
+// the gather from the source rank's buffer, "move" the rank shift, "unpack" the
+// placement at the destination; with all ranks in one memory the three are one
+// copy, so each payload byte is read once and written once per hop.
 //
-// Work is partitioned by bytes, not by blocks: the destination stream of a list
-// (blocks in receive-side order, each padded to 16 bytes) is cut into equal
-// chunks, one CTA per chunk, and a precomputed table gives the first descriptor
-// of every chunk.  A block larger than a chunk is therefore spread over several
-// CTAs, and a chunk of tiny blocks is shared out over the threads of one CTA.
+// Work is partitioned by bytes, not by blocks: a list's stream (its blocks in
+// receive-side order, padded to 16 bytes) is cut into equal chunks, one CTA per
+// chunk, and a precomputed table gives the first descriptor of every chunk.  A
+// block larger than a chunk is spread over several CTAs; a chunk of tiny blocks
+// is shared out over the threads of one CTA, which walk the chunk as one run of
+// 16-byte vectors: a small table in shared memory says which block owns which
+// vector, so that consecutive threads copy consecutive vectors whatever the
+// block boundaries are, several loads in flight per thread before the first store.
 //
-// Inside a CTA every piece of a block takes one of two routes:
-//   direct  - source and destination both 16-byte aligned and the piece is large:
-//             the pieces are laid end to end as one run of 16-byte vectors and
-//             every thread copies a strided share of that run, four loads in
-//             flight before the first store.
-//   staged  - small pieces and pieces whose two ends are aligned differently: all
-//             of them are gathered into shared memory first (every thread again
-//             takes a strided share of the vectors, whatever block they belong
-//             to), placed so that the shared-memory address is congruent to the
-//             destination address modulo 16; after a barrier the same vectors
-//             are written out with aligned 16-byte stores, partial ones at the
-//             two ends of a block with the widest aligned stores that fit.  No
-//             byte outside a block's destination range is written, and no byte
-//             outside the source buffer's extent is read.
+//   tuna_round_kernel    KEEP lists.  The stream IS the destination, so stores
+//                        are contiguous aligned vectors; sources are aligned
+//                        workspace blocks or arbitrarily aligned send-buffer
+//                        blocks (read as aligned words merged by funnel shifts).
+//   tuna_deliver_kernel, tuna_rotate_kernel, tuna_direct_kernel
+//                        DELIVER lists.  A vector whose destination is aligned and
+//                        whole goes straight to global memory.  Everything else
+//                        is gathered into shared memory at the destination's
+//                        alignment and written out after a barrier: whole
+//                        vectors with 16-byte stores, the partial first and last
+//                        vector of a block in the widest aligned pieces that fit.
+//                        No byte outside a block's destination range is written.
+// No byte outside a source buffer's extent is read: blocks within 19 bytes of
+// either end of their buffer are read byte by byte instead of by aligned windows.
 #include "tuna_internal.h"
 
 namespace {
 
 constexpr int kThreads = TUNA_MOVE_THREADS;
-constexpr int kWarps = kThreads / 32;
-constexpr int kBatch = kThreads;      // descriptors handled per batch (one per thread)
-constexpr int kStage = 32768;         // bytes of staging buffer
-constexpr int kStageVec = kStage / 16;
-constexpr int kDirectMin = 4096;      // aligned pieces at least this long skip the staging buffer
+constexpr int kBatch = kThreads;        // descriptors handled per batch (one per thread)
+constexpr int kKeepVec = 4096;          // vectors per chunk of a KEEP list, at most (64 KiB)
+constexpr int kKeepSpan = kKeepVec / kThreads;
+constexpr int kStageVec = 2048;         // vectors of the staging window of a DELIVER list (32 KiB)
+constexpr int kStageSpan = kStageVec / kThreads;
+constexpr int kClampVec = 1 << 26;      // |vector index| beyond which only "far away" matters
 
 __device__ __forceinline__ uint4 ld16(const char *p) { return *reinterpret_cast<const uint4 *>(p); }
 __device__ __forceinline__ void st16(char *p, uint4 v) { *reinterpret_cast<uint4 *>(p) = v; }
@@ -47,6 +53,9 @@ __device__ __forceinline__ void st16(char *p, uint4 v) { *reinterpret_cast<uint4
 // (a select, not an index: indexing a kernel parameter array spills it to local memory)
 __device__ __forceinline__ char *base_of(const TunaMoveArgs &a, int buf) {
   return buf == TUNA_BUF_SEND ? a.base[0] : (buf == TUNA_BUF_RECV ? a.base[1] : a.base[2]);
+}
+__device__ __forceinline__ int64_t extent_of(const TunaMoveArgs &a, int buf) {
+  return buf == TUNA_BUF_SEND ? a.extent[0] : (buf == TUNA_BUF_RECV ? a.extent[1] : a.extent[2]);
 }
 
 // Largest t < cnt with start[t] <= v (start is non-decreasing, start[0] <= v).
@@ -58,273 +67,302 @@ __device__ __forceinline__ int find_entry(const int *start, int cnt, int v) {
   return lo;
 }
 
-// Exclusive prefix sum over the CTA (one value per thread); *total gets the sum.
-__device__ __forceinline__ int block_exclusive_scan(int x, int *s_warp, int *total) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  int incl = x;
-#pragma unroll
-  for (int d = 1; d < 32; d <<= 1) {
-    const int y = __shfl_up_sync(0xffffffffu, incl, d);
-    if (lane >= d) incl += y;
+// Owner table: who[v - v_first] = the descriptor owning vector v, for the vectors
+// [v_first, v_last) of the current batch.  Each thread resolves SPAN consecutive
+// vectors: one binary search for its last vector, then a walk down.
+template <int SPAN>
+__device__ __forceinline__ void fill_owner(unsigned char *who, const int *start, int cnt,
+                                           int v_first, int v_last) {
+  const int v0 = v_first + (int)threadIdx.x * SPAN;
+  if (v0 >= v_last) return;
+  const int vend = (v0 + SPAN < v_last) ? v0 + SPAN : v_last;
+  int t = find_entry(start, cnt, vend - 1);
+  for (int v = vend - 1; v >= v0; v--) {
+    while (start[t] > v) t--;
+    who[v - v_first] = (unsigned char)t;
   }
-  if (lane == 31) s_warp[warp] = incl;
-  __syncthreads();
-  int woff = 0, tot = 0;
-#pragma unroll
-  for (int k = 0; k < kWarps; k++) {
-    const int w = s_warp[k];
-    if (k < warp) woff += w;
-    tot += w;
-  }
-  *total = tot;
-  __syncthreads();
-  return woff + incl - x;
 }
 
-// The 16 source bytes starting at sa (any alignment), read with aligned accesses.
-// [lo, hi) is the extent of the buffer sa points into; if the aligned window would
-// leave it, only the bytes [b0, b1) of the vector are read, one by one.
-__device__ __forceinline__ uint4 load16_any(const char *sa, const char *lo, const char *hi, int b0,
-                                            int b1) {
-  const unsigned r = (unsigned)(reinterpret_cast<uintptr_t>(sa) & 15);
+// The 16 bytes at sa (any alignment) from five aligned words merged by funnel shifts.
+// Reads [sa - (sa & 3), +20).
+__device__ __forceinline__ uint4 load16_funnel(const char *sa) {
+  const unsigned sh = (unsigned)(reinterpret_cast<uintptr_t>(sa) & 3);
+  const uint32_t *w = reinterpret_cast<const uint32_t *>(sa - sh);
+  const uint32_t w0 = w[0], w1 = w[1], w2 = w[2], w3 = w[3], w4 = w[4];
+  const unsigned bits = sh * 8;
   uint4 v;
-  if (r == 0) {
-    if (sa >= lo && sa + 16 <= hi) return ld16(sa);
-  } else if ((r & 3) == 0) {
-    if (sa >= lo && sa + 16 <= hi) {
-      const uint32_t *w = reinterpret_cast<const uint32_t *>(sa);
-      v.x = w[0];
-      v.y = w[1];
-      v.z = w[2];
-      v.w = w[3];
-      return v;
-    }
-  } else {
-    const unsigned sh = r & 3;
-    const char *wb = sa - sh;
-    if (wb >= lo && wb + 20 <= hi) {
-      const uint32_t *w = reinterpret_cast<const uint32_t *>(wb);
-      const uint32_t w0 = w[0], w1 = w[1], w2 = w[2], w3 = w[3], w4 = w[4];
-      const unsigned bits = sh * 8;
-      v.x = __funnelshift_r(w0, w1, bits);
-      v.y = __funnelshift_r(w1, w2, bits);
-      v.z = __funnelshift_r(w2, w3, bits);
-      v.w = __funnelshift_r(w3, w4, bits);
-      return v;
-    }
-  }
-  // at the very edge of the buffer: only the bytes that belong to the block
-  unsigned char b[16];
-#pragma unroll
-  for (int i = 0; i < 16; i++) b[i] = (i >= b0 && i < b1) ? (unsigned char)sa[i] : 0;
-  v.x = b[0] | (b[1] << 8) | (b[2] << 16) | ((unsigned)b[3] << 24);
-  v.y = b[4] | (b[5] << 8) | (b[6] << 16) | ((unsigned)b[7] << 24);
-  v.z = b[8] | (b[9] << 8) | (b[10] << 16) | ((unsigned)b[11] << 24);
-  v.w = b[12] | (b[13] << 8) | (b[14] << 16) | ((unsigned)b[15] << 24);
+  v.x = __funnelshift_r(w0, w1, bits);
+  v.y = __funnelshift_r(w1, w2, bits);
+  v.z = __funnelshift_r(w2, w3, bits);
+  v.w = __funnelshift_r(w3, w4, bits);
   return v;
 }
 
-// Store bytes [b0, b1) of the vector v to the 16-byte aligned address p, using the
-// widest naturally aligned stores that stay inside the range.
-__device__ __forceinline__ void store16_partial(char *p, uint4 v, int b0, int b1) {
-  const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-  for (int q = 0; q < 2; q++) {  // the two 8-byte halves
-    const int h0 = q * 8;
-    if (b0 <= h0 && b1 >= h0 + 8) {
-      *reinterpret_cast<uint2 *>(p + h0) = make_uint2(w[2 * q], w[2 * q + 1]);
-      continue;
+// Only the bytes [b0, b1) of the vector at sa, one by one (for blocks at the very
+// ends of their source buffer, where an aligned window would leave it).
+__device__ __noinline__ uint4 load16_bytes(const char *sa, int b0, int b1) {
+  uint32_t w[4] = {0, 0, 0, 0};
+  for (int i = b0; i < b1; i++) w[i >> 2] |= (uint32_t)(unsigned char)sa[i] << (8 * (i & 3));
+  return make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+// Store bytes [b0, b1) of the 16-byte vector at shared address sp to the 16-byte
+// aligned global address gp, in the widest naturally aligned pieces that fit.
+__device__ __forceinline__ void store_pieces(char *gp, const char *sp, int b0, int b1) {
+  int pos = b0;
+  while (pos < b1) {
+    if (!(pos & 7) && pos + 8 <= b1) {
+      *reinterpret_cast<uint2 *>(gp + pos) = *reinterpret_cast<const uint2 *>(sp + pos);
+      pos += 8;
+    } else if (!(pos & 3) && pos + 4 <= b1) {
+      *reinterpret_cast<uint32_t *>(gp + pos) = *reinterpret_cast<const uint32_t *>(sp + pos);
+      pos += 4;
+    } else if (!(pos & 1) && pos + 2 <= b1) {
+      *reinterpret_cast<unsigned short *>(gp + pos) = *reinterpret_cast<const unsigned short *>(sp + pos);
+      pos += 2;
+    } else {
+      gp[pos] = sp[pos];
+      pos += 1;
     }
+  }
+}
+
+// ------------------------------------------------------------------ KEEP lists
+
+__device__ __forceinline__ void keep_body(const TunaMoveArgs &a) {
+  __shared__ int s_vs[kBatch];             // first vector of the block, relative to the chunk
+  __shared__ const char *s_sadj[kBatch];   // source address of chunk vector v is s_sadj + 16 v
+  __shared__ unsigned char s_careful[kBatch];
+  __shared__ __align__(16) unsigned char s_who[kKeepVec];
+
+  const int tid = threadIdx.x, lane = tid & 31;
+  const int64_t c = blockIdx.x;
+  const int64_t cA = c * a.chunk;
+  const int64_t cB = (cA + a.chunk < a.total) ? cA + a.chunk : a.total;
+  const int nv = (int)((cB - cA) >> 4);
+  const int64_t e_lo = a.chunk_first[c];
+  const int64_t e_hi = (c + 1 < a.nchunks) ? (int64_t)a.chunk_first[c + 1] : a.n - 1;
+  char *const out = a.base[2] + a.keep_base + cA;
+
+  for (int64_t b = e_lo; b <= e_hi; b += kBatch) {
+    const int cnt = (int)((e_hi - b + 1 < kBatch) ? e_hi - b + 1 : kBatch);
+    if (b > e_lo) __syncthreads();  // the previous batch is done with the tables
+    if (tid < cnt) {
+      const int64_t e = b + tid;
+      const int64_t p = a.pos[e], pn = a.pos[e + 1];
+      const int64_t s = a.src[e];
+      const int sb = TUNA_LOC_BUF(s);
+      const char *sbase = base_of(a, sb);
+      const char *sp = sbase + TUNA_LOC_OFF(s);
+      const int64_t rel = p - cA;
+      int64_t vs = rel >> 4;
+      if (vs < -kClampVec) vs = -kClampVec;
+      s_vs[tid] = (int)vs;
+      s_sadj[tid] = sp - rel;
+      s_careful[tid] = (sp - 3 < sbase || sp + (pn - p) + 4 > sbase + extent_of(a, sb)) ? 1 : 0;
+    }
+    // vectors of the chunk this batch covers
+    const int64_t first_rel = a.pos[b] - cA, next_rel = a.pos[b + cnt] - cA;
+    const int vlo = first_rel > 0 ? (int)(first_rel >> 4) : 0;
+    const int vhi = (next_rel >> 4) < nv ? (int)(next_rel >> 4) : nv;
+    __syncthreads();
+    const bool single = cnt == 1;
+    if (!single) {
+      fill_owner<kKeepSpan>(s_who, s_vs, cnt, vlo, vhi);
+      __syncthreads();
+    }
+    for (int v = vlo + tid; v - lane < vhi; v += 4 * kThreads) {  // whole warps stay in the loop
+      uint4 x[4];
 #pragma unroll
-    for (int k = 0; k < 2; k++) {  // the 4-byte words of this half
-      const int w0 = h0 + k * 4;
-      const uint32_t x = w[2 * q + k];
-      if (b0 <= w0 && b1 >= w0 + 4) {
-        *reinterpret_cast<uint32_t *>(p + w0) = x;
-        continue;
+      for (int k = 0; k < 4; k++) {
+        const int vv = v + k * kThreads;
+        const bool on = vv < vhi;
+        const char *sa = nullptr;
+        bool careful = false;
+        int t = 0;
+        if (on) {
+          if (!single) t = s_who[vv - vlo];
+          sa = s_sadj[t] + ((int64_t)vv << 4);
+          careful = s_careful[t] != 0;
+        }
+        const bool aligned = (reinterpret_cast<uintptr_t>(sa) & 15) == 0;
+        if (__all_sync(0xffffffffu, !on || (aligned && !careful))) {
+          if (on) x[k] = ld16(sa);
+        } else if (on) {
+          if (!careful) {
+            x[k] = load16_funnel(sa);
+          } else {
+            const int64_t e = b + t;
+            const int64_t rem = a.len[e] - (cA + ((int64_t)vv << 4) - a.pos[e]);
+            x[k] = load16_bytes(sa, 0, rem < 16 ? (int)(rem > 0 ? rem : 0) : 16);
+          }
+        }
       }
 #pragma unroll
-      for (int j = 0; j < 2; j++) {  // the 2-byte halves of this word
-        const int s0 = w0 + j * 2;
-        const uint32_t y = (x >> (16 * j)) & 0xffffu;
-        if (b0 <= s0 && b1 >= s0 + 2) {
-          *reinterpret_cast<unsigned short *>(p + s0) = (unsigned short)y;
-        } else {
-          if (b0 <= s0 && b1 > s0) p[s0] = (char)(y & 0xff);
-          if (b0 <= s0 + 1 && b1 > s0 + 1) p[s0 + 1] = (char)(y >> 8);
-        }
+      for (int k = 0; k < 4; k++) {
+        const int vv = v + k * kThreads;
+        if (vv < vhi) st16(out + ((int64_t)vv << 4), x[k]);
       }
     }
   }
 }
 
-__device__ __forceinline__ void move_body(const TunaMoveArgs &a) {
-  __shared__ __align__(16) char s_buf[kStage];
-  __shared__ const char *s_src[kBatch];
-  __shared__ char *s_dst[kBatch];
-  __shared__ int s_n[kBatch];         // clipped length of the piece in bytes
-  __shared__ int s_dvec[kBatch];      // direct route: first vector of the piece in the run
-  __shared__ int s_svec[kBatch];      // staged route: first vector of the piece in the staging stream
-  __shared__ unsigned char s_who[kStageVec];  // staged route: piece that owns each staged vector
-  __shared__ int s_warp[kWarps];
+// ------------------------------------------------------------------ DELIVER lists
 
-  const int tid = threadIdx.x;
+__device__ __forceinline__ void deliver_body(const TunaMoveArgs &a) {
+  __shared__ __align__(16) char s_buf[kStageVec * 16];
+  __shared__ int s_vs[kBatch];             // first vector of the block, relative to the chunk
+  __shared__ int s_org[kBatch];            // chunk-relative byte position of the block's first byte
+  __shared__ int s_end[kBatch];            // ... and one past its last byte (clamped when far away)
+  __shared__ const char *s_sadj[kBatch];   // source address of chunk vector v is s_sadj + 16 v
+  __shared__ char *s_dadj[kBatch];         // destination address likewise (16-byte aligned)
+  __shared__ unsigned char s_careful[kBatch];
+  __shared__ __align__(16) unsigned char s_who[kStageVec];
+
+  const int tid = threadIdx.x, lane = tid & 31;
   const int64_t c = blockIdx.x;
-  const int64_t lo_pos = c * a.chunk;
-  const int64_t hi_pos = (lo_pos + a.chunk < a.total) ? lo_pos + a.chunk : a.total;
+  const int64_t cA = c * a.chunk;
+  const int64_t cB = (cA + a.chunk < a.total) ? cA + a.chunk : a.total;
+  const int nv = (int)((cB - cA) >> 4);
   const int64_t e_lo = a.chunk_first[c];
   const int64_t e_hi = (c + 1 < a.nchunks) ? (int64_t)a.chunk_first[c + 1] : a.n - 1;
 
   for (int64_t b = e_lo; b <= e_hi; b += kBatch) {
     const int cnt = (int)((e_hi - b + 1 < kBatch) ? e_hi - b + 1 : kBatch);
-    // ---- one descriptor per thread: clip to the chunk, classify ----
-    int n = 0, dvec = 0, svec = 0;
-    bool src_is_send = false, dst_is_work = false;
-    const char *src = nullptr;
-    char *dst = nullptr;
+    if (b > e_lo) __syncthreads();  // the previous batch is done with the tables
+    bool my_stage = false;
+    int my_org = 0, my_end = 0;
     if (tid < cnt) {
       const int64_t e = b + tid;
-      const int64_t p0 = a.pos[e];
+      const int64_t p = a.pos[e];
       const int64_t L = a.len[e];
-      const int64_t lo = (p0 > lo_pos ? p0 : lo_pos) - p0;
-      const int64_t hi = (p0 + L < hi_pos ? p0 + L : hi_pos) - p0;
-      if (hi > lo) {
-        n = (int)(hi - lo);
-        const int64_t s = a.src[e], d = a.dst[e];
-        src = base_of(a, TUNA_LOC_BUF(s)) + TUNA_LOC_OFF(s) + lo;
-        dst = base_of(a, TUNA_LOC_BUF(d)) + TUNA_LOC_OFF(d) + lo;
-        src_is_send = TUNA_LOC_BUF(s) == TUNA_BUF_SEND;
-        dst_is_work = TUNA_LOC_BUF(d) == TUNA_BUF_WORK;
-        const unsigned al = (unsigned)((reinterpret_cast<uintptr_t>(src) | reinterpret_cast<uintptr_t>(dst)) & 15);
-        if (al == 0 && n >= kDirectMin)
-          dvec = n >> 4;  // whole vectors go direct; a ragged tail (< 16 bytes) is staged
-      }
+      const int64_t s = a.src[e], d = a.dst[e];
+      const int sb = TUNA_LOC_BUF(s);
+      const char *sbase = base_of(a, sb);
+      const char *sp = sbase + TUNA_LOC_OFF(s);
+      char *dp = base_of(a, TUNA_LOC_BUF(d)) + TUNA_LOC_OFF(d);
+      const int ad = (int)(reinterpret_cast<uintptr_t>(dp) & 15);
+      const int64_t rel = p - cA;
+      int64_t vs = rel >> 4;
+      if (vs < -kClampVec) vs = -kClampVec;
+      const int64_t org = rel + ad;  // exact chunk-relative position of byte 0
+      int64_t end = org + L;
+      if (end > ((int64_t)kClampVec << 4)) end = (int64_t)kClampVec << 4;
+      my_org = (int)(vs << 4) + ad;
+      my_end = (int)end;
+      s_vs[tid] = (int)vs;
+      s_org[tid] = my_org;
+      s_end[tid] = my_end;
+      s_sadj[tid] = sp - org;
+      s_dadj[tid] = dp - org;
+      s_careful[tid] = (L > 0 && (sp - 19 < sbase || sp + L + 19 > sbase + extent_of(a, sb))) ? 1 : 0;
+      my_stage = L > 0 && (ad != 0 || (L & 15) != 0);
     }
-    const int a_dst = (int)(reinterpret_cast<uintptr_t>(dst) & 15);
-    // what is left for the staging route: everything, or only the ragged tail
-    int stage_n = n, stage_skip = 0;
-    if (dvec > 0) {
-      stage_skip = dvec << 4;
-      stage_n = n - stage_skip;
-    }
-    if (stage_n > 0) svec = (stage_n + a_dst + 15) >> 4;
-    int dtotal, stotal;
-    const int dstart = block_exclusive_scan(dvec, s_warp, &dtotal);
-    const int sstart = block_exclusive_scan(svec, s_warp, &stotal);
-    s_src[tid] = src;
-    s_dst[tid] = dst;
-    // flags packed beside the length: bit 30 = destination is the workspace,
-    // bit 29 = source is the send buffer; lengths are below 2^29 by construction
-    s_n[tid] = n | (dst_is_work ? (1 << 30) : 0) | (src_is_send ? (1 << 29) : 0);
-    s_dvec[tid] = dstart;
-    s_svec[tid] = sstart;
-    __syncthreads();
+    const int64_t first_rel = a.pos[b] - cA, next_rel = a.pos[b + cnt] - cA;
+    const int vlo = first_rel > 0 ? (int)(first_rel >> 4) : 0;
+    const int vhi = (next_rel >> 4) < nv ? (int)(next_rel >> 4) : nv;
+    const int any_stage = __syncthreads_or(my_stage ? 1 : 0);
+    const bool single = cnt == 1;
 
-    // ---- direct route: one run of aligned vectors ----
-    if (dtotal > 0) {
-      int v = tid;
-      for (; v + 3 * kThreads < dtotal; v += 4 * kThreads) {
+    for (int w_lo = vlo; w_lo < vhi; w_lo += kStageVec) {
+      const int w_hi = (w_lo + kStageVec < vhi) ? w_lo + kStageVec : vhi;
+      if (w_lo > vlo) __syncthreads();  // the previous window is done with s_who and s_buf
+      if (!single) {
+        fill_owner<kStageSpan>(s_who, s_vs, cnt, w_lo, w_hi);
+        __syncthreads();
+      }
+      // load a few vectors per thread, then store them: straight to global memory if
+      // the destination is aligned and the vector whole, else into the staging buffer
+      for (int v = w_lo + tid; v - lane < w_hi; v += 4 * kThreads) {  // whole warps stay in the loop
         uint4 x[4];
         char *out[4];
 #pragma unroll
         for (int k = 0; k < 4; k++) {
           const int vv = v + k * kThreads;
-          const int t = find_entry(s_dvec, cnt, vv);
-          const int64_t off = (int64_t)(vv - s_dvec[t]) << 4;
-          x[k] = ld16(s_src[t] + off);
-          out[k] = s_dst[t] + off;
+          bool on = vv < w_hi;
+          const char *sa = nullptr;
+          bool careful = false;
+          int b0 = 0, b1 = 16;
+          out[k] = nullptr;
+          if (on) {
+            const int t = single ? 0 : s_who[vv - w_lo];
+            const int org = s_org[t], end = s_end[t];
+            const int vb = vv << 4;
+            b0 = org - vb;
+            b1 = end - vb;
+            if (b1 <= 0) {
+              on = false;  // the spare vector behind a block: nothing to move
+            } else {
+              sa = s_sadj[t] + (int64_t)vb;
+              careful = s_careful[t] != 0;
+              if ((org & 15) == 0 && b0 <= 0 && b1 >= 16) out[k] = s_dadj[t] + (int64_t)vb;
+            }
+          }
+          const bool aligned = (reinterpret_cast<uintptr_t>(sa) & 15) == 0;
+          if (__all_sync(0xffffffffu, !on || (aligned && !careful))) {
+            if (on) x[k] = ld16(sa);
+          } else if (on) {
+            if (!careful)
+              x[k] = load16_funnel(sa);
+            else
+              x[k] = load16_bytes(sa, b0 > 0 ? b0 : 0, b1 < 16 ? b1 : 16);
+          }
+          if (!on) out[k] = reinterpret_cast<char *>(1);  // marks "skip"
         }
-#pragma unroll
-        for (int k = 0; k < 4; k++) st16(out[k], x[k]);
-      }
-      for (; v < dtotal; v += kThreads) {
-        const int t = find_entry(s_dvec, cnt, v);
-        const int64_t off = (int64_t)(v - s_dvec[t]) << 4;
-        st16(s_dst[t] + off, ld16(s_src[t] + off));
-      }
-    }
-
-    // ---- staged route, one window of the staging stream at a time ----
-    for (int w0 = 0; w0 < stotal; w0 += kStageVec) {
-      const int wn = (stotal - w0 < kStageVec) ? stotal - w0 : kStageVec;
-      if (w0 > 0) __syncthreads();  // the previous window has been written out
-      // gather
-      for (int v = tid; v < wn; v += 4 * kThreads) {
-        uint4 x[4];
 #pragma unroll
         for (int k = 0; k < 4; k++) {
           const int vv = v + k * kThreads;
-          if (vv < wn) {
-            const int g = w0 + vv;
-            const int t = find_entry(s_svec, cnt, g);
-            const int nn = s_n[t];
-            const int len = nn & ((1 << 29) - 1);
-            const bool whole_direct = false;
-            (void)whole_direct;
-            const char *sp = s_src[t];
-            const int ad = (int)(reinterpret_cast<uintptr_t>(s_dst[t]) & 15);
-            // bytes of the piece that go through staging start at `skip`
-            const int dv = (t + 1 < cnt ? s_dvec[t + 1] : dtotal) - s_dvec[t];
-            const int skip = dv << 4;
-            const int off = ((g - s_svec[t]) << 4) - ad;  // first byte of this vector, relative to skip
-            const int b0 = off < 0 ? -off : 0;
-            const int rem = (len - skip) - off;
-            const int b1 = rem < 16 ? rem : 16;
-            const char *sa = sp + skip + off;
-            const bool from_send = (nn >> 29) & 1;
-            const char *elo = from_send ? a.base[0] : a.base[2];
-            const char *ehi = elo + (from_send ? a.extent[0] : a.extent[2]);
-            x[k] = load16_any(sa, elo, ehi, b0, b1);
-            s_who[vv] = (unsigned char)t;
+          if (out[k] == nullptr)
+            *reinterpret_cast<uint4 *>(s_buf + ((vv - w_lo) << 4)) = x[k];
+          else if (out[k] != reinterpret_cast<char *>(1))
+            st16(out[k], x[k]);
+        }
+      }
+      if (any_stage) {
+        __syncthreads();
+        // whole vectors of blocks with an unaligned destination
+        for (int vv = w_lo + tid; vv < w_hi; vv += kThreads) {
+          const int t = single ? 0 : s_who[vv - w_lo];
+          const int org = s_org[t];
+          if (org & 15) {
+            const int vb = vv << 4;
+            if (org <= vb && s_end[t] >= vb + 16)
+              st16(s_dadj[t] + (int64_t)vb, *reinterpret_cast<const uint4 *>(s_buf + ((vv - w_lo) << 4)));
           }
         }
-#pragma unroll
-        for (int k = 0; k < 4; k++) {
-          const int vv = v + k * kThreads;
-          if (vv < wn) *reinterpret_cast<uint4 *>(s_buf + (vv << 4)) = x[k];
+        // the partial first and last vector of a block: its own thread
+        if (my_stage) {
+          const int vh = my_org >> 4, vt = (my_end - 1) >> 4;
+          if (vh >= w_lo && vh < w_hi && ((my_org & 15) != 0 || my_end < (vh << 4) + 16))
+            store_pieces(s_dadj[tid] + ((int64_t)vh << 4), s_buf + ((vh - w_lo) << 4), my_org - (vh << 4),
+                         my_end - (vh << 4) < 16 ? my_end - (vh << 4) : 16);
+          if (vt > vh && vt >= w_lo && vt < w_hi && (my_end & 15) != 0)
+            store_pieces(s_dadj[tid] + ((int64_t)vt << 4), s_buf + ((vt - w_lo) << 4), 0, my_end - (vt << 4));
         }
       }
-      __syncthreads();
-      // scatter
-      for (int vv = tid; vv < wn; vv += kThreads) {
-        const int g = w0 + vv;
-        const int t = s_who[vv];
-        const int nn = s_n[t];
-        const int len = nn & ((1 << 29) - 1);
-        char *dp = s_dst[t];
-        const int ad = (int)(reinterpret_cast<uintptr_t>(dp) & 15);
-        const int dv = (t + 1 < cnt ? s_dvec[t + 1] : dtotal) - s_dvec[t];
-        const int skip = dv << 4;
-        const int off = ((g - s_svec[t]) << 4) - ad;
-        const int b0 = off < 0 ? -off : 0;
-        const int rem = (len - skip) - off;
-        const int b1 = rem < 16 ? rem : 16;
-        const uint4 x = *reinterpret_cast<const uint4 *>(s_buf + (vv << 4));
-        char *da = dp + skip + off;
-        if ((b0 == 0 && b1 == 16) || ((nn >> 30) & 1))
-          st16(da, x);  // whole vector, or padding of our own workspace
-        else
-          store16_partial(da, x, b0, b1);
-      }
     }
-    __syncthreads();  // shared tables are rewritten by the next batch
   }
 }
 
-__global__ void __launch_bounds__(kThreads) tuna_round_kernel(const TunaMoveArgs a) { move_body(a); }
-__global__ void __launch_bounds__(kThreads) tuna_rotate_kernel(const TunaMoveArgs a) { move_body(a); }
-__global__ void __launch_bounds__(kThreads) tuna_direct_kernel(const TunaMoveArgs a) { move_body(a); }
+__global__ void __launch_bounds__(kThreads) tuna_round_kernel(const TunaMoveArgs a) { keep_body(a); }
+__global__ void __launch_bounds__(kThreads) tuna_deliver_kernel(const TunaMoveArgs a) { deliver_body(a); }
+__global__ void __launch_bounds__(kThreads) tuna_rotate_kernel(const TunaMoveArgs a) { deliver_body(a); }
+__global__ void __launch_bounds__(kThreads) tuna_direct_kernel(const TunaMoveArgs a) { deliver_body(a); }
 
 }  // namespace
 
-cudaError_t tuna_launch_move(int kind, const TunaMoveArgs &a, cudaStream_t stream) {
+cudaError_t tuna_launch_move(int kernel, const TunaMoveArgs &a, cudaStream_t stream) {
   if (a.nchunks <= 0 || a.n <= 0) return cudaSuccess;
   const dim3 grid((unsigned)a.nchunks), block(kThreads);
-  switch (kind) {
-    case TUNA_MOVE_ROUND:
+  switch (kernel) {
+    case TUNA_K_ROUND:
+      if (a.chunk > (int64_t)kKeepVec * 16) return cudaErrorInvalidValue;
       tuna_round_kernel<<<grid, block, 0, stream>>>(a);
       break;
-    case TUNA_MOVE_ROTATE:
+    case TUNA_K_DELIVER:
+      tuna_deliver_kernel<<<grid, block, 0, stream>>>(a);
+      break;
+    case TUNA_K_ROTATE:
       tuna_rotate_kernel<<<grid, block, 0, stream>>>(a);
       break;
     default:

@@ -40,8 +40,17 @@ __device__ __forceinline__ int64_t compact_of(int64_t v, int64_t stride, int rad
 
 struct PhaseDev {
   int level, radix, count;
-  int64_t stride, moving, per_rank;
+  int64_t stride, moving, per_rank, finals;
 };
+
+// Row position of a moving slot among the blocks its rank receives in a phase
+// (slot order), and the descriptor it maps to: the first `finals` positions of
+// every rank's row are the blocks that have arrived (DELIVER list, `finals` per
+// rank), the others travel on (KEEP list, per_rank - finals per rank).
+__device__ __forceinline__ int64_t row_position(const TunaTopo &t, const PhaseDev &ph, int io, int jo) {
+  return ph.level == 0 ? (int64_t)io * ph.moving + compact_of(jo, ph.stride, ph.radix)
+                       : compact_of(io, ph.stride, ph.radix) * t.Q + jo;
+}
 
 // Initial tables (before any phase): every block is in its owner's send region.
 // Also fills the direct list (receive-side order (d, s)) and the self entries of
@@ -85,8 +94,8 @@ __global__ void tuna_init_tables_kernel(TunaTopo t, const int64_t *__restrict__ 
 // per-round byte totals (round z = the slots whose digit equals z).
 __global__ void tuna_meta_exchange_kernel(TunaTopo t, PhaseDev ph, const int64_t *__restrict__ sz_cur,
                                           const int64_t *__restrict__ loc_cur, int64_t *sz_next,
-                                          int64_t *len, int64_t *src,
-                                          unsigned long long *round_bytes) {
+                                          int64_t *keep_len, int64_t *keep_src, int64_t *del_len,
+                                          int64_t *del_src, unsigned long long *round_bytes) {
   extern __shared__ unsigned long long s_hist[];
   const bool use_smem = ph.radix <= 4096;
   if (use_smem) {
@@ -104,19 +113,21 @@ __global__ void tuna_meta_exchange_kernel(TunaTopo t, PhaseDev ph, const int64_t
       sz_next[idx] = sz_cur[idx];
     } else {
       const int64_t dist = dig * ph.stride;
-      int sender;
-      int64_t e;
-      if (ph.level == 0) {
-        sender = n * t.Q + (int)(((q - dist) % t.Q + t.Q) % t.Q);
-        e = (int64_t)p * ph.per_rank + (int64_t)io * ph.moving + compact_of(jo, ph.stride, ph.radix);
-      } else {
-        sender = (int)(((n - dist) % t.N + t.N) % t.N) * t.Q + q;
-        e = (int64_t)p * ph.per_rank + compact_of(io, ph.stride, ph.radix) * t.Q + jo;
-      }
+      const int sender = ph.level == 0 ? n * t.Q + (int)(((q - dist) % t.Q + t.Q) % t.Q)
+                                       : (int)(((n - dist) % t.N + t.N) % t.N) * t.Q + q;
+      const int64_t c = row_position(t, ph, io, jo);
       const int64_t bytes = sz_cur[(int64_t)sender * t.P + sigma];
+      const int64_t where = loc_cur[(int64_t)sender * t.P + sigma];
       sz_next[idx] = bytes;
-      len[e] = bytes;
-      src[e] = loc_cur[(int64_t)sender * t.P + sigma];
+      if (c < ph.finals) {
+        const int64_t e = (int64_t)p * ph.finals + c;
+        del_len[e] = bytes;
+        del_src[e] = where;
+      } else {
+        const int64_t e = (int64_t)p * (ph.per_rank - ph.finals) + (c - ph.finals);
+        keep_len[e] = bytes;
+        keep_src[e] = where;
+      }
       if (bytes > 0) {
         if (use_smem)
           atomicAdd(&s_hist[dig], (unsigned long long)bytes);
@@ -133,10 +144,11 @@ __global__ void tuna_meta_exchange_kernel(TunaTopo t, PhaseDev ph, const int64_t
 }
 
 // Segmented exclusive prefix sum, one warp per segment, warp-shuffle scan over
-// 32-wide tiles with a running carry.  PAD rounds every value up to 16 first.
-// seg_total[s] receives the segment's (padded) sum, seg_raw[s] (optional) the
-// unpadded sum.
-template <bool PAD>
+// 32-wide tiles with a running carry.  MODE 0 sums the values as they are; MODE 1
+// (KEEP lists) rounds every value up to 16 first; MODE 2 (DELIVER lists) also
+// adds 16 spare bytes behind every non-zero value.  seg_total[s] receives the
+// segment's sum, seg_raw[s] (optional) the sum of the unmodified values.
+template <int MODE>
 __global__ void tuna_segscan_kernel(const int64_t *__restrict__ val, int64_t *out,
                                     int64_t *seg_total, int64_t *seg_raw, int64_t seglen,
                                     int64_t nseg) {
@@ -150,7 +162,8 @@ __global__ void tuna_segscan_kernel(const int64_t *__restrict__ val, int64_t *ou
     const int64_t i = base + lane;
     int64_t x = i < seglen ? v[i] : 0;
     raw += x;
-    if (PAD) x = pad16(x);
+    if (MODE >= 1) x = pad16(x);
+    if (MODE == 2 && x > 0) x += 16;
     int64_t incl = x;
 #pragma unroll
     for (int d = 1; d < 32; d <<= 1) {
@@ -174,7 +187,8 @@ __global__ void tuna_segscan_kernel(const int64_t *__restrict__ val, int64_t *ou
 // or wbase[0] when the phase keeps nothing in the workspace.
 __global__ void tuna_segbase_kernel(const int64_t *__restrict__ seg_total,
                                     const int64_t *__restrict__ seg_raw, int64_t *seg_base,
-                                    int64_t nseg, int64_t *scal, int64_t *wbase, int uses_work) {
+                                    int64_t nseg, int64_t *scal, int64_t *wbase, int uses_work,
+                                    int64_t *pos_end) {
   __shared__ int64_t s_warp[32];
   __shared__ int64_t s_carry;
   __shared__ int64_t s_raw[32];
@@ -211,6 +225,7 @@ __global__ void tuna_segbase_kernel(const int64_t *__restrict__ seg_total,
     for (int k = 0; k < nw; k++) r += s_raw[k];
     scal[0] = s_carry;
     scal[1] = r;
+    if (pos_end) *pos_end = s_carry;  // pos[n]: one past the last block
     if (wbase) wbase[1] = wbase[0] + (uses_work ? ((s_carry + 255) & ~(int64_t)255) : 0);
   }
 }
@@ -222,15 +237,17 @@ __global__ void tuna_add_base_kernel(int64_t *pos, const int64_t *__restrict__ s
   if (e < n) pos[e] += seg_base[e / seglen];
 }
 
-// Second half of a digit phase, after the prefix sums: destination of every
-// moving block, and the location table for the next phase.  A block whose
-// remaining digits are all zero has arrived: its destination is its place in
-// the receive buffer (direct-to-R) or, in classic mode, still the workspace,
-// with a rotation descriptor recorded for the final reorder.
+// Second half of a digit phase, after the prefix sums: stream positions become
+// global, every moving block gets its destination, and the location table for
+// the next phase is written.  A block whose remaining digits are all zero has
+// arrived: in direct-to-R mode it is in the DELIVER list and goes to its place in
+// the receive buffer; in classic mode every block stays in the workspace and a
+// rotation descriptor is recorded for the final reorder.
 __global__ void tuna_place_kernel(TunaTopo t, PhaseDev ph, const int64_t *__restrict__ loc_cur,
-                                  int64_t *loc_next, int64_t *pos,
-                                  const int64_t *__restrict__ seg_base,
-                                  const int64_t *__restrict__ len, int64_t *dst,
+                                  int64_t *loc_next, int64_t *keep_pos,
+                                  const int64_t *__restrict__ keep_base,
+                                  const int64_t *__restrict__ keep_len, int64_t *del_pos,
+                                  const int64_t *__restrict__ del_base, int64_t *del_dst,
                                   const int64_t *__restrict__ wbase,
                                   const int64_t *__restrict__ rdispls,
                                   const int64_t *__restrict__ recvbase, int classic,
@@ -246,33 +263,29 @@ __global__ void tuna_place_kernel(TunaTopo t, PhaseDev ph, const int64_t *__rest
     loc_next[idx] = loc_cur[idx];
     return;
   }
-  int64_t e;
-  bool fin;
-  if (ph.level == 0) {
-    e = (int64_t)p * ph.per_rank + (int64_t)io * ph.moving + compact_of(jo, ph.stride, ph.radix);
-    fin = (io == 0) && (jo / (ph.stride * ph.radix) == 0);
+  const int64_t c = row_position(t, ph, io, jo);
+  const bool fin = ph.level == 0 ? (io == 0 && jo / (ph.stride * ph.radix) == 0)
+                                 : io / (ph.stride * ph.radix) == 0;
+  const int origin = ((n - io + t.N) % t.N) * t.Q + (q - jo + t.Q) % t.Q;
+  const int64_t rloc =
+      TUNA_LOC(TUNA_BUF_RECV, (recvbase[p] + rdispls[(int64_t)p * t.P + origin]) * t.elem);
+  if (c < ph.finals) {  // DELIVER list (only in direct-to-R mode; these blocks have arrived)
+    const int64_t e = (int64_t)p * ph.finals + c;
+    del_pos[e] += del_base[p];
+    del_dst[e] = rloc;
+    loc_next[idx] = rloc;
   } else {
-    e = (int64_t)p * ph.per_rank + compact_of(io, ph.stride, ph.radix) * t.Q + jo;
-    fin = io / (ph.stride * ph.radix) == 0;
-  }
-  const int64_t w = pos[e] + seg_base[p];
-  pos[e] = w;
-  const int64_t wloc = TUNA_LOC(TUNA_BUF_WORK, wbase[0] + w);
-  int64_t d = wloc;
-  if (fin) {
-    const int origin = ((n - io + t.N) % t.N) * t.Q + (q - jo + t.Q) % t.Q;
-    const int64_t rloc =
-        TUNA_LOC(TUNA_BUF_RECV, (recvbase[p] + rdispls[(int64_t)p * t.P + origin]) * t.elem);
-    if (classic) {
-      rot_len[idx] = len[e];
+    const int64_t e = (int64_t)p * (ph.per_rank - ph.finals) + (c - ph.finals);
+    const int64_t w = keep_pos[e] + keep_base[p];
+    keep_pos[e] = w;
+    const int64_t wloc = TUNA_LOC(TUNA_BUF_WORK, wbase[0] + w);
+    loc_next[idx] = wloc;
+    if (fin && classic) {
+      rot_len[idx] = keep_len[e];
       rot_src[idx] = wloc;
       rot_dst[idx] = rloc;
-    } else {
-      d = rloc;
     }
   }
-  dst[e] = d;
-  loc_next[idx] = d;
 }
 
 // First descriptor of every chunk: the last e with pos[e] <= c * chunk.
@@ -312,7 +325,8 @@ struct tuna_plan {
   int last_launches = 0;
 
   std::vector<TunaPhase> phases;
-  std::vector<TunaList> lists;  // one per phase
+  std::vector<TunaList> keep;     // per phase: blocks that travel on (workspace)
+  std::vector<TunaList> deliver;  // per phase: blocks that have arrived (receive buffer)
   TunaList rot, dir;
 
   struct Round {
@@ -337,6 +351,7 @@ struct tuna_plan {
   unsigned long long *d_round_bytes = nullptr;
   int64_t stats_n = 0;
 
+  std::vector<int64_t> h_wbase;  // workspace offset of every phase's KEEP stream
   int64_t workspace_need = 0;
   char *workspace = nullptr;
   size_t workspace_bytes = 0;
@@ -449,12 +464,13 @@ void free_list(TunaList &l) {
   l = TunaList();
 }
 
-int alloc_list(tuna_plan *pl, TunaList &l, int64_t n) {
+int alloc_list(tuna_plan *pl, TunaList &l, int kind, int64_t n) {
+  l.kind = kind;
   l.n = n;
   TUNA_CUDA(pl, dev_alloc(&l.len, n));
-  TUNA_CUDA(pl, dev_alloc(&l.pos, n));
+  TUNA_CUDA(pl, dev_alloc(&l.pos, n + 1));
   TUNA_CUDA(pl, dev_alloc(&l.src, n));
-  TUNA_CUDA(pl, dev_alloc(&l.dst, n));
+  if (kind == TUNA_LIST_DELIVER) TUNA_CUDA(pl, dev_alloc(&l.dst, n));
   return TUNA_OK;
 }
 
@@ -467,16 +483,17 @@ int64_t env_i64(const char *name, int64_t dflt) {
 // Bytes of destination stream per CTA: enough chunks to fill the machine several
 // times over, but no smaller than a few KiB (descriptor overhead) and no larger
 // than 128 KiB (tail effect).
-int64_t pick_chunk(int64_t total) {
-  const int64_t forced = env_i64("TUNA_CHUNK_BYTES", 0);
-  if (forced >= 1024) return std::min<int64_t>((forced + 15) & ~(int64_t)15, (int64_t)1 << 24);
+int64_t pick_chunk(int64_t total, int kind) {
+  const int64_t forced = env_i64(kind == TUNA_LIST_KEEP ? "TUNA_CHUNK_BYTES_KEEP" : "TUNA_CHUNK_BYTES_DELIVER", 0);
+  const int64_t cap = kind == TUNA_LIST_KEEP ? 65536 : ((int64_t)1 << 24);
+  if (forced >= 1024) return std::min<int64_t>((forced + 15) & ~(int64_t)15, cap);
   int64_t c = 8192;
   while (c < 65536 && total / c > 148 * 32) c <<= 1;
   return c;
 }
 
 int build_chunks(tuna_plan *pl, TunaList &l, cudaStream_t st) {
-  l.chunk = pick_chunk(l.total);
+  l.chunk = pick_chunk(l.total, l.kind);
   l.nchunks = l.total > 0 ? (l.total + l.chunk - 1) / l.chunk : 0;
   if (l.nchunks > l.chunk_cap) {
     cudaFree(l.chunk_first);
@@ -496,22 +513,28 @@ int build_chunks(tuna_plan *pl, TunaList &l, cudaStream_t st) {
 
 // scan of one list: per-rank warp scans, segment bases, (optionally) add bases
 int scan_list(tuna_plan *pl, TunaList &l, int64_t seglen, int64_t nseg, int list_id,
-              int64_t *wbase_slot, int uses_work, bool add_base, cudaStream_t st) {
+              int64_t *wbase_slot, int uses_work, bool add_base, cudaStream_t st, int slot = 0) {
+  int64_t *seg_total = pl->d_seg_total + (int64_t)slot * pl->topo.P;
+  int64_t *seg_base = pl->d_seg_base + (int64_t)slot * pl->topo.P;
   if (nseg > 0 && seglen > 0) {
     const int th = 256;
     const int64_t blocks = (nseg * 32 + th - 1) / th;
-    tuna_segscan_kernel<true><<<(unsigned)blocks, th, 0, st>>>(l.len, l.pos, pl->d_seg_total,
-                                                                pl->d_seg_raw, seglen, nseg);
+    if (l.kind == TUNA_LIST_KEEP)
+      tuna_segscan_kernel<1><<<(unsigned)blocks, th, 0, st>>>(l.len, l.pos, seg_total, pl->d_seg_raw,
+                                                               seglen, nseg);
+    else
+      tuna_segscan_kernel<2><<<(unsigned)blocks, th, 0, st>>>(l.len, l.pos, seg_total, pl->d_seg_raw,
+                                                               seglen, nseg);
     TUNA_LAUNCHED(pl);
   }
-  tuna_segbase_kernel<<<1, 1024, 0, st>>>(pl->d_seg_total, pl->d_seg_raw, pl->d_seg_base,
+  tuna_segbase_kernel<<<1, 1024, 0, st>>>(seg_total, pl->d_seg_raw, seg_base,
                                           (nseg > 0 && seglen > 0) ? nseg : 0,
-                                          pl->d_scal + 2 * list_id, wbase_slot, uses_work);
+                                          pl->d_scal + 2 * list_id, wbase_slot, uses_work,
+                                          l.pos + l.n);
   TUNA_LAUNCHED(pl);
   if (add_base && l.n > 0) {
     const int th = 256;
-    tuna_add_base_kernel<<<(unsigned)((l.n + th - 1) / th), th, 0, st>>>(l.pos, pl->d_seg_base,
-                                                                          seglen, l.n);
+    tuna_add_base_kernel<<<(unsigned)((l.n + th - 1) / th), th, 0, st>>>(l.pos, seg_base, seglen, l.n);
     TUNA_LAUNCHED(pl);
   }
   return TUNA_OK;
@@ -583,8 +606,8 @@ int build_tables(tuna_plan *pl, const int64_t *counts, const int64_t *sdispls,
   if (sdispls) {
     TUNA_CUDA(pl, cudaMemcpyAsync(pl->d_sdispls, sdispls, PP * 8, cudaMemcpyHostToDevice, st));
   } else {  // packed: exclusive scan of every rank's row of counts
-    tuna_segscan_kernel<false><<<gseg, th, 0, st>>>(pl->d_counts, pl->d_sdispls, pl->d_seg_total,
-                                                     nullptr, P, P);
+    tuna_segscan_kernel<0><<<gseg, th, 0, st>>>(pl->d_counts, pl->d_sdispls, pl->d_seg_total,
+                                                 nullptr, P, P);
     TUNA_LAUNCHED(pl);
   }
   if (rdispls) {
@@ -592,8 +615,8 @@ int build_tables(tuna_plan *pl, const int64_t *counts, const int64_t *sdispls,
   } else {  // packed: scan of the receive counts = rows of the transposed matrix
     tuna_transpose_kernel<<<gPP, th, 0, st>>>(pl->d_counts, pl->d_tmp, P);
     TUNA_LAUNCHED(pl);
-    tuna_segscan_kernel<false><<<gseg, th, 0, st>>>(pl->d_tmp, pl->d_rdispls, pl->d_seg_total,
-                                                     nullptr, P, P);
+    tuna_segscan_kernel<0><<<gseg, th, 0, st>>>(pl->d_tmp, pl->d_rdispls, pl->d_seg_total,
+                                                 nullptr, P, P);
     TUNA_LAUNCHED(pl);
   }
 
@@ -615,53 +638,60 @@ int build_tables(tuna_plan *pl, const int64_t *counts, const int64_t *sdispls,
   int cur = 0;
   for (int f = 0; f < nph; f++) {
     const TunaPhase &ph = pl->phases[f];
-    TunaList &l = pl->lists[f];
-    PhaseDev pd{ph.level, ph.radix, ph.count, ph.stride, ph.moving, ph.per_rank};
+    TunaList &k = pl->keep[f];
+    TunaList &d = pl->deliver[f];
+    PhaseDev pd{ph.level, ph.radix, ph.count, ph.stride, ph.moving, ph.per_rank, ph.finals};
     const size_t smem = ph.radix <= 4096 ? (size_t)ph.radix * 8 : 0;
     tuna_meta_exchange_kernel<<<gPP, th, smem, st>>>(t, pd, pl->d_sz[cur], pl->d_loc[cur],
-                                                     pl->d_sz[cur ^ 1], l.len, l.src,
+                                                     pl->d_sz[cur ^ 1], k.len, k.src, d.len, d.src,
                                                      pl->d_round_bytes + ph.stats_off);
     TUNA_LAUNCHED(pl);
-    // in direct-to-R mode the last phase delivers everything: it keeps nothing
-    const int uses_work = (pl->classic || f + 1 < nph) ? 1 : 0;
-    rc = scan_list(pl, l, ph.per_rank, P, f, pl->d_wbase + f, uses_work, false, st);
+    // per-rank prefix sums of both lists; the KEEP stream is this phase's workspace region
+    rc = scan_list(pl, k, ph.per_rank - ph.finals, P, f, pl->d_wbase + f, 1, false, st, 0);
     if (rc) return rc;
-    tuna_place_kernel<<<gPP, th, 0, st>>>(t, pd, pl->d_loc[cur], pl->d_loc[cur ^ 1], l.pos,
-                                          pl->d_seg_base, l.len, l.dst, pl->d_wbase + f,
-                                          pl->d_rdispls, pl->d_recvbase, pl->classic ? 1 : 0,
-                                          pl->rot.len, pl->rot.src, pl->rot.dst);
+    rc = scan_list(pl, d, ph.finals, P, nph + f, nullptr, 0, false, st, 1);
+    if (rc) return rc;
+    tuna_place_kernel<<<gPP, th, 0, st>>>(t, pd, pl->d_loc[cur], pl->d_loc[cur ^ 1], k.pos,
+                                          pl->d_seg_base, k.len, d.pos, pl->d_seg_base + P, d.dst,
+                                          pl->d_wbase + f, pl->d_rdispls, pl->d_recvbase,
+                                          pl->classic ? 1 : 0, pl->rot.len, pl->rot.src, pl->rot.dst);
     TUNA_LAUNCHED(pl);
     cur ^= 1;
   }
   // work partitions of the rotation and direct lists
-  rc = scan_list(pl, pl->rot, pl->classic ? P : 1, P, nph, nullptr, 0, true, st);
+  rc = scan_list(pl, pl->rot, pl->classic ? P : 1, P, 2 * nph, nullptr, 0, true, st);
   if (rc) return rc;
-  rc = scan_list(pl, pl->dir, P, P, nph + 1, nullptr, 0, true, st);
+  rc = scan_list(pl, pl->dir, P, P, 2 * nph + 1, nullptr, 0, true, st);
   if (rc) return rc;
 
   plan_timer.stop();  // the chunk tables below are timed separately, after the read-back
   // one read-back: stream totals, workspace offsets, per-round bytes
-  std::vector<int64_t> scal(2 * (nph + 2)), wbase(nph + 1);
+  std::vector<int64_t> scal(2 * (2 * nph + 2)), wbase(nph + 1);
   std::vector<unsigned long long> rbytes(std::max<int64_t>(pl->stats_n, 1));
   TUNA_CUDA(pl, cudaMemcpyAsync(scal.data(), pl->d_scal, scal.size() * 8, cudaMemcpyDeviceToHost, st));
   TUNA_CUDA(pl, cudaMemcpyAsync(wbase.data(), pl->d_wbase, wbase.size() * 8, cudaMemcpyDeviceToHost, st));
   TUNA_CUDA(pl, cudaMemcpyAsync(rbytes.data(), pl->d_round_bytes, rbytes.size() * 8,
                                 cudaMemcpyDeviceToHost, st));
   TUNA_CUDA(pl, cudaStreamSynchronize(st));
+  pl->h_wbase = wbase;
+  auto take = [&](TunaList &l, int id) {
+    l.total = scal[2 * id];
+    l.bytes = scal[2 * id + 1];
+  };
   for (int f = 0; f < nph; f++) {
-    pl->lists[f].total = scal[2 * f];
-    pl->lists[f].bytes = scal[2 * f + 1];
+    take(pl->keep[f], f);
+    take(pl->deliver[f], nph + f);
   }
-  pl->rot.total = scal[2 * nph];
-  pl->rot.bytes = scal[2 * nph + 1];
-  pl->dir.total = scal[2 * (nph + 1)];
-  pl->dir.bytes = scal[2 * (nph + 1) + 1];
+  take(pl->rot, 2 * nph);
+  take(pl->dir, 2 * nph + 1);
   pl->workspace_need = wbase[nph];
   for (auto &r : pl->rounds) r.bytes = (int64_t)rbytes[pl->phases[r.phase].stats_off + r.z];
 
   Timed chunk_timer(pl, TUNA_TIMER_PLAN, 0, st);
   for (int f = 0; f < nph; f++) {
-    rc = build_chunks(pl, pl->lists[f], st);
+    rc = build_chunks(pl, pl->keep[f], st);
+    if (rc) return rc;
+    rc = build_chunks(pl, pl->deliver[f], st);
     if (rc) return rc;
   }
   rc = build_chunks(pl, pl->rot, st);
@@ -683,6 +713,10 @@ void add_level(tuna_plan *pl, int level, int count, int radix, int other) {
     ph.stride = ipow64(radix, x);
     ph.moving = count - count_digit(count, radix, x, 0);
     ph.per_rank = ph.moving * other;
+    // blocks whose higher digits are all zero arrive in this phase: the offsets
+    // below radix^(x+1) with a non-zero digit x (own group only, for local phases)
+    const int64_t arrive = std::min<int64_t>(count, ph.stride * radix) - std::min<int64_t>(count, ph.stride);
+    ph.finals = pl->classic ? 0 : (level == 0 ? arrive : arrive * other);
     ph.stats_off = pl->stats_n;
     pl->stats_n += radix;
     const int phase = (int)pl->phases.size();
@@ -763,6 +797,7 @@ TunaMoveArgs move_args(const tuna_plan *pl, const TunaList &l, const void *send,
   a.extent[TUNA_BUF_SEND] = pl->send_extent;
   a.extent[TUNA_BUF_RECV] = pl->recv_extent;
   a.extent[TUNA_BUF_WORK] = work ? pl->workspace_need : 0;
+  a.keep_base = 0;
   return a;
 }
 
@@ -771,19 +806,26 @@ int run_tuna(tuna_plan *pl, const void *send, void *recv, cudaStream_t st) {
       (!pl->workspace || pl->workspace_bytes < (size_t)pl->workspace_need))
     return TUNA_ERR_WORKSPACE;
   int launches = 0;
-  for (size_t f = 0; f < pl->lists.size(); f++) {
-    const TunaList &l = pl->lists[f];
-    if (l.nchunks == 0) continue;
-    {
-      Timed tm(pl, pl->phases[f].level == 0 ? TUNA_TIMER_ROUND_LOCAL : TUNA_TIMER_ROUND_GLOBAL,
-               l.bytes, st);
-      TUNA_CUDA(pl, tuna_launch_move(TUNA_MOVE_ROUND, move_args(pl, l, send, recv, pl->workspace), st));
+  for (size_t f = 0; f < pl->phases.size(); f++) {
+    const int kind = pl->phases[f].level == 0 ? TUNA_TIMER_ROUND_LOCAL : TUNA_TIMER_ROUND_GLOBAL;
+    const TunaList &k = pl->keep[f];
+    if (k.nchunks > 0) {
+      Timed tm(pl, kind, k.bytes, st);
+      TunaMoveArgs a = move_args(pl, k, send, recv, pl->workspace);
+      a.keep_base = pl->h_wbase[f];
+      TUNA_CUDA(pl, tuna_launch_move(TUNA_K_ROUND, a, st));
+      launches++;
     }
-    launches++;
+    const TunaList &d = pl->deliver[f];
+    if (d.nchunks > 0) {
+      Timed tm(pl, kind, d.bytes, st);
+      TUNA_CUDA(pl, tuna_launch_move(TUNA_K_DELIVER, move_args(pl, d, send, recv, pl->workspace), st));
+      launches++;
+    }
   }
   if (pl->rot.nchunks > 0) {
     Timed tm(pl, TUNA_TIMER_ROTATE, pl->rot.bytes, st);
-    TUNA_CUDA(pl, tuna_launch_move(TUNA_MOVE_ROTATE, move_args(pl, pl->rot, send, recv, pl->workspace), st));
+    TUNA_CUDA(pl, tuna_launch_move(TUNA_K_ROTATE, move_args(pl, pl->rot, send, recv, pl->workspace), st));
     launches++;
   }
   pl->last_launches = launches;
@@ -795,7 +837,7 @@ int run_direct(tuna_plan *pl, const void *send, void *recv, cudaStream_t st) {
   int launches = 0;
   if (pl->dir.nchunks > 0) {
     Timed tm(pl, TUNA_TIMER_DIRECT, pl->dir.bytes, st);
-    TUNA_CUDA(pl, tuna_launch_move(TUNA_MOVE_DIRECT, move_args(pl, pl->dir, send, recv, nullptr), st));
+    TUNA_CUDA(pl, tuna_launch_move(TUNA_K_DIRECT, move_args(pl, pl->dir, send, recv, nullptr), st));
     launches++;
   }
   pl->last_launches = launches;
@@ -831,7 +873,8 @@ const char *tuna_strerror(int status) {
 
 int tuna_plan_destroy(tuna_plan_t *pl) {
   if (!pl) return TUNA_OK;
-  for (auto &l : pl->lists) free_list(l);
+  for (auto &l : pl->keep) free_list(l);
+  for (auto &l : pl->deliver) free_list(l);
   free_list(pl->rot);
   free_list(pl->dir);
   cudaFree(pl->d_counts);
@@ -907,22 +950,29 @@ int tuna_plan_create(tuna_plan_t **out, int P, int radix, int radix_global, int 
     TUNA_TRY(dev_alloc(&pl->d_sz[i], PP));
     TUNA_TRY(dev_alloc(&pl->d_loc[i], PP));
   }
-  TUNA_TRY(dev_alloc(&pl->d_seg_total, P));
+  TUNA_TRY(dev_alloc(&pl->d_seg_total, 2 * P));
   TUNA_TRY(dev_alloc(&pl->d_seg_raw, P));
-  TUNA_TRY(dev_alloc(&pl->d_seg_base, P));
+  TUNA_TRY(dev_alloc(&pl->d_seg_base, 2 * P));
   TUNA_TRY(dev_alloc(&pl->d_tmp, PP));
-  TUNA_TRY(dev_alloc(&pl->d_scal, 2 * (nph + 2)));
+  TUNA_TRY(dev_alloc(&pl->d_scal, 2 * (2 * nph + 2)));
   TUNA_TRY(dev_alloc(&pl->d_wbase, nph + 1));
   TUNA_TRY(dev_alloc(&pl->d_round_bytes, pl->stats_n));
-  pl->lists.resize(nph);
+  pl->keep.resize(nph);
+  pl->deliver.resize(nph);
+  auto nomem = [&](int code) {
+    return fail(pl->cuda_err == (int)cudaErrorMemoryAllocation ? TUNA_ERR_NOMEM : code);
+  };
   for (int f = 0; f < nph; f++) {
-    rc = alloc_list(pl, pl->lists[f], (int64_t)P * pl->phases[f].per_rank);
-    if (rc) return fail(pl->cuda_err == (int)cudaErrorMemoryAllocation ? TUNA_ERR_NOMEM : rc);
+    const TunaPhase &ph = pl->phases[f];
+    rc = alloc_list(pl, pl->keep[f], TUNA_LIST_KEEP, (int64_t)P * (ph.per_rank - ph.finals));
+    if (rc) return nomem(rc);
+    rc = alloc_list(pl, pl->deliver[f], TUNA_LIST_DELIVER, (int64_t)P * ph.finals);
+    if (rc) return nomem(rc);
   }
-  rc = alloc_list(pl, pl->rot, pl->classic ? PP : P);
-  if (rc) return fail(rc);
-  rc = alloc_list(pl, pl->dir, PP);
-  if (rc) return fail(rc);
+  rc = alloc_list(pl, pl->rot, TUNA_LIST_DELIVER, pl->classic ? PP : P);
+  if (rc) return nomem(rc);
+  rc = alloc_list(pl, pl->dir, TUNA_LIST_DELIVER, PP);
+  if (rc) return nomem(rc);
 #undef TUNA_TRY
   rc = build_tables(pl, sendcounts, sdispls, rdispls, sendbase, recvbase, st);
   if (rc) return fail(rc);
@@ -1036,14 +1086,20 @@ int tuna_plan_num_phases(const tuna_plan_t *pl, int *n) {
   return TUNA_OK;
 }
 
-int tuna_plan_phase_info(const tuna_plan_t *pl, int phase, int *level, int *x, int64_t *entries,
-                         int64_t *bytes, int64_t *stream_bytes) {
+static const TunaList *pick_list(const tuna_plan *pl, int phase, int part) {
+  if (phase == -1) return &pl->rot;
+  if (phase == -2) return &pl->dir;
+  if (phase < 0 || phase >= (int)pl->phases.size()) return nullptr;
+  if (part == TUNA_PART_KEEP) return &pl->keep[phase];
+  if (part == TUNA_PART_DELIVER) return &pl->deliver[phase];
+  return nullptr;
+}
+
+int tuna_plan_phase_info(const tuna_plan_t *pl, int phase, int part, int *level, int *x,
+                         int64_t *entries, int64_t *bytes, int64_t *stream_bytes) {
   if (!pl) return TUNA_ERR_INVALID_ARG;
-  const TunaList *l;
-  if (phase == -1) l = &pl->rot;
-  else if (phase == -2) l = &pl->dir;
-  else if (phase >= 0 && phase < (int)pl->phases.size()) l = &pl->lists[phase];
-  else return TUNA_ERR_RANGE;
+  const TunaList *l = pick_list(pl, phase, part);
+  if (!l) return TUNA_ERR_RANGE;
   if (level) *level = phase >= 0 ? pl->phases[phase].level : -1;
   if (x) *x = phase >= 0 ? pl->phases[phase].x : -1;
   if (entries) *entries = l->n;
@@ -1052,14 +1108,11 @@ int tuna_plan_phase_info(const tuna_plan_t *pl, int phase, int *level, int *x, i
   return TUNA_OK;
 }
 
-int tuna_plan_phase_tables(const tuna_plan_t *pl, int phase, int64_t cap, int64_t *len,
+int tuna_plan_phase_tables(const tuna_plan_t *pl, int phase, int part, int64_t cap, int64_t *len,
                            int64_t *pos, int64_t *src, int64_t *dst, int64_t *rows) {
   if (!pl) return TUNA_ERR_INVALID_ARG;
-  const TunaList *l;
-  if (phase == -1) l = &pl->rot;
-  else if (phase == -2) l = &pl->dir;
-  else if (phase >= 0 && phase < (int)pl->phases.size()) l = &pl->lists[phase];
-  else return TUNA_ERR_RANGE;
+  const TunaList *l = pick_list(pl, phase, part);
+  if (!l) return TUNA_ERR_RANGE;
   if (rows) *rows = l->n;
   const int64_t n = std::min(cap, l->n);
   if (n <= 0) return TUNA_OK;
@@ -1068,7 +1121,15 @@ int tuna_plan_phase_tables(const tuna_plan_t *pl, int phase, int64_t cap, int64_
   if (len) TUNA_CUDA(m, cudaMemcpy(len, l->len, n * 8, cudaMemcpyDeviceToHost));
   if (pos) TUNA_CUDA(m, cudaMemcpy(pos, l->pos, n * 8, cudaMemcpyDeviceToHost));
   if (src) TUNA_CUDA(m, cudaMemcpy(src, l->src, n * 8, cudaMemcpyDeviceToHost));
-  if (dst) TUNA_CUDA(m, cudaMemcpy(dst, l->dst, n * 8, cudaMemcpyDeviceToHost));
+  if (dst) {
+    if (l->kind == TUNA_LIST_DELIVER) {
+      TUNA_CUDA(m, cudaMemcpy(dst, l->dst, n * 8, cudaMemcpyDeviceToHost));
+    } else {  // a KEEP list's stream is its destination: workspace offset of the phase + position
+      std::vector<int64_t> p(n);
+      TUNA_CUDA(m, cudaMemcpy(p.data(), l->pos, n * 8, cudaMemcpyDeviceToHost));
+      for (int64_t i = 0; i < n; i++) dst[i] = TUNA_LOC(TUNA_BUF_WORK, pl->h_wbase[phase] + p[i]);
+    }
+  }
   return TUNA_OK;
 }
 

@@ -141,29 +141,46 @@ def test_metadata_and_prefix_sums(P, r):
     assert plan.num_phases() == sizes.shape[0]
     work_off = 0
     for x in range(plan.num_phases()):
-        t = plan.phase_tables(x)
         moving = [o for o in range(P) if (o // r ** x) % r != 0]
-        exp_len = sizes[x][:, moving]                        # receive-side order (rank, offset)
-        assert np.array_equal(t["len"].reshape(P, len(moving)), exp_len)
+        arrived = [o for o in moving if o < r ** (x + 1)]      # no non-zero digit above x
+        onward = [o for o in moving if o >= r ** (x + 1)]
+        assert moving == arrived + onward                      # the arrived ones come first
+        # blocks that travel on: this phase's region of the workspace
+        t = plan.phase_tables(x, B.PART_KEEP)
+        exp_len = sizes[x][:, onward]                          # receive-side order (rank, offset)
+        assert np.array_equal(t["len"].reshape(P, len(onward)), exp_len)
         scan, tot = oracle.segmented_exclusive_scan(exp_len, 16)
         base, _ = oracle.segmented_exclusive_scan(tot.reshape(1, P), 1)
         exp_pos = scan + base.reshape(P, 1)
-        assert np.array_equal(t["pos"].reshape(P, len(moving)), exp_pos)
-        info = plan.phase_info(x)
+        assert np.array_equal(t["pos"].reshape(P, len(onward)), exp_pos)
+        info = plan.phase_info(x, B.PART_KEEP)
         assert info["bytes"] == exp_len.sum() and info["stream_bytes"] == tot.sum()
-        # destinations: final blocks in the receive buffer, the rest at their stream position
-        dst = t["dst"].reshape(P, len(moving))
+        assert np.array_equal(t["dst"].reshape(P, len(onward)), (2 << 56) | (work_off + exp_pos))
+        work_off += (int(tot.sum()) + 255) // 256 * 256
+        # blocks that have arrived: straight into the receive buffer
+        t = plan.phase_tables(x, B.PART_DELIVER)
+        exp_len = sizes[x][:, arrived]
+        assert np.array_equal(t["len"].reshape(P, len(arrived)), exp_len)
+        spaced = (exp_len + 15) // 16 * 16 + 16 * (exp_len > 0)
+        scan, tot = oracle.segmented_exclusive_scan(spaced, 1)
+        base, _ = oracle.segmented_exclusive_scan(tot.reshape(1, P), 1)
+        assert np.array_equal(t["pos"].reshape(P, len(arrived)), scan + base.reshape(P, 1))
+        assert plan.phase_info(x, B.PART_DELIVER)["bytes"] == exp_len.sum()
+        dst = t["dst"].reshape(P, len(arrived))
         for p in range(P):
-            for j, o in enumerate(moving):
-                if o < r ** (x + 1):
-                    s = (p - o) % P
-                    want = (1 << 56) | int(wl.recvbase[p] + wl.rdispls[p, s]) * wl.elem_size
-                else:
-                    want = (2 << 56) | (work_off + int(exp_pos[p, j]))
-                assert dst[p, j] == want
-        if x + 1 < plan.num_phases():
-            work_off += (int(tot.sum()) + 255) // 256 * 256
+            for j, o in enumerate(arrived):
+                s = (p - o) % P
+                assert dst[p, j] == (1 << 56) | int(wl.recvbase[p] + wl.rdispls[p, s]) * wl.elem_size
     assert plan.workspace_bytes() == work_off
+    # classic mode keeps every block in the workspace and rotates at the end
+    classic = B.plan_for(wl, r, flags=B.FLAG_CLASSIC_ROTATE)
+    for x in range(classic.num_phases()):
+        moving = [o for o in range(P) if (o // r ** x) % r != 0]
+        t = classic.phase_tables(x, B.PART_KEEP)
+        assert np.array_equal(t["len"].reshape(P, len(moving)), sizes[x][:, moving])
+        assert classic.phase_info(x, B.PART_DELIVER)["entries"] == 0
+    rot = classic.phase_tables(-1)
+    assert np.array_equal(rot["len"].reshape(P, P), sizes[-1])   # every block, in slot order
 
 
 def test_packed_layout_defaults_match_explicit():
