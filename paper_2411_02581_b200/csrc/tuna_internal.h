@@ -19,6 +19,7 @@
 
 #define TUNA_ALIGN 16  // every block in the workspace starts on this boundary
 #define TUNA_MOVE_THREADS 256
+#define TUNA_MAX_CHUNK_BYTES (256 * 1024)  // stream bytes one CTA handles, at most
 
 // Ranks and slots: rank p = n*Q + q; slot sigma = io*Q + jo names the block whose
 // destination is (n + io mod N, q + jo mod Q).  Flat TuNA is N = 1.

@@ -485,8 +485,7 @@ int64_t env_i64(const char *name, int64_t dflt) {
 // than 128 KiB (tail effect).
 int64_t pick_chunk(int64_t total, int kind) {
   const int64_t forced = env_i64(kind == TUNA_LIST_KEEP ? "TUNA_CHUNK_BYTES_KEEP" : "TUNA_CHUNK_BYTES_DELIVER", 0);
-  const int64_t cap = kind == TUNA_LIST_KEEP ? 65536 : ((int64_t)1 << 24);
-  if (forced >= 1024) return std::min<int64_t>((forced + 15) & ~(int64_t)15, cap);
+  if (forced >= 1024) return std::min<int64_t>((forced + 15) & ~(int64_t)15, TUNA_MAX_CHUNK_BYTES);
   int64_t c = 8192;
   while (c < 65536 && total / c > 148 * 32) c <<= 1;
   return c;
