@@ -76,7 +76,7 @@ def lib() -> ctypes.CDLL:
     """Load the CUDA library (built in-tree); raise if it does not exist."""
     global _lib
     if _lib is None:
-        path = _build.LIB_PATH
+        path = os.environ.get("TUNA_LIBRARY") or _build.LIB_PATH  # override: another build of the library
         if not os.path.exists(path):
             raise RuntimeError(
                 f"{path} is missing: build it with `python -m paper_2411_02581_b200.build` "

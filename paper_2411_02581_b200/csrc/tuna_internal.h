@@ -63,6 +63,7 @@ struct TunaList {
   int64_t bytes = 0;      // bytes moved (host copy)
   int64_t chunk = 0;      // bytes of stream per CTA
   int64_t nchunks = 0;
+  bool small_blocks = false;  // mean block far below a chunk (host copy, from bytes / n)
 };
 
 struct TunaMoveArgs {
@@ -81,7 +82,8 @@ enum TunaMoveKernel {
   TUNA_K_DIRECT = 3    // single-pass direct exchange
 };
 
-// Launches one mover kernel over one list (tuna_move.cu).
-cudaError_t tuna_launch_move(int kernel, const TunaMoveArgs &a, cudaStream_t stream);
+// Launches one mover kernel over one list (tuna_move.cu).  `small_blocks` picks
+// the build tuned for lists whose blocks are far smaller than a chunk.
+cudaError_t tuna_launch_move(int kernel, const TunaMoveArgs &a, bool small_blocks, cudaStream_t stream);
 
 #endif

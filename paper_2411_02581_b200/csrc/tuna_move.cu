@@ -272,14 +272,20 @@ __device__ __forceinline__ void move_body(const TunaMoveArgs &a) {
   }
 }
 
+// Two builds of every DELIVER kernel: lists of large blocks run best with four
+// CTAs per SM and all the registers the copy loop wants; lists of tiny blocks are
+// bound by latency and gain from a fifth resident CTA.
 __global__ void __launch_bounds__(kThreads) tuna_round_kernel(const TunaMoveArgs a) { move_body<false>(a); }
 __global__ void __launch_bounds__(kThreads) tuna_deliver_kernel(const TunaMoveArgs a) { move_body<true>(a); }
 __global__ void __launch_bounds__(kThreads) tuna_rotate_kernel(const TunaMoveArgs a) { move_body<true>(a); }
 __global__ void __launch_bounds__(kThreads) tuna_direct_kernel(const TunaMoveArgs a) { move_body<true>(a); }
+__global__ void __launch_bounds__(kThreads, 5) tuna_deliver_small_kernel(const TunaMoveArgs a) { move_body<true>(a); }
+__global__ void __launch_bounds__(kThreads, 5) tuna_rotate_small_kernel(const TunaMoveArgs a) { move_body<true>(a); }
+__global__ void __launch_bounds__(kThreads, 5) tuna_direct_small_kernel(const TunaMoveArgs a) { move_body<true>(a); }
 
 }  // namespace
 
-cudaError_t tuna_launch_move(int kernel, const TunaMoveArgs &a, cudaStream_t stream) {
+cudaError_t tuna_launch_move(int kernel, const TunaMoveArgs &a, bool small_blocks, cudaStream_t stream) {
   if (a.nchunks <= 0 || a.n <= 0) return cudaSuccess;
   if (a.chunk > TUNA_MAX_CHUNK_BYTES || (a.chunk & 15)) return cudaErrorInvalidValue;
   const dim3 grid((unsigned)a.nchunks), block(kThreads);
@@ -288,13 +294,22 @@ cudaError_t tuna_launch_move(int kernel, const TunaMoveArgs &a, cudaStream_t str
       tuna_round_kernel<<<grid, block, 0, stream>>>(a);
       break;
     case TUNA_K_DELIVER:
-      tuna_deliver_kernel<<<grid, block, 0, stream>>>(a);
+      if (small_blocks)
+        tuna_deliver_small_kernel<<<grid, block, 0, stream>>>(a);
+      else
+        tuna_deliver_kernel<<<grid, block, 0, stream>>>(a);
       break;
     case TUNA_K_ROTATE:
-      tuna_rotate_kernel<<<grid, block, 0, stream>>>(a);
+      if (small_blocks)
+        tuna_rotate_small_kernel<<<grid, block, 0, stream>>>(a);
+      else
+        tuna_rotate_kernel<<<grid, block, 0, stream>>>(a);
       break;
     default:
-      tuna_direct_kernel<<<grid, block, 0, stream>>>(a);
+      if (small_blocks)
+        tuna_direct_small_kernel<<<grid, block, 0, stream>>>(a);
+      else
+        tuna_direct_kernel<<<grid, block, 0, stream>>>(a);
       break;
   }
   return cudaGetLastError();

@@ -483,16 +483,24 @@ int64_t env_i64(const char *name, int64_t dflt) {
 // Bytes of destination stream per CTA: enough chunks to fill the machine several
 // times over, but no smaller than a few KiB (descriptor overhead) and no larger
 // than 128 KiB (tail effect).
-int64_t pick_chunk(int64_t total, int kind) {
-  const int64_t forced = env_i64(kind == TUNA_LIST_KEEP ? "TUNA_CHUNK_BYTES_KEEP" : "TUNA_CHUNK_BYTES_DELIVER", 0);
+constexpr int64_t kSmallBlockBytes = 2048;  // mean block size below which a list counts as "small blocks"
+
+// Bytes of stream per CTA.  Large blocks: 64 KiB, the best measured size for
+// multi-MiB blocks (smaller chunks pay the per-chunk set-up more often, larger
+// ones leave a longer tail).  Small blocks: 32 KiB, so that one batch of 256
+// descriptors covers a chunk.  Small lists: fewer bytes per CTA, to fill the SMs.
+int64_t pick_chunk(const TunaList &l) {
+  const int64_t forced = env_i64(l.kind == TUNA_LIST_KEEP ? "TUNA_CHUNK_BYTES_KEEP" : "TUNA_CHUNK_BYTES_DELIVER", 0);
   if (forced >= 1024) return std::min<int64_t>((forced + 15) & ~(int64_t)15, TUNA_MAX_CHUNK_BYTES);
+  const int64_t top = l.small_blocks ? 32768 : 65536;
   int64_t c = 8192;
-  while (c < 65536 && total / c > 148 * 32) c <<= 1;
+  while (c < top && l.total / c > 148 * 32) c <<= 1;
   return c;
 }
 
 int build_chunks(tuna_plan *pl, TunaList &l, cudaStream_t st) {
-  l.chunk = pick_chunk(l.total, l.kind);
+  l.small_blocks = l.n > 0 && l.bytes / l.n < kSmallBlockBytes;
+  l.chunk = pick_chunk(l);
   l.nchunks = l.total > 0 ? (l.total + l.chunk - 1) / l.chunk : 0;
   if (l.nchunks > l.chunk_cap) {
     cudaFree(l.chunk_first);
@@ -812,19 +820,19 @@ int run_tuna(tuna_plan *pl, const void *send, void *recv, cudaStream_t st) {
       Timed tm(pl, kind, k.bytes, st);
       TunaMoveArgs a = move_args(pl, k, send, recv, pl->workspace);
       a.keep_base = pl->h_wbase[f];
-      TUNA_CUDA(pl, tuna_launch_move(TUNA_K_ROUND, a, st));
+      TUNA_CUDA(pl, tuna_launch_move(TUNA_K_ROUND, a, k.small_blocks, st));
       launches++;
     }
     const TunaList &d = pl->deliver[f];
     if (d.nchunks > 0) {
       Timed tm(pl, kind, d.bytes, st);
-      TUNA_CUDA(pl, tuna_launch_move(TUNA_K_DELIVER, move_args(pl, d, send, recv, pl->workspace), st));
+      TUNA_CUDA(pl, tuna_launch_move(TUNA_K_DELIVER, move_args(pl, d, send, recv, pl->workspace), d.small_blocks, st));
       launches++;
     }
   }
   if (pl->rot.nchunks > 0) {
     Timed tm(pl, TUNA_TIMER_ROTATE, pl->rot.bytes, st);
-    TUNA_CUDA(pl, tuna_launch_move(TUNA_K_ROTATE, move_args(pl, pl->rot, send, recv, pl->workspace), st));
+    TUNA_CUDA(pl, tuna_launch_move(TUNA_K_ROTATE, move_args(pl, pl->rot, send, recv, pl->workspace), pl->rot.small_blocks, st));
     launches++;
   }
   pl->last_launches = launches;
@@ -836,7 +844,7 @@ int run_direct(tuna_plan *pl, const void *send, void *recv, cudaStream_t st) {
   int launches = 0;
   if (pl->dir.nchunks > 0) {
     Timed tm(pl, TUNA_TIMER_DIRECT, pl->dir.bytes, st);
-    TUNA_CUDA(pl, tuna_launch_move(TUNA_K_DIRECT, move_args(pl, pl->dir, send, recv, nullptr), st));
+    TUNA_CUDA(pl, tuna_launch_move(TUNA_K_DIRECT, move_args(pl, pl->dir, send, recv, nullptr), pl->dir.small_blocks, st));
     launches++;
   }
   pl->last_launches = launches;
