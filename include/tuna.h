@@ -153,6 +153,44 @@ int tuna_direct_alltoallv(tuna_plan_t *plan, const void *sendbuf, const int64_t 
                           const int64_t *rdispls, void *stream);
 
 /*
+ * tuna_direct_alltoallv_static - the direct exchange for callers that must not
+ * allocate device memory.  (The paper has no counterpart: this entry point exists
+ * for the library's users, not for the algorithm.)
+ *
+ * Who needs it: a process whose framework has already claimed the whole GPU for
+ * its own memory pool, so that a cudaMalloc from a library fails or fragments the
+ * pool; a serving or real-time loop in which cudaMalloc/cudaFree are banned after
+ * start-up because they synchronise the device and stall every stream; code that
+ * runs under a fixed memory budget and is audited for allocations.  Such callers
+ * cannot create a plan (a plan owns descriptor tables obtained with cudaMalloc).
+ *
+ * This call takes the layout and the buffers in one go and keeps every table it
+ * needs (counts, displacements, descriptors, prefix sums, chunk table: about
+ * 1.1 MiB) in a fixed array that is part of the library image on every GPU that
+ * loads it.  It calls no cudaMalloc, cudaFree or other allocating routine.
+ *
+ *   P            1 <= P <= TUNA_STATIC_MAX_P, else TUNA_ERR_RANGE.
+ *   elem_size, sendcounts, sdispls, rdispls, sendbase, recvbase
+ *                host arrays as for tuna_plan_create (NULL = packed).
+ *   sendbuf, recvbuf   device; must not overlap.
+ *   limit        the work stream (every non-empty block rounded up to 16 bytes plus
+ *                16) may not exceed TUNA_STATIC_MAX_CHUNKS * 256 KiB = 4 GiB, else
+ *                TUNA_ERR_RANGE; nothing is launched in that case.
+ * The first call on a device looks up the array's device address; make that call
+ * before starting a stream capture on that device.  All calls share the one array
+ * and it keeps the previous call's tables; every table a call reads it first
+ * rewrites, so nothing needs clearing, but two calls whose kernels can overlap on
+ * the GPU (different streams, no ordering between them) race on it: order them.
+ * Asynchronous on `stream`.  Results are byte-identical to tuna_direct_alltoallv.
+ */
+#define TUNA_STATIC_MAX_P 128
+#define TUNA_STATIC_MAX_CHUNKS 16384
+int tuna_direct_alltoallv_static(int P, int elem_size, const int64_t *sendcounts,
+                                 const int64_t *sdispls, const int64_t *rdispls,
+                                 const int64_t *sendbase, const int64_t *recvbase,
+                                 const void *sendbuf, void *recvbuf, void *stream);
+
+/*
  * tuna_alltoallv_host - the same exchange on HOST buffers: copies
  * [0, send_bytes) of host_send to the device, runs the chosen schedule
  * (TUNA_SCHEDULE_*), copies [0, recv_bytes) back into host_recv, all on `stream`,

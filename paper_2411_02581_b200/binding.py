@@ -47,6 +47,7 @@ SIGNATURES = {
     "tuna_alltoallv": (ctypes.c_int, [_VP, _VP, _I64P, _I64P, _VP, _I64P, _I64P, _VP]),
     "tuna_direct_alltoallv": (ctypes.c_int, [_VP, _VP, _I64P, _I64P, _VP, _I64P, _I64P, _VP]),
     "tuna_alltoallv_host": (ctypes.c_int, [_VP, _VP, _VP, ctypes.c_int, _VP]),
+    "tuna_direct_alltoallv_static": (ctypes.c_int, [ctypes.c_int, ctypes.c_int] + [_I64P] * 5 + [_VP, _VP, _VP]),
     "tuna_plan_num_rounds": (ctypes.c_int, [_VP, _INTP]),
     "tuna_plan_round_info": (ctypes.c_int, [_VP, ctypes.c_int, _INTP, _INTP, _INTP, _I64P, _I64P]),
     "tuna_plan_num_phases": (ctypes.c_int, [_VP, _INTP]),
@@ -266,6 +267,22 @@ class Plan:
         by = (ctypes.c_int64 * TIMER_KINDS)()
         self._check(lib().tuna_plan_get_timing(self._h, int(bool(reset)), ms, ln, by), "tuna_plan_get_timing")
         return {name: dict(ms=ms[i], launches=ln[i], bytes=by[i]) for i, name in enumerate(TIMER_NAMES)}
+
+
+STATIC_MAX_P = 128
+
+
+def direct_alltoallv_static(P, elem_size, sendcounts, sendbuf, recvbuf, sdispls=None, rdispls=None,
+                            sendbase=None, recvbase=None, stream=None):
+    """The direct exchange without a plan and without any device allocation: for
+    callers whose process may not call cudaMalloc (a framework owns all device
+    memory, or allocation is banned inside a latency-critical loop).  Limits: P up
+    to STATIC_MAX_P and about 4 GiB of payload; calls must not overlap on the GPU."""
+    keep = [_h(x) for x in (sendcounts, sdispls, rdispls, sendbase, recvbase)]
+    rc = lib().tuna_direct_alltoallv_static(P, elem_size, *[k[1] for k in keep], _ptr(sendbuf),
+                                            _ptr(recvbuf), _stream(stream))
+    if rc != 0:
+        raise TunaError(rc, "tuna_direct_alltoallv_static")
 
 
 def plan_for(wl, radix, l=None, g=1, radix_global=2, flags=0, explicit_layout=True, stream=None) -> Plan:
