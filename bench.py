@@ -30,12 +30,12 @@ if ROOT not in sys.path:
 METRIC = "alltoallv_payload_throughput"
 UNIT = "GB/s"
 
-# DRAM traffic of the dominant kernel from an ncu capture
+# DRAM traffic of the dominant kernels from ncu captures
 # (dram__bytes_read.sum + dram__bytes_write.sum per launch) divided by the payload
 # bytes that launch moved, keyed by the SHA-256 of the kernel source the capture
-# was taken with.  A changed source makes the figure stale: it is then reported
-# as null.
-NCU_TRAFFIC_PER_PAYLOAD_BYTE: dict[str, float] = {}
+# was taken with, then by kernel.  A changed source makes the figures stale: the
+# traffic is then reported as null.
+NCU_TRAFFIC_PER_PAYLOAD_BYTE: dict[str, dict[str, float]] = {}
 
 
 def parse_args():
@@ -334,23 +334,28 @@ def ours_arm(args):
     ms_per_step = elapsed_ms / args.steps
     value = world * payload / (ms_per_step * 1e-3) / 1e9
 
-    # roofline of the dominant kernel: the fused round kernel
+    # roofline of the dominant kernel: whichever of the fused pack-move-unpack
+    # kernels (blocks travelling on / blocks arriving) took the most time
     peak, peak_kind = measured_peaks()
-    rk = timing["round_local"]
-    rk_ms = rk["ms"] + timing["round_global"]["ms"]
-    rk_launches = rk["launches"] + timing["round_global"]["launches"]
-    rk_bytes = rk["bytes"] + timing["round_global"]["bytes"]
+    keep_ms = timing["round_local"]["ms"] + timing["round_global"]["ms"]
+    if keep_ms >= timing["deliver"]["ms"]:
+        kname = "tuna_round_kernel"
+        rk_ms = keep_ms
+        rk_launches = timing["round_local"]["launches"] + timing["round_global"]["launches"]
+        rk_bytes = timing["round_local"]["bytes"] + timing["round_global"]["bytes"]
+    else:
+        kname = "tuna_deliver_kernel"
+        rk_ms, rk_launches, rk_bytes = (timing["deliver"][k] for k in ("ms", "launches", "bytes"))
     achieved = 2.0 * rk_bytes / (rk_ms * 1e-3) / 1e9 if rk_ms > 0 else 0.0
-    per_byte = NCU_TRAFFIC_PER_PAYLOAD_BYTE.get(kernel_source_sha())
+    per_byte = NCU_TRAFFIC_PER_PAYLOAD_BYTE.get(kernel_source_sha(), {}).get(kname)
     roofline = {
-        "bound": "hbm", "kernel": "tuna_round_kernel", "achieved": achieved, "peak": peak,
+        "bound": "hbm", "kernel": kname, "achieved": achieved, "peak": peak,
         "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,
         "traffic": (per_byte * rk_bytes / rk_launches) if per_byte and rk_launches else None,
         "algorithmic_bytes_per_launch": 2.0 * rk_bytes / rk_launches if rk_launches else 0,
         "avg_launch_ms": rk_ms / rk_launches if rk_launches else None,
         "launches": rk_launches,
-        "plan_ms_per_step": timing["plan"]["ms"] / args.steps,
-        "rotate_ms_per_step": timing["rotate"]["ms"] / args.steps,
+        "ms_per_step": {k: v["ms"] / args.steps for k, v in timing.items()},
     }
 
     # end to end through the host-buffer entry point (pinned host memory)

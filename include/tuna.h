@@ -248,10 +248,12 @@ int tuna_plan_launch_count(const tuna_plan_t *plan, int64_t *launches);
  * metadata, data, replace, rearrange and inter-node cost).  With timing enabled
  * every launch is bracketed by CUDA events on the caller's stream:
  *   TUNA_TIMER_PLAN          metadata exchange + prefix sums (prepare + metadata)
- *   TUNA_TIMER_ROUND_LOCAL   flat / local digit phases (data; "replace" is fused away)
- *   TUNA_TIMER_ROUND_GLOBAL  global digit phases (inter-group cost)
+ *   TUNA_TIMER_ROUND_LOCAL   flat / local digit phases, blocks that travel on (data;
+ *                            "replace" is fused away)
+ *   TUNA_TIMER_ROUND_GLOBAL  global digit phases, blocks that travel on (inter-group cost)
  *   TUNA_TIMER_ROTATE        final rotation (rearrange)
  *   TUNA_TIMER_DIRECT        the single-pass direct exchange
+ *   TUNA_TIMER_DELIVER       blocks that arrive in a digit phase of either level (data)
  * tuna_plan_get_timing waits for the recorded events and returns, per kind
  * (arrays of TUNA_TIMER_KINDS, any may be NULL), accumulated milliseconds,
  * launches and payload bytes moved; `reset` non-zero clears the accumulators.
@@ -261,7 +263,8 @@ int tuna_plan_launch_count(const tuna_plan_t *plan, int64_t *launches);
 #define TUNA_TIMER_ROUND_GLOBAL 2
 #define TUNA_TIMER_ROTATE 3
 #define TUNA_TIMER_DIRECT 4
-#define TUNA_TIMER_KINDS 5
+#define TUNA_TIMER_DELIVER 5
+#define TUNA_TIMER_KINDS 6
 int tuna_plan_enable_timing(tuna_plan_t *plan, int on);
 int tuna_plan_get_timing(tuna_plan_t *plan, int reset, double *ms, int64_t *launches,
                          int64_t *bytes);

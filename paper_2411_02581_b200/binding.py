@@ -25,7 +25,7 @@ PART_DELIVER = 1
 SCHEDULE_TUNA = 0
 SCHEDULE_DIRECT = 1
 
-TIMER_NAMES = ("plan", "round_local", "round_global", "rotate", "direct")
+TIMER_NAMES = ("plan", "round_local", "round_global", "rotate", "direct", "deliver")
 TIMER_KINDS = len(TIMER_NAMES)
 
 STATUS = {

@@ -368,9 +368,9 @@ struct tuna_plan {
   };
   std::vector<Stamp> stamps;
   std::vector<cudaEvent_t> event_pool;
-  double t_ms[TUNA_TIMER_KINDS] = {0, 0, 0, 0, 0};
-  int64_t t_launches[TUNA_TIMER_KINDS] = {0, 0, 0, 0, 0};
-  int64_t t_bytes[TUNA_TIMER_KINDS] = {0, 0, 0, 0, 0};
+  double t_ms[TUNA_TIMER_KINDS] = {};
+  int64_t t_launches[TUNA_TIMER_KINDS] = {};
+  int64_t t_bytes[TUNA_TIMER_KINDS] = {};
 };
 
 namespace {
@@ -826,7 +826,7 @@ int run_tuna(tuna_plan *pl, const void *send, void *recv, cudaStream_t st) {
     }
     const TunaList &d = pl->deliver[f];
     if (d.nchunks > 0) {
-      Timed tm(pl, kind, d.bytes, st);
+      Timed tm(pl, TUNA_TIMER_DELIVER, d.bytes, st);
       TUNA_CUDA(pl, tuna_launch_move(TUNA_K_DELIVER, move_args(pl, d, send, recv, pl->workspace), d.small_blocks, st));
       launches++;
     }
