@@ -142,6 +142,21 @@ class ClockSampler:
                 "reasons": sorted(self.reasons), "samples": len(self.samples)}
 
 
+def max_over_ranks(ms, dist=None, device="cpu"):
+    """Slowest rank's time: the job is over when the last replica is."""
+    if dist is None or not dist.is_initialized() or dist.get_world_size() == 1:
+        return float(ms)
+    import torch
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_throughput(payload_bytes_per_rank, world, ms_per_step):
+    """Whole-job GB/s: what all replicas moved in a step over the slowest replica's time."""
+    return world * payload_bytes_per_rank / (ms_per_step * 1e-3) / 1e9
+
+
 def kernel_source_sha():
     h = hashlib.sha256()
     with open(os.path.join(ROOT, "paper_2411_02581_b200", "csrc", "tuna_move.cu"), "rb") as f:
@@ -327,12 +342,9 @@ def ours_arm(args):
     launches = plan.launch_count() - launches0
     timing = plan.get_timing(reset=True)
     plan.enable_timing(False)
-    if dist:
-        t = torch.tensor([elapsed_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(t.item())
+    elapsed_ms = max_over_ranks(elapsed_ms, dist, dev)
     ms_per_step = elapsed_ms / args.steps
-    value = world * payload / (ms_per_step * 1e-3) / 1e9
+    value = job_throughput(payload, world, ms_per_step)
 
     # roofline of the dominant kernel: whichever of the fused pack-move-unpack
     # kernels (blocks travelling on / blocks arriving) took the most time
@@ -378,11 +390,8 @@ def ours_arm(args):
         for _ in range(e_steps):
             estep()
         e_ms = (time.perf_counter() - t0) * 1e3 / e_steps
-        if dist:
-            t = torch.tensor([e_ms], dtype=torch.float64, device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e_ms = float(t.item())
-        e2e = {"value": world * payload / (e_ms * 1e-3) / 1e9, "unit": UNIT,
+        e_ms = max_over_ranks(e_ms, dist, dev)
+        e2e = {"value": job_throughput(payload, world, e_ms), "unit": UNIT,
                "h2d_bytes_per_step": wl.send_bytes + 8 * (3 * wl.P * wl.P + 2 * wl.P),
                "d2h_bytes_per_step": wl.recv_bytes, "ms_per_step": e_ms, "steps": e_steps}
         del hs, hr

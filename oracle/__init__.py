@@ -17,6 +17,12 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "tuna_oracle.c")
 _OUT_DIR = os.path.join(_HERE, "_build")
 _LIB = os.path.join(_OUT_DIR, "libtuna_oracle.so")
+# The mutation tests point this at a deliberately broken copy of the source to
+# check that the pins notice; nothing else sets it.
+if os.environ.get("TUNA_ORACLE_SOURCE"):
+    _SRC = os.environ["TUNA_ORACLE_SOURCE"]
+    _OUT_DIR = os.path.dirname(_SRC)
+    _LIB = os.path.splitext(_SRC)[0] + ".so"
 _lock = threading.Lock()
 _lib = None
 

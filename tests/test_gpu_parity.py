@@ -343,3 +343,61 @@ def test_c5_full_hier_and_direct():
     check_rounds(plan, rounds)
     got, _ = gpu_run(wl, 2, direct=True, pass_args=False)
     assert np.array_equal(got, ref)
+
+
+def _block_sums(buf_words, base, displs, counts, elem_words):
+    """Wrapping 64-bit sum of every block's words, via one cumulative sum."""
+    cs = torch.cumsum(buf_words, 0)
+    cs = torch.cat([torch.zeros(1, dtype=torch.int64, device=buf_words.device), cs])
+    start = torch.from_numpy(((base[:, None] + displs) * elem_words).astype(np.int64)).to(buf_words.device)
+    end = start + torch.from_numpy((counts * elem_words).astype(np.int64)).to(buf_words.device)
+    return cs[end] - cs[start]
+
+
+@pytest.mark.parametrize("schedule", ["r64", "r2", "r8_classic", "direct"])
+def test_c4_full_size(schedule):
+    """The 8 GiB token-dispatch shape in the configuration the benchmark times.
+    The oracle cannot run it in seconds, so the check is (a) sampled received bytes
+    against the definition of the exchange applied to the generator, and (b) a
+    property that holds at any size: every one of the P^2 received blocks has the
+    same 64-bit word sum as the block that was sent."""
+    free, _ = torch.cuda.mem_get_info()
+    if free < 70 * 2**30:
+        pytest.skip("needs about 70 GiB of free device memory")
+    wl = W.make_c4()
+    assert wl.payload_bytes_total == 8 * 2**30
+    send = wl.make_send("cuda")
+    recv = wl.make_recv("cuda", fill=CANARY)
+    kw = dict(r64=dict(radix=64), r2=dict(radix=2), r8_classic=dict(radix=8, flags=B.FLAG_CLASSIC_ROTATE),
+              direct=dict(radix=64))[schedule]
+    plan = B.plan_for(wl, **kw)
+    plan.alloc_workspace()
+    if schedule == "direct":
+        plan.direct_alltoallv(send, recv)
+    else:
+        plan.alltoallv(send, recv)
+    torch.cuda.synchronize()
+    # (a) samples
+    rng = np.random.default_rng(2024)
+    n = 1 << 20
+    s = rng.integers(0, wl.P, n)
+    d = rng.integers(0, wl.P, n)
+    k = (rng.random(n) * (wl.sendcounts[s, d] * wl.elem_size)).astype(np.int64)
+    src = torch.from_numpy((wl.sendbase[s] + wl.sdispls[s, d]) * wl.elem_size + k).cuda()
+    dst = torch.from_numpy((wl.recvbase[d] + wl.rdispls[d, s]) * wl.elem_size + k).cuda()
+    assert torch.equal(recv[dst], W.payload_byte_at(wl.seed, src))
+    # (b) all blocks, by checksum
+    ew = wl.elem_size // 8
+    sent = _block_sums(send.view(torch.int64), wl.sendbase, wl.sdispls, wl.sendcounts, ew)
+    got = _block_sums(recv.view(torch.int64), wl.recvbase, wl.rdispls, wl.recvcounts, ew)
+    assert torch.equal(got, sent.T)
+    # the schedule's byte counts: every block is moved once per non-zero digit of its offset
+    if schedule != "direct":
+        r = kw["radix"]
+        offs = (np.arange(wl.P)[None, :] - np.arange(wl.P)[:, None]) % wl.P
+        nz = np.zeros_like(offs)
+        t = offs.copy()
+        while t.any():
+            nz += (t % r) != 0
+            t //= r
+        assert sum(x["bytes"] for x in plan.rounds()) == int((wl.sendcounts * nz).sum()) * wl.elem_size
