@@ -191,14 +191,22 @@ int tuna_direct_alltoallv_static(int P, int elem_size, const int64_t *sendcounts
                                  const void *sendbuf, void *recvbuf, void *stream);
 
 /*
- * tuna_alltoallv_host - the same exchange on HOST buffers: copies
- * [0, send_bytes) of host_send to the device, runs the chosen schedule
- * (TUNA_SCHEDULE_*), copies [0, recv_bytes) back into host_recv, all on `stream`,
- * and returns without synchronising (pinned host memory makes the copies
- * asynchronous).  The workspace must hold workspace_bytes + host_staging_bytes.
- * Receive-buffer bytes that no block covers are overwritten with unspecified
- * values by the copy back.
+ * tuna_alltoallv_host - the same exchange on HOST buffers, all on `stream`,
+ * returning without synchronising.  `schedule` is TUNA_SCHEDULE_TUNA or
+ * TUNA_SCHEDULE_DIRECT, optionally OR-ed with TUNA_HOST_STAGED.
+ *   - Both buffers pinned and mapped into the device's address space (cudaHostAlloc
+ *     or cudaHostRegister memory under unified addressing): the kernels read
+ *     host_send and write host_recv in place over the host link, both directions
+ *     at once; blocks hop through the device workspace in between.  Needs only
+ *     workspace_bytes of workspace; receive-buffer bytes that no block covers are
+ *     left untouched.
+ *   - Otherwise, or with TUNA_HOST_STAGED: [0, send_bytes) of host_send is copied
+ *     to the device, the schedule runs there, and [0, recv_bytes) is copied back
+ *     into host_recv.  The workspace must then hold workspace_bytes +
+ *     host_staging_bytes, and receive-buffer bytes that no block covers are
+ *     overwritten with unspecified values by the copy back.
  */
+#define TUNA_HOST_STAGED 0x100
 int tuna_alltoallv_host(tuna_plan_t *plan, const void *host_send, void *host_recv, int schedule,
                         void *stream);
 

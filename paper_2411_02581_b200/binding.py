@@ -24,6 +24,7 @@ PART_KEEP = 0
 PART_DELIVER = 1
 SCHEDULE_TUNA = 0
 SCHEDULE_DIRECT = 1
+HOST_STAGED = 0x100
 
 TIMER_NAMES = ("plan", "round_local", "round_global", "rotate", "direct", "deliver")
 TIMER_KINDS = len(TIMER_NAMES)

@@ -564,43 +564,87 @@ int validate_layout(int P, const int64_t *counts, const int64_t *sdispls, const 
   return TUNA_OK;
 }
 
+// What the host works out from a layout before anything touches the GPU.
+struct HostLayout {
+  std::vector<int64_t> sendbase, recvbase;  // elements
+  int64_t payload = 0, send_extent = 0, recv_extent = 0;  // elements
+};
+
+// One pass over the P x P matrices: rejects negative entries, sums the payload and
+// finds every rank's region size.  rdispls is indexed [dst][src] while the counts
+// are [src][dst], so the pass walks 64 x 64 tiles to keep both in cache.
+int host_layout(int P, const int64_t *counts, const int64_t *sdispls, const int64_t *rdispls,
+                const int64_t *sendbase, const int64_t *recvbase, HostLayout *out) {
+  if (!counts) return TUNA_ERR_INVALID_ARG;
+  std::vector<int64_t> sreg(P, 0), rreg(P, 0);
+  int64_t payload = 0;
+  bool bad = false;
+  constexpr int T = 64;
+  for (int s0 = 0; s0 < P; s0 += T)
+    for (int d0 = 0; d0 < P; d0 += T) {
+      const int s1 = std::min(P, s0 + T), d1 = std::min(P, d0 + T);
+      for (int s = s0; s < s1; s++) {
+        const int64_t *crow = counts + (int64_t)s * P;
+        int64_t sr = sreg[s];
+        for (int d = d0; d < d1; d++) {
+          const int64_t c = crow[d];
+          bad |= c < 0;
+          payload += c;
+          if (sdispls) {
+            const int64_t x = sdispls[(int64_t)s * P + d];
+            bad |= x < 0;
+            sr = std::max(sr, x + c);
+          } else {
+            sr += c;
+          }
+          if (rdispls) {
+            const int64_t x = rdispls[(int64_t)d * P + s];
+            bad |= x < 0;
+            rreg[d] = std::max(rreg[d], x + c);
+          } else {
+            rreg[d] += c;
+          }
+        }
+        sreg[s] = sr;
+      }
+    }
+  for (int p = 0; p < P; p++) bad |= (sendbase && sendbase[p] < 0) || (recvbase && recvbase[p] < 0);
+  if (bad) return TUNA_ERR_INVALID_ARG;
+  out->sendbase.resize(P);
+  out->recvbase.resize(P);
+  int64_t se = 0, re = 0, acc_s = 0, acc_r = 0;
+  for (int p = 0; p < P; p++) {
+    out->sendbase[p] = sendbase ? sendbase[p] : acc_s;
+    out->recvbase[p] = recvbase ? recvbase[p] : acc_r;
+    acc_s += sreg[p];
+    acc_r += rreg[p];
+    se = std::max(se, out->sendbase[p] + sreg[p]);
+    re = std::max(re, out->recvbase[p] + rreg[p]);
+  }
+  out->payload = payload;
+  out->send_extent = se;
+  out->recv_extent = re;
+  return TUNA_OK;
+}
+
 // Uploads the layout, runs every plan kernel, reads the totals back.
-int build_tables(tuna_plan *pl, const int64_t *counts, const int64_t *sdispls,
-                 const int64_t *rdispls, const int64_t *sendbase, const int64_t *recvbase,
-                 cudaStream_t st) {
+int build_tables(tuna_plan *pl, const HostLayout &hl, const int64_t *counts, const int64_t *sdispls,
+                 const int64_t *rdispls, cudaStream_t st) {
   const TunaTopo &t = pl->topo;
   const int P = t.P;
   const int64_t PP = (int64_t)P * P;
-  int rc = validate_layout(P, counts, sdispls, rdispls, sendbase, recvbase);
-  if (rc) return rc;
+  int rc = TUNA_OK;
 
-  // host bookkeeping: copies for later validation, region sizes, extents
+  // host copies for the checks at call time
   pl->h_counts.assign(counts, counts + PP);
   pl->have_sdispls = sdispls != nullptr;
   pl->have_rdispls = rdispls != nullptr;
   if (sdispls) pl->h_sdispls.assign(sdispls, sdispls + PP); else pl->h_sdispls.clear();
   if (rdispls) pl->h_rdispls.assign(rdispls, rdispls + PP); else pl->h_rdispls.clear();
-  std::vector<int64_t> sreg(P, 0), rreg(P, 0), sb(P), rb(P);
-  int64_t payload = 0;
-  for (int s = 0; s < P; s++)
-    for (int d = 0; d < P; d++) {
-      const int64_t c = counts[(int64_t)s * P + d];
-      payload += c;
-      if (sdispls) sreg[s] = std::max(sreg[s], sdispls[(int64_t)s * P + d] + c); else sreg[s] += c;
-      if (rdispls) rreg[d] = std::max(rreg[d], rdispls[(int64_t)d * P + s] + c); else rreg[d] += c;
-    }
-  int64_t se = 0, re = 0, acc_s = 0, acc_r = 0;
-  for (int p = 0; p < P; p++) {
-    sb[p] = sendbase ? sendbase[p] : acc_s;
-    rb[p] = recvbase ? recvbase[p] : acc_r;
-    acc_s += sreg[p];
-    acc_r += rreg[p];
-    se = std::max(se, sb[p] + sreg[p]);
-    re = std::max(re, rb[p] + rreg[p]);
-  }
-  pl->payload = payload * t.elem;
-  pl->send_extent = se * t.elem;
-  pl->recv_extent = re * t.elem;
+  const std::vector<int64_t> &sb = hl.sendbase, &rb = hl.recvbase;
+  pl->payload = hl.payload * t.elem;
+  pl->send_extent = hl.send_extent * t.elem;
+  pl->recv_extent = hl.recv_extent * t.elem;
 
   Timed plan_timer(pl, TUNA_TIMER_PLAN, 0, st);
   TUNA_CUDA(pl, cudaMemcpyAsync(pl->d_counts, counts, PP * 8, cudaMemcpyHostToDevice, st));
@@ -920,7 +964,8 @@ int tuna_plan_create(tuna_plan_t **out, int P, int radix, int radix_global, int 
   if ((int64_t)l * g != P) return TUNA_ERR_BAD_HIERARCHY;
   if (radix < 2 || radix > std::max(2, l)) return TUNA_ERR_BAD_RADIX;
   if (g > 1 && (radix_global < 2 || radix_global > std::max(2, g))) return TUNA_ERR_BAD_RADIX;
-  int rc = validate_layout(P, sendcounts, sdispls, rdispls, sendbase, recvbase);
+  HostLayout hl;
+  int rc = host_layout(P, sendcounts, sdispls, rdispls, sendbase, recvbase, &hl);
   if (rc) return rc;
 
   tuna_plan *pl = new (std::nothrow) tuna_plan();
@@ -982,7 +1027,7 @@ int tuna_plan_create(tuna_plan_t **out, int P, int radix, int radix_global, int 
   rc = alloc_list(pl, pl->dir, TUNA_LIST_DELIVER, PP);
   if (rc) return nomem(rc);
 #undef TUNA_TRY
-  rc = build_tables(pl, sendcounts, sdispls, rdispls, sendbase, recvbase, st);
+  rc = build_tables(pl, hl, sendcounts, sdispls, rdispls, st);
   if (rc) return fail(rc);
   *out = pl;
   return TUNA_OK;
@@ -992,7 +1037,10 @@ int tuna_plan_update_counts(tuna_plan_t *pl, const int64_t *sendcounts, const in
                             const int64_t *rdispls, const int64_t *sendbase,
                             const int64_t *recvbase, void *stream) {
   if (!pl || !sendcounts) return TUNA_ERR_INVALID_ARG;
-  return build_tables(pl, sendcounts, sdispls, rdispls, sendbase, recvbase, (cudaStream_t)stream);
+  HostLayout hl;
+  const int rc = host_layout(pl->topo.P, sendcounts, sdispls, rdispls, sendbase, recvbase, &hl);
+  if (rc) return rc;
+  return build_tables(pl, hl, sendcounts, sdispls, rdispls, (cudaStream_t)stream);
 }
 
 int tuna_plan_workspace_bytes(const tuna_plan_t *pl, size_t *bytes) {
@@ -1048,15 +1096,41 @@ int tuna_direct_alltoallv(tuna_plan_t *pl, const void *sendbuf, const int64_t *s
   return run_direct(pl, sendbuf, recvbuf, (cudaStream_t)stream);
 }
 
+// Device-side alias of a pinned, mapped host buffer, or nullptr if the kernels
+// cannot address it (pageable memory, or a null / empty buffer).
+static void *mapped_alias(const void *host) {
+  if (!host) return nullptr;
+  cudaPointerAttributes at;
+  if (cudaPointerGetAttributes(&at, host) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return nullptr;
+  }
+  if (at.type != cudaMemoryTypeHost || !at.devicePointer) return nullptr;
+  return at.devicePointer;
+}
+
 int tuna_alltoallv_host(tuna_plan_t *pl, const void *host_send, void *host_recv, int schedule,
                         void *stream) {
   if (!pl) return TUNA_ERR_INVALID_ARG;
   if ((!host_send && pl->send_extent > 0) || (!host_recv && pl->recv_extent > 0)) return TUNA_ERR_INVALID_ARG;
+  const bool force_staging = (schedule & TUNA_HOST_STAGED) != 0;
+  schedule &= ~TUNA_HOST_STAGED;
   if (schedule != TUNA_SCHEDULE_TUNA && schedule != TUNA_SCHEDULE_DIRECT) return TUNA_ERR_INVALID_ARG;
+  if (ranges_overlap(host_send, (size_t)pl->send_extent, host_recv, (size_t)pl->recv_extent))
+    return TUNA_ERR_OVERLAP;
+  cudaStream_t st = (cudaStream_t)stream;
+  // Pinned, mapped host buffers: the kernels read the send buffer and write the
+  // receive buffer in place, so the two directions of the host link run at the
+  // same time and no block is copied twice.
+  if (!force_staging) {
+    void *zs = pl->send_extent > 0 ? mapped_alias(host_send) : (void *)host_send;
+    void *zr = pl->recv_extent > 0 ? mapped_alias(host_recv) : host_recv;
+    if ((zs || pl->send_extent == 0) && (zr || pl->recv_extent == 0))
+      return schedule == TUNA_SCHEDULE_TUNA ? run_tuna(pl, zs, zr, st) : run_direct(pl, zs, zr, st);
+  }
   const int64_t w = align256(pl->workspace_need);
   const int64_t need = w + align256(pl->send_extent) + align256(pl->recv_extent) + 256;
   if (!pl->workspace || pl->workspace_bytes < (size_t)need) return TUNA_ERR_WORKSPACE;
-  cudaStream_t st = (cudaStream_t)stream;
   char *d_send = pl->workspace + w;
   char *d_recv = d_send + align256(pl->send_extent);
   if (pl->send_extent > 0)

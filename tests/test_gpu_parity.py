@@ -243,20 +243,40 @@ def test_update_counts_and_rerun():
 
 
 def test_host_buffer_entry_point():
-    wl = W.make_random(9, 5000, seed=5, zero_frac=0.2)
-    ref = oracle_brute(wl)
+    wl = W.make_random(9, 5000, seed=5, zero_frac=0.2, gaps=True)
+    ref = oracle_brute(wl)                                   # canary 0xA5 in the gaps
     plan = B.plan_for(wl, 3)
     plan.alloc_workspace(host_staging=True)
     hs = wl.make_send().pin_memory()
+    covered = np.zeros(wl.recv_bytes, dtype=bool)
+    for d in range(wl.P):
+        for s in range(wl.P):
+            o = int(wl.recvbase[d] + wl.rdispls[d, s]) * wl.elem_size
+            covered[o:o + int(wl.sendcounts[s, d]) * wl.elem_size] = True
     for schedule in (B.SCHEDULE_TUNA, B.SCHEDULE_DIRECT):
-        hr = torch.zeros(wl.recv_bytes, dtype=torch.uint8).pin_memory()
+        # pinned buffers: the kernels work on host memory in place, gaps stay untouched
+        hr = torch.full((wl.recv_bytes,), CANARY, dtype=torch.uint8).pin_memory()
         plan.alltoallv_host(hs, hr, schedule)
         torch.cuda.synchronize()
         assert np.array_equal(hr.numpy(), ref)
+        # staged through device copies (forced, or because the memory is pageable)
+        for send_h, flag in ((hs, B.HOST_STAGED), (wl.make_send(), 0)):
+            hr2 = torch.zeros(wl.recv_bytes, dtype=torch.uint8)
+            if flag:
+                hr2 = hr2.pin_memory()
+            plan.alltoallv_host(send_h, hr2, schedule | flag)
+            torch.cuda.synchronize()
+            assert np.array_equal(hr2.numpy()[covered], ref[covered])
     small = B.plan_for(wl, 3)
     small.alloc_workspace(host_staging=False)
+    hr = torch.full((wl.recv_bytes,), CANARY, dtype=torch.uint8).pin_memory()
+    small.alltoallv_host(hs, hr, B.SCHEDULE_TUNA)            # in place: no staging space needed
+    torch.cuda.synchronize()
+    assert np.array_equal(hr.numpy(), ref)
     with pytest.raises(B.TunaError, match="WORKSPACE"):
-        small.alltoallv_host(hs, hr, B.SCHEDULE_TUNA)
+        small.alltoallv_host(hs, hr, B.SCHEDULE_TUNA | B.HOST_STAGED)
+    with pytest.raises(B.TunaError, match="OVERLAP"):
+        small.alltoallv_host(hs, hs, B.SCHEDULE_TUNA)
 
 
 def test_degenerate_inputs():
