@@ -403,7 +403,8 @@ def ours_arm(args):
             sstep()
         staged_ms = (time.perf_counter() - t0) * 1e3 / 2
         e2e = {"value": job_throughput(payload, world, e_ms), "unit": UNIT,
-               "path": "kernels read and write the pinned host buffers in place",
+               "path": "in place on the pinned host buffers for blocks of 2 KiB and more on average, "
+                       "staged through device copies below that",
                "staged_copies_ms_per_step": staged_ms,
                "h2d_bytes_per_step": wl.send_bytes + 8 * (3 * wl.P * wl.P + 2 * wl.P),
                "d2h_bytes_per_step": wl.recv_bytes, "ms_per_step": e_ms, "steps": e_steps}

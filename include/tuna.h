@@ -195,7 +195,8 @@ int tuna_direct_alltoallv_static(int P, int elem_size, const int64_t *sendcounts
  * returning without synchronising.  `schedule` is TUNA_SCHEDULE_TUNA or
  * TUNA_SCHEDULE_DIRECT, optionally OR-ed with TUNA_HOST_STAGED.
  *   - Both buffers pinned and mapped into the device's address space (cudaHostAlloc
- *     or cudaHostRegister memory under unified addressing): the kernels read
+ *     or cudaHostRegister memory under unified addressing), and blocks of 2 KiB or
+ *     more on average (or no room for staging in the workspace): the kernels read
  *     host_send and write host_recv in place over the host link, both directions
  *     at once; blocks hop through the device workspace in between.  Needs only
  *     workspace_bytes of workspace; receive-buffer bytes that no block covers are

@@ -243,7 +243,7 @@ def test_update_counts_and_rerun():
 
 
 def test_host_buffer_entry_point():
-    wl = W.make_random(9, 5000, seed=5, zero_frac=0.2, gaps=True)
+    wl = W.make_random(9, 20000, seed=5, zero_frac=0.2, gaps=True)   # mean block over 2 KiB
     ref = oracle_brute(wl)                                   # canary 0xA5 in the gaps
     plan = B.plan_for(wl, 3)
     plan.alloc_workspace(host_staging=True)
