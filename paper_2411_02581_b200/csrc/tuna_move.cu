@@ -45,7 +45,6 @@ namespace {
 
 constexpr int kThreads = TUNA_MOVE_THREADS;
 constexpr int kBatch = kThreads;        // descriptors handled per batch (one per thread)
-constexpr int kChunkVec = TUNA_MAX_CHUNK_BYTES / 16;  // vectors per chunk, at most
 constexpr int kClampVec = 1 << 26;      // |vector index| beyond which only "far away" matters
 
 __device__ __forceinline__ uint4 ld16(const char *p) { return *reinterpret_cast<const uint4 *>(p); }
@@ -141,7 +140,7 @@ __device__ __forceinline__ uint4 load16_any(const char *sa, bool careful, int b0
 
 // ------------------------------------------------------------------ the mover
 
-template <bool DELIVER>
+template <bool DELIVER, int kUnroll>  // kUnroll: vectors a thread has in flight
 __device__ __forceinline__ void move_body(const TunaMoveArgs &a) {
   __shared__ int s_vs[kBatch];             // first vector of the block, relative to the chunk
   __shared__ int s_org[kBatch];            // DELIVER: chunk-relative position of the block's first byte
@@ -149,7 +148,7 @@ __device__ __forceinline__ void move_body(const TunaMoveArgs &a) {
   __shared__ const char *s_sadj[kBatch];   // source address of chunk vector v is s_sadj + 16 v
   __shared__ char *s_dadj[kBatch];         // DELIVER: destination address likewise (16-byte aligned)
   __shared__ unsigned char s_careful[kBatch];
-  __shared__ __align__(16) unsigned char s_who[kChunkVec];
+  extern __shared__ __align__(16) unsigned char s_who[];  // owner of every vector of the chunk (chunk / 16 bytes)
 
   const int tid = threadIdx.x, lane = tid & 31;
   const int64_t c = blockIdx.x;
@@ -208,12 +207,12 @@ __device__ __forceinline__ void move_body(const TunaMoveArgs &a) {
       fill_owner(s_who, s_vs, cnt, vlo, vhi);
       __syncthreads();
     }
-    // every thread takes a strided share of the vectors: four loads, then four stores
-    for (int v = vlo + tid; v - lane < vhi; v += 4 * kThreads) {  // whole warps stay in the loop
-      uint4 x[4];
-      char *out[4];
+    // every thread takes a strided share of the vectors: a few loads, then as many stores
+    for (int v = vlo + tid; v - lane < vhi; v += kUnroll * kThreads) {  // whole warps stay in the loop
+      uint4 x[kUnroll];
+      char *out[kUnroll];
 #pragma unroll
-      for (int k = 0; k < 4; k++) {
+      for (int k = 0; k < kUnroll; k++) {
         const int vv = v + k * kThreads;
         bool on = vv < vhi;
         const char *sa = nullptr;
@@ -250,7 +249,7 @@ __device__ __forceinline__ void move_body(const TunaMoveArgs &a) {
         }
       }
 #pragma unroll
-      for (int k = 0; k < 4; k++)
+      for (int k = 0; k < kUnroll; k++)
         if (out[k]) st16(out[k], x[k]);
     }
     // DELIVER: the partial first and last vector of a block, by the block's own thread
@@ -272,16 +271,19 @@ __device__ __forceinline__ void move_body(const TunaMoveArgs &a) {
   }
 }
 
-// Two builds of every DELIVER kernel: lists of large blocks run best with four
-// CTAs per SM and all the registers the copy loop wants; lists of tiny blocks are
-// bound by latency and gain from a fifth resident CTA.
-__global__ void __launch_bounds__(kThreads) tuna_round_kernel(const TunaMoveArgs a) { move_body<false>(a); }
-__global__ void __launch_bounds__(kThreads) tuna_deliver_kernel(const TunaMoveArgs a) { move_body<true>(a); }
-__global__ void __launch_bounds__(kThreads) tuna_rotate_kernel(const TunaMoveArgs a) { move_body<true>(a); }
-__global__ void __launch_bounds__(kThreads) tuna_direct_kernel(const TunaMoveArgs a) { move_body<true>(a); }
-__global__ void __launch_bounds__(kThreads, 5) tuna_deliver_small_kernel(const TunaMoveArgs a) { move_body<true>(a); }
-__global__ void __launch_bounds__(kThreads, 5) tuna_rotate_small_kernel(const TunaMoveArgs a) { move_body<true>(a); }
-__global__ void __launch_bounds__(kThreads, 5) tuna_direct_small_kernel(const TunaMoveArgs a) { move_body<true>(a); }
+// Two builds of every kernel.  Lists of large blocks run best with four vectors in
+// flight per thread and the registers that takes (4-5 CTAs per SM).  Lists of tiny
+// blocks spend much of a CTA's life on the dependent loads of its set-up (chunk
+// table, descriptors, then data), so they gain from eight resident CTAs per SM
+// with two vectors in flight each (measured on 180-byte blocks: 1.15-1.4x).
+__global__ void __launch_bounds__(kThreads) tuna_round_kernel(const TunaMoveArgs a) { move_body<false, 4>(a); }
+__global__ void __launch_bounds__(kThreads) tuna_deliver_kernel(const TunaMoveArgs a) { move_body<true, 4>(a); }
+__global__ void __launch_bounds__(kThreads) tuna_rotate_kernel(const TunaMoveArgs a) { move_body<true, 4>(a); }
+__global__ void __launch_bounds__(kThreads) tuna_direct_kernel(const TunaMoveArgs a) { move_body<true, 4>(a); }
+__global__ void __launch_bounds__(kThreads, 8) tuna_round_small_kernel(const TunaMoveArgs a) { move_body<false, 2>(a); }
+__global__ void __launch_bounds__(kThreads, 8) tuna_deliver_small_kernel(const TunaMoveArgs a) { move_body<true, 2>(a); }
+__global__ void __launch_bounds__(kThreads, 8) tuna_rotate_small_kernel(const TunaMoveArgs a) { move_body<true, 2>(a); }
+__global__ void __launch_bounds__(kThreads, 8) tuna_direct_small_kernel(const TunaMoveArgs a) { move_body<true, 2>(a); }
 
 }  // namespace
 
@@ -289,27 +291,31 @@ cudaError_t tuna_launch_move(int kernel, const TunaMoveArgs &a, bool small_block
   if (a.nchunks <= 0 || a.n <= 0) return cudaSuccess;
   if (a.chunk > TUNA_MAX_CHUNK_BYTES || (a.chunk & 15)) return cudaErrorInvalidValue;
   const dim3 grid((unsigned)a.nchunks), block(kThreads);
+  const size_t who_bytes = (size_t)(a.chunk >> 4);  // one owner byte per 16-byte vector of a chunk (<= 16 KiB)
   switch (kernel) {
     case TUNA_K_ROUND:
-      tuna_round_kernel<<<grid, block, 0, stream>>>(a);
+      if (small_blocks)
+        tuna_round_small_kernel<<<grid, block, who_bytes, stream>>>(a);
+      else
+        tuna_round_kernel<<<grid, block, who_bytes, stream>>>(a);
       break;
     case TUNA_K_DELIVER:
       if (small_blocks)
-        tuna_deliver_small_kernel<<<grid, block, 0, stream>>>(a);
+        tuna_deliver_small_kernel<<<grid, block, who_bytes, stream>>>(a);
       else
-        tuna_deliver_kernel<<<grid, block, 0, stream>>>(a);
+        tuna_deliver_kernel<<<grid, block, who_bytes, stream>>>(a);
       break;
     case TUNA_K_ROTATE:
       if (small_blocks)
-        tuna_rotate_small_kernel<<<grid, block, 0, stream>>>(a);
+        tuna_rotate_small_kernel<<<grid, block, who_bytes, stream>>>(a);
       else
-        tuna_rotate_kernel<<<grid, block, 0, stream>>>(a);
+        tuna_rotate_kernel<<<grid, block, who_bytes, stream>>>(a);
       break;
     default:
       if (small_blocks)
-        tuna_direct_small_kernel<<<grid, block, 0, stream>>>(a);
+        tuna_direct_small_kernel<<<grid, block, who_bytes, stream>>>(a);
       else
-        tuna_direct_kernel<<<grid, block, 0, stream>>>(a);
+        tuna_direct_kernel<<<grid, block, who_bytes, stream>>>(a);
       break;
   }
   return cudaGetLastError();
