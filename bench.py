@@ -346,18 +346,13 @@ def ours_arm(args):
     ms_per_step = elapsed_ms / args.steps
     value = job_throughput(payload, world, ms_per_step)
 
-    # roofline of the dominant kernel: whichever of the fused pack-move-unpack
-    # kernels (blocks travelling on / blocks arriving) took the most time
+    # roofline of the dominant kernel: the fused pack-move-unpack kernel, one launch
+    # per digit phase
     peak, peak_kind = measured_peaks()
-    keep_ms = timing["round_local"]["ms"] + timing["round_global"]["ms"]
-    if keep_ms >= timing["deliver"]["ms"]:
-        kname = "tuna_round_kernel"
-        rk_ms = keep_ms
-        rk_launches = timing["round_local"]["launches"] + timing["round_global"]["launches"]
-        rk_bytes = timing["round_local"]["bytes"] + timing["round_global"]["bytes"]
-    else:
-        kname = "tuna_deliver_kernel"
-        rk_ms, rk_launches, rk_bytes = (timing["deliver"][k] for k in ("ms", "launches", "bytes"))
+    kname = "tuna_round_kernel"
+    rk_ms = timing["round_local"]["ms"] + timing["round_global"]["ms"]
+    rk_launches = timing["round_local"]["launches"] + timing["round_global"]["launches"]
+    rk_bytes = timing["round_local"]["bytes"] + timing["round_global"]["bytes"]
     achieved = 2.0 * rk_bytes / (rk_ms * 1e-3) / 1e9 if rk_ms > 0 else 0.0
     per_byte = NCU_TRAFFIC_PER_PAYLOAD_BYTE.get(kernel_source_sha(), {}).get(kname)
     roofline = {

@@ -125,10 +125,10 @@ int tuna_plan_extents(const tuna_plan_t *plan, size_t *send_bytes, size_t *recv_
 
 /*
  * tuna_alltoallv - run the plan's TuNA schedule (Algorithm 1, or Sec. IV /
- * Algorithm 3 when g > 1): per digit phase one fused pack-move-unpack launch for
- * the blocks that travel on and one for the blocks that have arrived (all rounds
- * z of one digit position x touch disjoint blocks, so they share a launch), then
- * one rotation launch (self blocks; in TUNA_FLAG_CLASSIC_ROTATE mode every block).
+ * Algorithm 3 when g > 1): one fused pack-move-unpack launch per digit phase (all
+ * rounds z of one digit position x touch disjoint blocks, so they share it; the
+ * self blocks ride along in the first one), and in TUNA_FLAG_CLASSIC_ROTATE mode
+ * one rotation launch at the end.
  *
  *   sendbuf, recvbuf   device; must not overlap.
  *   sendcounts, sdispls, recvcounts, rdispls
@@ -220,7 +220,7 @@ int tuna_alltoallv_host(tuna_plan_t *plan, const void *host_send, void *host_rec
  * has two descriptor lists, selected by `part`: TUNA_PART_KEEP, the blocks that
  * travel on in a later phase and land in the workspace, and TUNA_PART_DELIVER, the
  * blocks that have arrived and land in the receive buffer (empty in
- * TUNA_FLAG_CLASSIC_ROTATE mode); each non-empty list is one kernel launch.
+ * TUNA_FLAG_CLASSIC_ROTATE mode); the two lists of a phase share one kernel launch.
  * phase -1 selects the rotation list and -2 the direct list (`part` ignored).
  * `entries` descriptor rows, `bytes` moved, `stream_bytes` the padded length of the
  * list's stream (for a KEEP list: the size of its workspace region).
@@ -257,12 +257,11 @@ int tuna_plan_launch_count(const tuna_plan_t *plan, int64_t *launches);
  * metadata, data, replace, rearrange and inter-node cost).  With timing enabled
  * every launch is bracketed by CUDA events on the caller's stream:
  *   TUNA_TIMER_PLAN          metadata exchange + prefix sums (prepare + metadata)
- *   TUNA_TIMER_ROUND_LOCAL   flat / local digit phases, blocks that travel on (data;
- *                            "replace" is fused away)
- *   TUNA_TIMER_ROUND_GLOBAL  global digit phases, blocks that travel on (inter-group cost)
- *   TUNA_TIMER_ROTATE        final rotation (rearrange)
+ *   TUNA_TIMER_ROUND_LOCAL   flat / local digit phases (data; "replace" is fused away;
+ *                            the first phase's launch also copies the self blocks)
+ *   TUNA_TIMER_ROUND_GLOBAL  global digit phases (inter-group cost)
+ *   TUNA_TIMER_ROTATE        final rotation when it has a launch of its own (rearrange)
  *   TUNA_TIMER_DIRECT        the single-pass direct exchange
- *   TUNA_TIMER_DELIVER       blocks that arrive in a digit phase of either level (data)
  * tuna_plan_get_timing waits for the recorded events and returns, per kind
  * (arrays of TUNA_TIMER_KINDS, any may be NULL), accumulated milliseconds,
  * launches and payload bytes moved; `reset` non-zero clears the accumulators.
@@ -272,8 +271,7 @@ int tuna_plan_launch_count(const tuna_plan_t *plan, int64_t *launches);
 #define TUNA_TIMER_ROUND_GLOBAL 2
 #define TUNA_TIMER_ROTATE 3
 #define TUNA_TIMER_DIRECT 4
-#define TUNA_TIMER_DELIVER 5
-#define TUNA_TIMER_KINDS 6
+#define TUNA_TIMER_KINDS 5
 int tuna_plan_enable_timing(tuna_plan_t *plan, int on);
 int tuna_plan_get_timing(tuna_plan_t *plan, int reset, double *ms, int64_t *launches,
                          int64_t *bytes);

@@ -26,7 +26,7 @@ SCHEDULE_TUNA = 0
 SCHEDULE_DIRECT = 1
 HOST_STAGED = 0x100
 
-TIMER_NAMES = ("plan", "round_local", "round_global", "rotate", "direct", "deliver")
+TIMER_NAMES = ("plan", "round_local", "round_global", "rotate", "direct")
 TIMER_KINDS = len(TIMER_NAMES)
 
 STATUS = {

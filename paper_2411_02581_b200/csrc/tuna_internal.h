@@ -66,24 +66,32 @@ struct TunaList {
   bool small_blocks = false;  // mean block far below a chunk (host copy, from bytes / n)
 };
 
-struct TunaMoveArgs {
+// Device view of one list.
+struct TunaListArgs {
   const int64_t *len, *pos, *src, *dst;
   const int32_t *chunk_first;
-  int64_t n, total, chunk, nchunks;
+  int64_t n, total, chunk, nchunks;  // nchunks == 0: the list takes no part in the launch
+};
+
+// One launch moves up to three independent lists: the CTAs [0, keep.nchunks) take
+// the KEEP list, the next del.nchunks the first DELIVER list, the rest the second.
+struct TunaMoveArgs {
+  TunaListArgs keep;  // blocks of a digit phase that travel on (workspace)
+  TunaListArgs del;   // blocks of a digit phase that have arrived, or the direct list
+  TunaListArgs rot;   // rotation list (self blocks, or every block in classic mode)
   char *base[3];
   int64_t extent[3];  // bytes of each buffer that may be accessed, from its base
-  int64_t keep_base;  // KEEP lists: workspace offset of stream position 0
+  int64_t keep_base;  // workspace offset of stream position 0 of the KEEP list
 };
 
 enum TunaMoveKernel {
-  TUNA_K_ROUND = 0,    // KEEP list of a digit phase: blocks that travel on
-  TUNA_K_DELIVER = 1,  // DELIVER list of a digit phase: blocks that have arrived
-  TUNA_K_ROTATE = 2,   // final rotation / self blocks
-  TUNA_K_DIRECT = 3    // single-pass direct exchange
+  TUNA_K_ROUND = 0,   // a digit phase (with the self blocks riding along in the first one)
+  TUNA_K_ROTATE = 1,  // the rotation list alone
+  TUNA_K_DIRECT = 2   // single-pass direct exchange
 };
 
-// Launches one mover kernel over one list (tuna_move.cu).  `small_blocks` picks
-// the build tuned for lists whose blocks are far smaller than a chunk.
+// Launches one mover kernel (tuna_move.cu).  `small_blocks` picks the build tuned
+// for lists whose blocks are far smaller than a chunk.
 cudaError_t tuna_launch_move(int kernel, const TunaMoveArgs &a, bool small_blocks, cudaStream_t stream);
 
 #endif

@@ -21,14 +21,18 @@
 // vector, so that consecutive threads copy consecutive vectors whatever the
 // block boundaries are, several loads in flight per thread before the first store.
 //
-//   tuna_round_kernel    KEEP lists.  The stream IS the destination, so stores
+// A launch carries up to three independent lists (the block index picks list and
+// chunk): a digit phase is ONE tuna_round_kernel launch over its KEEP list, its
+// DELIVER list and, in the first phase, the self blocks; tuna_rotate_kernel runs a
+// rotation list alone (classic mode), tuna_direct_kernel the direct list.
+//
+//   KEEP lists.          The stream IS the destination, so stores
 //                        are contiguous aligned vectors (a block's padding is
 //                        written too: it is the library's own memory); sources are
 //                        aligned workspace blocks or arbitrarily aligned
 //                        send-buffer blocks (read as aligned words merged by
 //                        funnel shifts).
-//   tuna_deliver_kernel, tuna_rotate_kernel, tuna_direct_kernel
-//                        DELIVER lists.  The stream spaces the blocks so that
+//   DELIVER lists.       The stream spaces the blocks so that
 //                        block e can be thought of as sitting at its destination's
 //                        alignment: vector v of the stream then corresponds to
 //                        one 16-byte aligned vector of the destination.  Vectors
@@ -141,7 +145,7 @@ __device__ __forceinline__ uint4 load16_any(const char *sa, bool careful, int b0
 // ------------------------------------------------------------------ the mover
 
 template <bool DELIVER, int kUnroll>  // kUnroll: vectors a thread has in flight
-__device__ __forceinline__ void move_body(const TunaMoveArgs &a) {
+__device__ __forceinline__ void move_body(const TunaListArgs &l, const TunaMoveArgs &a, int64_t c) {
   __shared__ int s_vs[kBatch];             // first vector of the block, relative to the chunk
   __shared__ int s_org[kBatch];            // DELIVER: chunk-relative position of the block's first byte
   __shared__ int s_end[kBatch];            // DELIVER: ... and one past its last byte (clamped when far)
@@ -151,12 +155,11 @@ __device__ __forceinline__ void move_body(const TunaMoveArgs &a) {
   extern __shared__ __align__(16) unsigned char s_who[];  // owner of every vector of the chunk (chunk / 16 bytes)
 
   const int tid = threadIdx.x, lane = tid & 31;
-  const int64_t c = blockIdx.x;
-  const int64_t cA = c * a.chunk;
-  const int64_t cB = (cA + a.chunk < a.total) ? cA + a.chunk : a.total;
+  const int64_t cA = c * l.chunk;
+  const int64_t cB = (cA + l.chunk < l.total) ? cA + l.chunk : l.total;
   const int nv = (int)((cB - cA) >> 4);
-  const int64_t e_lo = a.chunk_first[c];
-  const int64_t e_hi = (c + 1 < a.nchunks) ? (int64_t)a.chunk_first[c + 1] : a.n - 1;
+  const int64_t e_lo = l.chunk_first[c];
+  const int64_t e_hi = (c + 1 < l.nchunks) ? (int64_t)l.chunk_first[c + 1] : l.n - 1;
   char *const keep_out = DELIVER ? nullptr : a.base[2] + a.keep_base + cA;
 
   for (int64_t b = e_lo; b <= e_hi; b += kBatch) {
@@ -166,8 +169,8 @@ __device__ __forceinline__ void move_body(const TunaMoveArgs &a) {
     bool my_edges = false;
     if (tid < cnt) {
       const int64_t e = b + tid;
-      const int64_t p = a.pos[e];
-      const int64_t s = a.src[e];
+      const int64_t p = l.pos[e];
+      const int64_t s = l.src[e];
       const int sb = TUNA_LOC_BUF(s);
       const char *sbase = base_of(a, sb);
       const char *sp = sbase + TUNA_LOC_OFF(s);
@@ -176,8 +179,8 @@ __device__ __forceinline__ void move_body(const TunaMoveArgs &a) {
       if (vs < -kClampVec) vs = -kClampVec;
       s_vs[tid] = (int)vs;
       if (DELIVER) {
-        const int64_t L = a.len[e];
-        const int64_t d = a.dst[e];
+        const int64_t L = l.len[e];
+        const int64_t d = l.dst[e];
         char *dp = base_of(a, TUNA_LOC_BUF(d)) + TUNA_LOC_OFF(d);
         const int ad = (int)(reinterpret_cast<uintptr_t>(dp) & 15);
         const int64_t org = rel + ad;  // exact chunk-relative position of byte 0
@@ -192,13 +195,13 @@ __device__ __forceinline__ void move_body(const TunaMoveArgs &a) {
         s_careful[tid] = (L > 0 && (sp - 19 < sbase || sp + L + 19 > sbase + extent_of(a, sb))) ? 1 : 0;
         my_edges = L > 0 && (ad != 0 || (L & 15) != 0);
       } else {
-        const int64_t pn = a.pos[e + 1];
+        const int64_t pn = l.pos[e + 1];
         s_sadj[tid] = sp - rel;
         s_careful[tid] = (sp - 3 < sbase || sp + (pn - p) + 4 > sbase + extent_of(a, sb)) ? 1 : 0;
       }
     }
     // vectors of the chunk this batch covers
-    const int64_t first_rel = a.pos[b] - cA, next_rel = a.pos[b + cnt] - cA;
+    const int64_t first_rel = l.pos[b] - cA, next_rel = l.pos[b + cnt] - cA;
     const int vlo = first_rel > 0 ? (int)(first_rel >> 4) : 0;
     const int vhi = (next_rel >> 4) < nv ? (int)(next_rel >> 4) : nv;
     __syncthreads();
@@ -243,7 +246,7 @@ __device__ __forceinline__ void move_body(const TunaMoveArgs &a) {
             x[k] = load16_bytes(sa, 0, 16);
           } else {
             const int64_t e = b + t;
-            const int64_t rem = a.len[e] - (cA + ((int64_t)vv << 4) - a.pos[e]);
+            const int64_t rem = l.len[e] - (cA + ((int64_t)vv << 4) - l.pos[e]);
             x[k] = load16_bytes(sa, 0, rem < 16 ? (int)(rem > 0 ? rem : 0) : 16);
           }
         }
@@ -271,39 +274,53 @@ __device__ __forceinline__ void move_body(const TunaMoveArgs &a) {
   }
 }
 
+// One launch, up to three lists: the block index picks the list and the chunk.
+template <int kUnroll>
+__device__ __forceinline__ void launch_body(const TunaMoveArgs &a) {
+  int64_t c = blockIdx.x;
+  if (c < a.keep.nchunks) {
+    move_body<false, kUnroll>(a.keep, a, c);
+    return;
+  }
+  c -= a.keep.nchunks;
+  if (c < a.del.nchunks)
+    move_body<true, kUnroll>(a.del, a, c);
+  else
+    move_body<true, kUnroll>(a.rot, a, c - a.del.nchunks);
+}
+
 // Two builds of every kernel.  Lists of large blocks run best with four vectors in
-// flight per thread and the registers that takes (4-5 CTAs per SM).  Lists of tiny
+// flight per thread and the registers that takes (4 CTAs per SM).  Lists of tiny
 // blocks spend much of a CTA's life on the dependent loads of its set-up (chunk
 // table, descriptors, then data), so they gain from eight resident CTAs per SM
 // with two vectors in flight each (measured on 180-byte blocks: 1.15-1.4x).
-__global__ void __launch_bounds__(kThreads) tuna_round_kernel(const TunaMoveArgs a) { move_body<false, 4>(a); }
-__global__ void __launch_bounds__(kThreads) tuna_deliver_kernel(const TunaMoveArgs a) { move_body<true, 4>(a); }
-__global__ void __launch_bounds__(kThreads) tuna_rotate_kernel(const TunaMoveArgs a) { move_body<true, 4>(a); }
-__global__ void __launch_bounds__(kThreads) tuna_direct_kernel(const TunaMoveArgs a) { move_body<true, 4>(a); }
-__global__ void __launch_bounds__(kThreads, 8) tuna_round_small_kernel(const TunaMoveArgs a) { move_body<false, 2>(a); }
-__global__ void __launch_bounds__(kThreads, 8) tuna_deliver_small_kernel(const TunaMoveArgs a) { move_body<true, 2>(a); }
-__global__ void __launch_bounds__(kThreads, 8) tuna_rotate_small_kernel(const TunaMoveArgs a) { move_body<true, 2>(a); }
-__global__ void __launch_bounds__(kThreads, 8) tuna_direct_small_kernel(const TunaMoveArgs a) { move_body<true, 2>(a); }
+__global__ void __launch_bounds__(kThreads) tuna_round_kernel(const TunaMoveArgs a) { launch_body<4>(a); }
+__global__ void __launch_bounds__(kThreads) tuna_rotate_kernel(const TunaMoveArgs a) { launch_body<4>(a); }
+__global__ void __launch_bounds__(kThreads) tuna_direct_kernel(const TunaMoveArgs a) { launch_body<4>(a); }
+__global__ void __launch_bounds__(kThreads, 8) tuna_round_small_kernel(const TunaMoveArgs a) { launch_body<2>(a); }
+__global__ void __launch_bounds__(kThreads, 8) tuna_rotate_small_kernel(const TunaMoveArgs a) { launch_body<2>(a); }
+__global__ void __launch_bounds__(kThreads, 8) tuna_direct_small_kernel(const TunaMoveArgs a) { launch_body<2>(a); }
 
 }  // namespace
 
 cudaError_t tuna_launch_move(int kernel, const TunaMoveArgs &a, bool small_blocks, cudaStream_t stream) {
-  if (a.nchunks <= 0 || a.n <= 0) return cudaSuccess;
-  if (a.chunk > TUNA_MAX_CHUNK_BYTES || (a.chunk & 15)) return cudaErrorInvalidValue;
-  const dim3 grid((unsigned)a.nchunks), block(kThreads);
-  const size_t who_bytes = (size_t)(a.chunk >> 4);  // one owner byte per 16-byte vector of a chunk (<= 16 KiB)
+  const TunaListArgs *ls[3] = {&a.keep, &a.del, &a.rot};
+  int64_t nchunks = 0, max_chunk = 0;
+  for (const TunaListArgs *l : ls) {
+    if (l->nchunks <= 0) continue;
+    if (l->chunk > TUNA_MAX_CHUNK_BYTES || (l->chunk & 15)) return cudaErrorInvalidValue;
+    nchunks += l->nchunks;
+    max_chunk = l->chunk > max_chunk ? l->chunk : max_chunk;
+  }
+  if (nchunks <= 0) return cudaSuccess;
+  const dim3 grid((unsigned)nchunks), block(kThreads);
+  const size_t who_bytes = (size_t)(max_chunk >> 4);  // one owner byte per 16-byte vector of a chunk (<= 16 KiB)
   switch (kernel) {
     case TUNA_K_ROUND:
       if (small_blocks)
         tuna_round_small_kernel<<<grid, block, who_bytes, stream>>>(a);
       else
         tuna_round_kernel<<<grid, block, who_bytes, stream>>>(a);
-      break;
-    case TUNA_K_DELIVER:
-      if (small_blocks)
-        tuna_deliver_small_kernel<<<grid, block, who_bytes, stream>>>(a);
-      else
-        tuna_deliver_kernel<<<grid, block, who_bytes, stream>>>(a);
       break;
     case TUNA_K_ROTATE:
       if (small_blocks)

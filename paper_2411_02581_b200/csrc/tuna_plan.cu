@@ -831,9 +831,8 @@ bool ranges_overlap(const void *a, size_t na, const void *b, size_t nb) {
   return na > 0 && nb > 0 && a0 < b0 + nb && b0 < a0 + na;
 }
 
-TunaMoveArgs move_args(const tuna_plan *pl, const TunaList &l, const void *send, void *recv,
-                       char *work) {
-  TunaMoveArgs a{};
+TunaListArgs list_args(const TunaList &l) {
+  TunaListArgs a{};
   a.len = l.len;
   a.pos = l.pos;
   a.src = l.src;
@@ -842,7 +841,12 @@ TunaMoveArgs move_args(const tuna_plan *pl, const TunaList &l, const void *send,
   a.n = l.n;
   a.total = l.total;
   a.chunk = l.chunk;
-  a.nchunks = l.nchunks;
+  a.nchunks = l.n > 0 ? l.nchunks : 0;
+  return a;
+}
+
+TunaMoveArgs move_args(const tuna_plan *pl, const void *send, void *recv, char *work) {
+  TunaMoveArgs a{};
   a.base[TUNA_BUF_SEND] = (char *)const_cast<void *>(send);
   a.base[TUNA_BUF_RECV] = (char *)recv;
   a.base[TUNA_BUF_WORK] = work;
@@ -853,31 +857,42 @@ TunaMoveArgs move_args(const tuna_plan *pl, const TunaList &l, const void *send,
   return a;
 }
 
+// One launch per digit phase: its KEEP list, its DELIVER list and, riding along in
+// the first launch, the self blocks (they depend on nothing).  In classic mode
+// the rotation list needs every phase finished and gets a launch of its own.
 int run_tuna(tuna_plan *pl, const void *send, void *recv, cudaStream_t st) {
   if (pl->workspace_need > 0 &&
       (!pl->workspace || pl->workspace_bytes < (size_t)pl->workspace_need))
     return TUNA_ERR_WORKSPACE;
   int launches = 0;
+  bool rot_done = pl->rot.nchunks == 0;
   for (size_t f = 0; f < pl->phases.size(); f++) {
     const int kind = pl->phases[f].level == 0 ? TUNA_TIMER_ROUND_LOCAL : TUNA_TIMER_ROUND_GLOBAL;
     const TunaList &k = pl->keep[f];
-    if (k.nchunks > 0) {
-      Timed tm(pl, kind, k.bytes, st);
-      TunaMoveArgs a = move_args(pl, k, send, recv, pl->workspace);
-      a.keep_base = pl->h_wbase[f];
-      TUNA_CUDA(pl, tuna_launch_move(TUNA_K_ROUND, a, k.small_blocks, st));
-      launches++;
-    }
     const TunaList &d = pl->deliver[f];
-    if (d.nchunks > 0) {
-      Timed tm(pl, TUNA_TIMER_DELIVER, d.bytes, st);
-      TUNA_CUDA(pl, tuna_launch_move(TUNA_K_DELIVER, move_args(pl, d, send, recv, pl->workspace), d.small_blocks, st));
-      launches++;
+    const bool with_rot = !rot_done && !pl->classic;
+    if (k.nchunks == 0 && d.nchunks == 0 && !with_rot) continue;
+    TunaMoveArgs a = move_args(pl, send, recv, pl->workspace);
+    a.keep = list_args(k);
+    a.del = list_args(d);
+    a.keep_base = pl->h_wbase[f];
+    int64_t bytes = k.bytes + d.bytes;
+    bool small = (k.nchunks == 0 || k.small_blocks) && (d.nchunks == 0 || d.small_blocks);
+    if (with_rot) {
+      a.rot = list_args(pl->rot);
+      bytes += pl->rot.bytes;
+      small = small && pl->rot.small_blocks;
+      rot_done = true;
     }
+    Timed tm(pl, kind, bytes, st);
+    TUNA_CUDA(pl, tuna_launch_move(TUNA_K_ROUND, a, small, st));
+    launches++;
   }
-  if (pl->rot.nchunks > 0) {
+  if (!rot_done) {
     Timed tm(pl, TUNA_TIMER_ROTATE, pl->rot.bytes, st);
-    TUNA_CUDA(pl, tuna_launch_move(TUNA_K_ROTATE, move_args(pl, pl->rot, send, recv, pl->workspace), pl->rot.small_blocks, st));
+    TunaMoveArgs a = move_args(pl, send, recv, pl->workspace);
+    a.rot = list_args(pl->rot);
+    TUNA_CUDA(pl, tuna_launch_move(TUNA_K_ROTATE, a, pl->rot.small_blocks, st));
     launches++;
   }
   pl->last_launches = launches;
@@ -889,7 +904,9 @@ int run_direct(tuna_plan *pl, const void *send, void *recv, cudaStream_t st) {
   int launches = 0;
   if (pl->dir.nchunks > 0) {
     Timed tm(pl, TUNA_TIMER_DIRECT, pl->dir.bytes, st);
-    TUNA_CUDA(pl, tuna_launch_move(TUNA_K_DIRECT, move_args(pl, pl->dir, send, recv, nullptr), pl->dir.small_blocks, st));
+    TunaMoveArgs a = move_args(pl, send, recv, nullptr);
+    a.del = list_args(pl->dir);
+    TUNA_CUDA(pl, tuna_launch_move(TUNA_K_DIRECT, a, pl->dir.small_blocks, st));
     launches++;
   }
   pl->last_launches = launches;
@@ -1438,15 +1455,15 @@ int tuna_direct_alltoallv_static(int P, int elem_size, const int64_t *sendcounts
                                                                              t.chunk_first);
   TUNA_STATIC_CUDA(cudaGetLastError());
   TunaMoveArgs a{};
-  a.len = t.len;
-  a.pos = t.pos;
-  a.src = t.src;
-  a.dst = t.dst;
-  a.chunk_first = t.chunk_first;
-  a.n = PP;
-  a.total = stream_bytes;
-  a.chunk = chunk;
-  a.nchunks = nchunks;
+  a.del.len = t.len;
+  a.del.pos = t.pos;
+  a.del.src = t.src;
+  a.del.dst = t.dst;
+  a.del.chunk_first = t.chunk_first;
+  a.del.n = PP;
+  a.del.total = stream_bytes;
+  a.del.chunk = chunk;
+  a.del.nchunks = nchunks;
   a.base[TUNA_BUF_SEND] = (char *)const_cast<void *>(sendbuf);
   a.base[TUNA_BUF_RECV] = (char *)recvbuf;
   a.base[TUNA_BUF_WORK] = nullptr;
