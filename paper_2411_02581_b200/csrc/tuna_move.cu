@@ -63,27 +63,39 @@ __device__ __forceinline__ int64_t extent_of(const TunaMoveArgs &a, int buf) {
 }
 
 // Largest t < cnt with start[t] <= v (start is non-decreasing, start[0] <= v).
+// Branch-free: eight select steps.
 __device__ __forceinline__ int find_entry(const int *start, int cnt, int v) {
   int lo = 0;
 #pragma unroll
-  for (int step = kBatch / 2; step > 0; step >>= 1)
-    if (lo + step < cnt && start[lo + step] <= v) lo += step;
+  for (int step = kBatch / 2; step > 0; step >>= 1) {
+    const int i = lo + step;
+    const bool in = i < cnt;
+    lo = (in && start[in ? i : 0] <= v) ? i : lo;
+  }
   return lo;
 }
 
-// Owner table: who[v - v_first] = the descriptor owning vector v, for the vectors
-// [v_first, v_last) of the current batch.  Each thread resolves a run of consecutive
-// vectors: one binary search for its last vector, then a walk down.
-__device__ __forceinline__ void fill_owner(unsigned char *who, const int *start, int cnt,
-                                           int v_first, int v_last) {
-  const int span = (v_last - v_first + kThreads - 1) / kThreads;
-  const int v0 = v_first + (int)threadIdx.x * span;
-  if (v0 >= v_last) return;
-  const int vend = (v0 + span < v_last) ? v0 + span : v_last;
-  int t = find_entry(start, cnt, vend - 1);
-  for (int v = vend - 1; v >= v0; v--) {
-    while (start[t] > v) t--;
-    who[v - v_first] = (unsigned char)t;
+// Owner table: who[v] = the descriptor (index in the batch) owning chunk vector v,
+// for v in [vlo, vhi).  Every descriptor with vectors has already written its index
+// at its first vector into the zeroed table; what is left is a running maximum
+// (indices grow with position).  Each thread takes a run of vectors, starts from
+// the owner of the run's first vector (one binary search) and sweeps four table
+// bytes at a time with packed byte maxima.
+__device__ __forceinline__ void fill_owner(unsigned char *who, const int *start, int cnt, int vlo,
+                                           int vhi) {
+  const int a0 = vlo & ~3;
+  const int span = (((vhi - a0) + kThreads - 1) / kThreads + 3) & ~3;
+  const int v0 = a0 + (int)threadIdx.x * span;
+  if (v0 >= vhi) return;
+  const int vend = (v0 + span < vhi) ? v0 + span : vhi;
+  unsigned carry = (unsigned)find_entry(start, cnt, v0 > vlo ? v0 : vlo);
+  for (int v = v0; v < vend; v += 4) {
+    unsigned w = *reinterpret_cast<unsigned *>(who + v);
+    w = __vmaxu4(w, carry);    // the owner so far enters at byte 0
+    w = __vmaxu4(w, w << 8);   // prefix maximum over the four bytes
+    w = __vmaxu4(w, w << 16);
+    *reinterpret_cast<unsigned *>(who + v) = w;
+    carry = w >> 24;
   }
 }
 
@@ -167,6 +179,9 @@ __device__ __forceinline__ void move_body(const TunaListArgs &l, const TunaMoveA
     if (b > e_lo) __syncthreads();  // the previous batch is done with the tables
     int my_org = 0, my_end = 0;
     bool my_edges = false;
+    for (int i = tid * 16; i < nv + 4; i += kThreads * 16)  // the owner table starts out empty
+      *reinterpret_cast<uint4 *>(s_who + i) = make_uint4(0, 0, 0, 0);
+    int mark_at = -1;  // chunk vector at which this thread's block starts, if it has vectors in the chunk
     if (tid < cnt) {
       const int64_t e = b + tid;
       const int64_t p = l.pos[e];
@@ -194,8 +209,10 @@ __device__ __forceinline__ void move_body(const TunaListArgs &l, const TunaMoveA
         s_dadj[tid] = dp - org;
         s_careful[tid] = (L > 0 && (sp - 19 < sbase || sp + L + 19 > sbase + extent_of(a, sb))) ? 1 : 0;
         my_edges = L > 0 && (ad != 0 || (L & 15) != 0);
+        if (L > 0 && tid > 0 && vs < nv) mark_at = (int)vs;
       } else {
         const int64_t pn = l.pos[e + 1];
+        if (pn > p && tid > 0 && vs < nv) mark_at = (int)vs;
         s_sadj[tid] = sp - rel;
         s_careful[tid] = (sp - 3 < sbase || sp + (pn - p) + 4 > sbase + extent_of(a, sb)) ? 1 : 0;
       }
@@ -207,6 +224,8 @@ __device__ __forceinline__ void move_body(const TunaListArgs &l, const TunaMoveA
     __syncthreads();
     const bool single = cnt == 1;
     if (!single) {
+      if (mark_at >= 0) s_who[mark_at] = (unsigned char)tid;
+      __syncthreads();
       fill_owner(s_who, s_vs, cnt, vlo, vhi);
       __syncthreads();
     }
@@ -223,7 +242,7 @@ __device__ __forceinline__ void move_body(const TunaListArgs &l, const TunaMoveA
         int t = 0;
         out[k] = nullptr;
         if (on) {
-          if (!single) t = s_who[vv - vlo];
+          if (!single) t = s_who[vv];
           const int64_t vb = (int64_t)vv << 4;
           if (DELIVER) {
             // only vectors that lie wholly inside the block; its edges come later
@@ -314,7 +333,7 @@ cudaError_t tuna_launch_move(int kernel, const TunaMoveArgs &a, bool small_block
   }
   if (nchunks <= 0) return cudaSuccess;
   const dim3 grid((unsigned)nchunks), block(kThreads);
-  const size_t who_bytes = (size_t)(max_chunk >> 4);  // one owner byte per 16-byte vector of a chunk (<= 16 KiB)
+  const size_t who_bytes = (size_t)(max_chunk >> 4) + 32;  // one owner byte per 16-byte vector of a chunk (<= 16 KiB)
   switch (kernel) {
     case TUNA_K_ROUND:
       if (small_blocks)
