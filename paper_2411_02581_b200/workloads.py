@@ -23,6 +23,9 @@ shapes below follow those, plus a mixture-of-experts token dispatch):
 * ``c4``  P=64,   8192 tokens per rank routed top-2 by Gaussian logits; a
           block is the chosen tokens' rows of ``hidden`` bf16 values.
 * ``c5``  P=2048, bytes, 30 % of pairs empty, the rest U{0..512}.
+
+plus the paper's other patterns at P=4096: ``normal`` and ``powerlaw`` block
+sizes capped at 1024 bytes, and the two FFT transposes ``fft_n1`` / ``fft_n2``.
 """
 from __future__ import annotations
 
@@ -308,4 +311,48 @@ def make_random(P: int, max_count: int, elem_size: int = 1, seed: int = 11,
     return _finish("random", P, elem_size, seed, c.reshape(P, P), gaps=gaps)
 
 
-FULL = {"c1": make_c1, "c2": make_c2, "c3": make_c3, "c4": make_c4, "c5": make_c5}
+# ---- the paper's other count patterns (Sec. VI-A and VI-C), all closed-form or seeded ----
+
+def make_normal(seed: int | None = None, P: int = 4096, mean: float = 1000.0, sd: float = 240.0,
+                cap: int = 1024) -> Workload:
+    """Block sizes N(mean, sd) in bytes, clipped to [0, cap] (Sec. VI-C: mean 1000,
+    standard deviation 240, blocks of at most 1024 bytes, P = 4096)."""
+    seed = bench_seed(6) if seed is None else seed
+    u1 = uniform_unit(seed, S_COUNTS, P * P).numpy()
+    u2 = uniform_unit(seed, S_ZERO, P * P).numpy()
+    z = np.sqrt(-2.0 * np.log(1.0 - u1)) * np.cos(2.0 * math.pi * u2)
+    c = np.clip(np.rint(mean + sd * z), 0, cap).astype(np.int64).reshape(P, P)
+    return _finish("normal", P, 1, seed, c, radices=tuple(r for r in (2, 64, P) if r <= P))
+
+
+def make_powerlaw(seed: int | None = None, P: int = 4096, exponent: float = 0.95,
+                  cap: int = 1024) -> Workload:
+    """Block sizes with Pr[c] proportional to (c+1)^-exponent on {0..cap} bytes
+    (Sec. VI-C: exponent 0.95; large blocks are rare, many are empty or tiny)."""
+    seed = bench_seed(7) if seed is None else seed
+    c = zipf_counts(seed, P * P, exponent, cap).reshape(P, P)
+    return _finish("powerlaw", P, 1, seed, c, radices=tuple(r for r in (2, 64, P) if r <= P))
+
+
+def make_fft_n1(P: int = 4096) -> Workload:
+    """FFT transpose with N1 = ceil(0.78125 P) * ceil(0.625 P) * 8 (Sec. VI-A): the
+    ranks below ceil(0.625 P) each send 8 FP64 values in each of their first
+    ceil(0.78125 P) blocks; everything else is empty."""
+    workers, filled = math.ceil(0.625 * P), math.ceil(0.78125 * P)
+    c = np.zeros((P, P), dtype=np.int64)
+    c[:workers, :filled] = 8
+    return _finish("fft_n1", P, 8, bench_seed(8), c, radices=tuple(r for r in (2, 64, P) if r <= P))
+
+
+def make_fft_n2(P: int = 4096) -> Workload:
+    """FFT transpose with N2 = ((P-1) * 32 + 8) * P complex values (Sec. VI-A): per
+    sender P-1 blocks of 32 complex = 64 FP64 values and a last block of 8 complex
+    = 16 FP64 values."""
+    c = np.full((P, P), 64, dtype=np.int64)
+    c[:, P - 1] = 16
+    return _finish("fft_n2", P, 8, bench_seed(9), c, radices=tuple(r for r in (2, 64, P) if r <= P))
+
+
+FULL = {"c1": make_c1, "c2": make_c2, "c3": make_c3, "c4": make_c4, "c5": make_c5,
+        "normal": make_normal, "powerlaw": make_powerlaw, "fft_n1": make_fft_n1,
+        "fft_n2": make_fft_n2}

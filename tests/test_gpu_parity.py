@@ -421,3 +421,19 @@ def test_c4_full_size(schedule):
             nz += (t % r) != 0
             t //= r
         assert sum(x["bytes"] for x in plan.rounds()) == int((wl.sendcounts * nz).sum()) * wl.elem_size
+
+
+@pytest.mark.parametrize("name", ["normal", "powerlaw", "fft_n1", "fft_n2"])
+def test_paper_count_patterns(name):
+    """Normal and power-law block sizes and the two FFT transposes, at P = 512."""
+    wl = W.FULL[name](P=512)
+    ref, rounds, _, _ = oracle_flat(wl, 8)
+    got, plan = gpu_run(wl, 8, pass_args=False)
+    assert np.array_equal(got, ref)
+    check_rounds(plan, rounds)
+    ref_h, rounds_h, _, _ = oracle_hier(wl, 32, 16, 32, 16)
+    got, plan = gpu_run(wl, 32, l=32, g=16, rg=16, pass_args=False)
+    assert np.array_equal(got, ref_h) and np.array_equal(ref_h, ref)
+    check_rounds(plan, rounds_h)
+    got, _ = gpu_run(wl, 2, direct=True, pass_args=False)
+    assert np.array_equal(got, ref)

@@ -404,3 +404,27 @@ def test_segmented_scan_against_numpy():
         assert np.array_equal(tot, pv.sum(axis=1))
         assert np.all(scan[:, 0] == 0)
         assert np.array_equal(scan[:, -1] + pv[:, -1], tot)      # last displacement + size = total
+
+
+# ---------------------------------------------------------------- the paper's other count patterns
+
+def test_paper_count_patterns_small():
+    """Normal / power-law sizes (Sec. VI-C) and the two FFT transposes (Sec. VI-A),
+    scaled down: shapes as stated in the paper, results equal to the definition."""
+    P = 32
+    n = W.make_normal(P=P)
+    assert n.sendcounts.max() <= 1024 and 850 < n.sendcounts.mean() < 1000    # clipped at the cap
+    pl = W.make_powerlaw(P=P)
+    assert pl.sendcounts.max() <= 1024 and np.median(pl.sendcounts) < pl.sendcounts.mean()
+    f1 = W.make_fft_n1(P=P)
+    assert f1.sendcounts.sum() * 1 == math.ceil(0.78125 * P) * math.ceil(0.625 * P) * 8   # = N1
+    assert np.all(f1.sendcounts[math.ceil(0.625 * P):] == 0)
+    f2 = W.make_fft_n2(P=P)
+    assert f2.sendcounts.sum() == ((P - 1) * 32 + 8) * P * 2      # N2 complex values = 2 FP64 each
+    for wl in (n, pl, f1, f2):
+        ref = brute(wl)
+        for r in (2, 8, P):
+            _, recv, _, _, _ = run_flat(wl, r)
+            assert np.array_equal(recv, ref)
+        recv, _, _, _ = run_hier(wl, 8, 4, 8, 4)
+        assert np.array_equal(recv, ref)
