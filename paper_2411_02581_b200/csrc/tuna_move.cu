@@ -171,12 +171,12 @@ __device__ __forceinline__ void move_body(const TunaListArgs &l, const TunaMoveA
   const int64_t cB = (cA + l.chunk < l.total) ? cA + l.chunk : l.total;
   const int nv = (int)((cB - cA) >> 4);
   const int64_t e_lo = l.chunk_first[c];
-  const int64_t e_hi = (c + 1 < l.nchunks) ? (int64_t)l.chunk_first[c + 1] : l.n - 1;
+  const int64_t e_hi = l.chunk_first[c + 1];  // the table has nchunks + 1 entries
   char *const keep_out = DELIVER ? nullptr : a.base[2] + a.keep_base + cA;
 
   for (int64_t b = e_lo; b <= e_hi; b += kBatch) {
     const int cnt = (int)((e_hi - b + 1 < kBatch) ? e_hi - b + 1 : kBatch);
-    if (b > e_lo) __syncthreads();  // the previous batch is done with the tables
+    __syncthreads();  // the previous batch is done with the tables
     int my_org = 0, my_end = 0;
     bool my_edges = false;
     for (int i = tid * 16; i < nv + 4; i += kThreads * 16)  // the owner table starts out empty
@@ -217,11 +217,12 @@ __device__ __forceinline__ void move_body(const TunaListArgs &l, const TunaMoveA
         s_careful[tid] = (sp - 3 < sbase || sp + (pn - p) + 4 > sbase + extent_of(a, sb)) ? 1 : 0;
       }
     }
-    // vectors of the chunk this batch covers
+    // vectors of the chunk this batch covers; a batch of empty blocks has none
     const int64_t first_rel = l.pos[b] - cA, next_rel = l.pos[b + cnt] - cA;
     const int vlo = first_rel > 0 ? (int)(first_rel >> 4) : 0;
     const int vhi = (next_rel >> 4) < nv ? (int)(next_rel >> 4) : nv;
     __syncthreads();
+    if (vhi <= vlo) continue;
     const bool single = cnt == 1;
     if (!single) {
       if (mark_at >= 0) s_who[mark_at] = (unsigned char)tid;

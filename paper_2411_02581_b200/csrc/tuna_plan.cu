@@ -289,12 +289,14 @@ __global__ void tuna_place_kernel(TunaTopo t, PhaseDev ph, const int64_t *__rest
   }
 }
 
-// First descriptor of every chunk: the last e with pos[e] <= c * chunk.
+// First descriptor of every chunk: the last e with pos[e] <= c * chunk.  One more
+// entry closes the table: the last descriptor that has any bytes (so that a tail
+// of empty blocks behind it is not walked by the last chunk's CTA).
 __global__ void tuna_chunk_index_kernel(const int64_t *__restrict__ pos, int64_t n, int64_t chunk,
-                                        int64_t nchunks, int32_t *first) {
+                                        int64_t nchunks, int64_t total, int32_t *first) {
   const int64_t c = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (c >= nchunks) return;
-  const int64_t target = c * chunk;
+  if (c > nchunks) return;
+  const int64_t target = c < nchunks ? c * chunk : total - 1;
   int64_t lo = 0, hi = n;  // first index with pos > target
   while (lo < hi) {
     const int64_t mid = (lo + hi) >> 1;
@@ -507,13 +509,13 @@ int build_chunks(tuna_plan *pl, TunaList &l, cudaStream_t st) {
     cudaFree(l.chunk_first);
     l.chunk_first = nullptr;
     l.chunk_cap = 0;
-    TUNA_CUDA(pl, dev_alloc(&l.chunk_first, l.nchunks));
+    TUNA_CUDA(pl, dev_alloc(&l.chunk_first, l.nchunks + 1));
     l.chunk_cap = l.nchunks;
   }
   if (l.nchunks > 0) {
     const int th = 128;
-    tuna_chunk_index_kernel<<<(unsigned)((l.nchunks + th - 1) / th), th, 0, st>>>(
-        l.pos, l.n, l.chunk, l.nchunks, l.chunk_first);
+    tuna_chunk_index_kernel<<<(unsigned)((l.nchunks + th) / th), th, 0, st>>>(
+        l.pos, l.n, l.chunk, l.nchunks, l.total, l.chunk_first);
     TUNA_LAUNCHED(pl);
   }
   return TUNA_OK;
@@ -1296,7 +1298,7 @@ constexpr int64_t kStaticPP = (int64_t)TUNA_STATIC_MAX_P * TUNA_STATIC_MAX_P;
 constexpr int64_t kStaticWords = 8 * kStaticPP + 1      // counts, sdispls, rdispls, tmp, len, pos(+1), src, dst
                                  + 5 * TUNA_STATIC_MAX_P  // sendbase, recvbase, seg_total, seg_raw, seg_base
                                  + 2                      // stream totals
-                                 + TUNA_STATIC_MAX_CHUNKS / 2;  // chunk table (32-bit entries)
+                                 + TUNA_STATIC_MAX_CHUNKS / 2 + 1;  // chunk table (32-bit entries)
 static __device__ __align__(256) int64_t tuna_static_scratch[kStaticWords];
 
 struct StaticTables {
@@ -1347,7 +1349,7 @@ cudaError_t static_tables(StaticTables *t) {
   t->seg_raw = take(TUNA_STATIC_MAX_P);
   t->seg_base = take(TUNA_STATIC_MAX_P);
   t->scal = take(2);
-  t->chunk_first = (int32_t *)take(TUNA_STATIC_MAX_CHUNKS / 2);
+  t->chunk_first = (int32_t *)take(TUNA_STATIC_MAX_CHUNKS / 2 + 1);
   return cudaSuccess;
 }
 
@@ -1451,8 +1453,8 @@ int tuna_direct_alltoallv_static(int P, int elem_size, const int64_t *sendcounts
   TUNA_STATIC_CUDA(cudaGetLastError());
   tuna_add_base_kernel<<<gPP, th, 0, st>>>(t.pos, t.seg_base, P, PP);
   TUNA_STATIC_CUDA(cudaGetLastError());
-  tuna_chunk_index_kernel<<<(unsigned)((nchunks + 127) / 128), 128, 0, st>>>(t.pos, PP, chunk, nchunks,
-                                                                             t.chunk_first);
+  tuna_chunk_index_kernel<<<(unsigned)((nchunks + 128) / 128), 128, 0, st>>>(t.pos, PP, chunk, nchunks,
+                                                                             stream_bytes, t.chunk_first);
   TUNA_STATIC_CUDA(cudaGetLastError());
   TunaMoveArgs a{};
   a.del.len = t.len;
