@@ -30,12 +30,17 @@ if ROOT not in sys.path:
 METRIC = "alltoallv_payload_throughput"
 UNIT = "GB/s"
 
-# DRAM traffic of the dominant kernels from ncu captures
+# DRAM traffic of the dominant kernel from ncu captures
 # (dram__bytes_read.sum + dram__bytes_write.sum per launch) divided by the payload
 # bytes that launch moved, keyed by the SHA-256 of the kernel source the capture
-# was taken with, then by kernel.  A changed source makes the figures stale: the
-# traffic is then reported as null.
-NCU_TRAFFIC_PER_PAYLOAD_BYTE: dict[str, dict[str, float]] = {}
+# was taken with, then by workload (at its default radix).  Traffic grows in
+# proportion to the bytes moved, so the full-size figure is this ratio times the
+# launch's bytes.  A changed source makes the figures stale: the traffic is then
+# reported as null.  Captures: profiles/round_kernel_c4_reduced.md (c4, reduced to
+# 2 GiB) and profiles/round_small_kernel_c5.md (c5 at full size).
+NCU_TRAFFIC_PER_PAYLOAD_BYTE: dict[str, dict[str, float]] = {
+    "f2c6995a4e14b17a72802978cc99e82f9f9bded42bf508a4106cbb153c523ecd": {"c4": 1.980, "c5": 2.311},
+}
 
 
 def parse_args():
@@ -354,7 +359,8 @@ def ours_arm(args):
     rk_launches = timing["round_local"]["launches"] + timing["round_global"]["launches"]
     rk_bytes = timing["round_local"]["bytes"] + timing["round_global"]["bytes"]
     achieved = 2.0 * rk_bytes / (rk_ms * 1e-3) / 1e9 if rk_ms > 0 else 0.0
-    per_byte = NCU_TRAFFIC_PER_PAYLOAD_BYTE.get(kernel_source_sha(), {}).get(kname)
+    per_byte = NCU_TRAFFIC_PER_PAYLOAD_BYTE.get(kernel_source_sha(), {}).get(wl.name) \
+        if not args.radix else None
     roofline = {
         "bound": "hbm", "kernel": kname, "achieved": achieved, "peak": peak,
         "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,
