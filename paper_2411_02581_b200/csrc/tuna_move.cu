@@ -224,6 +224,28 @@ __device__ __forceinline__ void move_body(const TunaListArgs &l, const TunaMoveA
     __syncthreads();
     if (vhi <= vlo) continue;
     const bool single = cnt == 1;
+    if (single) {
+      // One block covers the whole range (a chunk inside a large block).  If both
+      // ends are 16-byte aligned and no vector of the range is partial, this is a
+      // plain strided copy: no table look-ups in the loop.
+      const char *src = s_sadj[0] + ((int64_t)vlo << 4);
+      char *dst = (DELIVER ? s_dadj[0] : keep_out) + ((int64_t)vlo << 4);
+      bool plain = (reinterpret_cast<uintptr_t>(src) & 15) == 0 && s_careful[0] == 0;
+      if (DELIVER) plain = plain && s_org[0] <= (vlo << 4) && s_end[0] >= (vhi << 4);
+      if (plain) {
+        const int m = vhi - vlo;
+        int i = tid;
+        for (; i + (kUnroll - 1) * kThreads < m; i += kUnroll * kThreads) {
+          uint4 x[kUnroll];
+#pragma unroll
+          for (int k = 0; k < kUnroll; k++) x[k] = ld16(src + ((int64_t)(i + k * kThreads) << 4));
+#pragma unroll
+          for (int k = 0; k < kUnroll; k++) st16(dst + ((int64_t)(i + k * kThreads) << 4), x[k]);
+        }
+        for (; i < m; i += kThreads) st16(dst + ((int64_t)i << 4), ld16(src + ((int64_t)i << 4)));
+        continue;
+      }
+    }
     if (!single) {
       if (mark_at >= 0) s_who[mark_at] = (unsigned char)tid;
       __syncthreads();
