@@ -441,6 +441,7 @@ def ours_arm(args):
             entry(f"flat r={r}", make_plan(r))
         if wl.radices:
             entry(f"flat r={wl.radices[0]} classic-rotate", make_plan(wl.radices[0], flags=B.FLAG_CLASSIC_ROTATE))
+            entry(f"flat r={wl.radices[-1]} bulk-copy route", make_plan(wl.radices[-1], flags=B.FLAG_BULK_COPY))
         if wl.hier:
             l, g = wl.hier
             for rl, rg in wl.hier_radices:

@@ -53,6 +53,9 @@ typedef enum tuna_status {
 /* flags for tuna_plan_create */
 #define TUNA_FLAG_DIRECT_TO_R 0u    /* default: a block's last hop writes straight into the receive buffer */
 #define TUNA_FLAG_CLASSIC_ROTATE 1u /* last hops land in the workspace; one final rotation pass reorders them */
+#define TUNA_FLAG_BULK_COPY 2u      /* chunks inside one large 16-byte aligned block go through the SM's bulk
+                                       copy engine (cp.async.bulk through shared memory) instead of vector loads
+                                       and stores; same result, measured about 1 % slower, hence optional */
 
 /* schedules for the host-buffer entry point */
 #define TUNA_SCHEDULE_TUNA 0
@@ -278,6 +281,11 @@ int tuna_plan_get_timing(tuna_plan_t *plan, int reset, double *ms, int64_t *laun
 
 /* The cudaError_t of the most recent failing runtime call (0 if none). */
 int tuna_plan_cuda_error(const tuna_plan_t *plan);
+
+/* Synchronises the device and reports in *gave_up whether any kernel of this plan
+ * abandoned a bounded wait (only the TUNA_FLAG_BULK_COPY route waits: on the
+ * barriers of its bulk copies); the receive buffer is then incomplete. */
+int tuna_plan_device_status(tuna_plan_t *plan, int *gave_up);
 
 /* Static string for a status code. */
 const char *tuna_strerror(int status);

@@ -20,6 +20,7 @@ _VP = ctypes.c_void_p
 
 FLAG_DIRECT_TO_R = 0
 FLAG_CLASSIC_ROTATE = 1
+FLAG_BULK_COPY = 2
 PART_KEEP = 0
 PART_DELIVER = 1
 SCHEDULE_TUNA = 0
@@ -59,6 +60,7 @@ SIGNATURES = {
     "tuna_plan_enable_timing": (ctypes.c_int, [_VP, ctypes.c_int]),
     "tuna_plan_get_timing": (ctypes.c_int, [_VP, ctypes.c_int, ctypes.POINTER(ctypes.c_double), _I64P, _I64P]),
     "tuna_plan_cuda_error": (ctypes.c_int, [_VP]),
+    "tuna_plan_device_status": (ctypes.c_int, [_VP, _INTP]),
     "tuna_strerror": (ctypes.c_char_p, [ctypes.c_int]),
     "tuna_version": (ctypes.c_int, []),
 }
@@ -252,6 +254,12 @@ class Plan:
         self._check(lib().tuna_plan_last_launches(self._h, ctypes.byref(n)), "tuna_plan_last_launches")
         return n.value
 
+
+    def device_status(self) -> int:
+        """0, or 1 if a kernel of this plan gave up a bounded wait (synchronises the device)."""
+        n = ctypes.c_int()
+        self._check(lib().tuna_plan_device_status(self._h, ctypes.byref(n)), "tuna_plan_device_status")
+        return n.value
 
     def launch_count(self) -> int:
         n = ctypes.c_int64()

@@ -82,6 +82,9 @@ struct TunaMoveArgs {
   char *base[3];
   int64_t extent[3];  // bytes of each buffer that may be accessed, from its base
   int64_t keep_base;  // workspace offset of stream position 0 of the KEEP list
+  int *error;         // device flag raised when a bounded wait inside a kernel gave up (may be null)
+  int bulk_off;       // in: non-zero asks for the bulk-copy route; the launcher turns it into the offset
+                      // of the staging area in dynamic shared memory (0 = route off)
 };
 
 enum TunaMoveKernel {

@@ -154,9 +154,62 @@ __device__ __forceinline__ uint4 load16_any(const char *sa, bool careful, int b0
   return load16_funnel(sa);
 }
 
+// ------------------------------------------------------------------ bulk copies (TMA)
+//
+// Optional route (TUNA_FLAG_BULK_COPY).  A chunk that lies inside one large aligned
+// block needs no SM work at all: one thread hands it to the copy engine of the SM
+// in pieces (cp.async.bulk, global ->
+// shared, completion counted in bytes on an mbarrier) and, as each piece lands,
+// sends it on (cp.async.bulk, shared -> global).  Addresses and sizes are
+// multiples of 16 bytes by construction.  Every wait is bounded: if a barrier does
+// not complete, the CTA raises the launch's error flag and leaves.  Measured on
+// 2 MiB blocks this route reaches 6.58 TB/s against 6.65 TB/s for the plain vector
+// loop (64 KiB of staging leave three CTAs per SM), so it is off by default.
+
+constexpr int kBulkPiece = 16384;
+constexpr int kBulkPieces = 4;                       // pieces in flight: one 64 KiB chunk
+constexpr int kBulkBytes = kBulkPiece * kBulkPieces;
+constexpr int kBulkMin = 16384;                      // shorter ranges are copied by the threads
+
+__device__ __forceinline__ unsigned smem_u32(const void *p) {
+  return (unsigned)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void mbar_init(unsigned bar, unsigned count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(unsigned bar, unsigned bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity) {
+  for (int it = 0; it < (1 << 20); it++) {  // each try_wait sleeps for a while by itself
+    unsigned ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    if (ok) return true;
+  }
+  return false;
+}
+__device__ __forceinline__ void bulk_load(unsigned smem_dst, const void *gsrc, unsigned bytes, unsigned bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(smem_dst),
+               "l"(gsrc), "r"(bytes), "r"(bar)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_store(void *gdst, unsigned smem_src, unsigned bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gdst), "r"(smem_src), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// waits until the committed stores have been written (not only read out of shared memory)
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
 // ------------------------------------------------------------------ the mover
 
-template <bool DELIVER, int kUnroll>  // kUnroll: vectors a thread has in flight
+template <bool DELIVER, int kUnroll, bool kBulk>  // kUnroll: vectors a thread has in flight
 __device__ __forceinline__ void move_body(const TunaListArgs &l, const TunaMoveArgs &a, int64_t c) {
   __shared__ int s_vs[kBatch];             // first vector of the block, relative to the chunk
   __shared__ int s_org[kBatch];            // DELIVER: chunk-relative position of the block's first byte
@@ -166,7 +219,14 @@ __device__ __forceinline__ void move_body(const TunaListArgs &l, const TunaMoveA
   __shared__ unsigned char s_careful[kBatch];
   extern __shared__ __align__(16) unsigned char s_who[];  // owner of every vector of the chunk (chunk / 16 bytes)
 
+  // bulk route (builds with kBulk only): barriers, their phase, the staging area behind the owner table
+  __shared__ __align__(8) unsigned long long s_bar[kBulkPieces];
+  __shared__ int s_abort;
+  unsigned bulk_phase = 0;  // bit j: parity of barrier j's current phase
+  bool bar_ready = false;
+
   const int tid = threadIdx.x, lane = tid & 31;
+  if (kBulk && tid == 0) s_abort = 0;
   const int64_t cA = c * l.chunk;
   const int64_t cB = (cA + l.chunk < l.total) ? cA + l.chunk : l.total;
   const int nv = (int)((cB - cA) >> 4);
@@ -177,6 +237,7 @@ __device__ __forceinline__ void move_body(const TunaListArgs &l, const TunaMoveA
   for (int64_t b = e_lo; b <= e_hi; b += kBatch) {
     const int cnt = (int)((e_hi - b + 1 < kBatch) ? e_hi - b + 1 : kBatch);
     __syncthreads();  // the previous batch is done with the tables
+    if (kBulk && s_abort) return;
     int my_org = 0, my_end = 0;
     bool my_edges = false;
     for (int i = tid * 16; i < nv + 4; i += kThreads * 16)  // the owner table starts out empty
@@ -232,6 +293,43 @@ __device__ __forceinline__ void move_body(const TunaListArgs &l, const TunaMoveA
       char *dst = (DELIVER ? s_dadj[0] : keep_out) + ((int64_t)vlo << 4);
       bool plain = (reinterpret_cast<uintptr_t>(src) & 15) == 0 && s_careful[0] == 0;
       if (DELIVER) plain = plain && s_org[0] <= (vlo << 4) && s_end[0] >= (vhi << 4);
+      if (kBulk && a.bulk_off > 0 && plain && ((vhi - vlo) << 4) >= kBulkMin && ((vhi - vlo) << 4) <= kBulkBytes) {
+        if (tid == 0) {
+          const unsigned bytes = (unsigned)(vhi - vlo) << 4;
+          const int np = (int)((bytes + kBulkPiece - 1) / kBulkPiece);
+          char *stage = reinterpret_cast<char *>(s_who) + a.bulk_off;
+          if (!bar_ready) {
+            for (int j = 0; j < kBulkPieces; j++) mbar_init(smem_u32(&s_bar[j]), 1);
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+          }
+          for (int j = 0; j < np; j++) {
+            const unsigned off = (unsigned)j * kBulkPiece;
+            const unsigned sz = bytes - off < (unsigned)kBulkPiece ? bytes - off : (unsigned)kBulkPiece;
+            mbar_expect_tx(smem_u32(&s_bar[j]), sz);
+            bulk_load(smem_u32(stage + off), src + off, sz, smem_u32(&s_bar[j]));
+          }
+          bool ok = true;
+          for (int j = 0; j < np; j++) {
+            const unsigned off = (unsigned)j * kBulkPiece;
+            const unsigned sz = bytes - off < (unsigned)kBulkPiece ? bytes - off : (unsigned)kBulkPiece;
+            if (ok && !mbar_wait(smem_u32(&s_bar[j]), (bulk_phase >> j) & 1)) ok = false;
+            if (ok) {
+              bulk_store(dst + off, smem_u32(stage + off), sz);
+              bulk_commit();
+            } else {
+              (void)mbar_wait(smem_u32(&s_bar[j]), (bulk_phase >> j) & 1);  // one more bounded wait for the copy in flight
+            }
+          }
+          bulk_wait_all();
+          if (!ok) {
+            if (a.error) atomicExch(a.error, 1);
+            s_abort = 1;
+          }
+        }
+        bar_ready = true;
+        bulk_phase ^= (1u << ((((vhi - vlo) << 4) + kBulkPiece - 1) / kBulkPiece)) - 1;  // the barriers used
+        continue;
+      }
       if (plain) {
         const int m = vhi - vlo;
         int i = tid;
@@ -317,18 +415,18 @@ __device__ __forceinline__ void move_body(const TunaListArgs &l, const TunaMoveA
 }
 
 // One launch, up to three lists: the block index picks the list and the chunk.
-template <int kUnroll>
+template <int kUnroll, bool kBulk>
 __device__ __forceinline__ void launch_body(const TunaMoveArgs &a) {
   int64_t c = blockIdx.x;
   if (c < a.keep.nchunks) {
-    move_body<false, kUnroll>(a.keep, a, c);
+    move_body<false, kUnroll, kBulk>(a.keep, a, c);
     return;
   }
   c -= a.keep.nchunks;
   if (c < a.del.nchunks)
-    move_body<true, kUnroll>(a.del, a, c);
+    move_body<true, kUnroll, kBulk>(a.del, a, c);
   else
-    move_body<true, kUnroll>(a.rot, a, c - a.del.nchunks);
+    move_body<true, kUnroll, kBulk>(a.rot, a, c - a.del.nchunks);
 }
 
 // Two builds of every kernel.  Lists of large blocks run best with four vectors in
@@ -336,16 +434,17 @@ __device__ __forceinline__ void launch_body(const TunaMoveArgs &a) {
 // blocks spend much of a CTA's life on the dependent loads of its set-up (chunk
 // table, descriptors, then data), so they gain from eight resident CTAs per SM
 // with two vectors in flight each (measured on 180-byte blocks: 1.15-1.4x).
-__global__ void __launch_bounds__(kThreads) tuna_round_kernel(const TunaMoveArgs a) { launch_body<4>(a); }
-__global__ void __launch_bounds__(kThreads) tuna_rotate_kernel(const TunaMoveArgs a) { launch_body<4>(a); }
-__global__ void __launch_bounds__(kThreads) tuna_direct_kernel(const TunaMoveArgs a) { launch_body<4>(a); }
-__global__ void __launch_bounds__(kThreads, 8) tuna_round_small_kernel(const TunaMoveArgs a) { launch_body<2>(a); }
-__global__ void __launch_bounds__(kThreads, 8) tuna_rotate_small_kernel(const TunaMoveArgs a) { launch_body<2>(a); }
-__global__ void __launch_bounds__(kThreads, 8) tuna_direct_small_kernel(const TunaMoveArgs a) { launch_body<2>(a); }
+__global__ void __launch_bounds__(kThreads) tuna_round_kernel(const TunaMoveArgs a) { launch_body<4, true>(a); }
+__global__ void __launch_bounds__(kThreads) tuna_rotate_kernel(const TunaMoveArgs a) { launch_body<4, true>(a); }
+__global__ void __launch_bounds__(kThreads) tuna_direct_kernel(const TunaMoveArgs a) { launch_body<4, true>(a); }
+__global__ void __launch_bounds__(kThreads, 8) tuna_round_small_kernel(const TunaMoveArgs a) { launch_body<2, false>(a); }
+__global__ void __launch_bounds__(kThreads, 8) tuna_rotate_small_kernel(const TunaMoveArgs a) { launch_body<2, false>(a); }
+__global__ void __launch_bounds__(kThreads, 8) tuna_direct_small_kernel(const TunaMoveArgs a) { launch_body<2, false>(a); }
 
 }  // namespace
 
-cudaError_t tuna_launch_move(int kernel, const TunaMoveArgs &a, bool small_blocks, cudaStream_t stream) {
+cudaError_t tuna_launch_move(int kernel, const TunaMoveArgs &a_in, bool small_blocks, cudaStream_t stream) {
+  TunaMoveArgs a = a_in;
   const TunaListArgs *ls[3] = {&a.keep, &a.del, &a.rot};
   int64_t nchunks = 0, max_chunk = 0;
   for (const TunaListArgs *l : ls) {
@@ -356,7 +455,21 @@ cudaError_t tuna_launch_move(int kernel, const TunaMoveArgs &a, bool small_block
   }
   if (nchunks <= 0) return cudaSuccess;
   const dim3 grid((unsigned)nchunks), block(kThreads);
-  const size_t who_bytes = (size_t)(max_chunk >> 4) + 32;  // one owner byte per 16-byte vector of a chunk (<= 16 KiB)
+  size_t who_bytes = (size_t)(max_chunk >> 4) + 32;  // one owner byte per 16-byte vector of a chunk (<= 16 KiB)
+  const bool bulk = a.bulk_off != 0 && !small_blocks;  // the caller asks for the bulk-copy route
+  a.bulk_off = 0;
+  if (bulk) {  // the bulk staging area follows the owner table
+    a.bulk_off = (int)((who_bytes + 127) & ~(size_t)127);
+    who_bytes = a.bulk_off + kBulkBytes;
+    static bool raised = false;  // opt in to more than 48 KiB of dynamic shared memory, once
+    if (!raised) {
+      cudaError_t e = cudaFuncSetAttribute(tuna_round_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
+      if (e == cudaSuccess) e = cudaFuncSetAttribute(tuna_rotate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
+      if (e == cudaSuccess) e = cudaFuncSetAttribute(tuna_direct_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
+      if (e != cudaSuccess) return e;
+      raised = true;
+    }
+  }
   switch (kernel) {
     case TUNA_K_ROUND:
       if (small_blocks)

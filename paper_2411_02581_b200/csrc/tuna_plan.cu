@@ -353,6 +353,7 @@ struct tuna_plan {
   int64_t *d_wbase = nullptr;    // phases + 1 workspace offsets
   unsigned long long *d_round_bytes = nullptr;
   int64_t stats_n = 0;
+  int *d_error = nullptr;        // raised by a kernel whose bounded wait gave up
 
   std::vector<int64_t> h_wbase;  // workspace offset of every phase's KEEP stream
   int64_t workspace_need = 0;
@@ -856,6 +857,8 @@ TunaMoveArgs move_args(const tuna_plan *pl, const void *send, void *recv, char *
   a.extent[TUNA_BUF_RECV] = pl->recv_extent;
   a.extent[TUNA_BUF_WORK] = work ? pl->workspace_need : 0;
   a.keep_base = 0;
+  a.error = pl->d_error;
+  a.bulk_off = (pl->flags & TUNA_FLAG_BULK_COPY) ? 1 : 0;
   return a;
 }
 
@@ -964,6 +967,7 @@ int tuna_plan_destroy(tuna_plan_t *pl) {
   cudaFree(pl->d_scal);
   cudaFree(pl->d_wbase);
   cudaFree(pl->d_round_bytes);
+  cudaFree(pl->d_error);
   for (auto &s : pl->stamps) {
     cudaEventDestroy(s.a);
     cudaEventDestroy(s.b);
@@ -1029,6 +1033,8 @@ int tuna_plan_create(tuna_plan_t **out, int P, int radix, int radix_global, int 
   TUNA_TRY(dev_alloc(&pl->d_scal, 2 * (2 * nph + 2)));
   TUNA_TRY(dev_alloc(&pl->d_wbase, nph + 1));
   TUNA_TRY(dev_alloc(&pl->d_round_bytes, pl->stats_n));
+  TUNA_TRY(dev_alloc(&pl->d_error, 1));
+  TUNA_TRY(cudaMemset(pl->d_error, 0, sizeof(int)));
   pl->keep.resize(nph);
   pl->deliver.resize(nph);
   auto nomem = [&](int code) {
@@ -1284,6 +1290,13 @@ int tuna_plan_get_timing(tuna_plan_t *pl, int reset, double *ms, int64_t *launch
 }
 
 int tuna_plan_cuda_error(const tuna_plan_t *pl) { return pl ? pl->cuda_err : 0; }
+
+int tuna_plan_device_status(tuna_plan_t *pl, int *gave_up) {
+  if (!pl || !gave_up) return TUNA_ERR_INVALID_ARG;
+  TUNA_CUDA(pl, cudaDeviceSynchronize());
+  TUNA_CUDA(pl, cudaMemcpy(gave_up, pl->d_error, sizeof(int), cudaMemcpyDeviceToHost));
+  return TUNA_OK;
+}
 
 // ------------------------------------------------------------------ allocation-free direct exchange
 

@@ -115,6 +115,22 @@ def test_large_blocks_span_many_chunks():
     assert np.array_equal(got, ref)
 
 
+def test_bulk_copy_route():
+    """TUNA_FLAG_BULK_COPY: chunks inside large aligned blocks go through
+    cp.async.bulk; same bytes, and no kernel gives up a wait."""
+    aligned = W.make_c4(P=16, tokens=256, hidden=512)          # 1 KiB rows, blocks of ~32 KiB
+    ragged = W.make_random(6, 3_000_000, elem_size=1, seed=78, zero_frac=0.2)   # unaligned: falls back
+    for wl in (aligned, ragged):
+        ref = oracle_brute(wl)
+        for r, flags in ((2, B.FLAG_BULK_COPY), (4, B.FLAG_BULK_COPY | B.FLAG_CLASSIC_ROTATE),
+                         (wl.P, B.FLAG_BULK_COPY)):
+            got, plan = gpu_run(wl, r, flags=flags)
+            assert np.array_equal(got, ref)
+            assert plan.device_status() == 0
+        got, plan = gpu_run(wl, 2, flags=B.FLAG_BULK_COPY, direct=True)
+        assert np.array_equal(got, ref) and plan.device_status() == 0
+
+
 HIER = [(Q, N, rl, rg) for Q, N in [(1, 4), (4, 1), (2, 2), (3, 4), (5, 3), (4, 4), (8, 4), (6, 5)]
         for rl in sorted({2, max(2, Q)}) for rg in sorted({2, 3, max(2, N)})
         if rl <= max(2, Q) and rg <= max(2, N)]
