@@ -46,7 +46,7 @@ NCU_TRAFFIC_PER_PAYLOAD_BYTE: dict[str, dict[str, float]] = {
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c4", choices=["c1", "c2", "c3", "c4", "c4_skew", "c5", "normal", "powerlaw", "fft_n1", "fft_n2"])
@@ -236,7 +236,9 @@ def time_schedule(plan, wl, send, recv, steps, warmup, direct=False, replan=True
     """Median-free timing of `steps` back-to-back steps with CUDA events; returns ms per step."""
     import torch
     run = plan.direct_alltoallv if direct else plan.alltoallv
-    layout = (wl.sendcounts, wl.sdispls, wl.rdispls, wl.sendbase, wl.recvbase)
+    # the workloads are packed back to back, which is what "no displacement arrays" means
+    # to the library: only the counts cross to the device, the rest is computed there
+    layout = (wl.sendcounts, None, None, None, None)
 
     def step():
         if replan:
@@ -307,7 +309,7 @@ def ours_arm(args):
     payload = wl.payload_bytes_total
 
     def make_plan(r, l=None, g=1, rg=2, flags=0):
-        return B.plan_for(wl, r, l=l, g=g, radix_global=rg, flags=flags)
+        return B.plan_for(wl, r, l=l, g=g, radix_global=rg, flags=flags, explicit_layout=False)
 
     if hier_headline:
         l, g = wl.hier
@@ -318,7 +320,9 @@ def ours_arm(args):
         plan = make_plan(radix)
         sched = f"flat radix {radix}"
     plan.alloc_workspace(host_staging=not args.no_e2e, device=dev)
-    layout = (wl.sendcounts, wl.sdispls, wl.rdispls, wl.sendbase, wl.recvbase)
+    # the workloads are packed back to back, which is what "no displacement arrays" means
+    # to the library: only the counts cross to the device, the rest is computed there
+    layout = (wl.sendcounts, None, None, None, None)
 
     def step():
         plan.update_counts(*layout)
@@ -407,7 +411,7 @@ def ours_arm(args):
                "path": "in place on the pinned host buffers for blocks of 2 KiB and more on average, "
                        "staged through device copies below that",
                "staged_copies_ms_per_step": staged_ms,
-               "h2d_bytes_per_step": wl.send_bytes + 8 * (3 * wl.P * wl.P + 2 * wl.P),
+               "h2d_bytes_per_step": wl.send_bytes + 8 * (wl.P * wl.P + 2 * wl.P),
                "d2h_bytes_per_step": wl.recv_bytes, "ms_per_step": e_ms, "steps": e_steps}
         del hs, hr
 
