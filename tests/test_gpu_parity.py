@@ -453,3 +453,33 @@ def test_paper_count_patterns(name):
     check_rounds(plan, rounds_h)
     got, _ = gpu_run(wl, 2, direct=True, pass_args=False)
     assert np.array_equal(got, ref)
+
+
+def test_block_larger_than_4_gib():
+    """64-bit offsets end to end: one block of 5 GiB + 3 bytes (larger than any 32-bit
+    count or displacement), next to small unaligned ones, through a two-hop schedule."""
+    free, _ = torch.cuda.mem_get_info()
+    if free < 30 * 2**30:
+        pytest.skip("needs about 30 GiB of free device memory")
+    counts = np.array([[5, 7, 0, 11], [13, 0, 17, 19], [0, 23, 29, 31], [37, 41, 43, 0]], dtype=np.int64)
+    counts[1, 0] = 5 * 2**30 + 3
+    wl = W._finish("huge", 4, 1, 99, counts)
+    send = wl.make_send("cuda")
+    for kw, direct in ((dict(radix=2), False), (dict(radix=2, flags=B.FLAG_CLASSIC_ROTATE), False),
+                       (dict(radix=4), True)):
+        recv = wl.make_recv("cuda", fill=CANARY)
+        plan = B.plan_for(wl, **kw)
+        plan.alloc_workspace()
+        (plan.direct_alltoallv if direct else plan.alltoallv)(send, recv)
+        torch.cuda.synchronize()
+        for s in range(4):
+            for d in range(4):
+                n = int(wl.sendcounts[s, d])
+                a = int(wl.sendbase[s] + wl.sdispls[s, d])
+                b = int(wl.recvbase[d] + wl.rdispls[d, s])
+                assert torch.equal(recv[b:b + n], send[a:a + n]), (s, d)
+        assert int(wl.recv_bytes) == int(counts.sum())     # packed: every byte is covered
+        plan.set_workspace(None)
+        plan.destroy()
+        del recv
+        torch.cuda.empty_cache()
