@@ -295,7 +295,10 @@ def make_c5(seed: int | None = None, P: int = 2048, max_bytes: int = 512,
         hier = None
     return _finish("c5", P, 1, seed, c, gaps=gaps,
                    radices=tuple(r for r in (2, 8, 32, P) if r <= P), hier=hier,
-                   hier_radices=((hier[0], hier[1]),) if hier else ())
+                   hier_radices=tuple(dict.fromkeys(
+                       [(hier[0], hier[1])] + [(a, b) for a in (2, 8, 32) for b in (2, 8, 64)
+                                               if a <= max(2, hier[0]) and b <= max(2, hier[1])]))
+                   if hier else ())
 
 
 def make_uniform(P: int, count: int, elem_size: int = 1, seed: int = 7) -> Workload:
