@@ -39,7 +39,7 @@ UNIT = "GB/s"
 # reported as null.  Captures: profiles/round_kernel_c4_reduced.md (c4, reduced to
 # 2 GiB) and profiles/round_small_kernel_c5.md (c5 at full size).
 NCU_TRAFFIC_PER_PAYLOAD_BYTE: dict[str, dict[str, float]] = {
-    "f2c6995a4e14b17a72802978cc99e82f9f9bded42bf508a4106cbb153c523ecd": {"c4": 1.980, "c5": 2.311},
+    "442c90091d9441d762f294b36ceac07575e5bb0e657b145e09b9ca3cb6b54a2e": {"c4": 1.980, "c5": 2.314},
 }
 
 
