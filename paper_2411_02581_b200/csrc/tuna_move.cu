@@ -43,6 +43,8 @@
 //                        destination range is written.
 // No byte outside a source buffer's extent is read: blocks within 19 bytes of
 // either end of their buffer are read byte by byte instead of by aligned windows.
+#include <stdlib.h>
+
 #include "tuna_internal.h"
 
 namespace {
@@ -207,6 +209,17 @@ __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.comm
 // waits until the committed stores have been written (not only read out of shared memory)
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
+// ------------------------------------------------------------------ dependent launches
+//
+// The launches of one exchange form a chain on a stream.  Each is launched with
+// programmatic stream serialization: its CTAs may start while the previous launch
+// is still draining, do their set-up (which reads only the plan's tables), and
+// then block in hardware until the previous launch has completed and its writes
+// are visible.  Every launch lets its successor start early right away.
+
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ------------------------------------------------------------------ the mover
 
 template <bool DELIVER, int kUnroll, bool kBulk>  // kUnroll: vectors a thread has in flight
@@ -224,6 +237,7 @@ __device__ __forceinline__ void move_body(const TunaListArgs &l, const TunaMoveA
   __shared__ int s_abort;
   unsigned bulk_phase = 0;  // bit j: parity of barrier j's current phase
   bool bar_ready = false;
+  bool waited = false;      // has this CTA waited for the previous launch of the stream yet?
 
   const int tid = threadIdx.x, lane = tid & 31;
   if (kBulk && tid == 0) s_abort = 0;
@@ -284,6 +298,10 @@ __device__ __forceinline__ void move_body(const TunaListArgs &l, const TunaMoveA
     const int vhi = (next_rel >> 4) < nv ? (int)(next_rel >> 4) : nv;
     __syncthreads();
     if (vhi <= vlo) continue;
+    if (!waited) {  // everything above read only the plan's tables; the data may still be in the making
+      grid_dependency_wait();
+      waited = true;
+    }
     const bool single = cnt == 1;
     if (single) {
       // One block covers the whole range (a chunk inside a large block).  If both
@@ -417,16 +435,21 @@ __device__ __forceinline__ void move_body(const TunaListArgs &l, const TunaMoveA
 // One launch, up to three lists: the block index picks the list and the chunk.
 template <int kUnroll, bool kBulk>
 __device__ __forceinline__ void launch_body(const TunaMoveArgs &a) {
+  grid_launch_dependents();
   int64_t c = blockIdx.x;
   if (c < a.keep.nchunks) {
     move_body<false, kUnroll, kBulk>(a.keep, a, c);
-    return;
+  } else {
+    c -= a.keep.nchunks;
+    if (c < a.del.nchunks)
+      move_body<true, kUnroll, kBulk>(a.del, a, c);
+    else
+      move_body<true, kUnroll, kBulk>(a.rot, a, c - a.del.nchunks);
   }
-  c -= a.keep.nchunks;
-  if (c < a.del.nchunks)
-    move_body<true, kUnroll, kBulk>(a.del, a, c);
-  else
-    move_body<true, kUnroll, kBulk>(a.rot, a, c - a.del.nchunks);
+  // A CTA that found nothing to move has not waited yet.  Every CTA does before it
+  // leaves, so that this launch cannot complete before its predecessor has, and the
+  // next launch's wait covers the whole chain.
+  grid_dependency_wait();
 }
 
 // Two builds of every kernel.  Lists of large blocks (from about 64 KiB) run best
@@ -475,25 +498,33 @@ cudaError_t tuna_launch_move(int kernel, const TunaMoveArgs &a_in, bool small_bl
       if (dev >= 0 && dev < 64) raised[dev] = true;
     }
   }
+  void (*fn)(const TunaMoveArgs);
   switch (kernel) {
     case TUNA_K_ROUND:
-      if (small_blocks)
-        tuna_round_small_kernel<<<grid, block, who_bytes, stream>>>(a);
-      else
-        tuna_round_kernel<<<grid, block, who_bytes, stream>>>(a);
+      fn = small_blocks ? tuna_round_small_kernel : tuna_round_kernel;
       break;
     case TUNA_K_ROTATE:
-      if (small_blocks)
-        tuna_rotate_small_kernel<<<grid, block, who_bytes, stream>>>(a);
-      else
-        tuna_rotate_kernel<<<grid, block, who_bytes, stream>>>(a);
+      fn = small_blocks ? tuna_rotate_small_kernel : tuna_rotate_kernel;
       break;
     default:
-      if (small_blocks)
-        tuna_direct_small_kernel<<<grid, block, who_bytes, stream>>>(a);
-      else
-        tuna_direct_kernel<<<grid, block, who_bytes, stream>>>(a);
+      fn = small_blocks ? tuna_direct_small_kernel : tuna_direct_kernel;
       break;
   }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = who_bytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  static const bool chain = []() {  // TUNA_DEPENDENT_LAUNCH=0 turns the early start off
+    const char *e = getenv("TUNA_DEPENDENT_LAUNCH");
+    return !(e && e[0] == '0');
+  }();
+  cfg.attrs = attr;
+  cfg.numAttrs = chain ? 1 : 0;
+  const cudaError_t le = cudaLaunchKernelEx(&cfg, fn, a);
+  if (le != cudaSuccess) return le;
   return cudaGetLastError();
 }
