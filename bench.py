@@ -39,7 +39,7 @@ UNIT = "GB/s"
 # reported as null.  Captures: profiles/round_kernel_c4_reduced.md (c4, reduced to
 # 2 GiB) and profiles/round_small_kernel_c5.md (c5 at full size).
 NCU_TRAFFIC_PER_PAYLOAD_BYTE: dict[str, dict[str, float]] = {
-    "442c90091d9441d762f294b36ceac07575e5bb0e657b145e09b9ca3cb6b54a2e": {"c4": 1.980, "c5": 2.314},
+    "8ae500aca2f084ae5fc3b99ea0c685586cd50b1d5093301ea8d51ce848eded44": {"c4": 1.979, "c5": 2.336},
 }
 
 
@@ -368,6 +368,7 @@ def ours_arm(args):
     roofline = {
         "bound": "hbm", "kernel": kname, "achieved": achieved, "peak": peak,
         "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,
+        "frac_of_nominal_8000": achieved / 8000.0,
         "traffic": (per_byte * rk_bytes / rk_launches) if per_byte and rk_launches else None,
         "algorithmic_bytes_per_launch": 2.0 * rk_bytes / rk_launches if rk_launches else 0,
         "avg_launch_ms": rk_ms / rk_launches if rk_launches else None,
