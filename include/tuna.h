@@ -47,7 +47,9 @@ typedef enum tuna_status {
   TUNA_ERR_WORKSPACE = -6,      /* workspace missing, misaligned or too small */
   TUNA_ERR_CUDA = -7,           /* a CUDA runtime call failed; see tuna_plan_cuda_error */
   TUNA_ERR_NOMEM = -8,          /* host or device allocation of the plan's tables failed */
-  TUNA_ERR_RANGE = -9           /* index (round, phase, ...) out of range, or size above a stated limit */
+  TUNA_ERR_RANGE = -9,          /* index (round, phase, ...) out of range, or size above a stated limit */
+  TUNA_ERR_INTERNAL = -10       /* the plan's self-check failed: a descriptor would leave its buffers;
+                                   nothing has been moved and the plan must not be used */
 } tuna_status;
 
 /* flags for tuna_plan_create */
@@ -90,6 +92,10 @@ typedef enum tuna_status {
  *                 defaults are computed on the device by the same scan kernel.
  *   stream        the plan kernels run on it; the call synchronises it once to read
  *                 back the phase totals that size the workspace.
+ * Before returning, a device-side self-check verifies that every descriptor of
+ * every list reads inside [0, send_bytes) or the workspace and writes inside
+ * [0, recv_bytes) or the workspace (TUNA_ERR_INTERNAL otherwise): the exchange
+ * kernels touch only those ranges, so no exchange can access memory out of bounds.
  */
 int tuna_plan_create(tuna_plan_t **out, int P, int radix, int radix_global, int l, int g,
                      int elem_size, unsigned flags, const int64_t *sendcounts,

@@ -33,7 +33,7 @@ TIMER_KINDS = len(TIMER_NAMES)
 STATUS = {
     0: "TUNA_OK", -1: "TUNA_ERR_INVALID_ARG", -2: "TUNA_ERR_BAD_RADIX",
     -3: "TUNA_ERR_BAD_HIERARCHY", -4: "TUNA_ERR_COUNT_MISMATCH", -5: "TUNA_ERR_OVERLAP",
-    -6: "TUNA_ERR_WORKSPACE", -7: "TUNA_ERR_CUDA", -8: "TUNA_ERR_NOMEM", -9: "TUNA_ERR_RANGE",
+    -6: "TUNA_ERR_WORKSPACE", -7: "TUNA_ERR_CUDA", -8: "TUNA_ERR_NOMEM", -9: "TUNA_ERR_RANGE", -10: "TUNA_ERR_INTERNAL",
 }
 
 # name -> (restype, argtypes); must list every symbol include/tuna.h declares

@@ -308,6 +308,36 @@ __global__ void tuna_chunk_index_kernel(const int64_t *__restrict__ pos, int64_t
   first[c] = (int32_t)(lo > 0 ? lo - 1 : 0);
 }
 
+// Self-check of a finished list: every descriptor must read inside its source
+// buffer and write inside its destination.  The movers touch no other bytes than
+// these ranges (plus the documented aligned over-read inside the source buffer),
+// so a clean check bounds every access of the exchange.  Violations are counted.
+__global__ void tuna_check_list_kernel(const int64_t *__restrict__ len, const int64_t *__restrict__ pos,
+                                       const int64_t *__restrict__ src, const int64_t *__restrict__ dst,
+                                       int64_t n, int64_t send_extent, int64_t recv_extent,
+                                       const int64_t *__restrict__ work_extent, int64_t keep_base_index,
+                                       const int64_t *__restrict__ wbase, unsigned long long *violations) {
+  const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= n) return;
+  const int64_t L = len[e];
+  bool bad = L < 0 || pos[e + 1] < pos[e];
+  if (L > 0) {
+    const int64_t s = src[e];
+    const int sb = TUNA_LOC_BUF(s);
+    const int64_t so = TUNA_LOC_OFF(s);
+    const int64_t sext = sb == TUNA_BUF_SEND ? send_extent : (sb == TUNA_BUF_WORK ? *work_extent : -1);
+    bad = bad || so < 0 || so + L > sext;
+    if (dst) {  // DELIVER: into the receive buffer
+      const int64_t d = dst[e];
+      bad = bad || TUNA_LOC_BUF(d) != TUNA_BUF_RECV || TUNA_LOC_OFF(d) + L > recv_extent;
+    } else {    // KEEP: at its stream position in the phase's workspace region
+      const int64_t o = wbase[keep_base_index] + pos[e];
+      bad = bad || (o & (TUNA_ALIGN - 1)) != 0 || o + pad16(L) > *work_extent || pos[e + 1] - pos[e] != pad16(L);
+    }
+  }
+  if (bad) atomicAdd(violations, 1ULL);
+}
+
 __global__ void tuna_transpose_kernel(const int64_t *__restrict__ in, int64_t *out, int P) {
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= (int64_t)P * P) return;
@@ -354,6 +384,7 @@ struct tuna_plan {
   unsigned long long *d_round_bytes = nullptr;
   int64_t stats_n = 0;
   int *d_error = nullptr;        // raised by a kernel whose bounded wait gave up
+  unsigned long long *d_violations = nullptr;  // descriptors that failed the plan's self-check
 
   std::vector<int64_t> h_wbase;  // workspace offset of every phase's KEEP stream
   int64_t workspace_need = 0;
@@ -724,6 +755,27 @@ int build_tables(tuna_plan *pl, const HostLayout &hl, const int64_t *counts, con
   rc = scan_list(pl, pl->dir, P, P, 2 * nph + 1, nullptr, 0, true, st);
   if (rc) return rc;
 
+  // self-check: every descriptor of every list stays inside its buffers
+  TUNA_CUDA(pl, cudaMemsetAsync(pl->d_violations, 0, sizeof(unsigned long long), st));
+  auto check = [&](const TunaList &l, int keep_phase) -> int {
+    if (l.n <= 0) return TUNA_OK;
+    tuna_check_list_kernel<<<(unsigned)((l.n + th - 1) / th), th, 0, st>>>(
+        l.len, l.pos, l.src, l.kind == TUNA_LIST_DELIVER ? l.dst : nullptr, l.n, pl->send_extent,
+        pl->recv_extent, pl->d_wbase + nph, keep_phase, pl->d_wbase, pl->d_violations);
+    TUNA_LAUNCHED(pl);
+    return TUNA_OK;
+  };
+  for (int f = 0; f < nph; f++) {
+    rc = check(pl->keep[f], f);
+    if (rc) return rc;
+    rc = check(pl->deliver[f], 0);
+    if (rc) return rc;
+  }
+  rc = check(pl->rot, 0);
+  if (rc) return rc;
+  rc = check(pl->dir, 0);
+  if (rc) return rc;
+
   plan_timer.stop();  // the chunk tables below are timed separately, after the read-back
   // one read-back: stream totals, workspace offsets, per-round bytes
   std::vector<int64_t> scal(2 * (2 * nph + 2)), wbase(nph + 1);
@@ -732,7 +784,10 @@ int build_tables(tuna_plan *pl, const HostLayout &hl, const int64_t *counts, con
   TUNA_CUDA(pl, cudaMemcpyAsync(wbase.data(), pl->d_wbase, wbase.size() * 8, cudaMemcpyDeviceToHost, st));
   TUNA_CUDA(pl, cudaMemcpyAsync(rbytes.data(), pl->d_round_bytes, rbytes.size() * 8,
                                 cudaMemcpyDeviceToHost, st));
+  unsigned long long violations = 0;
+  TUNA_CUDA(pl, cudaMemcpyAsync(&violations, pl->d_violations, sizeof(violations), cudaMemcpyDeviceToHost, st));
   TUNA_CUDA(pl, cudaStreamSynchronize(st));
+  if (violations != 0) return TUNA_ERR_INTERNAL;
   pl->h_wbase = wbase;
   auto take = [&](TunaList &l, int id) {
     l.total = scal[2 * id];
@@ -946,6 +1001,7 @@ const char *tuna_strerror(int status) {
     case TUNA_ERR_CUDA: return "CUDA runtime error";
     case TUNA_ERR_NOMEM: return "out of memory";
     case TUNA_ERR_RANGE: return "index or size out of range";
+    case TUNA_ERR_INTERNAL: return "the plan's self-check found a descriptor outside its buffers";
     default: return "unknown status";
   }
 }
@@ -973,6 +1029,7 @@ int tuna_plan_destroy(tuna_plan_t *pl) {
   cudaFree(pl->d_wbase);
   cudaFree(pl->d_round_bytes);
   cudaFree(pl->d_error);
+  cudaFree(pl->d_violations);
   for (auto &s : pl->stamps) {
     cudaEventDestroy(s.a);
     cudaEventDestroy(s.b);
@@ -1039,6 +1096,7 @@ int tuna_plan_create(tuna_plan_t **out, int P, int radix, int radix_global, int 
   TUNA_TRY(dev_alloc(&pl->d_wbase, nph + 1));
   TUNA_TRY(dev_alloc(&pl->d_round_bytes, pl->stats_n));
   TUNA_TRY(dev_alloc(&pl->d_error, 1));
+  TUNA_TRY(dev_alloc(&pl->d_violations, 1));
   TUNA_TRY(cudaMemset(pl->d_error, 0, sizeof(int)));
   pl->keep.resize(nph);
   pl->deliver.resize(nph);

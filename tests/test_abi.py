@@ -36,7 +36,7 @@ def test_every_declared_symbol_is_exported_and_bound(lib):
 
 def test_version_and_strerror(lib):
     assert lib.tuna_version() >= 100
-    for code in range(0, -10, -1):
+    for code in range(0, -11, -1):
         s = lib.tuna_strerror(code)
         assert s and s != b"unknown status"
     assert lib.tuna_strerror(-99) == b"unknown status"
