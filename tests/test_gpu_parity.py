@@ -483,3 +483,32 @@ def test_block_larger_than_4_gib():
         plan.destroy()
         del recv
         torch.cuda.empty_cache()
+
+
+def test_random_configurations():
+    """Seeded sweep over rank counts, groupings, radices, element sizes, sparsity,
+    layouts with gaps, buffer misalignment and both placement modes."""
+    rng = np.random.default_rng(20241102)
+    for case in range(90):
+        P = int(rng.integers(1, 49))
+        divs = [d for d in range(1, P + 1) if P % d == 0]
+        l = int(rng.choice(divs))
+        g = P // l
+        r = int(rng.integers(2, max(2, l) + 1))
+        rg = int(rng.integers(2, max(2, g) + 1))
+        elem = int(rng.choice([1, 2, 3, 4, 8]))
+        maxc = int(rng.choice([0, 1, 17, 300, 5000]))
+        wl = W.make_random(P, maxc, elem_size=elem, seed=1000 + case,
+                           zero_frac=float(rng.choice([0.0, 0.3, 0.9])), gaps=bool(rng.integers(0, 2)))
+        flags = int(rng.choice([0, B.FLAG_CLASSIC_ROTATE, B.FLAG_BULK_COPY]))
+        mis = int(rng.choice([0, 0, 1, 5, 8]))
+        ref = oracle_brute(wl)
+        got, plan = gpu_run(wl, r, l=l, g=g, rg=rg, flags=flags, misalign=mis,
+                            explicit=True)
+        assert np.array_equal(got, ref), (case, P, l, g, r, rg, elem, maxc, flags, mis)
+        assert plan.device_status() == 0
+        if g == 1:
+            _, rounds, _, _ = oracle_flat(wl, r)
+        else:
+            _, rounds, _, _ = oracle_hier(wl, l, g, r, rg)
+        check_rounds(plan, rounds)
