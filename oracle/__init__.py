@@ -66,6 +66,9 @@ def _load():
             lib.oracle_tuna_hier.argtypes = (
                 [ctypes.c_int] * 5 + [_I64P] * 5 + [_U8P, _U8P, ctypes.c_int64, _U8P, _I64P,
                                                     ctypes.c_int, _IP])
+            lib.oracle_tuna_hier_staggered.argtypes = (
+                [ctypes.c_int] * 5 + [_I64P] * 5 + [_U8P, _U8P, ctypes.c_int64, _U8P, _I64P,
+                                                    ctypes.c_int, _IP, _IP])
             _lib = lib
     return _lib
 
@@ -183,3 +186,26 @@ def tuna_hier(wl, Q: int, N: int, rl: int, rg: int, send: np.ndarray, recv: np.n
                                 rounds.ctypes.data_as(_I64P), K, Ks), "oracle_tuna_hier")
     assert Ks[0] + Ks[1] == K
     return recv, rounds[:K], (Ks[0], Ks[1]), after
+
+
+def tuna_hier_staggered(wl, Q: int, N: int, rl: int, block_count: int, send: np.ndarray,
+                        recv: np.ndarray):
+    """Local phase, then the staggered inter-group exchange in batches of ``block_count``
+    steps.  Returns (recv, rounds, (K_local, K_global), batches)."""
+    lib = _load()
+    assert Q * N == wl.P
+    c, cp = _i64(wl.sendcounts)
+    sd, sdp = _i64(wl.sdispls)
+    rd, rdp = _i64(wl.rdispls)
+    sb, sbp = _i64(wl.sendbase)
+    rb, rbp = _i64(wl.recvbase)
+    K = lib.oracle_round_list(Q, rl, None, None, 0) + Q * (N - 1)
+    rounds = np.zeros((max(K, 1), RS_COLS), dtype=np.int64)
+    Ks = (ctypes.c_int * 2)()
+    batches = ctypes.c_int(0)
+    _check(lib.oracle_tuna_hier_staggered(Q, N, rl, block_count, wl.elem_size, cp, sdp, rdp, sbp,
+                                          rbp, _u8(send), _u8(recv), recv.nbytes, None,
+                                          rounds.ctypes.data_as(_I64P), K, Ks,
+                                          ctypes.byref(batches)), "oracle_tuna_hier_staggered")
+    assert Ks[0] + Ks[1] == K
+    return recv, rounds[:K], (Ks[0], Ks[1]), batches.value

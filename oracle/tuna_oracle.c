@@ -23,6 +23,10 @@
  *                            phase is itself a TuNA of radix rg over
  *                            super-blocks (rg = N gives Algorithm 3's N-1
  *                            rounds of Q blocks each).
+ *   oracle_tuna_hier_staggered
+ *                          - Sec. IV-B and Algorithm 2: the same local phase, then
+ *                            the staggered inter-group exchange, one block per
+ *                            step, block_count steps posted per batch.
  *
  * Readings taken where the printed text is ambiguous (each pinned by a test):
  *   - direction: a rank sends to the rank at distance +z*r^x (Sec. III-A and the
@@ -40,6 +44,11 @@
  *   - the self block is copied S -> R and never sent; zero-length blocks keep a
  *     metadata entry and move no bytes.
  *   - blocks inside a message are in ascending offset order.
+ *   - Algorithm 2 prints several names for the same quantities; here gi = ii / Q,
+ *     gr = ii % Q, the partner groups are (n + gi) mod N for receiving and
+ *     (n - gi) mod N for sending (as printed: the mirror image of Algorithm 3's
+ *     direction), partner ranks keep the local id q, and block index
+ *     group * Q + gr names the block whose original owner has local id gr.
  *
  * All counts and displacements are in elements of elem bytes; rank p's send
  * region starts sendbase[p] elements into `send`, block (p -> d) sits
@@ -388,23 +397,25 @@ done:
  * `recv_after_local` (may be NULL) receives a copy of the receive buffer as it
  * stands after the local phase.  K_out[0] = local rounds, K_out[1] = global.
  */
-int oracle_tuna_hier(int Q, int N, int rl, int rg, int elem, const int64_t *counts,
-                     const int64_t *sdispls, const int64_t *rdispls, const int64_t *sendbase,
-                     const int64_t *recvbase, const uint8_t *send, uint8_t *recv,
-                     int64_t recv_bytes, uint8_t *recv_after_local, int64_t *rounds,
-                     int rounds_cap, int *K_out) {
-  if (Q < 1 || N < 1 || rl < 2 || rg < 2 || elem < 1) return ORACLE_EARG;
+static int hier_impl(int Q, int N, int rl, int rg, int block_count, int elem,
+                     const int64_t *counts, const int64_t *sdispls, const int64_t *rdispls,
+                     const int64_t *sendbase, const int64_t *recvbase, const uint8_t *send,
+                     uint8_t *recv, int64_t recv_bytes, uint8_t *recv_after_local,
+                     int64_t *rounds, int rounds_cap, int *K_out, int *batches_out) {
+  if (Q < 1 || N < 1 || rl < 2 || rg < 2 || elem < 1 || block_count < 0) return ORACLE_EARG;
   const int P = Q * N;
   int rc = ORACLE_OK;
   const int wl = oracle_num_digits(Q, rl), wg = oracle_num_digits(N, rg);
   const int Kl = oracle_round_list(Q, rl, NULL, NULL, 0);
-  const int Kg = oracle_round_list(N, rg, NULL, NULL, 0);
-  const int Bg = N - (Kg + 1);
+  const int Kg = block_count > 0 ? Q * (N - 1) : oracle_round_list(N, rg, NULL, NULL, 0);
+  const int Bg = block_count > 0 ? 0 : N - (Kg + 1);
   if (Bg < 0) return ORACLE_ESCHED;
   if (K_out) {
     K_out[0] = Kl;
     K_out[1] = Kg;
   }
+  slot_t *box = NULL;     /* staggered exchange: blocks in flight within a batch */
+  int64_t *boxlen = NULL; /* and their sizes */
 
   /* local phase state: slot (i, jo) of rank (n, q) names the block for rank
      (i, (q + jo) % Q); sz holds its current size, L its bytes once it has moved */
@@ -517,6 +528,83 @@ int oracle_tuna_hier(int Q, int N, int rl, int rg, int elem, const int64_t *coun
     goto done;
   }
   if (recv_after_local) memcpy(recv_after_local, recv, (size_t)recv_bytes);
+
+  if (block_count > 0) {
+    /* Algorithm 2, the staggered inter-group exchange.  A step index ii runs
+       over [0, P) in batches of block_count; step ii stands for the pair
+       gi = ii / Q (group distance) and gr = ii % Q (local id of the block's
+       original owner).  In step (gi, gr) with gi >= 1, rank (n, q) sends the
+       single block that came from rank (n, gr) and is meant for rank
+       ((n - gi) mod N, q) to that rank, and receives from rank
+       ((n + gi) mod N, q) the block that came from ((n + gi) mod N, gr).  Steps
+       with gi = 0 name the rank's own group and do nothing.  The receiver knows
+       the size from its receive counts, so no metadata travels and nothing is
+       compacted.  Within a batch every receive and send is posted before any
+       completes: all ranks hand their blocks over, then all take delivery. */
+    int batches = 0;
+    box = (slot_t *)calloc((size_t)P * block_count, sizeof(slot_t));
+    boxlen = (int64_t *)calloc((size_t)P * block_count, sizeof(int64_t));
+    if (!box || !boxlen) {
+      rc = ORACLE_ENOMEM;
+      goto done;
+    }
+    for (int r0 = 0; r0 < Kg && rounds && Kl + r0 < rounds_cap; r0++) {
+      int64_t *row = rounds + (int64_t)(Kl + r0) * RS_COLS;
+      row[RS_LEVEL] = 1;
+      row[RS_X] = 1 + r0 / Q;
+      row[RS_Z] = r0 % Q;
+      row[RS_UNITS] = 0;
+      row[RS_BYTES_SENT] = 0;
+      row[RS_BYTES_RECV] = 0;
+    }
+    for (int ii = 0; ii < P; ii += block_count) {
+      int active = 0;
+      for (int p = 0; p < P; p++) {
+        int n = p / Q, q = p % Q;
+        for (int i = 0; i < block_count && ii + i < P; i++) {
+          int gi = (ii + i) / Q, gr = (ii + i) % Q;
+          int ndst = ((n - gi) % N + N) % N;
+          if (ndst == n) continue;
+          active = 1;
+          int jo = ((q - gr) % Q + Q) % Q;
+          int64_t nb = sz[(int64_t)p * P + ndst * Q + jo];
+          const uint8_t *src = (jo == 0)
+                                   ? send + (sendbase[p] + sdispls[(int64_t)p * P + ndst * Q + q]) * elem
+                                   : L[(int64_t)p * P + ndst * Q + jo].ptr;
+          rc = slot_put(&box[(int64_t)p * block_count + i], src, nb);
+          if (rc) goto done;
+          boxlen[(int64_t)p * block_count + i] = nb;
+          if (rounds && Kl + (gi - 1) * Q + gr < rounds_cap) {
+            int64_t *row = rounds + (int64_t)(Kl + (gi - 1) * Q + gr) * RS_COLS;
+            row[RS_UNITS] += 1;
+            row[RS_BYTES_SENT] += nb;
+          }
+        }
+      }
+      for (int p = 0; p < P; p++) {
+        int n = p / Q, q = p % Q;
+        for (int i = 0; i < block_count && ii + i < P; i++) {
+          int gi = (ii + i) / Q, gr = (ii + i) % Q;
+          int nsrc = (n + gi) % N;
+          if (nsrc == n) continue;
+          const slot_t *b = &box[(int64_t)(nsrc * Q + q) * block_count + i];
+          int64_t want = counts[(int64_t)(nsrc * Q + gr) * P + p] * elem;
+          if (boxlen[(int64_t)(nsrc * Q + q) * block_count + i] != want) {
+            rc = ORACLE_ESCHED;
+            goto done;
+          }
+          if (want > 0)
+            memcpy(recv + (recvbase[p] + rdispls[(int64_t)p * P + nsrc * Q + gr]) * elem, b->ptr,
+                   (size_t)want);
+          if (rounds && Kl + (gi - 1) * Q + gr < rounds_cap)
+            rounds[(int64_t)(Kl + (gi - 1) * Q + gr) * RS_COLS + RS_BYTES_RECV] += want;
+        }
+      }
+      batches += active;
+    }
+    if (batches_out) *batches_out = batches;
+    goto done;
+  }
 
   /* compaction: rank (n, q) gathers, for every other group i, the Q blocks
      (n, q') -> (i, q) in ascending q' into one contiguous super-block */
@@ -660,6 +748,10 @@ done:
   if (msg)
     for (int p = 0; p < P; p++) msg_free(&msg[p]);
   free(msg);
+  if (box)
+    for (int64_t i = 0; i < (int64_t)P * block_count; i++) free(box[i].ptr);
+  free(box);
+  free(boxlen);
   if (L)
     for (int64_t i = 0; i < (int64_t)P * P; i++) free(L[i].ptr);
   free(L);
@@ -672,4 +764,31 @@ done:
   free(usz);
   free(sz);
   return rc;
+}
+
+int oracle_tuna_hier(int Q, int N, int rl, int rg, int elem, const int64_t *counts,
+                     const int64_t *sdispls, const int64_t *rdispls, const int64_t *sendbase,
+                     const int64_t *recvbase, const uint8_t *send, uint8_t *recv,
+                     int64_t recv_bytes, uint8_t *recv_after_local, int64_t *rounds,
+                     int rounds_cap, int *K_out) {
+  return hier_impl(Q, N, rl, rg, 0, elem, counts, sdispls, rdispls, sendbase, recvbase, send, recv,
+                   recv_bytes, recv_after_local, rounds, rounds_cap, K_out, NULL);
+}
+
+/*
+ * Sec. IV-B and Algorithm 2: the local phase of Algorithm 3 followed by the
+ * staggered inter-group exchange, one block per step, block_count steps per
+ * batch.  K_out[1] = Q*(N-1) steps; *batches_out = batches that move anything.
+ * Round rows of the global level carry RS_X = gi and RS_Z = gr.
+ */
+int oracle_tuna_hier_staggered(int Q, int N, int rl, int block_count, int elem,
+                               const int64_t *counts, const int64_t *sdispls,
+                               const int64_t *rdispls, const int64_t *sendbase,
+                               const int64_t *recvbase, const uint8_t *send, uint8_t *recv,
+                               int64_t recv_bytes, uint8_t *recv_after_local, int64_t *rounds,
+                               int rounds_cap, int *K_out, int *batches_out) {
+  if (block_count < 1) return ORACLE_EARG;
+  return hier_impl(Q, N, rl, 2, block_count, elem, counts, sdispls, rdispls, sendbase, recvbase,
+                   send, recv, recv_bytes, recv_after_local, rounds, rounds_cap, K_out,
+                   batches_out);
 }

@@ -34,6 +34,15 @@ MUTATIONS = [
      "int from = (int)(((n - dist) % N + N) % N) * Q + q;", "int from = (int)((n + dist) % N) * Q + q;"),
     ("hier_own_group_blocks_kept_in_T",
      "if (local_final && i == n) {", "if (0) {"),
+    ("staggered_sends_the_wrong_way",
+     "          int ndst = ((n - gi) % N + N) % N;\n          if (ndst == n) continue;\n          active = 1;",
+     "          int ndst = (n + gi) % N;\n          if (ndst == n) continue;\n          active = 1;"),
+    ("staggered_mirrored_both_ways",     # consistent, but not the direction Algorithm 2 prints
+     ("int ndst = ((n - gi) % N + N) % N;", "int nsrc = (n + gi) % N;"),
+     ("int ndst = (n + gi) % N;", "int nsrc = ((n - gi) % N + N) % N;")),
+    ("staggered_owner_index_is_receiver",
+     "          int jo = ((q - gr) % Q + Q) % Q;\n          int64_t nb = sz[(int64_t)p * P + ndst * Q + jo];",
+     "          int jo = gr;\n          int64_t nb = sz[(int64_t)p * P + ndst * Q + jo];"),
     ("scan_inclusive",
      "      out[s * seglen + i] = run;\n      run += v;", "      run += v;\n      out[s * seglen + i] = run;"),
     ("dropped_self_block",
@@ -45,9 +54,12 @@ MUTATIONS = [
 @pytest.mark.parametrize("name,old,new", MUTATIONS, ids=[m[0] for m in MUTATIONS])
 def test_pins_catch_a_planted_mistake(tmp_path, name, old, new):
     text = open(SRC).read()
-    assert text.count(old) >= 1, f"mutation {name} no longer applies: update it"
+    olds, news = (old, new) if isinstance(old, tuple) else ((old,), (new,))
+    for o, n in zip(olds, news):
+        assert text.count(o) >= 1, f"mutation {name} no longer applies: update it"
+        text = text.replace(o, n, 1)
     mutated = tmp_path / "tuna_oracle_mutated.c"
-    mutated.write_text(text.replace(old, new, 1))
+    mutated.write_text(text)
     env = dict(os.environ, TUNA_ORACLE_SOURCE=str(mutated))
     r = subprocess.run([sys.executable, "-m", "pytest", os.path.join(ROOT, "tests", "test_oracle_pins.py"),
                         "-x", "-q", "-p", "no:cacheprovider"], cwd=ROOT, env=env, capture_output=True,

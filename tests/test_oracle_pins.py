@@ -334,6 +334,65 @@ def test_hier_equals_definition_and_conserves_bytes(Q, N, rl, rg):
         assert row[oracle.RS_BYTES_SENT] == tot
 
 
+# ---------------------------------------------------------------- staggered (Algorithm 2)
+
+def run_staggered(wl, Q, N, rl, bc):
+    send = wl.make_send().numpy()
+    recv = wl.make_recv(fill=CANARY).numpy().copy()
+    return oracle.tuna_hier_staggered(wl, Q, N, rl, bc, send, recv)
+
+
+STAGGERED_CASES = [(Q, N, rl, bc) for Q, N in [(1, 1), (1, 5), (5, 1), (2, 2), (3, 4), (4, 3), (6, 5)]
+                   for rl in sorted({2, max(2, Q)})
+                   for bc in sorted({1, 2, Q, Q + 1, Q * N, 3 * Q * N})]
+
+
+@pytest.mark.parametrize("Q,N,rl,bc", STAGGERED_CASES)
+def test_staggered_equals_definition(Q, N, rl, bc):
+    """Sec. IV-B (figure of the two inter-node patterns): the staggered exchange takes
+    (N - 1) * Q steps of one block per rank where the coalesced one takes N - 1 of Q
+    blocks; both end in the MPI_Alltoallv result."""
+    P = Q * N
+    wl = W.make_random(P, 23, elem_size=3, seed=11 * P + rl + bc, zero_frac=0.25, gaps=True)
+    recv, rounds, (Kl, Kg), batches = run_staggered(wl, Q, N, rl, bc)
+    assert np.array_equal(recv, brute(wl))
+    assert Kl == closed_form_K(Q, rl) and Kg == (N - 1) * Q
+    # batches of block_count consecutive step indices ii in [0, P); the first Q
+    # indices name the own group and move nothing
+    want_batches = sum(1 for lo in range(0, P, bc) if min(P, lo + bc) > Q)
+    assert batches == want_batches
+    gl = rounds[rounds[:, oracle.RS_LEVEL] == 1]
+    assert len(gl) == Kg
+    assert np.all(gl[:, oracle.RS_UNITS] == P)           # one block per rank per step
+    assert np.all(gl[:, oracle.RS_BYTES_SENT] == gl[:, oracle.RS_BYTES_RECV])
+    # step (gi, gr): every rank (n, q) receives the block that rank ((n + gi) mod N, gr)
+    # owns for it
+    C = wl.sendcounts * wl.elem_size
+    for row in gl:
+        gi, gr = int(row[oracle.RS_X]), int(row[oracle.RS_Z])
+        tot = sum(int(C[((n + gi) % N) * Q + gr, n * Q + q]) for n in range(N) for q in range(Q))
+        assert row[oracle.RS_BYTES_SENT] == tot
+    assert [(int(a), int(b)) for a, b in gl[:, [oracle.RS_X, oracle.RS_Z]]] == \
+        [(gi, gr) for gi in range(1, N) for gr in range(Q)]
+
+
+@pytest.mark.parametrize("Q,N", [(3, 4), (4, 3), (2, 5)])
+def test_staggered_steps_add_up_to_coalesced_rounds(Q, N):
+    """The Q steps of group distance gi carry what one coalesced round carries: the
+    super-blocks between groups gi apart.  Algorithm 2 sends towards (n - gi),
+    Algorithm 3 towards (n + z), so distance gi matches round z = N - gi."""
+    P = Q * N
+    wl = W.make_random(P, 31, elem_size=1, seed=77 + P, zero_frac=0.1)
+    _, rs, (Kl, _), _ = run_staggered(wl, Q, N, 2, 1)
+    _, rc, (Kl2, Kg2), _ = run_hier(wl, Q, N, 2, N)
+    assert Kl == Kl2 and Kg2 == N - 1
+    assert np.array_equal(rs[:Kl], rc[:Kl])              # same local phase
+    co = {int(r[oracle.RS_Z]): int(r[oracle.RS_BYTES_SENT]) for r in rc[Kl:]}
+    for gi in range(1, N):
+        steps = rs[Kl:][rs[Kl:, oracle.RS_X] == gi]
+        assert steps[:, oracle.RS_BYTES_SENT].sum() == co[N - gi]
+
+
 @pytest.mark.parametrize("P,r", [(6, 2), (9, 3), (16, 4), (13, 2)])
 def test_hier_reduces_to_flat(P, r):
     """One group (N = 1) is the flat exchange over Q = P ranks; one rank per
