@@ -308,8 +308,9 @@ def ours_arm(args):
     recv = wl.make_recv(dev)
     payload = wl.payload_bytes_total
 
-    def make_plan(r, l=None, g=1, rg=2, flags=0):
-        return B.plan_for(wl, r, l=l, g=g, radix_global=rg, flags=flags, explicit_layout=False)
+    def make_plan(r, l=None, g=1, rg=2, flags=0, block_count=0):
+        return B.plan_for(wl, r, l=l, g=g, radix_global=rg, flags=flags, explicit_layout=False,
+                          block_count=block_count)
 
     if hier_headline:
         l, g = wl.hier
@@ -451,6 +452,11 @@ def ours_arm(args):
             l, g = wl.hier
             for rl, rg in wl.hier_radices:
                 entry(f"hier {l}x{g} r={rl}/{rg}", make_plan(rl, l=l, g=g, rg=rg))
+            # staggered inter-group exchange: one block per step, block_count steps per launch
+            rl = max(a for a, _ in wl.hier_radices)
+            for bc in (1, l, wl.P):
+                entry(f"hier {l}x{g} r={rl} staggered block_count={bc}",
+                      make_plan(rl, l=l, g=g, block_count=bc))
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

@@ -103,6 +103,35 @@ int tuna_plan_create(tuna_plan_t **out, int P, int radix, int radix_global, int 
                      const int64_t *recvbase, void *stream);
 
 /*
+ * tuna_plan_create_staggered - hierarchical plan whose inter-group phase is the
+ * staggered exchange.
+ *
+ * Computes: the local phase of tuna_plan_create (Sec. IV-A), then Sec. IV-B's
+ * staggered pattern as Algorithm 2 states it: a step index ii = gi*l + gr runs over
+ * [0, P) in batches of `block_count`; in step (gi, gr), gi >= 1, rank (n, q) sends
+ * the single block whose original owner is rank (n, gr) to rank ((n - gi) mod g, q)
+ * and receives from rank ((n + gi) mod g, q) the block owned by ((n + gi) mod g, gr),
+ * straight into the receive buffer.  Nothing is compacted into super-blocks.  The
+ * steps of one batch share one kernel launch (the counterpart of the requests that
+ * are in flight together), so the exchange takes one launch per local digit phase
+ * plus one per batch that moves anything; block_count >= P gives a single batch.
+ *
+ *   block_count   steps per batch, >= 1.
+ *   radix         local radix in [2, max(2, l)].
+ *   flags         TUNA_FLAG_CLASSIC_ROTATE is not supported here (TUNA_ERR_INVALID_ARG).
+ * All other arguments, ownership and errors as tuna_plan_create.  Every function
+ * taking a plan accepts this one.  Its rounds of level 1 are the l*(g-1) steps in
+ * order, reported by tuna_plan_round_info with x = gi, z = gr and units = P (one
+ * block per rank); its phases of level 1 are the batches (x = batch number), each
+ * with an empty KEEP list and a DELIVER list of P rows, one per receiving rank,
+ * holding the batch's steps in ascending ii.
+ */
+int tuna_plan_create_staggered(tuna_plan_t **out, int P, int radix, int block_count, int l, int g,
+                               int elem_size, unsigned flags, const int64_t *sendcounts,
+                               const int64_t *sdispls, const int64_t *rdispls,
+                               const int64_t *sendbase, const int64_t *recvbase, void *stream);
+
+/*
  * tuna_plan_update_counts - same plan shape, new counts (e.g. routing that changes
  * every step): re-runs the metadata exchange and the prefix sums on the device.
  * Arguments as in tuna_plan_create.  Synchronises `stream` once.  The required

@@ -40,6 +40,8 @@ STATUS = {
 SIGNATURES = {
     "tuna_plan_create": (ctypes.c_int, [ctypes.POINTER(_VP)] + [ctypes.c_int] * 6 + [ctypes.c_uint]
                          + [_I64P] * 5 + [_VP]),
+    "tuna_plan_create_staggered": (ctypes.c_int, [ctypes.POINTER(_VP)] + [ctypes.c_int] * 6
+                                   + [ctypes.c_uint] + [_I64P] * 5 + [_VP]),
     "tuna_plan_update_counts": (ctypes.c_int, [_VP] + [_I64P] * 5 + [_VP]),
     "tuna_plan_destroy": (ctypes.c_int, [_VP]),
     "tuna_plan_workspace_bytes": (ctypes.c_int, [_VP, _SZP]),
@@ -127,16 +129,24 @@ class Plan:
 
     def __init__(self, P, radix, l=None, g=1, radix_global=2, elem_size=1, flags=0,
                  sendcounts=None, sdispls=None, rdispls=None, sendbase=None, recvbase=None,
-                 stream=None):
+                 stream=None, block_count=0):
+        """``block_count`` > 0 selects ``tuna_plan_create_staggered`` (``radix_global`` unused)."""
         self._h = _VP()
         self._ws = None
         l = P if l is None else l
         keep = [_h(x) for x in (sendcounts, sdispls, rdispls, sendbase, recvbase)]
-        rc = lib().tuna_plan_create(ctypes.byref(self._h), P, radix, radix_global, l, g, elem_size,
-                                    flags, *[k[1] for k in keep], _stream(stream))
+        if block_count:
+            what = "tuna_plan_create_staggered"
+            rc = lib().tuna_plan_create_staggered(ctypes.byref(self._h), P, radix, block_count, l, g,
+                                                  elem_size, flags, *[k[1] for k in keep],
+                                                  _stream(stream))
+        else:
+            what = "tuna_plan_create"
+            rc = lib().tuna_plan_create(ctypes.byref(self._h), P, radix, radix_global, l, g,
+                                        elem_size, flags, *[k[1] for k in keep], _stream(stream))
         if rc != 0:
             self._h = _VP()
-            raise TunaError(rc, "tuna_plan_create")
+            raise TunaError(rc, what)
         self.P, self.elem_size = P, elem_size
 
     def _check(self, rc, what):
@@ -294,10 +304,11 @@ def direct_alltoallv_static(P, elem_size, sendcounts, sendbuf, recvbuf, sdispls=
         raise TunaError(rc, "tuna_direct_alltoallv_static")
 
 
-def plan_for(wl, radix, l=None, g=1, radix_global=2, flags=0, explicit_layout=True, stream=None) -> Plan:
+def plan_for(wl, radix, l=None, g=1, radix_global=2, flags=0, explicit_layout=True, stream=None,
+             block_count=0) -> Plan:
     """A plan for a :class:`workloads.Workload`."""
     kw = dict(sendcounts=wl.sendcounts)
     if explicit_layout:
         kw.update(sdispls=wl.sdispls, rdispls=wl.rdispls, sendbase=wl.sendbase, recvbase=wl.recvbase)
     return Plan(wl.P, radix, l=l, g=g, radix_global=radix_global, elem_size=wl.elem_size,
-                flags=flags, stream=stream, **kw)
+                flags=flags, stream=stream, block_count=block_count, **kw)

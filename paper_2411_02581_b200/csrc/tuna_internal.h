@@ -39,6 +39,10 @@ struct TunaPhase {
   int64_t per_rank;  // blocks a rank receives in this phase
   int64_t finals;    // the first `finals` of them (in slot order) have arrived and are delivered
   int64_t stats_off; // first of `radix` counters in the stats array
+  // Staggered inter-group exchange: this "phase" is one batch of steps [stag_lo,
+  // stag_hi) of the step index ii = gi*Q + gr; every block it moves has arrived.
+  // stag_hi == 0 for an ordinary digit phase.
+  int stag_lo, stag_hi;
 };
 
 // How a list's stream positions are spaced.

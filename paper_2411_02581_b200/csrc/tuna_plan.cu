@@ -144,6 +144,37 @@ __global__ void tuna_meta_exchange_kernel(TunaTopo t, PhaseDev ph, const int64_t
   }
 }
 
+// Staggered inter-group exchange (Sec. IV-B, Algorithm 2), one batch: the steps
+// ii in [lo, hi) of the index ii = gi*Q + gr, gi >= 1.  In step (gi, gr) rank
+// (n, q) receives, from rank ((n + gi) mod N, q), the one block whose original
+// owner is ((n + gi) mod N, gr).  Every such block has arrived: descriptor
+// e = p*(hi - lo) + (ii - lo) of the batch's DELIVER list gets its size, where the
+// sender keeps it, and its place in the receive buffer.  step_bytes[ii] sums the
+// bytes of step ii over all ranks.
+__global__ void tuna_stagger_batch_kernel(TunaTopo t, int lo, int hi,
+                                          const int64_t *__restrict__ sz_cur,
+                                          const int64_t *__restrict__ loc_cur,
+                                          const int64_t *__restrict__ rdispls,
+                                          const int64_t *__restrict__ recvbase, int64_t *del_len,
+                                          int64_t *del_src, int64_t *del_dst,
+                                          unsigned long long *step_bytes) {
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int m = hi - lo;
+  if (idx >= (int64_t)t.P * m) return;
+  const int p = (int)(idx / m), ii = lo + (int)(idx % m);
+  const int n = p / t.Q, q = p % t.Q, gi = ii / t.Q, gr = ii % t.Q;
+  const int nsrc = (n + gi) % t.N;
+  const int sender = nsrc * t.Q + q, origin = nsrc * t.Q + gr;
+  // the slot of that block, in offset coordinates: group offset from its owner's
+  // group to this one, local offset from its owner to this rank
+  const int sigma = ((t.N - gi) % t.N) * t.Q + (q - gr + t.Q) % t.Q;
+  const int64_t bytes = sz_cur[(int64_t)sender * t.P + sigma];
+  del_len[idx] = bytes;
+  del_src[idx] = loc_cur[(int64_t)sender * t.P + sigma];
+  del_dst[idx] = TUNA_LOC(TUNA_BUF_RECV, (recvbase[p] + rdispls[(int64_t)p * t.P + origin]) * t.elem);
+  if (bytes > 0) atomicAdd(&step_bytes[ii], (unsigned long long)bytes);
+}
+
 // Segmented exclusive prefix sum, one warp per segment, warp-shuffle scan over
 // 32-wide tiles with a running carry.  MODE 0 sums the values as they are; MODE 1
 // (KEEP lists) rounds every value up to 16 first; MODE 2 (DELIVER lists) also
@@ -352,6 +383,7 @@ __global__ void tuna_transpose_kernel(const int64_t *__restrict__ in, int64_t *o
 struct tuna_plan {
   TunaTopo topo{};
   int radix_l = 2, radix_g = 2;
+  int block_count = 0;  // > 0: staggered inter-group exchange in batches of this many steps
   unsigned flags = 0;
   bool classic = false;
   int cuda_err = 0;
@@ -365,6 +397,7 @@ struct tuna_plan {
   struct Round {
     int level, x, z, phase;
     int64_t units, bytes;
+    int64_t stat;  // index of its byte counter in the stats array
   };
   std::vector<Round> rounds;
 
@@ -731,6 +764,18 @@ int build_tables(tuna_plan *pl, const HostLayout &hl, const int64_t *counts, con
     const TunaPhase &ph = pl->phases[f];
     TunaList &k = pl->keep[f];
     TunaList &d = pl->deliver[f];
+    if (ph.stag_hi > 0) {  // a batch of the staggered exchange: every block arrives
+      const int64_t nd = (int64_t)P * (ph.stag_hi - ph.stag_lo);
+      tuna_stagger_batch_kernel<<<(unsigned)((nd + th - 1) / th), th, 0, st>>>(
+          t, ph.stag_lo, ph.stag_hi, pl->d_sz[cur], pl->d_loc[cur], pl->d_rdispls, pl->d_recvbase,
+          d.len, d.src, d.dst, pl->d_round_bytes + ph.stats_off);
+      TUNA_LAUNCHED(pl);
+      rc = scan_list(pl, k, 0, P, f, pl->d_wbase + f, 1, false, st, 0);
+      if (rc) return rc;
+      rc = scan_list(pl, d, ph.finals, P, nph + f, nullptr, 0, true, st, 1);
+      if (rc) return rc;
+      continue;
+    }
     PhaseDev pd{ph.level, ph.radix, ph.count, ph.stride, ph.moving, ph.per_rank, ph.finals};
     const size_t smem = ph.radix <= 4096 ? (size_t)ph.radix * 8 : 0;
     tuna_meta_exchange_kernel<<<gPP, th, smem, st>>>(t, pd, pl->d_sz[cur], pl->d_loc[cur],
@@ -800,7 +845,7 @@ int build_tables(tuna_plan *pl, const HostLayout &hl, const int64_t *counts, con
   take(pl->rot, 2 * nph);
   take(pl->dir, 2 * nph + 1);
   pl->workspace_need = wbase[nph];
-  for (auto &r : pl->rounds) r.bytes = (int64_t)rbytes[pl->phases[r.phase].stats_off + r.z];
+  for (auto &r : pl->rounds) r.bytes = (int64_t)rbytes[r.stat];
 
   Timed chunk_timer(pl, TUNA_TIMER_PLAN, 0, st);
   for (int f = 0; f < nph; f++) {
@@ -843,8 +888,45 @@ void add_level(tuna_plan *pl, int level, int count, int radix, int other) {
       r.x = x;
       r.z = z;
       r.phase = phase;
+      r.stat = ph.stats_off + z;
       // level 0 counts blocks, level 1 super-blocks (Q blocks each)
       r.units = (int64_t)pl->topo.P * count_digit(count, radix, x, z) * (level == 0 ? other : 1);
+      pl->rounds.push_back(r);
+    }
+  }
+}
+
+// Staggered inter-group exchange (Algorithm 2): the step index ii = gi*Q + gr runs
+// over [0, P) in batches of block_count; the first Q indices (gi = 0) name the own
+// group and move nothing.  Every batch that moves something becomes one launch.
+void add_staggered(tuna_plan *pl, int block_count) {
+  const int P = pl->topo.P, Q = pl->topo.Q, N = pl->topo.N;
+  const int64_t stats_off = pl->stats_n;
+  pl->stats_n += P;
+  int batch = 0;
+  for (int64_t lo0 = 0; lo0 < P; lo0 += block_count) {
+    const int lo = (int)std::max<int64_t>(lo0, Q), hi = (int)std::min<int64_t>(P, lo0 + block_count);
+    if (hi <= lo) continue;
+    TunaPhase ph{};
+    ph.level = 1;
+    ph.x = batch++;
+    ph.radix = N;
+    ph.count = N;
+    ph.stride = 1;
+    ph.moving = ph.per_rank = ph.finals = hi - lo;
+    ph.stats_off = stats_off;
+    ph.stag_lo = lo;
+    ph.stag_hi = hi;
+    const int phase = (int)pl->phases.size();
+    pl->phases.push_back(ph);
+    for (int ii = lo; ii < hi; ii++) {
+      tuna_plan::Round r{};
+      r.level = 1;
+      r.x = ii / Q;  // gi
+      r.z = ii % Q;  // gr
+      r.phase = phase;
+      r.stat = stats_off + ii;
+      r.units = P;   // one block per rank
       pl->rounds.push_back(r);
     }
   }
@@ -1039,16 +1121,19 @@ int tuna_plan_destroy(tuna_plan_t *pl) {
   return TUNA_OK;
 }
 
-int tuna_plan_create(tuna_plan_t **out, int P, int radix, int radix_global, int l, int g,
-                     int elem_size, unsigned flags, const int64_t *sendcounts,
-                     const int64_t *sdispls, const int64_t *rdispls, const int64_t *sendbase,
-                     const int64_t *recvbase, void *stream) {
+static int plan_create(tuna_plan_t **out, int P, int radix, int radix_global, int block_count,
+                       int l, int g, int elem_size, unsigned flags, const int64_t *sendcounts,
+                       const int64_t *sdispls, const int64_t *rdispls, const int64_t *sendbase,
+                       const int64_t *recvbase, void *stream) {
   if (!out) return TUNA_ERR_INVALID_ARG;
   *out = nullptr;
   if (P < 1 || P > 32768 || elem_size < 1 || !sendcounts || l < 1 || g < 1) return TUNA_ERR_INVALID_ARG;
   if ((int64_t)l * g != P) return TUNA_ERR_BAD_HIERARCHY;
   if (radix < 2 || radix > std::max(2, l)) return TUNA_ERR_BAD_RADIX;
-  if (g > 1 && (radix_global < 2 || radix_global > std::max(2, g))) return TUNA_ERR_BAD_RADIX;
+  if (block_count == 0 && g > 1 && (radix_global < 2 || radix_global > std::max(2, g)))
+    return TUNA_ERR_BAD_RADIX;
+  if (block_count < 0 || (block_count > 0 && (flags & TUNA_FLAG_CLASSIC_ROTATE)))
+    return TUNA_ERR_INVALID_ARG;
   HostLayout hl;
   int rc = host_layout(P, sendcounts, sdispls, rdispls, sendbase, recvbase, &hl);
   if (rc) return rc;
@@ -1057,11 +1142,15 @@ int tuna_plan_create(tuna_plan_t **out, int P, int radix, int radix_global, int 
   if (!pl) return TUNA_ERR_NOMEM;
   pl->topo = TunaTopo{P, l, g, elem_size};
   pl->radix_l = radix;
-  pl->radix_g = g > 1 ? radix_global : 2;
+  pl->radix_g = (g > 1 && block_count == 0) ? radix_global : 2;
+  pl->block_count = block_count;
   pl->flags = flags;
   pl->classic = (flags & TUNA_FLAG_CLASSIC_ROTATE) != 0;
   add_level(pl, 0, l, radix, g);
-  if (g > 1) add_level(pl, 1, g, pl->radix_g, l);
+  if (g > 1 && block_count > 0)
+    add_staggered(pl, block_count);
+  else if (g > 1)
+    add_level(pl, 1, g, pl->radix_g, l);
 
   const int64_t PP = (int64_t)P * P;
   const int nph = (int)pl->phases.size();
@@ -1119,6 +1208,26 @@ int tuna_plan_create(tuna_plan_t **out, int P, int radix, int radix_global, int 
   if (rc) return fail(rc);
   *out = pl;
   return TUNA_OK;
+}
+
+int tuna_plan_create(tuna_plan_t **out, int P, int radix, int radix_global, int l, int g,
+                     int elem_size, unsigned flags, const int64_t *sendcounts,
+                     const int64_t *sdispls, const int64_t *rdispls, const int64_t *sendbase,
+                     const int64_t *recvbase, void *stream) {
+  return plan_create(out, P, radix, radix_global, 0, l, g, elem_size, flags, sendcounts, sdispls,
+                     rdispls, sendbase, recvbase, stream);
+}
+
+int tuna_plan_create_staggered(tuna_plan_t **out, int P, int radix, int block_count, int l, int g,
+                               int elem_size, unsigned flags, const int64_t *sendcounts,
+                               const int64_t *sdispls, const int64_t *rdispls,
+                               const int64_t *sendbase, const int64_t *recvbase, void *stream) {
+  if (block_count < 1) {
+    if (out) *out = nullptr;
+    return TUNA_ERR_INVALID_ARG;
+  }
+  return plan_create(out, P, radix, 2, block_count, l, g, elem_size, flags, sendcounts, sdispls,
+                     rdispls, sendbase, recvbase, stream);
 }
 
 int tuna_plan_update_counts(tuna_plan_t *pl, const int64_t *sendcounts, const int64_t *sdispls,

@@ -33,7 +33,7 @@ def oracle_brute(wl):
 
 
 def gpu_run(wl, radix, l=None, g=1, rg=2, flags=0, direct=False, explicit=True, pass_args=True,
-            misalign=0):
+            misalign=0, block_count=0):
     """Run the exchange on the GPU; returns (recv bytes as numpy, plan).
     ``misalign`` shifts both device buffers by that many bytes off 256-byte alignment."""
     send0 = wl.make_send("cuda")
@@ -46,7 +46,8 @@ def gpu_run(wl, radix, l=None, g=1, rg=2, flags=0, direct=False, explicit=True, 
         recv = rbuf[misalign:misalign + recv0.numel()]
     else:
         send, recv = send0, recv0
-    plan = B.plan_for(wl, radix, l=l, g=g, radix_global=rg, flags=flags, explicit_layout=explicit)
+    plan = B.plan_for(wl, radix, l=l, g=g, radix_global=rg, flags=flags, explicit_layout=explicit,
+                      block_count=block_count)
     plan.alloc_workspace()
     args = {}
     if pass_args and explicit:
@@ -512,3 +513,63 @@ def test_random_configurations():
         else:
             _, rounds, _, _ = oracle_hier(wl, l, g, r, rg)
         check_rounds(plan, rounds)
+
+
+# ---------------------------------------------------------------- staggered inter-group exchange
+
+def oracle_staggered(wl, Q, N, rl, bc):
+    send = wl.make_send().numpy()
+    recv = wl.make_recv(fill=CANARY).numpy().copy()
+    return oracle.tuna_hier_staggered(wl, Q, N, rl, bc, send, recv)
+
+
+STAGGERED = [(Q, N, rl, bc) for Q, N in [(1, 5), (5, 1), (2, 2), (3, 4), (4, 3), (8, 4), (16, 16)]
+             for rl in sorted({2, max(2, Q)})
+             for bc in sorted({1, 3, Q, Q + 1, Q * N, 2 * Q * N})]
+
+
+@pytest.mark.parametrize("Q,N,rl,bc", STAGGERED)
+def test_staggered_small(Q, N, rl, bc):
+    """Algorithm 2: result, the Q(N-1) steps with their bytes, one launch per batch."""
+    P = Q * N
+    wl = W.make_random(P, 300, elem_size=1, seed=3000 + P + bc, zero_frac=0.25, gaps=True)
+    ref, rounds, (Kl, Kg), batches = oracle_staggered(wl, Q, N, rl, bc)
+    got, plan = gpu_run(wl, rl, l=Q, g=N, block_count=bc, misalign=(bc % 3) * 5)
+    assert np.array_equal(got, ref)
+    check_rounds(plan, rounds)
+    assert plan.device_status() == 0
+    local_phases = sum(1 for f in range(plan.num_phases()) if plan.phase_info(f, B.PART_KEEP)["level"] == 0)
+    assert plan.num_phases() - local_phases == batches
+    # every batch is a launch of its own unless it moves no bytes at all
+    assert plan.last_launches() <= local_phases + batches
+    if wl.sendcounts.min() > 0:
+        assert plan.last_launches() == local_phases + batches
+
+
+def test_staggered_rejects_bad_arguments():
+    wl = W.make_random(12, 10, seed=5)
+    with pytest.raises(B.TunaError, match="INVALID_ARG"):
+        B.plan_for(wl, 2, l=4, g=3, block_count=-1)
+    with pytest.raises(B.TunaError, match="INVALID_ARG"):
+        B.plan_for(wl, 2, l=4, g=3, block_count=2, flags=B.FLAG_CLASSIC_ROTATE)
+    with pytest.raises(B.TunaError, match="BAD_HIERARCHY"):
+        B.plan_for(wl, 2, l=5, g=3, block_count=2)
+
+
+def test_staggered_update_counts_and_full_c3():
+    """New counts on a staggered plan; then the 16 x 16 Zipf configuration at full size."""
+    wl = W.make_random(12, 200, seed=8, gaps=True)
+    plan = B.plan_for(wl, 2, l=4, g=3, block_count=4)
+    wl2 = W.make_random(12, 500, seed=9, zero_frac=0.5, gaps=True)
+    plan.update_counts(wl2.sendcounts, wl2.sdispls, wl2.rdispls, wl2.sendbase, wl2.recvbase)
+    plan.alloc_workspace()
+    send = wl2.make_send("cuda")
+    recv = wl2.make_recv("cuda", fill=CANARY)
+    plan.alltoallv(send, recv)
+    torch.cuda.synchronize()
+    assert np.array_equal(recv.cpu().numpy(), oracle_brute(wl2))
+    c3 = W.make_c3()
+    ref, rounds, _, batches = oracle_staggered(c3, 16, 16, 16, 16)
+    got, plan3 = gpu_run(c3, 16, l=16, g=16, block_count=16)
+    assert np.array_equal(got, ref)
+    check_rounds(plan3, rounds)
