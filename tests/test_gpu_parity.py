@@ -440,6 +440,60 @@ def test_c4_full_size(schedule):
         assert sum(x["bytes"] for x in plan.rounds()) == int((wl.sendcounts * nz).sum()) * wl.elem_size
 
 
+@pytest.mark.parametrize("name,kw", [("normal", dict(radix=64)), ("normal", dict(radix=4096)),
+                                     ("powerlaw", dict(radix=2)),
+                                     ("powerlaw", dict(radix=64, l=64, g=64, radix_global=64)),
+                                     ("normal", dict(radix=64, l=64, g=64, block_count=64))])
+def test_paper_scale_4096_ranks(name, kw):
+    """Sec. VI-C's scale: P = 4096 ranks, 16.8 million blocks of at most 1 KiB.  Too
+    large for the oracle, so the received bytes are sampled against the definition of
+    the exchange applied to the generator, and the schedule's byte count is checked
+    against its closed form."""
+    free, _ = torch.cuda.mem_get_info()
+    if free < 80 * 2**30:
+        pytest.skip("needs about 80 GiB of free device memory")
+    wl = W.FULL[name]()
+    assert wl.P == 4096
+    send = wl.make_send("cuda")
+    recv = wl.make_recv("cuda", fill=CANARY)
+    plan = B.plan_for(wl, explicit_layout=False, **kw)
+    plan.alloc_workspace()
+    plan.alltoallv(send, recv)
+    torch.cuda.synchronize()
+    assert plan.device_status() == 0
+    rng = np.random.default_rng(4096)
+    n = 1 << 22
+    s = rng.integers(0, wl.P, n)
+    d = rng.integers(0, wl.P, n)
+    k = (rng.random(n) * wl.sendcounts[s, d]).astype(np.int64)
+    ok = wl.sendcounts[s, d] > 0
+    s, d, k = s[ok], d[ok], k[ok]
+    src = torch.from_numpy(wl.sendbase[s] + wl.sdispls[s, d] + k).cuda()
+    dst = torch.from_numpy(wl.recvbase[d] + wl.rdispls[d, s] + k).cuda()
+    assert torch.equal(recv[dst], W.payload_byte_at(wl.seed, src))
+    # first and last byte of every block of a few receivers
+    for rank in (0, 1777, 4095):
+        c = wl.sendcounts[:, rank]
+        nz = np.nonzero(c)[0]
+        for kk in (np.zeros_like(nz), c[nz] - 1):
+            src = torch.from_numpy(wl.sendbase[nz] + wl.sdispls[nz, rank] + kk).cuda()
+            dst = torch.from_numpy(wl.recvbase[rank] + wl.rdispls[rank, nz] + kk).cuda()
+            assert torch.equal(recv[dst], W.payload_byte_at(wl.seed, src))
+    # bytes moved: once per non-zero digit of the block's offset(s)
+    if "block_count" not in kw:
+        Q, N = (kw["l"], kw["g"]) if "l" in kw else (wl.P, 1)
+        idx = np.arange(wl.P)
+        jo = (idx[None, :] % Q - idx[:, None] % Q) % Q
+        io = (idx[None, :] // Q - idx[:, None] // Q) % N
+        hops = np.zeros((wl.P, wl.P), dtype=np.int64)
+        for t, r in ((jo, kw["radix"]), (io, kw.get("radix_global", 2))):
+            t = t.copy()
+            while t.any():
+                hops += (t % r) != 0
+                t //= r
+        assert sum(x["bytes"] for x in plan.rounds()) == int((wl.sendcounts * hops).sum())
+
+
 @pytest.mark.parametrize("name", ["normal", "powerlaw", "fft_n1", "fft_n2"])
 def test_paper_count_patterns(name):
     """Normal and power-law block sizes and the two FFT transposes, at P = 512."""
