@@ -69,6 +69,8 @@ def _load():
             lib.oracle_tuna_hier_staggered.argtypes = (
                 [ctypes.c_int] * 5 + [_I64P] * 5 + [_U8P, _U8P, ctypes.c_int64, _U8P, _I64P,
                                                     ctypes.c_int, _IP, _IP])
+            lib.oracle_rows_alltoallv.argtypes = ([ctypes.c_int, ctypes.c_int64] + [_I64P] * 7
+                                                  + [_U8P, ctypes.c_int64, _U8P, ctypes.c_int64])
             _lib = lib
     return _lib
 
@@ -209,3 +211,25 @@ def tuna_hier_staggered(wl, Q: int, N: int, rl: int, block_count: int, send: np.
                                           ctypes.byref(batches)), "oracle_tuna_hier_staggered")
     assert Ks[0] + Ks[1] == K
     return recv, rounds[:K], (Ks[0], Ks[1]), batches.value
+
+
+def rows_alltoallv(wl, gather, scatter, rows_in: np.ndarray, rows_out: np.ndarray) -> np.ndarray:
+    """Exchange of whole rows with a gather in front and a scatter behind (not in the
+    paper).  ``wl`` counts rows of ``wl.elem_size`` bytes; ``rows_in`` / ``rows_out`` are
+    2-D uint8 arrays [rows, elem_size]; ``gather`` / ``scatter`` are int64 row maps or None."""
+    lib = _load()
+    c, cp = _i64(wl.sendcounts)
+    sd, sdp = _i64(wl.sdispls)
+    rd, rdp = _i64(wl.rdispls)
+    sb, sbp = _i64(wl.sendbase)
+    rb, rbp = _i64(wl.recvbase)
+    g = gp = s = sp = None
+    if gather is not None:
+        g, gp = _i64(gather)
+    if scatter is not None:
+        s, sp = _i64(scatter)
+    assert rows_in.shape[1] == rows_out.shape[1] == wl.elem_size
+    _check(lib.oracle_rows_alltoallv(wl.P, wl.elem_size, cp, sdp, rdp, sbp, rbp, gp, sp, _u8(rows_in),
+                                     rows_in.shape[0], _u8(rows_out), rows_out.shape[0]),
+           "oracle_rows_alltoallv")
+    return rows_out

@@ -28,6 +28,13 @@
  *                            the staggered inter-group exchange, one block per
  *                            step, block_count steps posted per batch.
  *
+ *   oracle_rows_alltoallv  - NOT IN THE PAPER: the MPI_Alltoallv definition above with
+ *                            a row gather in front of it and a row scatter behind it
+ *                            (the token dispatch of a mixture-of-experts layer:
+ *                            rows leave in token order and arrive in expert order).
+ *                            It is the composition of three textbook definitions
+ *                            and is pinned against exactly that composition.
+ *
  * Readings taken where the printed text is ambiguous (each pinned by a test):
  *   - direction: a rank sends to the rank at distance +z*r^x (Sec. III-A and the
  *     Fig. 2 narrative: P1 sends to P2 and receives from P0); offsets are
@@ -791,4 +798,34 @@ int oracle_tuna_hier_staggered(int Q, int N, int rl, int block_count, int elem,
   return hier_impl(Q, N, rl, 2, block_count, elem, counts, sdispls, rdispls, sendbase, recvbase,
                    send, recv, recv_bytes, recv_after_local, rounds, rounds_cap, K_out,
                    batches_out);
+}
+
+/*
+ * Not in the paper.  Counts and displacements are in rows of row_bytes bytes.
+ * Row j of the (virtual) packed send buffer is row gather[j] of `in` (NULL: j
+ * itself); row j of the (virtual) receive buffer lands in row scatter[j] of `out`
+ * (NULL: j itself).  For every pair (s, d) and k < counts[s][d]:
+ *   out[scatter[recvbase[d] + rdispls[d][s] + k]] = in[gather[sendbase[s] + sdispls[s][d] + k]].
+ * Rows of `out` that no block reaches are left untouched.  Indices outside
+ * [0, in_rows) / [0, out_rows) are an argument error.
+ */
+int oracle_rows_alltoallv(int P, int64_t row_bytes, const int64_t *counts, const int64_t *sdispls,
+                          const int64_t *rdispls, const int64_t *sendbase,
+                          const int64_t *recvbase, const int64_t *gather, const int64_t *scatter,
+                          const uint8_t *in, int64_t in_rows, uint8_t *out, int64_t out_rows) {
+  if (P < 1 || row_bytes < 1) return ORACLE_EARG;
+  for (int s = 0; s < P; s++)
+    for (int d = 0; d < P; d++) {
+      int64_t n = counts[(int64_t)s * P + d];
+      if (n < 0) return ORACLE_EARG;
+      for (int64_t k = 0; k < n; k++) {
+        int64_t js = sendbase[s] + sdispls[(int64_t)s * P + d] + k;
+        int64_t jr = recvbase[d] + rdispls[(int64_t)d * P + s] + k;
+        int64_t from = gather ? gather[js] : js;
+        int64_t to = scatter ? scatter[jr] : jr;
+        if (from < 0 || from >= in_rows || to < 0 || to >= out_rows) return ORACLE_EARG;
+        memcpy(out + to * row_bytes, in + from * row_bytes, (size_t)row_bytes);
+      }
+    }
+  return ORACLE_OK;
 }

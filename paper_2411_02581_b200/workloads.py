@@ -248,15 +248,16 @@ def make_c3(seed: int | None = None, l: int = 16, g: int = 16, cmax: int = 8192,
                                       for b in rr if b <= max(2, g)))
 
 
-def moe_top2_counts(seed: int, P: int, tokens: int, skew: bool = False) -> np.ndarray:
-    """counts[s, d] = tokens of rank s whose two largest logits include d.
+def moe_top2_routing(seed: int, P: int, tokens: int, skew: bool = False):
+    """(first, second): the two destinations of every token, arrays [P, tokens].
 
     Logits are i.i.d. N(0,1) by Box-Muller on the counter-based generator; the
     softmax is monotone, so the two largest logits are the top-2 experts; ties
     go to the lower index.  ``skew`` adds one N(0,1) bias per destination,
     shared by all ranks.
     """
-    counts = np.zeros((P, P), dtype=np.int64)
+    first = np.zeros((P, tokens), dtype=np.int64)
+    second = np.zeros((P, tokens), dtype=np.int64)
     bias = None
     if skew:
         u1 = uniform_unit(seed, S_BIAS, 2 * P).numpy()
@@ -269,11 +270,50 @@ def moe_top2_counts(seed: int, P: int, tokens: int, skew: bool = False) -> np.nd
         z = np.sqrt(-2.0 * np.log(1.0 - u[0])) * np.cos(2.0 * math.pi * u[1])
         if bias is not None:
             z = z + bias[None, :]
-        first = np.argmax(z, axis=1)
-        z[np.arange(tokens), first] = -np.inf
-        second = np.argmax(z, axis=1)
-        counts[s] = np.bincount(first, minlength=P) + np.bincount(second, minlength=P)
+        first[s] = np.argmax(z, axis=1)
+        z[np.arange(tokens), first[s]] = -np.inf
+        second[s] = np.argmax(z, axis=1)
+    return first, second
+
+
+def moe_top2_counts(seed: int, P: int, tokens: int, skew: bool = False) -> np.ndarray:
+    """counts[s, d] = tokens of rank s whose two largest logits include d."""
+    first, second = moe_top2_routing(seed, P, tokens, skew)
+    counts = np.zeros((P, P), dtype=np.int64)
+    for s in range(P):
+        counts[s] = np.bincount(first[s], minlength=P) + np.bincount(second[s], minlength=P)
     return counts
+
+
+def moe_row_maps(first: np.ndarray, second: np.ndarray):
+    """Row maps of a token dispatch with packed buffers.
+
+    ``gather[j]``: the global token row (rank * tokens + token) that row j of the
+    packed send buffer holds: every rank's rows sorted by destination, ascending
+    token order inside a block.  ``scatter[j]``: where row j of the packed receive
+    buffer (grouped by source rank) goes in the expert's own order: sorted by
+    token index first, source rank second.  Both as int64 arrays of length
+    2 * P * tokens."""
+    P, tokens = first.shape
+    gather = np.empty(2 * P * tokens, dtype=np.int64)
+    dest = np.empty(2 * P * tokens, dtype=np.int64)
+    for s in range(P):
+        d = np.concatenate([first[s], second[s]])
+        t = np.concatenate([np.arange(tokens), np.arange(tokens)])
+        order = np.lexsort((t, d))                       # by destination, then token
+        gather[2 * s * tokens:2 * (s + 1) * tokens] = s * tokens + t[order]
+        dest[2 * s * tokens:2 * (s + 1) * tokens] = d[order]
+    # receive side: rows of rank d in (source, position) order are the send rows with
+    # destination d in ascending send position
+    send_pos = np.arange(2 * P * tokens)
+    recv_order = np.lexsort((send_pos, dest))            # receive row j holds send row recv_order[j]
+    tok = gather[recv_order] % tokens
+    src = gather[recv_order] // tokens
+    rdest = dest[recv_order]
+    expert_order = np.lexsort((src, tok, rdest))         # by receiver, then token, then source
+    scatter = np.empty_like(expert_order)
+    scatter[expert_order] = np.arange(2 * P * tokens)
+    return gather, scatter
 
 
 def make_c4(seed: int | None = None, P: int = 64, tokens: int = 8192, hidden: int = 4096,

@@ -43,6 +43,9 @@ MUTATIONS = [
     ("staggered_owner_index_is_receiver",
      "          int jo = ((q - gr) % Q + Q) % Q;\n          int64_t nb = sz[(int64_t)p * P + ndst * Q + jo];",
      "          int jo = gr;\n          int64_t nb = sz[(int64_t)p * P + ndst * Q + jo];"),
+    ("rows_maps_swapped",
+     "int64_t from = gather ? gather[js] : js;\n        int64_t to = scatter ? scatter[jr] : jr;",
+     "int64_t from = gather ? gather[jr] : js;\n        int64_t to = scatter ? scatter[js] : jr;"),
     ("scan_inclusive",
      "      out[s * seglen + i] = run;\n      run += v;", "      run += v;\n      out[s * seglen + i] = run;"),
     ("dropped_self_block",

@@ -487,3 +487,75 @@ def test_paper_count_patterns_small():
             assert np.array_equal(recv, ref)
         recv, _, _, _ = run_hier(wl, 8, 4, 8, 4)
         assert np.array_equal(recv, ref)
+
+
+# ---------------------------------------------------------------- rows with gather / scatter (not in the paper)
+
+def _rows_case(P, maxc, row_bytes, seed, gaps):
+    wl = W.make_random(P, maxc, elem_size=row_bytes, seed=seed, zero_frac=0.2, gaps=gaps)
+    rng = np.random.default_rng(seed)
+    send_rows = wl.send_bytes // row_bytes
+    recv_rows = wl.recv_bytes // row_bytes
+    in_rows = send_rows + 7
+    out_rows = recv_rows + 5
+    gather = rng.integers(0, in_rows, send_rows)                 # rows may repeat
+    scatter = rng.permutation(out_rows)[:recv_rows]              # injective
+    rows_in = rng.integers(0, 256, (in_rows, row_bytes), dtype=np.uint8)
+    return wl, gather, scatter, rows_in, out_rows
+
+
+@pytest.mark.parametrize("P,row_bytes,gaps", [(1, 4, False), (5, 3, True), (8, 16, False), (12, 40, True)])
+def test_rows_exchange_is_gather_then_definition_then_scatter(P, row_bytes, gaps):
+    wl, gather, scatter, rows_in, out_rows = _rows_case(P, 9, row_bytes, 50 + P, gaps)
+    out = np.full((out_rows, row_bytes), CANARY, dtype=np.uint8)
+    oracle.rows_alltoallv(wl, gather, scatter, rows_in, out)
+    # the same thing from library routines and the pinned definition: numpy take,
+    # MPI_Alltoallv on the gathered buffer, numpy fancy assignment
+    send = np.ascontiguousarray(rows_in[gather]).reshape(-1)
+    recv = oracle.bruteforce(wl, send, np.full(wl.recv_bytes, CANARY, dtype=np.uint8))
+    covered = oracle.bruteforce(wl, np.full(wl.send_bytes, 1, dtype=np.uint8),
+                                np.zeros(wl.recv_bytes, dtype=np.uint8)).reshape(-1, row_bytes)[:, 0] == 1
+    ref = np.full((out_rows, row_bytes), CANARY, dtype=np.uint8)
+    ref[scatter[covered]] = recv.reshape(-1, row_bytes)[covered]
+    assert np.array_equal(out, ref)
+    # identity maps: the plain exchange
+    out2 = np.full((wl.recv_bytes // row_bytes, row_bytes), CANARY, dtype=np.uint8)
+    rows_send = wl.make_send().numpy().reshape(-1, row_bytes)
+    oracle.rows_alltoallv(wl, None, None, rows_send, out2)
+    assert np.array_equal(out2.reshape(-1), brute(wl))
+
+
+def test_rows_exchange_rejects_indices_outside_the_buffers():
+    wl, gather, scatter, rows_in, out_rows = _rows_case(4, 5, 8, 3, False)
+    out = np.zeros((out_rows, 8), dtype=np.uint8)
+    bad = gather.copy()
+    bad[0] = rows_in.shape[0]
+    if wl.sendcounts[0, 0] == 0:
+        bad[:] = rows_in.shape[0]
+    with pytest.raises(RuntimeError):
+        oracle.rows_alltoallv(wl, bad, scatter, rows_in, out)
+
+
+def test_moe_row_maps_dispatch_tokens_into_expert_order():
+    """Token rows that name their (rank, token): after the exchange every expert holds
+    exactly the tokens routed to it, sorted by token index, then by source rank."""
+    P, tokens = 8, 64
+    wl = W.make_c4(P=P, tokens=tokens, hidden=4)                 # rows of 8 bytes
+    first, second = W.moe_top2_routing(wl.seed, P, tokens)
+    gather, scatter = W.moe_row_maps(first, second)
+    assert np.array_equal(np.bincount(gather, minlength=P * tokens), np.full(P * tokens, 2))
+    assert np.array_equal(np.sort(scatter), np.arange(2 * P * tokens))
+    rows_in = np.zeros((P * tokens, 8), dtype=np.uint8)
+    rows_in[:, 0] = np.repeat(np.arange(P), tokens)
+    rows_in[:, 1] = np.tile(np.arange(tokens), P)
+    out = np.full((2 * P * tokens, 8), CANARY, dtype=np.uint8)
+    oracle.rows_alltoallv(wl, gather, scatter, rows_in, out)
+    at = 0
+    for d in range(P):
+        want = sorted((t, s) for s in range(P) for t in range(tokens)
+                      if first[s, t] == d or second[s, t] == d)
+        n = len(want)
+        assert n == wl.recvcounts[d].sum()
+        got = [(int(r[1]), int(r[0])) for r in out[at:at + n]]
+        assert got == want
+        at += n
