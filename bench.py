@@ -257,6 +257,60 @@ def time_schedule(plan, wl, send, recv, steps, warmup, direct=False, replan=True
     return a.elapsed_time(b) / steps
 
 
+def token_dispatch_entry(wl, args, send, recv, payload):
+    """The token dispatch in one pass (gather from token order, exchange, scatter into
+    expert order) against the same thing as three passes; `send` and `recv` serve as
+    the intermediate buffers of the three-pass route."""
+    import numpy as np
+    import torch
+    from paper_2411_02581_b200 import binding as B, workloads as W
+    P, rb = wl.P, wl.elem_size
+    tokens = int(wl.sendcounts[0].sum()) // 2
+    first, second = W.moe_top2_routing(wl.seed, P, tokens, skew=args.workload == "c4_skew")
+    g_np, s_np = W.moe_row_maps(first, second)
+    gather, scatter = torch.from_numpy(g_np).cuda(), torch.from_numpy(s_np).cuda()
+    rows_in = torch.empty((P * tokens, rb), dtype=torch.uint8, device="cuda")
+    rows_in.view(torch.int64).random_()
+    rows_out = torch.empty((2 * P * tokens, rb), dtype=torch.uint8, device="cuda")
+    plan = B.plan_for(wl, P, explicit_layout=False)
+
+    def timed(fn, steps, warmup=3):
+        for _ in range(warmup):
+            fn()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(steps):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / steps
+
+    def fused_step():
+        plan.update_counts(wl.sendcounts, None, None, None, None)
+        plan.set_row_maps(gather, scatter, rows_in.shape[0], rows_out.shape[0])
+        plan.rows_alltoallv(rows_in, rows_out)
+
+    ms = timed(fused_step, args.sweep_steps)
+    ms_x = timed(lambda: plan.rows_alltoallv(rows_in, rows_out), args.sweep_steps, 1)
+    send2, recv2 = send.view(-1, rb), recv.view(-1, rb)
+
+    def three_passes():
+        torch.index_select(rows_in, 0, gather, out=send2)
+        plan.direct_alltoallv(send, recv)
+        rows_out.index_copy_(0, scatter, recv2)
+
+    fused = rows_out.clone()
+    ms_3 = timed(three_passes, args.sweep_steps, 1)
+    same = bool(torch.equal(fused, rows_out))
+    plan.destroy()
+    return {"schedule": "token dispatch in one pass: gather + exchange + scatter (rows)",
+            "ms_per_step": ms, "payload_GBps": payload / ms / 1e6, "exchange_only_ms": ms_x,
+            "rounds": 1, "launches": 1, "moved_over_payload": 1.0,
+            "effective_hbm_GBps": 2 * payload / ms_x / 1e6, "workspace_bytes": 0,
+            "three_passes_exchange_only_ms": ms_3, "matches_three_passes": same}
+
+
 def verify_samples(wl, recv, n=4096):
     """Sampled parity at full size: a received byte must equal the generator's byte
     at the position the exchange's definition says it came from."""
@@ -457,6 +511,9 @@ def ours_arm(args):
             for bc in (1, l, wl.P):
                 entry(f"hier {l}x{g} r={rl} staggered block_count={bc}",
                       make_plan(rl, l=l, g=g, block_count=bc))
+
+        if args.workload in ("c4", "c4_skew"):
+            sweep.append(token_dispatch_entry(wl, args, send, recv, payload))
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

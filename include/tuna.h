@@ -250,6 +250,39 @@ int tuna_alltoallv_host(tuna_plan_t *plan, const void *host_send, void *host_rec
                         void *stream);
 
 /*
+ * tuna_plan_set_row_maps, tuna_rows_alltoallv - the exchange of whole rows with a
+ * gather in front of it and a scatter behind it, in one pass.
+ *
+ * The paper has no counterpart: it exchanges contiguous blocks.  A token dispatch
+ * (mixture-of-experts routing) holds its rows in token order and wants them in the
+ * receiving expert's order; done as gather, exchange, scatter that is three passes
+ * over the payload, fused it is one.  The plan's counts and displacements are in
+ * rows (elem_size = bytes per row) and describe two VIRTUAL packed buffers; the maps
+ * tie them to the caller's real ones.  For every s, d and k < sendcounts[s][d]:
+ *   rows_out[scatter_rows[recvbase[d] + rdispls[d][s] + k]]
+ *       = rows_in[gather_rows[sendbase[s] + sdispls[s][d] + k]].
+ *
+ *   gather_rows   DEVICE, one int64 per row of the send layout (send extent in rows),
+ *                 or NULL for the identity.  Rows may repeat.
+ *   scatter_rows  DEVICE, one int64 per row of the receive layout, or NULL.  Must not
+ *                 send two received rows to the same place (not checked; the result
+ *                 for such a row is then one of the candidates).
+ *   in_rows, out_rows   rows of the two buffers; a map entry outside them, for a row
+ *                 that is exchanged, gives TUNA_ERR_RANGE and nothing is moved.
+ * set_row_maps reads the maps on `stream` and synchronises it once; the maps may be
+ * freed afterwards.  It must be called again after tuna_plan_update_counts.  The
+ * row list costs 32 bytes of device memory per exchanged row, owned by the plan.
+ * tuna_rows_alltoallv: rows_in, rows_out DEVICE, in_rows / out_rows rows of
+ * elem_size bytes, must not overlap (TUNA_ERR_OVERLAP); one launch, asynchronous on
+ * `stream`; TUNA_ERR_COUNT_MISMATCH if no maps are set for the current counts.  Rows
+ * of rows_out that no block reaches are left untouched.
+ */
+int tuna_plan_set_row_maps(tuna_plan_t *plan, const int64_t *gather_rows,
+                           const int64_t *scatter_rows, int64_t in_rows, int64_t out_rows,
+                           void *stream);
+int tuna_rows_alltoallv(tuna_plan_t *plan, const void *rows_in, void *rows_out, void *stream);
+
+/*
  * Schedule introspection (host values, filled at plan time).
  * Rounds are the paper's (x, z) pairs in execution order (Sec. III-A); `level` is 0
  * for flat/local rounds and 1 for global rounds; `units` counts blocks sent by all

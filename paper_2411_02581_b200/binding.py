@@ -43,6 +43,8 @@ SIGNATURES = {
     "tuna_plan_create_staggered": (ctypes.c_int, [ctypes.POINTER(_VP)] + [ctypes.c_int] * 6
                                    + [ctypes.c_uint] + [_I64P] * 5 + [_VP]),
     "tuna_plan_update_counts": (ctypes.c_int, [_VP] + [_I64P] * 5 + [_VP]),
+    "tuna_plan_set_row_maps": (ctypes.c_int, [_VP, _VP, _VP, ctypes.c_int64, ctypes.c_int64, _VP]),
+    "tuna_rows_alltoallv": (ctypes.c_int, [_VP, _VP, _VP, _VP]),
     "tuna_plan_destroy": (ctypes.c_int, [_VP]),
     "tuna_plan_workspace_bytes": (ctypes.c_int, [_VP, _SZP]),
     "tuna_plan_host_staging_bytes": (ctypes.c_int, [_VP, _SZP]),
@@ -215,6 +217,17 @@ class Plan:
         self._check(lib().tuna_direct_alltoallv(self._h, _ptr(sendbuf), keep[0][1], keep[1][1],
                                                 _ptr(recvbuf), keep[2][1], keep[3][1],
                                                 _stream(stream)), "tuna_direct_alltoallv")
+
+    def set_row_maps(self, gather_rows, scatter_rows, in_rows: int, out_rows: int, stream=None):
+        """``gather_rows`` / ``scatter_rows``: int64 CUDA tensors or None (identity)."""
+        self._check(lib().tuna_plan_set_row_maps(
+            self._h, _ptr(gather_rows) if gather_rows is not None else None,
+            _ptr(scatter_rows) if scatter_rows is not None else None, in_rows, out_rows,
+            _stream(stream)), "tuna_plan_set_row_maps")
+
+    def rows_alltoallv(self, rows_in, rows_out, stream=None):
+        self._check(lib().tuna_rows_alltoallv(self._h, _ptr(rows_in), _ptr(rows_out), _stream(stream)),
+                    "tuna_rows_alltoallv")
 
     def alltoallv_host(self, host_send, host_recv, schedule=SCHEDULE_TUNA, stream=None):
         self._check(lib().tuna_alltoallv_host(self._h, _ptr(host_send), _ptr(host_recv), schedule,

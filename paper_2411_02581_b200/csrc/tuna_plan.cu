@@ -175,6 +175,45 @@ __global__ void tuna_stagger_batch_kernel(TunaTopo t, int lo, int hi,
   if (bytes > 0) atomicAdd(&step_bytes[ii], (unsigned long long)bytes);
 }
 
+// Row list of the exchange with a gather in front and a scatter behind (no
+// counterpart in the paper): one descriptor per row.  One warp per block (d, s);
+// row k of the block is row sendbase[s] + sdispls[s][d] + k of the packed send
+// layout and row recvbase[d] + rdispls[d][s] + k of the receive layout; the maps
+// (identity when null) turn these into rows of the caller's two buffers.
+// row_start[d*P + s] = rows of all blocks before (d, s) in receive-side order.
+__global__ void tuna_rows_list_kernel(int P, int64_t row_bytes, const int64_t *__restrict__ counts,
+                                      const int64_t *__restrict__ sdispls,
+                                      const int64_t *__restrict__ rdispls,
+                                      const int64_t *__restrict__ sendbase,
+                                      const int64_t *__restrict__ recvbase,
+                                      const int64_t *__restrict__ row_start,
+                                      const int64_t *__restrict__ gather,
+                                      const int64_t *__restrict__ scatter, int64_t in_rows,
+                                      int64_t out_rows, int64_t n_rows, int64_t *len, int64_t *pos,
+                                      int64_t *src, int64_t *dst) {
+  const int64_t w = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  const int64_t stride = pad16(row_bytes) + 16;  // DELIVER spacing of equal-sized blocks
+  if (w == 0 && lane == 0) pos[n_rows] = n_rows * stride;
+  if (w >= (int64_t)P * P) return;
+  const int d = (int)(w / P), s = (int)(w % P);
+  const int64_t c = counts[(int64_t)s * P + d];
+  const int64_t js = sendbase[s] + sdispls[(int64_t)s * P + d];
+  const int64_t jr = recvbase[d] + rdispls[(int64_t)d * P + s];
+  const int64_t e0 = row_start[w];
+  for (int64_t k = lane; k < c; k += 32) {
+    const int64_t from = gather ? gather[js + k] : js + k;
+    const int64_t to = scatter ? scatter[jr + k] : jr + k;
+    const int64_t e = e0 + k;
+    len[e] = row_bytes;
+    pos[e] = e * stride;
+    // a row outside its buffer gets a location that the range check that follows
+    // rejects (the wrong buffer tag) instead of an offset that could wrap around
+    src[e] = (from < 0 || from >= in_rows) ? TUNA_LOC(TUNA_BUF_RECV, 0) : TUNA_LOC(TUNA_BUF_SEND, from * row_bytes);
+    dst[e] = (to < 0 || to >= out_rows) ? TUNA_LOC(TUNA_BUF_SEND, 0) : TUNA_LOC(TUNA_BUF_RECV, to * row_bytes);
+  }
+}
+
 // Segmented exclusive prefix sum, one warp per segment, warp-shuffle scan over
 // 32-wide tiles with a running carry.  MODE 0 sums the values as they are; MODE 1
 // (KEEP lists) rounds every value up to 16 first; MODE 2 (DELIVER lists) also
@@ -393,6 +432,12 @@ struct tuna_plan {
   std::vector<TunaList> keep;     // per phase: blocks that travel on (workspace)
   std::vector<TunaList> deliver;  // per phase: blocks that have arrived (receive buffer)
   TunaList rot, dir;
+  // exchange of rows through a gather and a scatter map (tuna_plan_set_row_maps)
+  TunaList rowsl;
+  int64_t rows_cap = 0;          // descriptors allocated in rowsl
+  int64_t *d_row_start = nullptr;
+  int64_t rows_in_bytes = 0, rows_out_bytes = 0;
+  bool rows_valid = false;
 
   struct Round {
     int level, x, z, phase;
@@ -707,6 +752,7 @@ int build_tables(tuna_plan *pl, const HostLayout &hl, const int64_t *counts, con
   const int64_t PP = (int64_t)P * P;
   int rc = TUNA_OK;
 
+  pl->rows_valid = false;  // a row list belongs to the counts it was built for
   // host copies for the checks at call time
   pl->h_counts.assign(counts, counts + PP);
   pl->have_sdispls = sdispls != nullptr;
@@ -1094,6 +1140,8 @@ int tuna_plan_destroy(tuna_plan_t *pl) {
   for (auto &l : pl->deliver) free_list(l);
   free_list(pl->rot);
   free_list(pl->dir);
+  free_list(pl->rowsl);
+  cudaFree(pl->d_row_start);
   cudaFree(pl->d_counts);
   cudaFree(pl->d_sdispls);
   cudaFree(pl->d_rdispls);
@@ -1181,7 +1229,7 @@ static int plan_create(tuna_plan_t **out, int P, int radix, int radix_global, in
   TUNA_TRY(dev_alloc(&pl->d_seg_raw, P));
   TUNA_TRY(dev_alloc(&pl->d_seg_base, 2 * P));
   TUNA_TRY(dev_alloc(&pl->d_tmp, PP));
-  TUNA_TRY(dev_alloc(&pl->d_scal, 2 * (2 * nph + 2)));
+  TUNA_TRY(dev_alloc(&pl->d_scal, 2 * (2 * nph + 3)));
   TUNA_TRY(dev_alloc(&pl->d_wbase, nph + 1));
   TUNA_TRY(dev_alloc(&pl->d_round_bytes, pl->stats_n));
   TUNA_TRY(dev_alloc(&pl->d_error, 1));
@@ -1343,6 +1391,91 @@ int tuna_alltoallv_host(tuna_plan_t *pl, const void *host_send, void *host_recv,
   if (rc) return rc;
   if (pl->recv_extent > 0)
     TUNA_CUDA(pl, cudaMemcpyAsync(host_recv, d_recv, (size_t)pl->recv_extent, cudaMemcpyDeviceToHost, st));
+  return TUNA_OK;
+}
+
+int tuna_plan_set_row_maps(tuna_plan_t *pl, const int64_t *gather_rows, const int64_t *scatter_rows,
+                           int64_t in_rows, int64_t out_rows, void *stream) {
+  if (!pl || in_rows < 0 || out_rows < 0) return TUNA_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  const TunaTopo &t = pl->topo;
+  const int P = t.P;
+  const int64_t PP = (int64_t)P * P;
+  const int64_t n = pl->payload / t.elem;  // rows exchanged
+  pl->rows_valid = false;
+  if (in_rows > (INT64_MAX >> 8) / t.elem || out_rows > (INT64_MAX >> 8) / t.elem) return TUNA_ERR_RANGE;
+  if (!pl->d_row_start) TUNA_CUDA(pl, dev_alloc(&pl->d_row_start, PP));
+  if (!pl->rowsl.len || n > pl->rows_cap) {
+    free_list(pl->rowsl);
+    pl->rows_cap = 0;
+    const int rc = alloc_list(pl, pl->rowsl, TUNA_LIST_DELIVER, n);
+    if (rc) return pl->cuda_err == (int)cudaErrorMemoryAllocation ? TUNA_ERR_NOMEM : rc;
+    pl->rows_cap = n;
+  }
+  TunaList &l = pl->rowsl;
+  l.n = n;
+  const int th = 256;
+  const unsigned gPP = (unsigned)((PP + th - 1) / th);
+  const unsigned gseg = (unsigned)(((int64_t)P * 32 + th - 1) / th);
+  const int nph = (int)pl->phases.size();
+  Timed plan_timer(pl, TUNA_TIMER_PLAN, 0, st);
+  // rows before every block in receive-side order: scan of the transposed counts
+  tuna_transpose_kernel<<<gPP, th, 0, st>>>(pl->d_counts, pl->d_tmp, P);
+  TUNA_LAUNCHED(pl);
+  tuna_segscan_kernel<0><<<gseg, th, 0, st>>>(pl->d_tmp, pl->d_row_start, pl->d_seg_total, nullptr, P, P);
+  TUNA_LAUNCHED(pl);
+  tuna_segbase_kernel<<<1, 1024, 0, st>>>(pl->d_seg_total, nullptr, pl->d_seg_base, P,
+                                          pl->d_scal + 2 * (2 * nph + 2), nullptr, 0, nullptr);
+  TUNA_LAUNCHED(pl);
+  tuna_add_base_kernel<<<gPP, th, 0, st>>>(pl->d_row_start, pl->d_seg_base, P, PP);
+  TUNA_LAUNCHED(pl);
+  const int64_t warps = PP;
+  tuna_rows_list_kernel<<<(unsigned)((warps * 32 + th - 1) / th), th, 0, st>>>(
+      P, t.elem, pl->d_counts, pl->d_sdispls, pl->d_rdispls, pl->d_sendbase, pl->d_recvbase,
+      pl->d_row_start, gather_rows, scatter_rows, in_rows, out_rows, n, l.len, l.pos, l.src, l.dst);
+  TUNA_LAUNCHED(pl);
+  pl->rows_in_bytes = in_rows * t.elem;
+  pl->rows_out_bytes = out_rows * t.elem;
+  l.bytes = n * t.elem;
+  l.total = n * (((int64_t)t.elem + 15) / 16 * 16 + 16);
+  // every row must lie inside the two buffers
+  TUNA_CUDA(pl, cudaMemsetAsync(pl->d_violations, 0, sizeof(unsigned long long), st));
+  if (n > 0) {
+    tuna_check_list_kernel<<<(unsigned)((n + th - 1) / th), th, 0, st>>>(
+        l.len, l.pos, l.src, l.dst, n, pl->rows_in_bytes, pl->rows_out_bytes, pl->d_wbase + nph, 0,
+        pl->d_wbase, pl->d_violations);
+    TUNA_LAUNCHED(pl);
+  }
+  int rc = build_chunks(pl, l, st);
+  if (rc) return rc;
+  unsigned long long violations = 0;
+  TUNA_CUDA(pl, cudaMemcpyAsync(&violations, pl->d_violations, sizeof(violations), cudaMemcpyDeviceToHost, st));
+  TUNA_CUDA(pl, cudaStreamSynchronize(st));
+  if (violations != 0) return TUNA_ERR_RANGE;
+  pl->rows_valid = true;
+  return TUNA_OK;
+}
+
+int tuna_rows_alltoallv(tuna_plan_t *pl, const void *rows_in, void *rows_out, void *stream) {
+  if (!pl) return TUNA_ERR_INVALID_ARG;
+  if (!pl->rows_valid) return TUNA_ERR_COUNT_MISMATCH;
+  const TunaList &l = pl->rowsl;
+  if (l.n > 0 && (!rows_in || !rows_out)) return TUNA_ERR_INVALID_ARG;
+  if (ranges_overlap(rows_in, (size_t)pl->rows_in_bytes, rows_out, (size_t)pl->rows_out_bytes))
+    return TUNA_ERR_OVERLAP;
+  int launches = 0;
+  if (l.nchunks > 0) {
+    cudaStream_t st = (cudaStream_t)stream;
+    Timed tm(pl, TUNA_TIMER_DIRECT, l.bytes, st);
+    TunaMoveArgs a = move_args(pl, rows_in, rows_out, nullptr);
+    a.extent[TUNA_BUF_SEND] = pl->rows_in_bytes;
+    a.extent[TUNA_BUF_RECV] = pl->rows_out_bytes;
+    a.del = list_args(l);
+    TUNA_CUDA(pl, tuna_launch_move(TUNA_K_DIRECT, a, l.small_blocks, st));
+    launches++;
+  }
+  pl->last_launches = launches;
+  pl->launch_count += launches;
   return TUNA_OK;
 }
 

@@ -627,3 +627,116 @@ def test_staggered_update_counts_and_full_c3():
     got, plan3 = gpu_run(c3, 16, l=16, g=16, block_count=16)
     assert np.array_equal(got, ref)
     check_rounds(plan3, rounds)
+
+
+# ---------------------------------------------------------------- rows with gather / scatter maps
+
+def _rows_inputs(wl, seed, identity_gather=False, identity_scatter=False):
+    rb = wl.elem_size
+    rng = np.random.default_rng(seed)
+    send_rows, recv_rows = wl.send_bytes // rb, wl.recv_bytes // rb
+    in_rows = send_rows + (0 if identity_gather else 7)
+    out_rows = recv_rows + (0 if identity_scatter else 5)
+    gather = None if identity_gather else rng.integers(0, in_rows, send_rows)
+    scatter = None if identity_scatter else rng.permutation(out_rows)[:recv_rows]
+    rows_in = rng.integers(0, 256, (max(in_rows, 1), rb), dtype=np.uint8)[:in_rows]
+    return gather, scatter, rows_in, out_rows
+
+
+def _rows_gpu(wl, gather, scatter, rows_in, out_rows):
+    rb = wl.elem_size
+    plan = B.plan_for(wl, 2)
+    dev = lambda a: None if a is None else torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    d_in = torch.from_numpy(rows_in).cuda()
+    d_out = torch.full((out_rows, rb), CANARY, dtype=torch.uint8, device="cuda")
+    plan.set_row_maps(dev(gather), dev(scatter), rows_in.shape[0], out_rows)
+    plan.rows_alltoallv(d_in, d_out)
+    torch.cuda.synchronize()
+    assert plan.device_status() == 0
+    return d_out.cpu().numpy(), plan
+
+
+@pytest.mark.parametrize("P,maxc,rb,gaps", [(1, 5, 16, False), (5, 9, 3, True), (8, 40, 16, False),
+                                            (12, 30, 40, True), (33, 20, 264, False),
+                                            (16, 12, 8192, False), (64, 3, 100, True)])
+@pytest.mark.parametrize("ident", [(False, False), (True, False), (False, True), (True, True)])
+def test_rows_exchange(P, maxc, rb, gaps, ident):
+    wl = W.make_random(P, maxc, elem_size=rb, seed=60 + P, zero_frac=0.2, gaps=gaps)
+    gather, scatter, rows_in, out_rows = _rows_inputs(wl, 7 * P + rb, *ident)
+    ref = np.full((out_rows, rb), CANARY, dtype=np.uint8)
+    oracle.rows_alltoallv(wl, gather, scatter, rows_in, ref)
+    got, plan = _rows_gpu(wl, gather, scatter, rows_in, out_rows)
+    assert np.array_equal(got, ref)
+    assert plan.last_launches() == (1 if wl.payload_bytes_total else 0)
+
+
+def test_rows_exchange_errors_and_recount():
+    wl = W.make_random(6, 10, elem_size=32, seed=2, gaps=False)
+    gather, scatter, rows_in, out_rows = _rows_inputs(wl, 5)
+    plan = B.plan_for(wl, 2)
+    d_in = torch.from_numpy(rows_in).cuda()
+    d_out = torch.full((out_rows, 32), CANARY, dtype=torch.uint8, device="cuda")
+    with pytest.raises(B.TunaError, match="COUNT_MISMATCH"):      # no maps yet
+        plan.rows_alltoallv(d_in, d_out)
+    s0, d0 = (int(v[0]) for v in np.nonzero(wl.sendcounts))       # a pair that exchanges rows
+    bad = gather.copy()
+    bad[wl.sdispls[s0, d0] + wl.sendbase[s0]] = rows_in.shape[0]  # one row past the end of rows_in
+    with pytest.raises(B.TunaError, match="RANGE"):
+        plan.set_row_maps(torch.from_numpy(bad).cuda(), torch.from_numpy(scatter).cuda(),
+                          rows_in.shape[0], out_rows)
+    bad = scatter.copy()
+    bad[wl.rdispls[d0, s0] + wl.recvbase[d0]] = -1
+    with pytest.raises(B.TunaError, match="RANGE"):
+        plan.set_row_maps(torch.from_numpy(gather).cuda(), torch.from_numpy(bad).cuda(),
+                          rows_in.shape[0], out_rows)
+    with pytest.raises(B.TunaError, match="COUNT_MISMATCH"):      # the failed call left no maps behind
+        plan.rows_alltoallv(d_in, d_out)
+    plan.set_row_maps(torch.from_numpy(gather).cuda(), torch.from_numpy(scatter).cuda(),
+                      rows_in.shape[0], out_rows)
+    with pytest.raises(B.TunaError, match="OVERLAP"):
+        plan.rows_alltoallv(d_in, d_in)
+    plan.rows_alltoallv(d_in, d_out)
+    torch.cuda.synchronize()
+    # new counts invalidate the maps
+    wl2 = W.make_random(6, 14, elem_size=32, seed=3)
+    plan.update_counts(wl2.sendcounts, wl2.sdispls, wl2.rdispls, wl2.sendbase, wl2.recvbase)
+    with pytest.raises(B.TunaError, match="COUNT_MISMATCH"):
+        plan.rows_alltoallv(d_in, d_out)
+    g2, s2, in2, out2 = _rows_inputs(wl2, 9)
+    ref = np.full((out2, 32), CANARY, dtype=np.uint8)
+    oracle.rows_alltoallv(wl2, g2, s2, in2, ref)
+    d_in2 = torch.from_numpy(in2).cuda()
+    d_out2 = torch.full((out2, 32), CANARY, dtype=torch.uint8, device="cuda")
+    plan.set_row_maps(torch.from_numpy(g2).cuda(), torch.from_numpy(s2).cuda(), in2.shape[0], out2)
+    plan.rows_alltoallv(d_in2, d_out2)
+    torch.cuda.synchronize()
+    assert np.array_equal(d_out2.cpu().numpy(), ref)
+
+
+def test_rows_exchange_token_dispatch():
+    """The token-dispatch shape, scaled down: P = 64 ranks, 256 tokens of 1 KiB per
+    rank, top-2 routing; tokens leave in token order and arrive in expert order."""
+    P, tokens, hidden = 64, 256, 512
+    wl = W.make_c4(P=P, tokens=tokens, hidden=hidden)
+    first, second = W.moe_top2_routing(wl.seed, P, tokens)
+    gather, scatter = W.moe_row_maps(first, second)
+    rng = np.random.default_rng(11)
+    rows_in = rng.integers(0, 256, (P * tokens, wl.elem_size), dtype=np.uint8)
+    ref = np.full((2 * P * tokens, wl.elem_size), CANARY, dtype=np.uint8)
+    oracle.rows_alltoallv(wl, gather, scatter, rows_in, ref)
+    plan = B.plan_for(wl, 64, explicit_layout=False)
+    d_in = torch.from_numpy(rows_in).cuda()
+    d_out = torch.full(ref.shape, CANARY, dtype=torch.uint8, device="cuda")
+    plan.set_row_maps(torch.from_numpy(gather).cuda(), torch.from_numpy(scatter).cuda(),
+                      rows_in.shape[0], ref.shape[0])
+    plan.rows_alltoallv(d_in, d_out)
+    torch.cuda.synchronize()
+    assert np.array_equal(d_out.cpu().numpy(), ref)
+    # the unfused route gives the same rows: gather, exchange, scatter
+    send = d_in[torch.from_numpy(gather).cuda()].contiguous()
+    recv = torch.empty_like(send)
+    plan.direct_alltoallv(send, recv)
+    out2 = torch.full(ref.shape, CANARY, dtype=torch.uint8, device="cuda")
+    out2[torch.from_numpy(scatter).cuda()] = recv
+    torch.cuda.synchronize()
+    assert torch.equal(out2, d_out)
