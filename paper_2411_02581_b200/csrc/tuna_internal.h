@@ -65,9 +65,10 @@ struct TunaList {
   int64_t chunk_cap = 0;  // allocated entries of chunk_first
   int64_t total = 0;      // stream bytes (host copy)
   int64_t bytes = 0;      // bytes moved (host copy)
+  int64_t unaligned_bytes = 0;  // ... of which in blocks whose source and destination differ modulo 16
   int64_t chunk = 0;      // bytes of stream per CTA
   int64_t nchunks = 0;
-  bool small_blocks = false;  // mean block far below a chunk (host copy, from bytes / n)
+  bool small_blocks = false;  // runs the small-block kernel build (tiny or mostly skewed blocks)
 };
 
 // Device view of one list.

@@ -386,11 +386,12 @@ __global__ void tuna_check_list_kernel(const int64_t *__restrict__ len, const in
                                        const int64_t *__restrict__ src, const int64_t *__restrict__ dst,
                                        int64_t n, int64_t send_extent, int64_t recv_extent,
                                        const int64_t *__restrict__ work_extent, int64_t keep_base_index,
-                                       const int64_t *__restrict__ wbase, unsigned long long *violations) {
+                                       const int64_t *__restrict__ wbase, unsigned long long *violations,
+                                       unsigned long long *unaligned_bytes) {
   const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (e >= n) return;
-  const int64_t L = len[e];
-  bool bad = L < 0 || pos[e + 1] < pos[e];
+  const int64_t L = e < n ? len[e] : 0;
+  bool bad = e < n && (L < 0 || pos[e + 1] < pos[e]);
+  int64_t skewed = 0;  // bytes of a block whose source and destination differ modulo 16
   if (L > 0) {
     const int64_t s = src[e];
     const int sb = TUNA_LOC_BUF(s);
@@ -400,12 +401,17 @@ __global__ void tuna_check_list_kernel(const int64_t *__restrict__ len, const in
     if (dst) {  // DELIVER: into the receive buffer
       const int64_t d = dst[e];
       bad = bad || TUNA_LOC_BUF(d) != TUNA_BUF_RECV || TUNA_LOC_OFF(d) + L > recv_extent;
+      if (((so - TUNA_LOC_OFF(d)) & 15) != 0) skewed = L;
     } else {    // KEEP: at its stream position in the phase's workspace region
       const int64_t o = wbase[keep_base_index] + pos[e];
       bad = bad || (o & (TUNA_ALIGN - 1)) != 0 || o + pad16(L) > *work_extent || pos[e + 1] - pos[e] != pad16(L);
+      if ((so & 15) != 0) skewed = L;
     }
   }
   if (bad) atomicAdd(violations, 1ULL);
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) skewed += __shfl_xor_sync(0xffffffffu, skewed, d);
+  if ((threadIdx.x & 31) == 0 && skewed > 0) atomicAdd(unaligned_bytes, (unsigned long long)skewed);
 }
 
 __global__ void tuna_transpose_kernel(const int64_t *__restrict__ in, int64_t *out, int P) {
@@ -462,7 +468,9 @@ struct tuna_plan {
   unsigned long long *d_round_bytes = nullptr;
   int64_t stats_n = 0;
   int *d_error = nullptr;        // raised by a kernel whose bounded wait gave up
-  unsigned long long *d_violations = nullptr;  // descriptors that failed the plan's self-check
+  unsigned long long *d_violations = nullptr;  // [0]: descriptors that failed the plan's self-check;
+                                               // [1 + list id]: bytes of that list's blocks whose source
+                                               // and destination differ modulo 16
 
   std::vector<int64_t> h_wbase;  // workspace offset of every phase's KEEP stream
   int64_t workspace_need = 0;
@@ -593,31 +601,41 @@ int64_t env_i64(const char *name, int64_t dflt) {
   return strtoll(s, nullptr, 10);
 }
 
-// Bytes of destination stream per CTA: enough chunks to fill the machine several
-// times over, but no smaller than a few KiB (descriptor overhead) and no larger
-// than 128 KiB (tail effect).
-// Mean block size below which a list runs the small-block kernel build.  Measured
-// with 16-byte aligned blocks: the small build wins up to 16 KiB blocks (6.06 vs
-// 5.94 TB/s), the large one from 128 KiB on (6.40 vs 6.30 TB/s).
-constexpr int64_t kSmallBlockBytes = 65536;
+// Which kernel build runs a list.  Measured on the direct exchange (TB/s of read +
+// write, large build / small build): blocks whose source and destination agree
+// modulo 16 (plain vector copies) 2.86 / 3.58 at 64-byte blocks, 4.20 / 4.84 at
+// 128 B, 5.37 / 5.22 at 256 B, 5.89 / 5.67 at 4 KiB, 6.40 / 6.07 at 128 KiB,
+// 6.56 / 6.12 at 1 MiB; blocks that need the funnel-shift loads 2.38 / 2.83 at 128 B,
+// 3.77 / 4.40 at 1 KiB, 4.23 / 4.93 at 32 KiB, 4.55 / 5.31 at 1 MiB.  So: the small
+// build for lists of tiny blocks and for lists that are mostly skewed, whatever
+// their block size; the large build otherwise.  Lists small enough to live in L2
+// are latency-bound rather than DRAM-bound and also do better with the small
+// build's higher occupancy (c3, 16 x 16 ranks, radix 16/2: 0.144 ms against 0.169 ms).
+constexpr int64_t kSmallBlockBytes = 256;
+constexpr int64_t kSmallListBytes = 64 << 20;
+constexpr int64_t kStaticSmallBlockBytes = 65536;  // the table-free entry point decides by size alone
 constexpr int64_t kHostStagingBlockBytes = 2048;  // mean block below which host buffers are staged
 
-// Bytes of stream per CTA.  Large blocks: 64 KiB, the best measured size for
+// Bytes of stream per CTA.  Large build: 64 KiB, the best measured size for
 // multi-MiB blocks (smaller chunks pay the per-chunk set-up more often, larger
-// ones leave a longer tail).  Small-block build: 32 KiB, so that one batch of 256
-// descriptors covers a chunk of tiny blocks.  Small lists: fewer bytes per CTA,
-// to fill the SMs.
+// ones leave a longer tail); 128 KiB for blocks of 1 to 32 KiB (measured: 6.03 vs
+// 5.89 TB/s at 4 KiB, 6.10 vs 5.96 at 16 KiB, 6.35 vs 6.00 on scattered 8 KiB
+// rows).  Small build: 32 KiB, so that one batch of 256 descriptors covers a chunk
+// of tiny blocks.  Small lists: fewer bytes per CTA, to fill the SMs.
 int64_t pick_chunk(const TunaList &l) {
   const int64_t forced = env_i64(l.kind == TUNA_LIST_KEEP ? "TUNA_CHUNK_BYTES_KEEP" : "TUNA_CHUNK_BYTES_DELIVER", 0);
   if (forced >= 1024) return std::min<int64_t>((forced + 15) & ~(int64_t)15, TUNA_MAX_CHUNK_BYTES);
-  const int64_t top = l.small_blocks ? 32768 : 65536;
+  const int64_t mean = l.n > 0 ? l.bytes / l.n : 0;
+  const int64_t top = l.small_blocks ? 32768 : ((mean >= 1024 && mean <= 32768) ? 131072 : 65536);
   int64_t c = 8192;
   while (c < top && l.total / c > 148 * 32) c <<= 1;
   return c;
 }
 
 int build_chunks(tuna_plan *pl, TunaList &l, cudaStream_t st) {
-  l.small_blocks = l.n > 0 && l.bytes / l.n < env_i64("TUNA_SMALL_BLOCK_BYTES", kSmallBlockBytes);
+  l.small_blocks = l.n > 0 && (l.bytes / l.n < env_i64("TUNA_SMALL_BLOCK_BYTES", kSmallBlockBytes) ||
+                               l.bytes < env_i64("TUNA_SMALL_LIST_BYTES", kSmallListBytes) ||
+                               (2 * l.unaligned_bytes > l.bytes && env_i64("TUNA_SKEWED_SMALL", 1) != 0));
   l.chunk = pick_chunk(l);
   l.nchunks = l.total > 0 ? (l.total + l.chunk - 1) / l.chunk : 0;
   if (l.nchunks > l.chunk_cap) {
@@ -847,24 +865,28 @@ int build_tables(tuna_plan *pl, const HostLayout &hl, const int64_t *counts, con
   if (rc) return rc;
 
   // self-check: every descriptor of every list stays inside its buffers
-  TUNA_CUDA(pl, cudaMemsetAsync(pl->d_violations, 0, sizeof(unsigned long long), st));
-  auto check = [&](const TunaList &l, int keep_phase) -> int {
+  // (the same pass sums, per list, the bytes of the blocks whose source and
+  // destination differ modulo 16: they pick the kernel build)
+  const int nlists = 2 * nph + 2;
+  TUNA_CUDA(pl, cudaMemsetAsync(pl->d_violations, 0, sizeof(unsigned long long) * (1 + nlists), st));
+  auto check = [&](const TunaList &l, int keep_phase, int id) -> int {
     if (l.n <= 0) return TUNA_OK;
     tuna_check_list_kernel<<<(unsigned)((l.n + th - 1) / th), th, 0, st>>>(
         l.len, l.pos, l.src, l.kind == TUNA_LIST_DELIVER ? l.dst : nullptr, l.n, pl->send_extent,
-        pl->recv_extent, pl->d_wbase + nph, keep_phase, pl->d_wbase, pl->d_violations);
+        pl->recv_extent, pl->d_wbase + nph, keep_phase, pl->d_wbase, pl->d_violations,
+        pl->d_violations + 1 + id);
     TUNA_LAUNCHED(pl);
     return TUNA_OK;
   };
   for (int f = 0; f < nph; f++) {
-    rc = check(pl->keep[f], f);
+    rc = check(pl->keep[f], f, f);
     if (rc) return rc;
-    rc = check(pl->deliver[f], 0);
+    rc = check(pl->deliver[f], 0, nph + f);
     if (rc) return rc;
   }
-  rc = check(pl->rot, 0);
+  rc = check(pl->rot, 0, 2 * nph);
   if (rc) return rc;
-  rc = check(pl->dir, 0);
+  rc = check(pl->dir, 0, 2 * nph + 1);
   if (rc) return rc;
 
   plan_timer.stop();  // the chunk tables below are timed separately, after the read-back
@@ -875,14 +897,15 @@ int build_tables(tuna_plan *pl, const HostLayout &hl, const int64_t *counts, con
   TUNA_CUDA(pl, cudaMemcpyAsync(wbase.data(), pl->d_wbase, wbase.size() * 8, cudaMemcpyDeviceToHost, st));
   TUNA_CUDA(pl, cudaMemcpyAsync(rbytes.data(), pl->d_round_bytes, rbytes.size() * 8,
                                 cudaMemcpyDeviceToHost, st));
-  unsigned long long violations = 0;
-  TUNA_CUDA(pl, cudaMemcpyAsync(&violations, pl->d_violations, sizeof(violations), cudaMemcpyDeviceToHost, st));
+  std::vector<unsigned long long> checked(1 + nlists);
+  TUNA_CUDA(pl, cudaMemcpyAsync(checked.data(), pl->d_violations, checked.size() * 8, cudaMemcpyDeviceToHost, st));
   TUNA_CUDA(pl, cudaStreamSynchronize(st));
-  if (violations != 0) return TUNA_ERR_INTERNAL;
+  if (checked[0] != 0) return TUNA_ERR_INTERNAL;
   pl->h_wbase = wbase;
   auto take = [&](TunaList &l, int id) {
     l.total = scal[2 * id];
     l.bytes = scal[2 * id + 1];
+    l.unaligned_bytes = (int64_t)checked[1 + id];
   };
   for (int f = 0; f < nph; f++) {
     take(pl->keep[f], f);
@@ -1070,13 +1093,15 @@ int run_tuna(tuna_plan *pl, const void *send, void *recv, cudaStream_t st) {
     a.del = list_args(d);
     a.keep_base = pl->h_wbase[f];
     int64_t bytes = k.bytes + d.bytes;
-    bool small = (k.nchunks == 0 || k.small_blocks) && (d.nchunks == 0 || d.small_blocks);
+    // the lists of a launch share one kernel build: the one most of its bytes want
+    int64_t small_bytes = (k.small_blocks ? k.bytes : 0) + (d.small_blocks ? d.bytes : 0);
     if (with_rot) {
       a.rot = list_args(pl->rot);
       bytes += pl->rot.bytes;
-      small = small && pl->rot.small_blocks;
+      small_bytes += pl->rot.small_blocks ? pl->rot.bytes : 0;
       rot_done = true;
     }
+    const bool small = 2 * small_bytes >= bytes;
     Timed tm(pl, kind, bytes, st);
     TUNA_CUDA(pl, tuna_launch_move(TUNA_K_ROUND, a, small, st));
     launches++;
@@ -1233,7 +1258,7 @@ static int plan_create(tuna_plan_t **out, int P, int radix, int radix_global, in
   TUNA_TRY(dev_alloc(&pl->d_wbase, nph + 1));
   TUNA_TRY(dev_alloc(&pl->d_round_bytes, pl->stats_n));
   TUNA_TRY(dev_alloc(&pl->d_error, 1));
-  TUNA_TRY(dev_alloc(&pl->d_violations, 1));
+  TUNA_TRY(dev_alloc(&pl->d_violations, 1 + 2 * nph + 3));
   TUNA_TRY(cudaMemset(pl->d_error, 0, sizeof(int)));
   pl->keep.resize(nph);
   pl->deliver.resize(nph);
@@ -1439,19 +1464,21 @@ int tuna_plan_set_row_maps(tuna_plan_t *pl, const int64_t *gather_rows, const in
   l.bytes = n * t.elem;
   l.total = n * (((int64_t)t.elem + 15) / 16 * 16 + 16);
   // every row must lie inside the two buffers
-  TUNA_CUDA(pl, cudaMemsetAsync(pl->d_violations, 0, sizeof(unsigned long long), st));
+  TUNA_CUDA(pl, cudaMemsetAsync(pl->d_violations, 0, 2 * sizeof(unsigned long long), st));
   if (n > 0) {
     tuna_check_list_kernel<<<(unsigned)((n + th - 1) / th), th, 0, st>>>(
         l.len, l.pos, l.src, l.dst, n, pl->rows_in_bytes, pl->rows_out_bytes, pl->d_wbase + nph, 0,
-        pl->d_wbase, pl->d_violations);
+        pl->d_wbase, pl->d_violations, pl->d_violations + 1);
     TUNA_LAUNCHED(pl);
   }
-  int rc = build_chunks(pl, l, st);
-  if (rc) return rc;
-  unsigned long long violations = 0;
-  TUNA_CUDA(pl, cudaMemcpyAsync(&violations, pl->d_violations, sizeof(violations), cudaMemcpyDeviceToHost, st));
+  unsigned long long checked[2] = {0, 0};
+  TUNA_CUDA(pl, cudaMemcpyAsync(checked, pl->d_violations, sizeof(checked), cudaMemcpyDeviceToHost, st));
   TUNA_CUDA(pl, cudaStreamSynchronize(st));
-  if (violations != 0) return TUNA_ERR_RANGE;
+  if (checked[0] != 0) return TUNA_ERR_RANGE;
+  l.unaligned_bytes = (int64_t)checked[1];
+  const int rc = build_chunks(pl, l, st);
+  if (rc) return rc;
+  TUNA_CUDA(pl, cudaStreamSynchronize(st));
   pl->rows_valid = true;
   return TUNA_OK;
 }
@@ -1791,7 +1818,7 @@ int tuna_direct_alltoallv_static(int P, int elem_size, const int64_t *sendcounts
   a.extent[TUNA_BUF_SEND] = se;
   a.extent[TUNA_BUF_RECV] = re;
   a.extent[TUNA_BUF_WORK] = 0;
-  TUNA_STATIC_CUDA(tuna_launch_move(TUNA_K_DIRECT, a, payload / PP < kSmallBlockBytes, st));
+  TUNA_STATIC_CUDA(tuna_launch_move(TUNA_K_DIRECT, a, payload / PP < kStaticSmallBlockBytes, st));
 #undef TUNA_STATIC_CUDA
   return TUNA_OK;
 }
