@@ -39,7 +39,7 @@ UNIT = "GB/s"
 # reported as null.  Captures: profiles/round_kernel_c4_reduced.md (c4, reduced to
 # 2 GiB) and profiles/round_small_kernel_c5.md (c5 at full size).
 NCU_TRAFFIC_PER_PAYLOAD_BYTE: dict[str, dict[str, float]] = {
-    "8ae500aca2f084ae5fc3b99ea0c685586cd50b1d5093301ea8d51ce848eded44": {"c4": 1.979, "c5": 2.336},
+    "6d329643b4d0f21852306ca2c777d1a1af07f22b26f4a5b65df95b9f9cd9df01": {"c4": 1.979, "c5": 2.329},
 }
 
 
