@@ -22,6 +22,7 @@
 #include <algorithm>
 #include <mutex>
 #include <new>
+#include <thread>
 
 #include "tuna_internal.h"
 
@@ -453,7 +454,15 @@ struct tuna_plan {
   std::vector<Round> rounds;
 
   // host copies for validation
-  std::vector<int64_t> h_counts, h_sdispls, h_rdispls;
+  // The count matrix on the host, for the checks at call time and as the source of
+  // the upload: two buffers (pinned when that can be had), so that new counts are
+  // validated and copied in one pass into the spare one and a rejected update
+  // leaves the plan as it was.
+  int64_t *h_counts = nullptr;  // the buffer that matches the device tables
+  int64_t *h_buf[2] = {nullptr, nullptr};
+  bool h_pinned = false;
+  int h_cur = 0;
+  std::vector<int64_t> h_sdispls, h_rdispls;
   bool have_sdispls = false, have_rdispls = false;
   int64_t send_extent = 0, recv_extent = 0, payload = 0;  // bytes
 
@@ -705,44 +714,87 @@ struct HostLayout {
   int64_t payload = 0, send_extent = 0, recv_extent = 0;  // elements
 };
 
-// One pass over the P x P matrices: rejects negative entries, sums the payload and
-// finds every rank's region size.  rdispls is indexed [dst][src] while the counts
-// are [src][dst], so the pass walks 64 x 64 tiles to keep both in cache.
+// The host's pass over the P x P matrices: rejects negative entries, sums the
+// payload, finds every rank's region size and (copy_to) keeps a copy of the counts.
+// Rows are walked in order, in bands shared out over a few threads; rdispls, which
+// is indexed [dst][src] against the counts' [src][dst], gets a second, tiled walk
+// (64 x 64) so that both stay in cache.
 int host_layout(int P, const int64_t *counts, const int64_t *sdispls, const int64_t *rdispls,
-                const int64_t *sendbase, const int64_t *recvbase, HostLayout *out) {
+                const int64_t *sendbase, const int64_t *recvbase, HostLayout *out,
+                int64_t *copy_to = nullptr) {
   if (!counts) return TUNA_ERR_INVALID_ARG;
-  std::vector<int64_t> sreg(P, 0), rreg(P, 0);
-  int64_t payload = 0;
-  bool bad = false;
-  constexpr int T = 64;
-  for (int s0 = 0; s0 < P; s0 += T)
-    for (int d0 = 0; d0 < P; d0 += T) {
-      const int s1 = std::min(P, s0 + T), d1 = std::min(P, d0 + T);
-      for (int s = s0; s < s1; s++) {
-        const int64_t *crow = counts + (int64_t)s * P;
-        int64_t sr = sreg[s];
-        for (int d = d0; d < d1; d++) {
-          const int64_t c = crow[d];
-          bad |= c < 0;
-          payload += c;
-          if (sdispls) {
-            const int64_t x = sdispls[(int64_t)s * P + d];
-            bad |= x < 0;
-            sr = std::max(sr, x + c);
-          } else {
-            sr += c;
-          }
-          if (rdispls) {
-            const int64_t x = rdispls[(int64_t)d * P + s];
-            bad |= x < 0;
-            rreg[d] = std::max(rreg[d], x + c);
-          } else {
-            rreg[d] += c;
+  const int64_t PP = (int64_t)P * P;
+  int nt = 1;
+  if (PP >= (1 << 20)) {
+    const unsigned hc = std::thread::hardware_concurrency();
+    nt = (int)std::min<unsigned>(8, hc ? hc : 1);
+    nt = std::max(1, std::min(nt, P / 64));
+  }
+  std::vector<int64_t> sreg(P, 0);
+  std::vector<std::vector<int64_t>> rpart(nt, std::vector<int64_t>(P, 0));
+  std::vector<int64_t> pay(nt, 0);
+  std::vector<char> badv(nt, 0);
+  auto band = [&](int t) {
+    const int s_lo = (int)((int64_t)P * t / nt), s_hi = (int)((int64_t)P * (t + 1) / nt);
+    int64_t payload = 0;
+    bool bad = false;
+    int64_t *rr = rpart[t].data();
+    for (int s = s_lo; s < s_hi; s++) {
+      const int64_t *crow = counts + (int64_t)s * P;
+      const int64_t *drow = sdispls ? sdispls + (int64_t)s * P : nullptr;
+      int64_t *keep = copy_to ? copy_to + (int64_t)s * P : nullptr;
+      int64_t sr = 0;
+      for (int d = 0; d < P; d++) {
+        const int64_t c = crow[d];
+        if (keep) keep[d] = c;
+        bad |= c < 0;
+        payload += c;
+        if (drow) {
+          bad |= drow[d] < 0;
+          sr = std::max(sr, drow[d] + c);
+        } else {
+          sr += c;
+        }
+        if (!rdispls) rr[d] += c;
+      }
+      sreg[s] = sr;
+    }
+    if (rdispls) {
+      constexpr int T = 64;
+      for (int s0 = s_lo; s0 < s_hi; s0 += T)
+        for (int d0 = 0; d0 < P; d0 += T) {
+          const int s1 = std::min(s_hi, s0 + T), d1 = std::min(P, d0 + T);
+          for (int d = d0; d < d1; d++) {
+            const int64_t *xrow = rdispls + (int64_t)d * P;
+            int64_t m = rr[d];
+            for (int s = s0; s < s1; s++) {
+              const int64_t x = xrow[s];
+              bad |= x < 0;
+              m = std::max(m, x + counts[(int64_t)s * P + d]);
+            }
+            rr[d] = m;
           }
         }
-        sreg[s] = sr;
-      }
     }
+    pay[t] = payload;
+    badv[t] = bad;
+  };
+  if (nt == 1) {
+    band(0);
+  } else {
+    std::vector<std::thread> th;
+    for (int t = 1; t < nt; t++) th.emplace_back(band, t);
+    band(0);
+    for (auto &x : th) x.join();
+  }
+  bool bad = false;
+  int64_t payload = 0;
+  std::vector<int64_t> rreg(P, 0);
+  for (int t = 0; t < nt; t++) {
+    bad |= badv[t] != 0;
+    payload += pay[t];
+    for (int d = 0; d < P; d++) rreg[d] = rdispls ? std::max(rreg[d], rpart[t][d]) : rreg[d] + rpart[t][d];
+  }
   for (int p = 0; p < P; p++) bad |= (sendbase && sendbase[p] < 0) || (recvbase && recvbase[p] < 0);
   if (bad) return TUNA_ERR_INVALID_ARG;
   out->sendbase.resize(P);
@@ -763,8 +815,9 @@ int host_layout(int P, const int64_t *counts, const int64_t *sdispls, const int6
 }
 
 // Uploads the layout, runs every plan kernel, reads the totals back.
-int build_tables(tuna_plan *pl, const HostLayout &hl, const int64_t *counts, const int64_t *sdispls,
-                 const int64_t *rdispls, cudaStream_t st) {
+int build_tables(tuna_plan *pl, const HostLayout &hl, const int64_t *sdispls, const int64_t *rdispls,
+                 cudaStream_t st) {
+  const int64_t *counts = pl->h_counts;  // validated and copied by host_layout
   const TunaTopo &t = pl->topo;
   const int P = t.P;
   const int64_t PP = (int64_t)P * P;
@@ -772,7 +825,6 @@ int build_tables(tuna_plan *pl, const HostLayout &hl, const int64_t *counts, con
 
   pl->rows_valid = false;  // a row list belongs to the counts it was built for
   // host copies for the checks at call time
-  pl->h_counts.assign(counts, counts + PP);
   pl->have_sdispls = sdispls != nullptr;
   pl->have_rdispls = rdispls != nullptr;
   if (sdispls) pl->h_sdispls.assign(sdispls, sdispls + PP); else pl->h_sdispls.clear();
@@ -1005,7 +1057,7 @@ int check_call_args(const tuna_plan *pl, const int64_t *sendcounts, const int64_
                     const int64_t *recvcounts, const int64_t *rdispls) {
   const int P = pl->topo.P;
   const int64_t PP = (int64_t)P * P;
-  if (sendcounts && memcmp(sendcounts, pl->h_counts.data(), PP * 8) != 0) return TUNA_ERR_COUNT_MISMATCH;
+  if (sendcounts && memcmp(sendcounts, pl->h_counts, PP * 8) != 0) return TUNA_ERR_COUNT_MISMATCH;
   if (recvcounts)
     for (int d = 0; d < P; d++)
       for (int s = 0; s < P; s++)
@@ -1167,6 +1219,12 @@ int tuna_plan_destroy(tuna_plan_t *pl) {
   free_list(pl->dir);
   free_list(pl->rowsl);
   cudaFree(pl->d_row_start);
+  for (int i = 0; i < 2; i++) {
+    if (pl->h_pinned)
+      cudaFreeHost(pl->h_buf[i]);
+    else
+      free(pl->h_buf[i]);
+  }
   cudaFree(pl->d_counts);
   cudaFree(pl->d_sdispls);
   cudaFree(pl->d_rdispls);
@@ -1207,12 +1265,37 @@ static int plan_create(tuna_plan_t **out, int P, int radix, int radix_global, in
     return TUNA_ERR_BAD_RADIX;
   if (block_count < 0 || (block_count > 0 && (flags & TUNA_FLAG_CLASSIC_ROTATE)))
     return TUNA_ERR_INVALID_ARG;
-  HostLayout hl;
-  int rc = host_layout(P, sendcounts, sdispls, rdispls, sendbase, recvbase, &hl);
-  if (rc) return rc;
-
   tuna_plan *pl = new (std::nothrow) tuna_plan();
   if (!pl) return TUNA_ERR_NOMEM;
+  // host buffers for the counts: pinned if possible (the upload then runs at the
+  // host link's rate and without a staging copy), plain memory otherwise
+  {
+    const size_t bytes = (size_t)P * P * sizeof(int64_t);
+    void *a = nullptr, *b = nullptr;
+    if (cudaHostAlloc(&a, bytes, cudaHostAllocDefault) == cudaSuccess &&
+        cudaHostAlloc(&b, bytes, cudaHostAllocDefault) == cudaSuccess) {
+      pl->h_pinned = true;
+    } else {
+      (void)cudaGetLastError();
+      if (a) cudaFreeHost(a);
+      a = malloc(bytes);
+      b = malloc(bytes);
+    }
+    pl->h_buf[0] = (int64_t *)a;
+    pl->h_buf[1] = (int64_t *)b;
+    if (!a || !b) {
+      tuna_plan_destroy(pl);
+      return TUNA_ERR_NOMEM;
+    }
+  }
+  HostLayout hl;
+  int rc = host_layout(P, sendcounts, sdispls, rdispls, sendbase, recvbase, &hl, pl->h_buf[0]);
+  if (rc) {
+    tuna_plan_destroy(pl);
+    return rc;
+  }
+  pl->h_cur = 0;
+  pl->h_counts = pl->h_buf[0];
   pl->topo = TunaTopo{P, l, g, elem_size};
   pl->radix_l = radix;
   pl->radix_g = (g > 1 && block_count == 0) ? radix_global : 2;
@@ -1277,7 +1360,7 @@ static int plan_create(tuna_plan_t **out, int P, int radix, int radix_global, in
   rc = alloc_list(pl, pl->dir, TUNA_LIST_DELIVER, PP);
   if (rc) return nomem(rc);
 #undef TUNA_TRY
-  rc = build_tables(pl, hl, sendcounts, sdispls, rdispls, st);
+  rc = build_tables(pl, hl, sdispls, rdispls, st);
   if (rc) return fail(rc);
   *out = pl;
   return TUNA_OK;
@@ -1308,9 +1391,13 @@ int tuna_plan_update_counts(tuna_plan_t *pl, const int64_t *sendcounts, const in
                             const int64_t *recvbase, void *stream) {
   if (!pl || !sendcounts) return TUNA_ERR_INVALID_ARG;
   HostLayout hl;
-  const int rc = host_layout(pl->topo.P, sendcounts, sdispls, rdispls, sendbase, recvbase, &hl);
-  if (rc) return rc;
-  return build_tables(pl, hl, sendcounts, sdispls, rdispls, (cudaStream_t)stream);
+  const int spare = pl->h_cur ^ 1;
+  const int rc = host_layout(pl->topo.P, sendcounts, sdispls, rdispls, sendbase, recvbase, &hl,
+                             pl->h_buf[spare]);
+  if (rc) return rc;  // the plan still holds its previous counts
+  pl->h_cur = spare;
+  pl->h_counts = pl->h_buf[spare];
+  return build_tables(pl, hl, sdispls, rdispls, (cudaStream_t)stream);
 }
 
 int tuna_plan_workspace_bytes(const tuna_plan_t *pl, size_t *bytes) {

@@ -259,6 +259,35 @@ def test_update_counts_and_rerun():
         check_rounds(plan, rounds)
 
 
+@pytest.mark.parametrize("P", [10, 1100])
+def test_rejected_update_leaves_the_plan_as_it_was(P):
+    """New counts with a negative entry are refused; the plan still checks calls against,
+    and exchanges, the counts it had.  P = 1100 takes the threaded host pass."""
+    wl = W.make_random(P, 40 if P > 100 else 400, seed=31, zero_frac=0.2, gaps=P < 100)
+    plan = B.plan_for(wl, 4)
+    plan.alloc_workspace()
+    bad = wl.sendcounts.copy()
+    bad[P - 1, P // 2] = -3
+    with pytest.raises(B.TunaError, match="INVALID_ARG"):
+        plan.update_counts(bad, wl.sdispls, wl.rdispls, wl.sendbase, wl.recvbase)
+    bad_d = wl.rdispls.copy()
+    bad_d[P // 3, P - 1] = -1
+    with pytest.raises(B.TunaError, match="INVALID_ARG"):
+        plan.update_counts(wl.sendcounts, wl.sdispls, bad_d, wl.sendbase, wl.recvbase)
+    send, recv = wl.make_send("cuda"), wl.make_recv("cuda", fill=CANARY)
+    plan.alltoallv(send, recv, sendcounts=wl.sendcounts, sdispls=wl.sdispls,
+                   recvcounts=wl.recvcounts, rdispls=wl.rdispls)
+    torch.cuda.synchronize()
+    assert np.array_equal(recv.cpu().numpy(), oracle_brute(wl))
+    other = wl.sendcounts.copy()
+    other[0, 0] += 1
+    with pytest.raises(B.TunaError, match="COUNT_MISMATCH"):
+        plan.alltoallv(send, recv, sendcounts=other)
+    # extents and payload from the threaded pass agree with the generator's
+    se, re_, payload = plan.extents()
+    assert (se, re_) == (wl.send_bytes, wl.recv_bytes) and payload == wl.payload_bytes_total
+
+
 def test_host_buffer_entry_point():
     wl = W.make_random(9, 20000, seed=5, zero_frac=0.2, gaps=True)   # mean block over 2 KiB
     ref = oracle_brute(wl)                                   # canary 0xA5 in the gaps
