@@ -394,15 +394,20 @@ def ours_arm(args):
         dist.barrier()
     torch.cuda.synchronize()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]  # end of every step
     with ClockSampler(local) as clocks:
         ev0.record()
-        for _ in range(args.steps):
+        for i in range(args.steps):
             step()
+            marks[i].record()
         ev1.record()
         torch.cuda.synchronize()
     if dist:
         dist.barrier()
     elapsed_ms = ev0.elapsed_time(ev1)
+    per_step = [a.elapsed_time(b) for a, b in zip([ev0] + marks[:-1], marks)]
+    step_ms = {"median": statistics.median(per_step), "min": min(per_step), "max": max(per_step),
+               "stddev": statistics.pstdev(per_step)} if per_step else None
     launches = plan.launch_count() - launches0
     timing = plan.get_timing(reset=True)
     plan.enable_timing(False)
@@ -539,7 +544,7 @@ def ours_arm(args):
                        "replicas": "one independent exchange per GPU" if world > 1 else "single GPU"},
             "gpu_launches": int(launches), "parity_samples_ok": ok,
             "clocks": clocks.summary(), "e2e": e2e, "roofline": roofline,
-            "cpu_baseline": cpu, "sweep": sweep,
+            "cpu_baseline": cpu, "step_ms": step_ms, "sweep": sweep,
         }
         print(json.dumps(line), flush=True)
     if dist:

@@ -175,7 +175,9 @@ int tuna_plan_extents(const tuna_plan_t *plan, size_t *send_bytes, size_t *recv_
  *                      copies drive the kernels.  recvcounts[d*P+s] must equal
  *                      sendcounts[s*P+d].
  * Asynchronous on `stream`; re-runnable; two calls on one plan must not overlap
- * in time (they share the workspace).
+ * in time (they share the workspace).  With timing off the call only enqueues
+ * kernels (no allocation, no synchronisation), so it may be captured into a CUDA
+ * graph and replayed while plan, workspace and buffers stay as they were.
  */
 int tuna_alltoallv(tuna_plan_t *plan, const void *sendbuf, const int64_t *sendcounts,
                    const int64_t *sdispls, void *recvbuf, const int64_t *recvcounts,

@@ -288,6 +288,31 @@ def test_rejected_update_leaves_the_plan_as_it_was(P):
     assert (se, re_) == (wl.send_bytes, wl.recv_bytes) and payload == wl.payload_bytes_total
 
 
+@pytest.mark.parametrize("kw", [dict(radix=2), dict(radix=3, l=3, g=4, rg=2), dict(radix=12, direct=True)])
+def test_exchange_replayed_from_a_cuda_graph(kw):
+    """The exchange only enqueues kernels, so it can be captured once and replayed."""
+    wl = W.make_random(12, 700, seed=41, zero_frac=0.2, gaps=True)
+    kw = dict(kw)
+    direct = kw.pop("direct", False)
+    plan = B.plan_for(wl, kw.pop("radix"), l=kw.pop("l", None), g=kw.pop("g", 1), radix_global=kw.pop("rg", 2))
+    plan.alloc_workspace()
+    send, recv = wl.make_send("cuda"), wl.make_recv("cuda", fill=CANARY)
+    run = plan.direct_alltoallv if direct else plan.alltoallv
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        run(send, recv)                         # warm-up outside the capture
+        stream.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            run(send, recv)
+        for _ in range(3):
+            recv.copy_(wl.make_recv("cuda", fill=CANARY))
+            graph.replay()
+            stream.synchronize()
+            assert np.array_equal(recv.cpu().numpy(), oracle_brute(wl))
+    assert plan.device_status() == 0
+
+
 def test_host_buffer_entry_point():
     wl = W.make_random(9, 20000, seed=5, zero_frac=0.2, gaps=True)   # mean block over 2 KiB
     ref = oracle_brute(wl)                                   # canary 0xA5 in the gaps
