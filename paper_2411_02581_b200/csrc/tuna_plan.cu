@@ -20,6 +20,7 @@
 #include <string.h>
 
 #include <algorithm>
+#include <atomic>
 #include <mutex>
 #include <new>
 #include <thread>
@@ -468,6 +469,8 @@ struct tuna_plan {
 
   // device tables
   int64_t *d_counts = nullptr, *d_sdispls = nullptr, *d_rdispls = nullptr;
+  int64_t *d_counts_buf[2] = {nullptr, nullptr};  // d_counts is one of them; an update fills the other
+  bool counts_uploaded = false;  // the host pass already sent the counts to d_counts
   int64_t *d_sendbase = nullptr, *d_recvbase = nullptr;
   int64_t *d_sz[2] = {nullptr, nullptr}, *d_loc[2] = {nullptr, nullptr};
   int64_t *d_seg_total = nullptr, *d_seg_raw = nullptr, *d_seg_base = nullptr;
@@ -714,78 +717,111 @@ struct HostLayout {
   int64_t payload = 0, send_extent = 0, recv_extent = 0;  // elements
 };
 
+// Where the validated counts go on the device while the host's pass is still
+// running (optional).
+struct CountUpload {
+  int64_t *d_dst = nullptr;
+  cudaStream_t st = nullptr;
+  bool done = false;       // out: every row has been handed to the copy engine
+  cudaError_t err = cudaSuccess;
+};
+
 // The host's pass over the P x P matrices: rejects negative entries, sums the
 // payload, finds every rank's region size and (copy_to) keeps a copy of the counts.
-// Rows are walked in order, in bands shared out over a few threads; rdispls, which
-// is indexed [dst][src] against the counts' [src][dst], gets a second, tiled walk
-// (64 x 64) so that both stay in cache.
+// Rows are walked in order, in blocks of rows that a few threads take in turn;
+// rdispls, which is indexed [dst][src] against the counts' [src][dst], gets a
+// second, tiled walk (64 x 64) so that both stay in cache.  With `up`, the calling
+// thread sends every finished block of the copy to the device at once, in order,
+// so the upload runs beside the pass instead of after it.
 int host_layout(int P, const int64_t *counts, const int64_t *sdispls, const int64_t *rdispls,
                 const int64_t *sendbase, const int64_t *recvbase, HostLayout *out,
-                int64_t *copy_to = nullptr) {
+                int64_t *copy_to = nullptr, CountUpload *up = nullptr) {
   if (!counts) return TUNA_ERR_INVALID_ARG;
   const int64_t PP = (int64_t)P * P;
   int nt = 1;
   if (PP >= (1 << 20)) {
     const unsigned hc = std::thread::hardware_concurrency();
-    nt = (int)std::min<unsigned>(8, hc ? hc : 1);
-    nt = std::max(1, std::min(nt, P / 64));
+    nt = (int)std::min<unsigned>(8, hc > 1 ? hc - 1 : 1);
+    nt = (int)env_i64("TUNA_HOST_THREADS", nt);
+    nt = std::max(1, std::min(std::min(nt, 64), P / 64));
   }
+  const int nblk = nt == 1 ? 1 : 4 * nt;  // blocks of rows; thread t takes t, t + nt, ...
+  auto row_of = [&](int k) { return (int)((int64_t)P * k / nblk); };
   std::vector<int64_t> sreg(P, 0);
   std::vector<std::vector<int64_t>> rpart(nt, std::vector<int64_t>(P, 0));
   std::vector<int64_t> pay(nt, 0);
   std::vector<char> badv(nt, 0);
-  auto band = [&](int t) {
-    const int s_lo = (int)((int64_t)P * t / nt), s_hi = (int)((int64_t)P * (t + 1) / nt);
+  std::vector<std::atomic<int>> ready(nblk);
+  for (auto &r : ready) r.store(0, std::memory_order_relaxed);
+  auto work = [&](int t) {
     int64_t payload = 0;
     bool bad = false;
     int64_t *rr = rpart[t].data();
-    for (int s = s_lo; s < s_hi; s++) {
-      const int64_t *crow = counts + (int64_t)s * P;
-      const int64_t *drow = sdispls ? sdispls + (int64_t)s * P : nullptr;
-      int64_t *keep = copy_to ? copy_to + (int64_t)s * P : nullptr;
-      int64_t sr = 0;
-      for (int d = 0; d < P; d++) {
-        const int64_t c = crow[d];
-        if (keep) keep[d] = c;
-        bad |= c < 0;
-        payload += c;
-        if (drow) {
-          bad |= drow[d] < 0;
-          sr = std::max(sr, drow[d] + c);
-        } else {
-          sr += c;
-        }
-        if (!rdispls) rr[d] += c;
-      }
-      sreg[s] = sr;
-    }
-    if (rdispls) {
-      constexpr int T = 64;
-      for (int s0 = s_lo; s0 < s_hi; s0 += T)
-        for (int d0 = 0; d0 < P; d0 += T) {
-          const int s1 = std::min(s_hi, s0 + T), d1 = std::min(P, d0 + T);
-          for (int d = d0; d < d1; d++) {
-            const int64_t *xrow = rdispls + (int64_t)d * P;
-            int64_t m = rr[d];
-            for (int s = s0; s < s1; s++) {
-              const int64_t x = xrow[s];
-              bad |= x < 0;
-              m = std::max(m, x + counts[(int64_t)s * P + d]);
-            }
-            rr[d] = m;
+    for (int k = t; k < nblk; k += nt) {
+      const int s_lo = row_of(k), s_hi = row_of(k + 1);
+      for (int s = s_lo; s < s_hi; s++) {
+        const int64_t *crow = counts + (int64_t)s * P;
+        const int64_t *drow = sdispls ? sdispls + (int64_t)s * P : nullptr;
+        int64_t *keep = copy_to ? copy_to + (int64_t)s * P : nullptr;
+        int64_t sr = 0;
+        for (int d = 0; d < P; d++) {
+          const int64_t c = crow[d];
+          if (keep) keep[d] = c;
+          bad |= c < 0;
+          payload += c;
+          if (drow) {
+            bad |= drow[d] < 0;
+            sr = std::max(sr, drow[d] + c);
+          } else {
+            sr += c;
           }
+          if (!rdispls) rr[d] += c;
         }
+        sreg[s] = sr;
+      }
+      ready[k].store(1, std::memory_order_release);  // the copy of these rows is complete
+      if (rdispls) {
+        constexpr int T = 64;
+        for (int s0 = s_lo; s0 < s_hi; s0 += T)
+          for (int d0 = 0; d0 < P; d0 += T) {
+            const int s1 = std::min(s_hi, s0 + T), d1 = std::min(P, d0 + T);
+            for (int d = d0; d < d1; d++) {
+              const int64_t *xrow = rdispls + (int64_t)d * P;
+              int64_t m = rr[d];
+              for (int s = s0; s < s1; s++) {
+                const int64_t x = xrow[s];
+                bad |= x < 0;
+                m = std::max(m, x + counts[(int64_t)s * P + d]);
+              }
+              rr[d] = m;
+            }
+          }
+      }
     }
     pay[t] = payload;
     badv[t] = bad;
   };
+  auto send_block = [&](int k) {  // rows of block k: host copy -> device
+    const int64_t lo = (int64_t)row_of(k) * P, hi = (int64_t)row_of(k + 1) * P;
+    if (hi > lo && up->err == cudaSuccess)
+      up->err = cudaMemcpyAsync(up->d_dst + lo, copy_to + lo, (size_t)(hi - lo) * 8, cudaMemcpyHostToDevice, up->st);
+  };
+  const bool streaming = up && copy_to && nt > 1;
   if (nt == 1) {
-    band(0);
+    work(0);
   } else {
     std::vector<std::thread> th;
-    for (int t = 1; t < nt; t++) th.emplace_back(band, t);
-    band(0);
+    for (int t = 0; t < nt; t++) th.emplace_back(work, t);
+    if (streaming)
+      for (int k = 0; k < nblk; k++) {
+        while (ready[k].load(std::memory_order_acquire) == 0) std::this_thread::yield();
+        send_block(k);
+      }
     for (auto &x : th) x.join();
+  }
+  if (streaming) {
+    if (up->err != cudaSuccess) return TUNA_ERR_CUDA;
+    up->done = true;
   }
   bool bad = false;
   int64_t payload = 0;
@@ -835,7 +871,9 @@ int build_tables(tuna_plan *pl, const HostLayout &hl, const int64_t *sdispls, co
   pl->recv_extent = hl.recv_extent * t.elem;
 
   Timed plan_timer(pl, TUNA_TIMER_PLAN, 0, st);
-  TUNA_CUDA(pl, cudaMemcpyAsync(pl->d_counts, counts, PP * 8, cudaMemcpyHostToDevice, st));
+  if (!pl->counts_uploaded)
+    TUNA_CUDA(pl, cudaMemcpyAsync(pl->d_counts, counts, PP * 8, cudaMemcpyHostToDevice, st));
+  pl->counts_uploaded = false;
   TUNA_CUDA(pl, cudaMemcpyAsync(pl->d_sendbase, sb.data(), P * 8, cudaMemcpyHostToDevice, st));
   TUNA_CUDA(pl, cudaMemcpyAsync(pl->d_recvbase, rb.data(), P * 8, cudaMemcpyHostToDevice, st));
   // sb/rb are pageable stack-owned vectors: the copies above are staged by the
@@ -1225,7 +1263,8 @@ int tuna_plan_destroy(tuna_plan_t *pl) {
     else
       free(pl->h_buf[i]);
   }
-  cudaFree(pl->d_counts);
+  cudaFree(pl->d_counts_buf[0]);
+  cudaFree(pl->d_counts_buf[1]);
   cudaFree(pl->d_sdispls);
   cudaFree(pl->d_rdispls);
   cudaFree(pl->d_sendbase);
@@ -1324,7 +1363,9 @@ static int plan_create(tuna_plan_t **out, int P, int radix, int radix_global, in
       return fail(code_);                               \
     }                                                   \
   } while (0)
-  TUNA_TRY(dev_alloc(&pl->d_counts, PP));
+  TUNA_TRY(dev_alloc(&pl->d_counts_buf[0], PP));
+  TUNA_TRY(dev_alloc(&pl->d_counts_buf[1], PP));
+  pl->d_counts = pl->d_counts_buf[0];
   TUNA_TRY(dev_alloc(&pl->d_sdispls, PP));
   TUNA_TRY(dev_alloc(&pl->d_rdispls, PP));
   TUNA_TRY(dev_alloc(&pl->d_sendbase, P));
@@ -1392,11 +1433,21 @@ int tuna_plan_update_counts(tuna_plan_t *pl, const int64_t *sendcounts, const in
   if (!pl || !sendcounts) return TUNA_ERR_INVALID_ARG;
   HostLayout hl;
   const int spare = pl->h_cur ^ 1;
+  CountUpload up;  // the spare device buffer takes the new counts while the pass is running
+  up.d_dst = pl->d_counts == pl->d_counts_buf[0] ? pl->d_counts_buf[1] : pl->d_counts_buf[0];
+  up.st = (cudaStream_t)stream;
   const int rc = host_layout(pl->topo.P, sendcounts, sdispls, rdispls, sendbase, recvbase, &hl,
-                             pl->h_buf[spare]);
-  if (rc) return rc;  // the plan still holds its previous counts
+                             pl->h_buf[spare], &up);
+  if (rc) {  // the plan still holds its previous counts, on the host and on the device
+    if (rc == TUNA_ERR_CUDA) pl->cuda_err = (int)up.err;
+    return rc;
+  }
   pl->h_cur = spare;
   pl->h_counts = pl->h_buf[spare];
+  if (up.done) {
+    pl->d_counts = up.d_dst;
+    pl->counts_uploaded = true;
+  }
   return build_tables(pl, hl, sdispls, rdispls, (cudaStream_t)stream);
 }
 
