@@ -18,9 +18,12 @@
 #include <stdio.h>
 #include <stdlib.h>
 #include <string.h>
+#include <unistd.h>
 
 #include <algorithm>
 #include <atomic>
+#include <condition_variable>
+#include <functional>
 #include <mutex>
 #include <new>
 #include <thread>
@@ -717,6 +720,67 @@ struct HostLayout {
   int64_t payload = 0, send_extent = 0, recv_extent = 0;  // elements
 };
 
+// A few parked host threads for the pass over large count matrices (starting
+// threads anew costs more than the pass itself).  One job at a time; created on
+// first use and never torn down.
+class HostPool {
+ public:
+  static HostPool &get() {
+    static HostPool *pool = new HostPool();
+    return *pool;
+  }
+  int size() const { return (int)workers_.size(); }
+  bool usable() const { return !workers_.empty() && owner_ == getpid(); }  // threads do not survive a fork
+  // Runs fn(i) for i in [0, n) on n of the parked threads and returns at once.
+  void start(int n, std::function<void(int)> fn) {
+    busy_.lock();
+    std::lock_guard<std::mutex> lk(m_);
+    job_ = std::move(fn);
+    want_ = n;
+    pending_ = n;
+    gen_++;
+    work_.notify_all();
+  }
+  void wait() {
+    {
+      std::unique_lock<std::mutex> lk(m_);
+      done_.wait(lk, [&] { return pending_ == 0; });
+    }
+    busy_.unlock();
+  }
+
+ private:
+  HostPool() : owner_(getpid()) {
+    const unsigned hc = std::thread::hardware_concurrency();
+    const int n = (int)std::min<unsigned>(8, hc > 1 ? hc - 1 : 0);
+    for (int i = 0; i < n; i++) {
+      workers_.emplace_back([this, i] { loop(i); });
+      workers_.back().detach();
+    }
+  }
+  void loop(int i) {
+    unsigned seen = 0;
+    for (;;) {
+      std::unique_lock<std::mutex> lk(m_);
+      work_.wait(lk, [&] { return gen_ != seen; });
+      seen = gen_;
+      if (i >= want_) continue;
+      std::function<void(int)> f = job_;
+      lk.unlock();
+      f(i);
+      lk.lock();
+      if (--pending_ == 0) done_.notify_all();
+    }
+  }
+  std::mutex m_, busy_;
+  std::condition_variable work_, done_;
+  std::function<void(int)> job_;
+  std::vector<std::thread> workers_;
+  unsigned gen_ = 0;
+  int want_ = 0, pending_ = 0;
+  pid_t owner_;
+};
+
 // Where the validated counts go on the device while the host's pass is still
 // running (optional).
 struct CountUpload {
@@ -739,11 +803,12 @@ int host_layout(int P, const int64_t *counts, const int64_t *sdispls, const int6
   if (!counts) return TUNA_ERR_INVALID_ARG;
   const int64_t PP = (int64_t)P * P;
   int nt = 1;
+  HostPool *pool = nullptr;
   if (PP >= (1 << 20)) {
-    const unsigned hc = std::thread::hardware_concurrency();
-    nt = (int)std::min<unsigned>(8, hc > 1 ? hc - 1 : 1);
-    nt = (int)env_i64("TUNA_HOST_THREADS", nt);
-    nt = std::max(1, std::min(std::min(nt, 64), P / 64));
+    pool = &HostPool::get();
+    nt = pool->usable() ? pool->size() : 1;
+    nt = (int)std::min<int64_t>(nt, env_i64("TUNA_HOST_THREADS", nt));
+    nt = std::max(1, std::min(nt, P / 64));
   }
   const int nblk = nt == 1 ? 1 : 4 * nt;  // blocks of rows; thread t takes t, t + nt, ...
   auto row_of = [&](int k) { return (int)((int64_t)P * k / nblk); };
@@ -810,14 +875,13 @@ int host_layout(int P, const int64_t *counts, const int64_t *sdispls, const int6
   if (nt == 1) {
     work(0);
   } else {
-    std::vector<std::thread> th;
-    for (int t = 0; t < nt; t++) th.emplace_back(work, t);
+    pool->start(nt, work);
     if (streaming)
       for (int k = 0; k < nblk; k++) {
         while (ready[k].load(std::memory_order_acquire) == 0) std::this_thread::yield();
         send_block(k);
       }
-    for (auto &x : th) x.join();
+    pool->wait();
   }
   if (streaming) {
     if (up->err != cudaSuccess) return TUNA_ERR_CUDA;
