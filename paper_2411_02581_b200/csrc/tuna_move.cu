@@ -41,7 +41,7 @@
 //                        afterwards by the block's own thread, in the widest
 //                        aligned pieces that fit.  No byte outside a block's
 //                        destination range is written.
-// No byte outside a source buffer's extent is read: blocks within 19 bytes of
+// No byte outside a source buffer's extent is read: blocks within 31 bytes of
 // either end of their buffer are read byte by byte instead of by aligned windows.
 #include <stdlib.h>
 
@@ -101,25 +101,10 @@ __device__ __forceinline__ void fill_owner(unsigned char *who, const int *start,
   }
 }
 
-// The 16 bytes at sa (any alignment) from five aligned words merged by funnel shifts.
-// Reads [sa - (sa & 3), +20).
-__device__ __forceinline__ uint4 load16_funnel(const char *sa) {
-  const unsigned sh = (unsigned)(reinterpret_cast<uintptr_t>(sa) & 3);
-  const uint32_t *w = reinterpret_cast<const uint32_t *>(sa - sh);
-  const uint32_t w0 = w[0], w1 = w[1], w2 = w[2], w3 = w[3], w4 = w[4];
-  const unsigned bits = sh * 8;
-  uint4 v;
-  v.x = __funnelshift_r(w0, w1, bits);
-  v.y = __funnelshift_r(w1, w2, bits);
-  v.z = __funnelshift_r(w2, w3, bits);
-  v.w = __funnelshift_r(w3, w4, bits);
-  return v;
-}
-
-// The same 16 bytes from the two 16-byte aligned vectors that hold them: word
+// The 16 bytes at sa (any alignment) from the two 16-byte aligned vectors that hold them: word
 // selection by the offset's bits 2 and 3, then funnel shifts by its low two bits.
-// Two wide loads put a fraction of the five narrow ones' load on the L1 data
-// pipe (a warp's 4-byte loads at a 16-byte stride use a quarter of every line
+// Two wide loads put far less load on the L1 data pipe than five aligned words
+// would (a warp's 4-byte loads at a 16-byte stride use a quarter of every line
 // they fetch).  Reads [sa - (sa & 15), +32).
 __device__ __forceinline__ uint4 load16_pair(const char *sa) {
   const uintptr_t a = reinterpret_cast<uintptr_t>(sa);
@@ -146,36 +131,45 @@ __device__ __noinline__ uint4 load16_bytes(const char *sa, int b0, int b1) {
   return make_uint4(w[0], w[1], w[2], w[3]);
 }
 
-// Store bytes [b0, b1) of the vector x to the 16-byte aligned global address gp, in
-// the widest naturally aligned pieces that fit.
-__device__ __forceinline__ void store_pieces(char *gp, uint4 x, int b0, int b1) {
-  const unsigned long long lo = x.x | ((unsigned long long)x.y << 32);
-  const unsigned long long hi = x.z | ((unsigned long long)x.w << 32);
-  int pos = b0;
-  while (pos < b1) {
-    const unsigned long long w = (pos < 8 ? lo : hi) >> (8 * (pos & 7));
-    if (!(pos & 7) && pos + 8 <= b1) {
-      *reinterpret_cast<unsigned long long *>(gp + pos) = w;
-      pos += 8;
-    } else if (!(pos & 3) && pos + 4 <= b1) {
-      *reinterpret_cast<uint32_t *>(gp + pos) = (uint32_t)w;
-      pos += 4;
-    } else if (!(pos & 1) && pos + 2 <= b1) {
-      *reinterpret_cast<unsigned short *>(gp + pos) = (unsigned short)w;
-      pos += 2;
-    } else {
-      gp[pos] = (char)w;
-      pos += 1;
-    }
+// Store bytes [b0, b1) of a vector parked in shared memory (sc, 16-byte aligned) to
+// the 16-byte aligned global address gp, in the widest naturally aligned pieces
+// that fit.  Every piece is a narrow shared load followed by a store of the same
+// width, so no byte is shifted in registers.  Straight-line: pieces of 1, 2, 4, 8
+// bytes while the position's alignment grows (each only if it still fits), then
+// 8, 4, 2, 1 bytes for what is left.
+__device__ __forceinline__ void store_pieces(char *gp, const unsigned char *sc, int b0, int b1) {
+  int p = b0;
+  if ((p & 1) && p + 1 <= b1) {
+    *reinterpret_cast<unsigned char *>(gp + p) = *reinterpret_cast<const unsigned char *>(sc + p);
+    p += 1;
   }
-}
-
-// One 16-byte vector from an arbitrary address; `careful` restricts the read to
-// the bytes [b0, b1).
-__device__ __forceinline__ uint4 load16_any(const char *sa, bool careful, int b0, int b1) {
-  if (careful) return load16_bytes(sa, b0, b1);
-  if ((reinterpret_cast<uintptr_t>(sa) & 15) == 0) return ld16(sa);
-  return load16_funnel(sa);  // (for these scattered single vectors the five narrow loads measured faster)
+  if ((p & 2) && p + 2 <= b1) {
+    *reinterpret_cast<unsigned short *>(gp + p) = *reinterpret_cast<const unsigned short *>(sc + p);
+    p += 2;
+  }
+  if ((p & 4) && p + 4 <= b1) {
+    *reinterpret_cast<uint32_t *>(gp + p) = *reinterpret_cast<const uint32_t *>(sc + p);
+    p += 4;
+  }
+  if ((p & 8) && p + 8 <= b1) {
+    *reinterpret_cast<unsigned long long *>(gp + p) = *reinterpret_cast<const unsigned long long *>(sc + p);
+    p += 8;
+  }
+  // p is now aligned to every size that is still to come
+  const int r = b1 - p;
+  if (r & 8) {
+    *reinterpret_cast<unsigned long long *>(gp + p) = *reinterpret_cast<const unsigned long long *>(sc + p);
+    p += 8;
+  }
+  if (r & 4) {
+    *reinterpret_cast<uint32_t *>(gp + p) = *reinterpret_cast<const uint32_t *>(sc + p);
+    p += 4;
+  }
+  if (r & 2) {
+    *reinterpret_cast<unsigned short *>(gp + p) = *reinterpret_cast<const unsigned short *>(sc + p);
+    p += 2;
+  }
+  if (r & 1) *reinterpret_cast<unsigned char *>(gp + p) = *reinterpret_cast<const unsigned char *>(sc + p);
 }
 
 // ------------------------------------------------------------------ bulk copies (TMA)
@@ -252,6 +246,7 @@ __device__ __forceinline__ void move_body(const TunaListArgs &l, const TunaMoveA
   __shared__ const char *s_sadj[kBatch];   // source address of chunk vector v is s_sadj + 16 v
   __shared__ char *s_dadj[kBatch];         // DELIVER: destination address likewise (16-byte aligned)
   __shared__ unsigned char s_careful[kBatch];
+  __shared__ __align__(16) unsigned char s_edge[DELIVER ? kBatch * 32 : 16];  // two parking slots per block: its partial first and last vector
   extern __shared__ __align__(16) unsigned char s_who[];  // owner of every vector of the chunk (chunk / 16 bytes)
 
   // bulk route (builds with kBulk only): barriers, their phase, the staging area behind the owner table
@@ -304,7 +299,7 @@ __device__ __forceinline__ void move_body(const TunaListArgs &l, const TunaMoveA
         s_end[tid] = my_end;
         s_sadj[tid] = sp - org;
         s_dadj[tid] = dp - org;
-        s_careful[tid] = (L > 0 && (sp - 19 < sbase || sp + L + 19 > sbase + extent_of(a, sb))) ? 1 : 0;
+        s_careful[tid] = (L > 0 && (sp - 31 < sbase || sp + L + 31 > sbase + extent_of(a, sb))) ? 1 : 0;
         my_edges = L > 0 && (ad != 0 || (L & 15) != 0);
         if (L > 0 && tid > 0 && vs < nv) mark_at = (int)vs;
       } else {
@@ -400,15 +395,23 @@ __device__ __forceinline__ void move_body(const TunaListArgs &l, const TunaMoveA
         bool on = vv < vhi;
         const char *sa = nullptr;
         bool careful = false;
-        int t = 0;
+        int t = 0, b0 = 0, b1 = 16;
         out[k] = nullptr;
         if (on) {
           if (!single) t = s_who[vv];
           const int64_t vb = (int64_t)vv << 4;
           if (DELIVER) {
-            // only vectors that lie wholly inside the block; its edges come later
-            on = s_org[t] <= (int)vb && s_end[t] >= (int)vb + 16;
-            out[k] = s_dadj[t] + vb;
+            // A vector that lies wholly inside the block goes straight to its place.
+            // The block's partial first and last vector are loaded here too, beside
+            // their neighbours (the same cache lines), and parked in the block's two
+            // slots of shared memory; the block's own thread stores their bytes later.
+            const int org = s_org[t], end = s_end[t];
+            b0 = org - (int)vb;
+            b1 = end - (int)vb;
+            const bool full = b0 <= 0 && b1 >= 16;
+            on = b0 < 16 && b1 > 0;
+            out[k] = full ? s_dadj[t] + vb
+                          : reinterpret_cast<char *>(s_edge) + t * 32 + (vv == (org >> 4) ? 0 : 16);
           } else {
             out[k] = keep_out + vb;
           }
@@ -423,7 +426,7 @@ __device__ __forceinline__ void move_body(const TunaListArgs &l, const TunaMoveA
           if (!careful) {
             x[k] = load16_pair(sa);
           } else if (DELIVER) {
-            x[k] = load16_bytes(sa, 0, 16);
+            x[k] = load16_bytes(sa, b0 > 0 ? b0 : 0, b1 < 16 ? b1 : 16);
           } else {
             const int64_t e = b + t;
             const int64_t rem = l.len[e] - (cA + ((int64_t)vv << 4) - l.pos[e]);
@@ -433,22 +436,21 @@ __device__ __forceinline__ void move_body(const TunaListArgs &l, const TunaMoveA
       }
 #pragma unroll
       for (int k = 0; k < kUnroll; k++)
-        if (out[k]) st16(out[k], x[k]);
+        if (out[k]) st16(out[k], x[k]);  // (a generic store: global memory or the parking slot)
     }
-    // DELIVER: the partial first and last vector of a block, by the block's own thread
-    if (DELIVER && my_edges) {
-      const int vh = my_org >> 4, vt = (my_end - 1) >> 4;
-      const bool careful = s_careful[tid] != 0;
-      if (vh >= vlo && vh < vhi && ((my_org & 15) != 0 || my_end < (vh << 4) + 16)) {
-        const int b0 = my_org - (vh << 4);
-        const int b1 = my_end - (vh << 4) < 16 ? my_end - (vh << 4) : 16;
-        const int64_t vb = (int64_t)vh << 4;
-        store_pieces(s_dadj[tid] + vb, load16_any(s_sadj[tid] + vb, careful, b0, b1), b0, b1);
-      }
-      if (vt > vh && vt >= vlo && vt < vhi && (my_end & 15) != 0) {
-        const int b1 = my_end - (vt << 4);
-        const int64_t vb = (int64_t)vt << 4;
-        store_pieces(s_dadj[tid] + vb, load16_any(s_sadj[tid] + vb, careful, 0, b1), 0, b1);
+    // DELIVER: the partial first and last vector of a block, by the block's own
+    // thread, out of the parking slots
+    if (DELIVER) {
+      __syncthreads();
+      if (my_edges) {
+        const int vh = my_org >> 4, vt = (my_end - 1) >> 4;
+        if (vh >= vlo && vh < vhi && ((my_org & 15) != 0 || my_end < (vh << 4) + 16)) {
+          const int b0 = my_org - (vh << 4);
+          const int b1 = my_end - (vh << 4) < 16 ? my_end - (vh << 4) : 16;
+          store_pieces(s_dadj[tid] + ((int64_t)vh << 4), s_edge + tid * 32, b0, b1);
+        }
+        if (vt > vh && vt >= vlo && vt < vhi && (my_end & 15) != 0)
+          store_pieces(s_dadj[tid] + ((int64_t)vt << 4), s_edge + tid * 32 + 16, 0, my_end - (vt << 4));
       }
     }
   }
