@@ -141,6 +141,28 @@ int tuna_plan_update_counts(tuna_plan_t *plan, const int64_t *sendcounts, const 
                             const int64_t *rdispls, const int64_t *sendbase,
                             const int64_t *recvbase, void *stream);
 
+/*
+ * tuna_plan_update_counts_device - as tuna_plan_update_counts, for counts that are
+ * already in device memory (routing decided on the GPU): the count-metadata
+ * exchange and the prefix sums of Sec. III-B/C then start from the device array
+ * and nothing crosses the host link but a few totals.
+ *   d_sendcounts  DEVICE pointer, P * P int64, [src][dst], in elements; read on
+ *                 `stream`; the plan keeps its own copy, so the array may be
+ *                 reused as soon as the call returns.
+ * The layout is the packed one (what tuna_plan_update_counts does with NULL
+ * displacements and bases): every rank's blocks back to back in ascending peer
+ * order, the ranks' regions back to back in both buffers.  Region bases, buffer
+ * extents and the payload size are computed on the device.
+ * Synchronises `stream` once.  The required workspace size may change; query it
+ * again.  Errors: a negative count gives TUNA_ERR_INVALID_ARG; unlike the
+ * host-array form, a failed update leaves the plan unusable (its tables have been
+ * rewritten; exchange calls return TUNA_ERR_INTERNAL) until an update succeeds.
+ * Count or displacement arrays passed to a later exchange call are still
+ * compared with the plan's: the first such call copies the counts to the host
+ * (one synchronous device-to-host copy).
+ */
+int tuna_plan_update_counts_device(tuna_plan_t *plan, const int64_t *d_sendcounts, void *stream);
+
 /* Frees the plan's device tables and the plan.  NULL is accepted. */
 int tuna_plan_destroy(tuna_plan_t *plan);
 

@@ -43,6 +43,7 @@ SIGNATURES = {
     "tuna_plan_create_staggered": (ctypes.c_int, [ctypes.POINTER(_VP)] + [ctypes.c_int] * 6
                                    + [ctypes.c_uint] + [_I64P] * 5 + [_VP]),
     "tuna_plan_update_counts": (ctypes.c_int, [_VP] + [_I64P] * 5 + [_VP]),
+    "tuna_plan_update_counts_device": (ctypes.c_int, [_VP, _VP, _VP]),
     "tuna_plan_set_row_maps": (ctypes.c_int, [_VP, _VP, _VP, ctypes.c_int64, ctypes.c_int64, _VP]),
     "tuna_rows_alltoallv": (ctypes.c_int, [_VP, _VP, _VP, _VP]),
     "tuna_plan_destroy": (ctypes.c_int, [_VP]),
@@ -171,6 +172,11 @@ class Plan:
         keep = [_h(x) for x in (sendcounts, sdispls, rdispls, sendbase, recvbase)]
         self._check(lib().tuna_plan_update_counts(self._h, *[k[1] for k in keep], _stream(stream)),
                     "tuna_plan_update_counts")
+
+    def update_counts_device(self, d_sendcounts, stream=None):
+        """New counts from a P x P int64 array in device memory (packed layout)."""
+        self._check(lib().tuna_plan_update_counts_device(self._h, _ptr(d_sendcounts), _stream(stream)),
+                    "tuna_plan_update_counts_device")
 
     def workspace_bytes(self) -> int:
         n = ctypes.c_size_t()

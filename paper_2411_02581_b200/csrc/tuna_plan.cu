@@ -389,41 +389,68 @@ __global__ void tuna_chunk_index_kernel(const int64_t *__restrict__ pos, int64_t
 // so a clean check bounds every access of the exchange.  Violations are counted.
 __global__ void tuna_check_list_kernel(const int64_t *__restrict__ len, const int64_t *__restrict__ pos,
                                        const int64_t *__restrict__ src, const int64_t *__restrict__ dst,
-                                       int64_t n, int64_t send_extent, int64_t recv_extent,
+                                       int64_t n, const int64_t *__restrict__ extents,
                                        const int64_t *__restrict__ work_extent, int64_t keep_base_index,
                                        const int64_t *__restrict__ wbase, unsigned long long *violations,
                                        unsigned long long *unaligned_bytes) {
-  const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  const int64_t L = e < n ? len[e] : 0;
-  bool bad = e < n && (L < 0 || pos[e + 1] < pos[e]);
-  int64_t skewed = 0;  // bytes of a block whose source and destination differ modulo 16
-  if (L > 0) {
-    const int64_t s = src[e];
-    const int sb = TUNA_LOC_BUF(s);
-    const int64_t so = TUNA_LOC_OFF(s);
-    const int64_t sext = sb == TUNA_BUF_SEND ? send_extent : (sb == TUNA_BUF_WORK ? *work_extent : -1);
-    bad = bad || so < 0 || so + L > sext;
-    if (dst) {  // DELIVER: into the receive buffer
-      const int64_t d = dst[e];
-      bad = bad || TUNA_LOC_BUF(d) != TUNA_BUF_RECV || TUNA_LOC_OFF(d) + L > recv_extent;
-      if (((so - TUNA_LOC_OFF(d)) & 15) != 0) skewed = L;
-    } else {    // KEEP: at its stream position in the phase's workspace region
-      const int64_t o = wbase[keep_base_index] + pos[e];
-      bad = bad || (o & (TUNA_ALIGN - 1)) != 0 || o + pad16(L) > *work_extent || pos[e + 1] - pos[e] != pad16(L);
-      if ((so & 15) != 0) skewed = L;
+  bool bad = false;
+  int64_t skewed = 0;  // bytes of blocks whose source and destination differ modulo 16
+  const int64_t send_extent = extents[0], recv_extent = extents[1];
+  for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < n; e += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t L = len[e];
+    bad = bad || L < 0 || pos[e + 1] < pos[e];
+    if (L > 0) {
+      const int64_t s = src[e];
+      const int sb = TUNA_LOC_BUF(s);
+      const int64_t so = TUNA_LOC_OFF(s);
+      const int64_t sext = sb == TUNA_BUF_SEND ? send_extent : (sb == TUNA_BUF_WORK ? *work_extent : -1);
+      bad = bad || so < 0 || so + L > sext;
+      if (dst) {  // DELIVER: into the receive buffer
+        const int64_t d = dst[e];
+        bad = bad || TUNA_LOC_BUF(d) != TUNA_BUF_RECV || TUNA_LOC_OFF(d) + L > recv_extent;
+        if (((so - TUNA_LOC_OFF(d)) & 15) != 0) skewed += L;
+      } else {    // KEEP: at its stream position in the phase's workspace region
+        const int64_t o = wbase[keep_base_index] + pos[e];
+        bad = bad || (o & (TUNA_ALIGN - 1)) != 0 || o + pad16(L) > *work_extent || pos[e + 1] - pos[e] != pad16(L);
+        if ((so & 15) != 0) skewed += L;
+      }
     }
   }
   if (bad) atomicAdd(violations, 1ULL);
+  // one atomic per CTA of a bounded grid: a list of millions of blocks would
+  // otherwise queue a hundred thousand of them on one address
+  __shared__ int64_t s_part[32];
 #pragma unroll
   for (int d = 16; d > 0; d >>= 1) skewed += __shfl_xor_sync(0xffffffffu, skewed, d);
-  if ((threadIdx.x & 31) == 0 && skewed > 0) atomicAdd(unaligned_bytes, (unsigned long long)skewed);
+  if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = skewed;
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    int64_t v = threadIdx.x < (blockDim.x + 31) / 32 ? s_part[threadIdx.x] : 0;
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(0xffffffffu, v, d);
+    if (threadIdx.x == 0 && v > 0) atomicAdd(unaligned_bytes, (unsigned long long)v);
+  }
 }
 
-__global__ void tuna_transpose_kernel(const int64_t *__restrict__ in, int64_t *out, int P) {
+// out = in^T.  With `negatives`, entries below zero are counted there (counts that
+// arrive in device memory are validated in this pass).
+__global__ void tuna_transpose_kernel(const int64_t *__restrict__ in, int64_t *out, int P, int64_t *negatives) {
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= (int64_t)P * P) return;
   const int r = (int)(idx / P), c = (int)(idx % P);
-  out[idx] = in[(int64_t)c * P + r];
+  const int64_t v = in[(int64_t)c * P + r];
+  out[idx] = v;
+  if (negatives && v < 0) atomicAdd(reinterpret_cast<unsigned long long *>(negatives), 1ULL);
+}
+
+// Packed layout worked out on the device: both buffers extend over the sum of all
+// counts (tot[0], in elements).
+__global__ void tuna_packed_extents_kernel(const int64_t *__restrict__ tot, int elem, int64_t *extents) {
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    extents[0] = tot[0] * elem;
+    extents[1] = tot[0] * elem;
+    extents[2] = tot[0];
+  }
 }
 
 }  // namespace
@@ -468,6 +495,8 @@ struct tuna_plan {
   int h_cur = 0;
   std::vector<int64_t> h_sdispls, h_rdispls;
   bool have_sdispls = false, have_rdispls = false;
+  bool h_counts_valid = true;   // false after an update from device counts, until they are read back
+  bool tables_valid = false;    // false while an update is under way and after one that failed
   int64_t send_extent = 0, recv_extent = 0, payload = 0;  // bytes
 
   // device tables
@@ -480,6 +509,8 @@ struct tuna_plan {
   int64_t *d_tmp = nullptr;      // P*P scratch (transpose)
   int64_t *d_scal = nullptr;     // per list: stream bytes, bytes moved
   int64_t *d_wbase = nullptr;    // phases + 1 workspace offsets
+  int64_t *d_extents = nullptr;  // send extent, receive extent (bytes), total of the counts (elements),
+                                 // number of negative counts seen
   unsigned long long *d_round_bytes = nullptr;
   int64_t stats_n = 0;
   int *d_error = nullptr;        // raised by a kernel whose bounded wait gave up
@@ -914,8 +945,10 @@ int host_layout(int P, const int64_t *counts, const int64_t *sdispls, const int6
   return TUNA_OK;
 }
 
-// Uploads the layout, runs every plan kernel, reads the totals back.
-int build_tables(tuna_plan *pl, const HostLayout &hl, const int64_t *sdispls, const int64_t *rdispls,
+// Uploads the layout, runs every plan kernel, reads the totals back.  Without a
+// host layout (`hl` null) the counts are already in pl->d_counts and the layout
+// is packed: region bases, extents and the payload are worked out on the device.
+int build_tables(tuna_plan *pl, const HostLayout *hl, const int64_t *sdispls, const int64_t *rdispls,
                  cudaStream_t st) {
   const int64_t *counts = pl->h_counts;  // validated and copied by host_layout
   const TunaTopo &t = pl->topo;
@@ -924,24 +957,30 @@ int build_tables(tuna_plan *pl, const HostLayout &hl, const int64_t *sdispls, co
   int rc = TUNA_OK;
 
   pl->rows_valid = false;  // a row list belongs to the counts it was built for
+  pl->tables_valid = false;
   // host copies for the checks at call time
   pl->have_sdispls = sdispls != nullptr;
   pl->have_rdispls = rdispls != nullptr;
   if (sdispls) pl->h_sdispls.assign(sdispls, sdispls + PP); else pl->h_sdispls.clear();
   if (rdispls) pl->h_rdispls.assign(rdispls, rdispls + PP); else pl->h_rdispls.clear();
-  const std::vector<int64_t> &sb = hl.sendbase, &rb = hl.recvbase;
-  pl->payload = hl.payload * t.elem;
-  pl->send_extent = hl.send_extent * t.elem;
-  pl->recv_extent = hl.recv_extent * t.elem;
+  pl->h_counts_valid = hl != nullptr;
 
   Timed plan_timer(pl, TUNA_TIMER_PLAN, 0, st);
-  if (!pl->counts_uploaded)
-    TUNA_CUDA(pl, cudaMemcpyAsync(pl->d_counts, counts, PP * 8, cudaMemcpyHostToDevice, st));
+  if (hl) {
+    pl->payload = hl->payload * t.elem;
+    pl->send_extent = hl->send_extent * t.elem;
+    pl->recv_extent = hl->recv_extent * t.elem;
+    if (!pl->counts_uploaded)
+      TUNA_CUDA(pl, cudaMemcpyAsync(pl->d_counts, counts, PP * 8, cudaMemcpyHostToDevice, st));
+    TUNA_CUDA(pl, cudaMemcpyAsync(pl->d_sendbase, hl->sendbase.data(), P * 8, cudaMemcpyHostToDevice, st));
+    TUNA_CUDA(pl, cudaMemcpyAsync(pl->d_recvbase, hl->recvbase.data(), P * 8, cudaMemcpyHostToDevice, st));
+    const int64_t ext[4] = {pl->send_extent, pl->recv_extent, hl->payload, 0};
+    TUNA_CUDA(pl, cudaMemcpyAsync(pl->d_extents, ext, sizeof(ext), cudaMemcpyHostToDevice, st));
+    // (pageable sources: the runtime stages these copies before it returns)
+  } else {
+    TUNA_CUDA(pl, cudaMemsetAsync(pl->d_extents, 0, 4 * 8, st));
+  }
   pl->counts_uploaded = false;
-  TUNA_CUDA(pl, cudaMemcpyAsync(pl->d_sendbase, sb.data(), P * 8, cudaMemcpyHostToDevice, st));
-  TUNA_CUDA(pl, cudaMemcpyAsync(pl->d_recvbase, rb.data(), P * 8, cudaMemcpyHostToDevice, st));
-  // sb/rb are pageable stack-owned vectors: the copies above are staged by the
-  // runtime before returning, so they may go out of scope.
   const int th = 256;
   const unsigned gPP = (unsigned)((PP + th - 1) / th);
   const unsigned gseg = (unsigned)(((int64_t)P * 32 + th - 1) / th);
@@ -951,15 +990,27 @@ int build_tables(tuna_plan *pl, const HostLayout &hl, const int64_t *sdispls, co
     tuna_segscan_kernel<0><<<gseg, th, 0, st>>>(pl->d_counts, pl->d_sdispls, pl->d_seg_total,
                                                  nullptr, P, P);
     TUNA_LAUNCHED(pl);
+    if (!hl) {  // send regions laid end to end: bases = scan of the row sums
+      tuna_segbase_kernel<<<1, 1024, 0, st>>>(pl->d_seg_total, nullptr, pl->d_sendbase, P, pl->d_scal, nullptr, 0,
+                                              nullptr);
+      TUNA_LAUNCHED(pl);
+      tuna_packed_extents_kernel<<<1, 32, 0, st>>>(pl->d_scal, t.elem, pl->d_extents);
+      TUNA_LAUNCHED(pl);
+    }
   }
   if (rdispls) {
     TUNA_CUDA(pl, cudaMemcpyAsync(pl->d_rdispls, rdispls, PP * 8, cudaMemcpyHostToDevice, st));
   } else {  // packed: scan of the receive counts = rows of the transposed matrix
-    tuna_transpose_kernel<<<gPP, th, 0, st>>>(pl->d_counts, pl->d_tmp, P);
+    tuna_transpose_kernel<<<gPP, th, 0, st>>>(pl->d_counts, pl->d_tmp, P, hl ? nullptr : pl->d_extents + 3);
     TUNA_LAUNCHED(pl);
     tuna_segscan_kernel<0><<<gseg, th, 0, st>>>(pl->d_tmp, pl->d_rdispls, pl->d_seg_total,
                                                  nullptr, P, P);
     TUNA_LAUNCHED(pl);
+    if (!hl) {  // receive regions likewise: scan of the column sums
+      tuna_segbase_kernel<<<1, 1024, 0, st>>>(pl->d_seg_total, nullptr, pl->d_recvbase, P, pl->d_scal, nullptr, 0,
+                                              nullptr);
+      TUNA_LAUNCHED(pl);
+    }
   }
 
   const int nph = (int)pl->phases.size();
@@ -1025,9 +1076,9 @@ int build_tables(tuna_plan *pl, const HostLayout &hl, const int64_t *sdispls, co
   TUNA_CUDA(pl, cudaMemsetAsync(pl->d_violations, 0, sizeof(unsigned long long) * (1 + nlists), st));
   auto check = [&](const TunaList &l, int keep_phase, int id) -> int {
     if (l.n <= 0) return TUNA_OK;
-    tuna_check_list_kernel<<<(unsigned)((l.n + th - 1) / th), th, 0, st>>>(
-        l.len, l.pos, l.src, l.kind == TUNA_LIST_DELIVER ? l.dst : nullptr, l.n, pl->send_extent,
-        pl->recv_extent, pl->d_wbase + nph, keep_phase, pl->d_wbase, pl->d_violations,
+    tuna_check_list_kernel<<<(unsigned)std::min<int64_t>((l.n + th - 1) / th, 148 * 8), th, 0, st>>>(
+        l.len, l.pos, l.src, l.kind == TUNA_LIST_DELIVER ? l.dst : nullptr, l.n, pl->d_extents,
+        pl->d_wbase + nph, keep_phase, pl->d_wbase, pl->d_violations,
         pl->d_violations + 1 + id);
     TUNA_LAUNCHED(pl);
     return TUNA_OK;
@@ -1053,7 +1104,15 @@ int build_tables(tuna_plan *pl, const HostLayout &hl, const int64_t *sdispls, co
                                 cudaMemcpyDeviceToHost, st));
   std::vector<unsigned long long> checked(1 + nlists);
   TUNA_CUDA(pl, cudaMemcpyAsync(checked.data(), pl->d_violations, checked.size() * 8, cudaMemcpyDeviceToHost, st));
+  int64_t ext[4] = {0, 0, 0, 0};
+  if (!hl) TUNA_CUDA(pl, cudaMemcpyAsync(ext, pl->d_extents, sizeof(ext), cudaMemcpyDeviceToHost, st));
   TUNA_CUDA(pl, cudaStreamSynchronize(st));
+  if (!hl) {
+    if (ext[3] != 0) return TUNA_ERR_INVALID_ARG;  // negative counts
+    pl->send_extent = ext[0];
+    pl->recv_extent = ext[1];
+    pl->payload = ext[2] * t.elem;
+  }
   if (checked[0] != 0) return TUNA_ERR_INTERNAL;
   pl->h_wbase = wbase;
   auto take = [&](TunaList &l, int id) {
@@ -1082,6 +1141,7 @@ int build_tables(tuna_plan *pl, const HostLayout &hl, const int64_t *sdispls, co
   rc = build_chunks(pl, pl->dir, st);
   if (rc) return rc;
   TUNA_CUDA(pl, cudaStreamSynchronize(st));
+  pl->tables_valid = true;
   return TUNA_OK;
 }
 
@@ -1155,10 +1215,17 @@ void add_staggered(tuna_plan *pl, int block_count) {
   }
 }
 
-int check_call_args(const tuna_plan *pl, const int64_t *sendcounts, const int64_t *sdispls,
+int check_call_args(tuna_plan *pl, const int64_t *sendcounts, const int64_t *sdispls,
                     const int64_t *recvcounts, const int64_t *rdispls) {
   const int P = pl->topo.P;
   const int64_t PP = (int64_t)P * P;
+  if (!pl->tables_valid) return TUNA_ERR_INTERNAL;  // the last update failed: the plan must not be used
+  if (!pl->h_counts_valid && (sendcounts || sdispls || recvcounts || rdispls)) {
+    // the counts came from device memory: fetch them for the comparison, once
+    TUNA_CUDA(pl, cudaMemcpy(pl->h_buf[pl->h_cur], pl->d_counts, (size_t)PP * 8, cudaMemcpyDeviceToHost));
+    pl->h_counts = pl->h_buf[pl->h_cur];
+    pl->h_counts_valid = true;
+  }
   if (sendcounts && memcmp(sendcounts, pl->h_counts, PP * 8) != 0) return TUNA_ERR_COUNT_MISMATCH;
   if (recvcounts)
     for (int d = 0; d < P; d++)
@@ -1343,6 +1410,7 @@ int tuna_plan_destroy(tuna_plan_t *pl) {
   cudaFree(pl->d_tmp);
   cudaFree(pl->d_scal);
   cudaFree(pl->d_wbase);
+  cudaFree(pl->d_extents);
   cudaFree(pl->d_round_bytes);
   cudaFree(pl->d_error);
   cudaFree(pl->d_violations);
@@ -1444,6 +1512,7 @@ static int plan_create(tuna_plan_t **out, int P, int radix, int radix_global, in
   TUNA_TRY(dev_alloc(&pl->d_tmp, PP));
   TUNA_TRY(dev_alloc(&pl->d_scal, 2 * (2 * nph + 3)));
   TUNA_TRY(dev_alloc(&pl->d_wbase, nph + 1));
+  TUNA_TRY(dev_alloc(&pl->d_extents, 6));  // [4], [5]: extents of the row exchange's buffers
   TUNA_TRY(dev_alloc(&pl->d_round_bytes, pl->stats_n));
   TUNA_TRY(dev_alloc(&pl->d_error, 1));
   TUNA_TRY(dev_alloc(&pl->d_violations, 1 + 2 * nph + 3));
@@ -1465,7 +1534,7 @@ static int plan_create(tuna_plan_t **out, int P, int radix, int radix_global, in
   rc = alloc_list(pl, pl->dir, TUNA_LIST_DELIVER, PP);
   if (rc) return nomem(rc);
 #undef TUNA_TRY
-  rc = build_tables(pl, hl, sdispls, rdispls, st);
+  rc = build_tables(pl, &hl, sdispls, rdispls, st);
   if (rc) return fail(rc);
   *out = pl;
   return TUNA_OK;
@@ -1512,7 +1581,21 @@ int tuna_plan_update_counts(tuna_plan_t *pl, const int64_t *sendcounts, const in
     pl->d_counts = up.d_dst;
     pl->counts_uploaded = true;
   }
-  return build_tables(pl, hl, sdispls, rdispls, (cudaStream_t)stream);
+  return build_tables(pl, &hl, sdispls, rdispls, (cudaStream_t)stream);
+}
+
+int tuna_plan_update_counts_device(tuna_plan_t *pl, const int64_t *d_sendcounts, void *stream) {
+  if (!pl || !d_sendcounts) return TUNA_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  const int64_t PP = (int64_t)pl->topo.P * pl->topo.P;
+  // the plan keeps its own copy (the caller may reuse its array at once); it goes
+  // into the spare buffer, like an upload from the host
+  int64_t *spare = pl->d_counts == pl->d_counts_buf[0] ? pl->d_counts_buf[1] : pl->d_counts_buf[0];
+  if (d_sendcounts != spare)
+    TUNA_CUDA(pl, cudaMemcpyAsync(spare, d_sendcounts, (size_t)PP * 8, cudaMemcpyDeviceToDevice, st));
+  pl->d_counts = spare;
+  pl->counts_uploaded = true;
+  return build_tables(pl, nullptr, nullptr, nullptr, st);
 }
 
 int tuna_plan_workspace_bytes(const tuna_plan_t *pl, size_t *bytes) {
@@ -1588,6 +1671,7 @@ int tuna_alltoallv_host(tuna_plan_t *pl, const void *host_send, void *host_recv,
   const bool force_staging = (schedule & TUNA_HOST_STAGED) != 0;
   schedule &= ~TUNA_HOST_STAGED;
   if (schedule != TUNA_SCHEDULE_TUNA && schedule != TUNA_SCHEDULE_DIRECT) return TUNA_ERR_INVALID_ARG;
+  if (!pl->tables_valid) return TUNA_ERR_INTERNAL;
   if (ranges_overlap(host_send, (size_t)pl->send_extent, host_recv, (size_t)pl->recv_extent))
     return TUNA_ERR_OVERLAP;
   cudaStream_t st = (cudaStream_t)stream;
@@ -1624,6 +1708,7 @@ int tuna_alltoallv_host(tuna_plan_t *pl, const void *host_send, void *host_recv,
 int tuna_plan_set_row_maps(tuna_plan_t *pl, const int64_t *gather_rows, const int64_t *scatter_rows,
                            int64_t in_rows, int64_t out_rows, void *stream) {
   if (!pl || in_rows < 0 || out_rows < 0) return TUNA_ERR_INVALID_ARG;
+  if (!pl->tables_valid) return TUNA_ERR_INTERNAL;
   cudaStream_t st = (cudaStream_t)stream;
   const TunaTopo &t = pl->topo;
   const int P = t.P;
@@ -1647,7 +1732,7 @@ int tuna_plan_set_row_maps(tuna_plan_t *pl, const int64_t *gather_rows, const in
   const int nph = (int)pl->phases.size();
   Timed plan_timer(pl, TUNA_TIMER_PLAN, 0, st);
   // rows before every block in receive-side order: scan of the transposed counts
-  tuna_transpose_kernel<<<gPP, th, 0, st>>>(pl->d_counts, pl->d_tmp, P);
+  tuna_transpose_kernel<<<gPP, th, 0, st>>>(pl->d_counts, pl->d_tmp, P, nullptr);
   TUNA_LAUNCHED(pl);
   tuna_segscan_kernel<0><<<gseg, th, 0, st>>>(pl->d_tmp, pl->d_row_start, pl->d_seg_total, nullptr, P, P);
   TUNA_LAUNCHED(pl);
@@ -1666,10 +1751,12 @@ int tuna_plan_set_row_maps(tuna_plan_t *pl, const int64_t *gather_rows, const in
   l.bytes = n * t.elem;
   l.total = n * (((int64_t)t.elem + 15) / 16 * 16 + 16);
   // every row must lie inside the two buffers
+  const int64_t row_ext[2] = {pl->rows_in_bytes, pl->rows_out_bytes};
+  TUNA_CUDA(pl, cudaMemcpyAsync(pl->d_extents + 4, row_ext, sizeof(row_ext), cudaMemcpyHostToDevice, st));
   TUNA_CUDA(pl, cudaMemsetAsync(pl->d_violations, 0, 2 * sizeof(unsigned long long), st));
   if (n > 0) {
-    tuna_check_list_kernel<<<(unsigned)((n + th - 1) / th), th, 0, st>>>(
-        l.len, l.pos, l.src, l.dst, n, pl->rows_in_bytes, pl->rows_out_bytes, pl->d_wbase + nph, 0,
+    tuna_check_list_kernel<<<(unsigned)std::min<int64_t>((n + th - 1) / th, 148 * 8), th, 0, st>>>(
+        l.len, l.pos, l.src, l.dst, n, pl->d_extents + 4, pl->d_wbase + nph, 0,
         pl->d_wbase, pl->d_violations, pl->d_violations + 1);
     TUNA_LAUNCHED(pl);
   }
@@ -1986,7 +2073,7 @@ int tuna_direct_alltoallv_static(int P, int elem_size, const int64_t *sendcounts
   if (rdispls) {
     TUNA_STATIC_CUDA(cudaMemcpyAsync(t.rdispls, rdispls, PP * 8, cudaMemcpyHostToDevice, st));
   } else {
-    tuna_transpose_kernel<<<gPP, th, 0, st>>>(t.counts, t.tmp, P);
+    tuna_transpose_kernel<<<gPP, th, 0, st>>>(t.counts, t.tmp, P, nullptr);
     TUNA_STATIC_CUDA(cudaGetLastError());
     tuna_segscan_kernel<0><<<gseg, th, 0, st>>>(t.tmp, t.rdispls, t.seg_total, nullptr, P, P);
     TUNA_STATIC_CUDA(cudaGetLastError());

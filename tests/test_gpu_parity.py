@@ -288,6 +288,93 @@ def test_rejected_update_leaves_the_plan_as_it_was(P):
     assert (se, re_) == (wl.send_bytes, wl.recv_bytes) and payload == wl.payload_bytes_total
 
 
+@pytest.mark.parametrize("kw", [dict(radix=3), dict(radix=2, flags=B.FLAG_CLASSIC_ROTATE),
+                                dict(radix=2, l=4, g=3, radix_global=3), dict(radix=4, l=4, g=3, block_count=5),
+                                dict(radix=12, direct=True)])
+def test_update_counts_from_device_memory(kw):
+    """Counts that live on the GPU (packed layout worked out there): every schedule
+    must give what the oracle gives for those counts, and the plan's extents, payload
+    and per-round byte counts must be those of the new counts."""
+    kw = dict(kw)
+    direct = kw.pop("direct", False)
+    first = W.make_random(12, 300, seed=61, zero_frac=0.1)
+    plan = B.plan_for(first, explicit_layout=False, **kw)
+    for seed, top, zf in ((62, 900, 0.4), (63, 17, 0.0), (64, 5000, 0.8)):
+        wl = W.make_random(12, top, seed=seed, zero_frac=zf)      # packed, like the device layout
+        d_counts = torch.from_numpy(wl.sendcounts).cuda()
+        plan.update_counts_device(d_counts)
+        d_counts.fill_(-7)                                        # the plan kept its own copy
+        plan.alloc_workspace()
+        assert plan.extents() == (wl.send_bytes, wl.recv_bytes, wl.payload_bytes_total)
+        send, recv = wl.make_send("cuda"), wl.make_recv("cuda", fill=CANARY)
+        (plan.direct_alltoallv if direct else plan.alltoallv)(send, recv)
+        torch.cuda.synchronize()
+        assert np.array_equal(recv.cpu().numpy(), oracle_brute(wl))
+        if not direct and "l" not in kw:
+            _, rounds, _, _ = oracle_flat(wl, kw["radix"])
+            check_rounds(plan, rounds)
+        # arrays given at call time are still compared with the plan's (fetched from the device)
+        recv.fill_(CANARY)
+        (plan.direct_alltoallv if direct else plan.alltoallv)(
+            send, recv, sendcounts=wl.sendcounts, sdispls=wl.sdispls, recvcounts=wl.recvcounts, rdispls=wl.rdispls)
+        torch.cuda.synchronize()
+        assert np.array_equal(recv.cpu().numpy(), oracle_brute(wl))
+        other = wl.sendcounts.copy()
+        other[3, 4] += 1
+        with pytest.raises(B.TunaError, match="COUNT_MISMATCH"):
+            plan.alltoallv(send, recv, sendcounts=other)
+    # and back to counts from the host, with gaps
+    wl = W.make_random(12, 200, seed=65, zero_frac=0.3, gaps=True)
+    plan.update_counts(wl.sendcounts, wl.sdispls, wl.rdispls, wl.sendbase, wl.recvbase)
+    plan.alloc_workspace()
+    send, recv = wl.make_send("cuda"), wl.make_recv("cuda", fill=CANARY)
+    (plan.direct_alltoallv if direct else plan.alltoallv)(send, recv)
+    torch.cuda.synchronize()
+    assert np.array_equal(recv.cpu().numpy(), oracle_brute(wl))
+
+
+def test_negative_device_counts_are_refused_and_the_plan_recovers():
+    wl = W.make_random(9, 300, seed=71, zero_frac=0.2)
+    plan = B.plan_for(wl, 3, explicit_layout=False)
+    plan.alloc_workspace()
+    bad = wl.sendcounts.copy()
+    bad[8, 2] = -1
+    with pytest.raises(B.TunaError, match="INVALID_ARG"):
+        plan.update_counts_device(torch.from_numpy(bad).cuda())
+    send, recv = wl.make_send("cuda"), wl.make_recv("cuda", fill=CANARY)
+    with pytest.raises(B.TunaError, match="INTERNAL"):             # its tables were rewritten
+        plan.alltoallv(send, recv)
+    with pytest.raises(B.TunaError, match="INTERNAL"):
+        plan.direct_alltoallv(send, recv)
+    torch.cuda.synchronize()
+    assert bool((recv == CANARY).all())                            # nothing was moved
+    plan.update_counts_device(torch.from_numpy(wl.sendcounts).cuda())
+    plan.alloc_workspace()
+    plan.alltoallv(send, recv)
+    torch.cuda.synchronize()
+    assert np.array_equal(recv.cpu().numpy(), oracle_brute(wl))
+
+
+def test_device_counts_at_p2048_match_the_host_path():
+    """c5's count matrix (4.2 million pairs) through both update paths: same tables."""
+    wl = W.make_c5()
+    plan_h = B.plan_for(wl, wl.P, explicit_layout=False)
+    plan_d = B.plan_for(W.make_uniform(wl.P, 1), wl.P, explicit_layout=False)
+    plan_d.update_counts_device(torch.from_numpy(wl.sendcounts).cuda())
+    assert plan_d.extents() == plan_h.extents() == (wl.send_bytes, wl.recv_bytes, wl.payload_bytes_total)
+    th, td = plan_h.phase_tables(0, B.PART_DELIVER), plan_d.phase_tables(0, B.PART_DELIVER)
+    for key in ("len", "pos", "src", "dst"):
+        assert np.array_equal(th[key], td[key])
+    send = wl.make_send("cuda")
+    got = []
+    for plan in (plan_h, plan_d):
+        recv = wl.make_recv("cuda", fill=CANARY)
+        plan.alltoallv(send, recv)
+        torch.cuda.synchronize()
+        got.append(recv)
+    assert torch.equal(got[0], got[1])
+
+
 @pytest.mark.parametrize("kw", [dict(radix=2), dict(radix=3, l=3, g=4, rg=2), dict(radix=12, direct=True)])
 def test_exchange_replayed_from_a_cuda_graph(kw):
     """The exchange only enqueues kernels, so it can be captured once and replayed."""
