@@ -39,7 +39,7 @@ UNIT = "GB/s"
 # reported as null.  Captures: profiles/round_kernel_c4_reduced.md (c4, reduced to
 # 2 GiB) and profiles/round_small_kernel_c5.md (c5 at full size).
 NCU_TRAFFIC_PER_PAYLOAD_BYTE: dict[str, dict[str, float]] = {
-    "6d329643b4d0f21852306ca2c777d1a1af07f22b26f4a5b65df95b9f9cd9df01": {"c4": 1.979, "c5": 2.329},
+    "e8b927e2be251e873da404b7fab3ba1a57fdcd82f5f946d4ed134e4c6211542a": {"c4": 1.979, "c5": 2.179},
 }
 
 
@@ -438,20 +438,6 @@ def ours_arm(args):
         "ms_per_step": {k: v["ms"] / args.steps for k, v in timing.items()},
     }
 
-    # the re-plan alone (count-metadata exchange + prefix sums), wall clock: from the
-    # device-resident counts and from a host array
-    def wall(fn, n):
-        fn()
-        torch.cuda.synchronize()
-        t0 = time.perf_counter()
-        for _ in range(n):
-            fn()
-        torch.cuda.synchronize()
-        return (time.perf_counter() - t0) * 1e3 / n
-
-    replan = {"from_device_counts_ms": wall(lambda: plan.update_counts_device(d_counts), 5),
-              "from_host_counts_ms": wall(lambda: plan.update_counts(*layout), 5)}
-
     # end to end through the host-buffer entry point (pinned host memory)
     e2e = None
     if not args.no_e2e:
@@ -491,6 +477,22 @@ def ours_arm(args):
                "h2d_bytes_per_step": wl.send_bytes + 8 * (wl.P * wl.P + 2 * wl.P),
                "d2h_bytes_per_step": wl.recv_bytes, "ms_per_step": e_ms, "steps": e_steps}
         del hs, hr
+
+    # the re-plan alone (count-metadata exchange + prefix sums), wall clock: from the
+    # device-resident counts and from a host array
+    replan = None
+    if not args.no_sweep:
+        def wall(fn, n):
+            fn()
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            for _ in range(n):
+                fn()
+            torch.cuda.synchronize()
+            return (time.perf_counter() - t0) * 1e3 / n
+
+        replan = {"from_device_counts_ms": wall(lambda: plan.update_counts_device(d_counts), 5),
+                  "from_host_counts_ms": wall(lambda: plan.update_counts(*layout), 5)}
 
     # the other schedules of the workload, timed the same way (exchange + re-plan)
     sweep = []

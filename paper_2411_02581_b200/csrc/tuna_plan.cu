@@ -39,9 +39,10 @@ __device__ __forceinline__ int64_t pad16(int64_t v) { return (v + (TUNA_ALIGN - 
 // Compact index of offset v among the offsets whose digit (v / stride) % radix is
 // non-zero, ascending.  Only called for such v.
 __device__ __forceinline__ int64_t compact_of(int64_t v, int64_t stride, int radix) {
-  const int64_t hi = v / (stride * radix);
-  const int64_t rem = v - hi * stride * radix;  // z*stride + lo
-  return hi * (radix - 1) * stride + (rem - stride);
+  const unsigned sr = (unsigned)stride * (unsigned)radix;  // at most P * radix < 2^31: 32-bit division
+  const unsigned hi = (unsigned)v / sr;
+  const int64_t rem = v - (int64_t)hi * sr;  // z*stride + lo
+  return (int64_t)hi * (radix - 1) * stride + (rem - stride);
 }
 
 struct PhaseDev {
@@ -72,7 +73,7 @@ __global__ void tuna_init_tables_kernel(TunaTopo t, const int64_t *__restrict__ 
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   const int64_t PP = (int64_t)t.P * t.P;
   if (idx >= PP) return;
-  const int p = (int)(idx / t.P), sigma = (int)(idx % t.P);
+  const int p = (int)((unsigned)idx / (unsigned)t.P), sigma = (int)((unsigned)idx % (unsigned)t.P);  // (P * P < 2^31)
   const int n = p / t.Q, q = p % t.Q, io = sigma / t.Q, jo = sigma % t.Q;
   const int dest = ((n + io) % t.N) * t.Q + (q + jo) % t.Q;
   const int64_t bytes = counts[(int64_t)p * t.P + dest] * t.elem;
@@ -111,10 +112,10 @@ __global__ void tuna_meta_exchange_kernel(TunaTopo t, PhaseDev ph, const int64_t
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   const int64_t PP = (int64_t)t.P * t.P;
   if (idx < PP) {
-    const int p = (int)(idx / t.P), sigma = (int)(idx % t.P);
+    const int p = (int)((unsigned)idx / (unsigned)t.P), sigma = (int)((unsigned)idx % (unsigned)t.P);  // (P * P < 2^31)
     const int n = p / t.Q, q = p % t.Q, io = sigma / t.Q, jo = sigma % t.Q;
     const int v = ph.level == 0 ? jo : io;
-    const int dig = (int)((v / ph.stride) % ph.radix);
+    const int dig = (int)(((unsigned)v / (unsigned)ph.stride) % (unsigned)ph.radix);
     if (dig == 0) {
       sz_next[idx] = sz_cur[idx];
     } else {
@@ -220,7 +221,7 @@ __global__ void tuna_rows_list_kernel(int P, int64_t row_bytes, const int64_t *_
 }
 
 // Segmented exclusive prefix sum, one warp per segment, warp-shuffle scan over
-// 32-wide tiles with a running carry.  MODE 0 sums the values as they are; MODE 1
+// 128-wide tiles (four values per lane) with a running carry.  MODE 0 sums the values as they are; MODE 1
 // (KEEP lists) rounds every value up to 16 first; MODE 2 (DELIVER lists) also
 // adds 16 spare bytes behind every non-zero value.  seg_total[s] receives the
 // segment's sum, seg_raw[s] (optional) the sum of the unmodified values.
@@ -234,19 +235,33 @@ __global__ void tuna_segscan_kernel(const int64_t *__restrict__ val, int64_t *ou
   int64_t carry = 0, raw = 0;
   const int64_t *v = val + w * seglen;
   int64_t *o = out + w * seglen;
-  for (int64_t base = 0; base < seglen; base += 32) {
-    const int64_t i = base + lane;
-    int64_t x = i < seglen ? v[i] : 0;
-    raw += x;
-    if (MODE >= 1) x = pad16(x);
-    if (MODE == 2 && x > 0) x += 16;
-    int64_t incl = x;
+  // tiles of 128: every lane takes four consecutive values, sums them in registers,
+  // and only the lanes' sums go through the shuffle scan
+  constexpr int kPer = 4;
+  for (int64_t base = 0; base < seglen; base += 32 * kPer) {
+    const int64_t i0 = base + lane * kPer;
+    int64_t x[kPer], sum = 0;
+#pragma unroll
+    for (int k = 0; k < kPer; k++) {
+      int64_t y = i0 + k < seglen ? v[i0 + k] : 0;
+      raw += y;
+      if (MODE >= 1) y = pad16(y);
+      if (MODE == 2 && y > 0) y += 16;
+      x[k] = y;
+      sum += y;
+    }
+    int64_t incl = sum;
 #pragma unroll
     for (int d = 1; d < 32; d <<= 1) {
       const int64_t y = __shfl_up_sync(0xffffffffu, incl, d);
       if (lane >= d) incl += y;
     }
-    if (i < seglen) o[i] = carry + incl - x;
+    int64_t run = carry + incl - sum;  // exclusive prefix of this lane's first value
+#pragma unroll
+    for (int k = 0; k < kPer; k++) {
+      if (i0 + k < seglen) o[i0 + k] = run;
+      run += x[k];
+    }
     carry += __shfl_sync(0xffffffffu, incl, 31);
   }
 #pragma unroll
@@ -331,17 +346,17 @@ __global__ void tuna_place_kernel(TunaTopo t, PhaseDev ph, const int64_t *__rest
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   const int64_t PP = (int64_t)t.P * t.P;
   if (idx >= PP) return;
-  const int p = (int)(idx / t.P), sigma = (int)(idx % t.P);
+  const int p = (int)((unsigned)idx / (unsigned)t.P), sigma = (int)((unsigned)idx % (unsigned)t.P);  // (P * P < 2^31)
   const int n = p / t.Q, q = p % t.Q, io = sigma / t.Q, jo = sigma % t.Q;
   const int v = ph.level == 0 ? jo : io;
-  const int dig = (int)((v / ph.stride) % ph.radix);
+  const int dig = (int)(((unsigned)v / (unsigned)ph.stride) % (unsigned)ph.radix);
   if (dig == 0) {
     loc_next[idx] = loc_cur[idx];
     return;
   }
   const int64_t c = row_position(t, ph, io, jo);
-  const bool fin = ph.level == 0 ? (io == 0 && jo / (ph.stride * ph.radix) == 0)
-                                 : io / (ph.stride * ph.radix) == 0;
+  const unsigned sr = (unsigned)ph.stride * (unsigned)ph.radix;
+  const bool fin = ph.level == 0 ? (io == 0 && (unsigned)jo < sr) : (unsigned)io < sr;
   const int origin = ((n - io + t.N) % t.N) * t.Q + (q - jo + t.Q) % t.Q;
   const int64_t rloc =
       TUNA_LOC(TUNA_BUF_RECV, (recvbase[p] + rdispls[(int64_t)p * t.P + origin]) * t.elem);
@@ -437,7 +452,7 @@ __global__ void tuna_check_list_kernel(const int64_t *__restrict__ len, const in
 __global__ void tuna_transpose_kernel(const int64_t *__restrict__ in, int64_t *out, int P, int64_t *negatives) {
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= (int64_t)P * P) return;
-  const int r = (int)(idx / P), c = (int)(idx % P);
+  const int r = (int)((unsigned)idx / (unsigned)P), c = (int)((unsigned)idx % (unsigned)P);
   const int64_t v = in[(int64_t)c * P + r];
   out[idx] = v;
   if (negatives && v < 0) atomicAdd(reinterpret_cast<unsigned long long *>(negatives), 1ULL);
