@@ -135,11 +135,12 @@ int tuna_plan_create_staggered(tuna_plan_t **out, int P, int radix, int block_co
  * tuna_plan_update_counts - same plan shape, new counts (e.g. routing that changes
  * every step): re-runs the metadata exchange and the prefix sums on the device.
  * Arguments as in tuna_plan_create.  Synchronises `stream` once.  The required
- * workspace size may change; query it again.  The tables are rewritten in place:
- * an exchange enqueued with this plan must have finished before the update is
- * called (the update waits only for `stream`), or it would run on tables that
- * change under it.  To overlap the re-plan of one batch with the exchange of the
- * previous one, alternate between two plans.
+ * workspace size may change; query it again.  The tables are rewritten in place,
+ * so the update first waits (on the host) for the exchanges this plan has
+ * enqueued, whatever their stream; replays of an exchange captured into a CUDA
+ * graph are not tracked and must have finished before the call.  To overlap the
+ * re-plan of one batch with the exchange of the previous one, alternate between
+ * two plans.
  */
 int tuna_plan_update_counts(tuna_plan_t *plan, const int64_t *sendcounts, const int64_t *sdispls,
                             const int64_t *rdispls, const int64_t *sendbase,
@@ -158,8 +159,8 @@ int tuna_plan_update_counts(tuna_plan_t *plan, const int64_t *sendcounts, const 
  * order, the ranks' regions back to back in both buffers.  Region bases, buffer
  * extents and the payload size are computed on the device.
  * Synchronises `stream` once.  The required workspace size may change; query it
- * again.  As with tuna_plan_update_counts, no exchange of this plan may still be
- * running.  Errors: a negative count gives TUNA_ERR_INVALID_ARG; unlike the
+ * again.  Waits for this plan's exchanges in flight like tuna_plan_update_counts.
+ * Errors: a negative count gives TUNA_ERR_INVALID_ARG; unlike the
  * host-array form, a failed update leaves the plan unusable (its tables have been
  * rewritten; exchange calls return TUNA_ERR_INTERNAL) until an update succeeds.
  * Count or displacement arrays passed to a later exchange call are still

@@ -539,6 +539,8 @@ struct tuna_plan {
   size_t workspace_bytes = 0;
 
   int64_t launch_count = 0;  // kernels launched by this plan since creation
+  cudaEvent_t in_flight = nullptr;  // end of the last exchange this plan enqueued (outside graph capture)
+  bool in_flight_set = false;
 
   // optional per-launch timing (CUDA events on the caller's stream)
   bool timing = false;
@@ -571,6 +573,31 @@ namespace {
     (plan)->launch_count++;                       \
     TUNA_CUDA(plan, cudaGetLastError());          \
   } while (0)
+
+// An exchange reads the plan's tables until it ends; an update rewrites them.  Every
+// exchange call marks its end on its stream, and an update waits for the mark.  A
+// stream that is being captured gets no mark (an event recorded there could not be
+// waited for later): replays of a captured exchange are the caller's to order.
+int mark_in_flight(tuna_plan *pl, cudaStream_t st) {
+  cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+  if (cudaStreamIsCapturing(st, &cap) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return TUNA_OK;
+  }
+  if (cap != cudaStreamCaptureStatusNone) return TUNA_OK;
+  if (!pl->in_flight) TUNA_CUDA(pl, cudaEventCreateWithFlags(&pl->in_flight, cudaEventDisableTiming));
+  TUNA_CUDA(pl, cudaEventRecord(pl->in_flight, st));
+  pl->in_flight_set = true;
+  return TUNA_OK;
+}
+
+int wait_in_flight(tuna_plan *pl) {
+  if (pl->in_flight_set) {
+    TUNA_CUDA(pl, cudaEventSynchronize(pl->in_flight));
+    pl->in_flight_set = false;
+  }
+  return TUNA_OK;
+}
 
 cudaEvent_t take_event(tuna_plan *pl) {
   cudaEvent_t e = nullptr;
@@ -971,6 +998,8 @@ int build_tables(tuna_plan *pl, const HostLayout *hl, const int64_t *sdispls, co
   const int64_t PP = (int64_t)P * P;
   int rc = TUNA_OK;
 
+  rc = wait_in_flight(pl);  // an exchange that is still running reads the tables rewritten below
+  if (rc) return rc;
   pl->rows_valid = false;  // a row list belongs to the counts it was built for
   pl->tables_valid = false;
   // host copies for the checks at call time
@@ -1351,7 +1380,7 @@ int run_tuna(tuna_plan *pl, const void *send, void *recv, cudaStream_t st) {
   }
   pl->last_launches = launches;
   pl->launch_count += launches;
-  return TUNA_OK;
+  return launches > 0 ? mark_in_flight(pl, st) : TUNA_OK;
 }
 
 int run_direct(tuna_plan *pl, const void *send, void *recv, cudaStream_t st) {
@@ -1365,7 +1394,7 @@ int run_direct(tuna_plan *pl, const void *send, void *recv, cudaStream_t st) {
   }
   pl->last_launches = launches;
   pl->launch_count += launches;
-  return TUNA_OK;
+  return launches > 0 ? mark_in_flight(pl, st) : TUNA_OK;
 }
 
 int64_t align256(int64_t v) { return (v + 255) & ~(int64_t)255; }
@@ -1397,6 +1426,10 @@ const char *tuna_strerror(int status) {
 
 int tuna_plan_destroy(tuna_plan_t *pl) {
   if (!pl) return TUNA_OK;
+  if (pl->in_flight) {
+    if (pl->in_flight_set) (void)cudaEventSynchronize(pl->in_flight);  // the tables are freed below
+    cudaEventDestroy(pl->in_flight);
+  }
   for (auto &l : pl->keep) free_list(l);
   for (auto &l : pl->deliver) free_list(l);
   free_list(pl->rot);
@@ -1729,6 +1762,10 @@ int tuna_plan_set_row_maps(tuna_plan_t *pl, const int64_t *gather_rows, const in
   const int P = t.P;
   const int64_t PP = (int64_t)P * P;
   const int64_t n = pl->payload / t.elem;  // rows exchanged
+  {
+    const int wrc = wait_in_flight(pl);  // a row exchange still running reads the list rewritten below
+    if (wrc) return wrc;
+  }
   pl->rows_valid = false;
   if (in_rows > (INT64_MAX >> 8) / t.elem || out_rows > (INT64_MAX >> 8) / t.elem) return TUNA_ERR_RANGE;
   if (!pl->d_row_start) TUNA_CUDA(pl, dev_alloc(&pl->d_row_start, PP));
@@ -1795,8 +1832,8 @@ int tuna_rows_alltoallv(tuna_plan_t *pl, const void *rows_in, void *rows_out, vo
   if (ranges_overlap(rows_in, (size_t)pl->rows_in_bytes, rows_out, (size_t)pl->rows_out_bytes))
     return TUNA_ERR_OVERLAP;
   int launches = 0;
+  cudaStream_t st = (cudaStream_t)stream;
   if (l.nchunks > 0) {
-    cudaStream_t st = (cudaStream_t)stream;
     Timed tm(pl, TUNA_TIMER_DIRECT, l.bytes, st);
     TunaMoveArgs a = move_args(pl, rows_in, rows_out, nullptr);
     a.extent[TUNA_BUF_SEND] = pl->rows_in_bytes;
@@ -1807,7 +1844,7 @@ int tuna_rows_alltoallv(tuna_plan_t *pl, const void *rows_in, void *rows_out, vo
   }
   pl->last_launches = launches;
   pl->launch_count += launches;
-  return TUNA_OK;
+  return launches > 0 ? mark_in_flight(pl, st) : TUNA_OK;
 }
 
 int tuna_plan_num_rounds(const tuna_plan_t *pl, int *K) {

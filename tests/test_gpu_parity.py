@@ -333,6 +333,37 @@ def test_update_counts_from_device_memory(kw):
     assert np.array_equal(recv.cpu().numpy(), oracle_brute(wl))
 
 
+def test_update_waits_for_the_plans_own_exchange_in_flight():
+    """An update issued on another stream while the plan's exchange is still running must
+    not disturb that exchange (the library waits for it before it rewrites the tables)."""
+    big = W.make_random(48, 1 << 20, seed=81, zero_frac=0.1)       # about 1 GB: a millisecond of exchange
+    small = W.make_random(48, 64, seed=82, zero_frac=0.5)
+    plan = B.plan_for(big, 48, explicit_layout=False)
+    send, recv = big.make_send("cuda"), big.make_recv("cuda", fill=CANARY)
+    d_small = torch.from_numpy(small.sendcounts).cuda()
+    s_x, s_p = torch.cuda.Stream(), torch.cuda.Stream(priority=-1)
+    torch.cuda.synchronize()
+    plan.alltoallv(send, recv, stream=s_x)
+    plan.update_counts_device(d_small, stream=s_p)                   # while the exchange runs
+    torch.cuda.synchronize()
+    ref_plan = B.plan_for(big, 48, explicit_layout=False)            # the same exchange, undisturbed
+    want = big.make_recv("cuda", fill=CANARY)
+    ref_plan.alltoallv(send, want)
+    torch.cuda.synchronize()
+    assert torch.equal(recv, want)
+    rng = np.random.default_rng(83)                                  # and pinned to the definition on samples
+    s_, d_ = rng.integers(0, 48, 4096), rng.integers(0, 48, 4096)
+    k_ = (rng.random(4096) * big.sendcounts[s_, d_]).astype(np.int64)
+    src = torch.from_numpy(big.sendbase[s_] + big.sdispls[s_, d_] + k_).cuda()
+    dst = torch.from_numpy(big.recvbase[d_] + big.rdispls[d_, s_] + k_).cuda()
+    ok = torch.from_numpy(big.sendcounts[s_, d_] > 0).cuda()
+    assert torch.equal(recv[dst][ok], send[src][ok])
+    send2, recv2 = small.make_send("cuda"), small.make_recv("cuda", fill=CANARY)
+    plan.alltoallv(send2, recv2)
+    torch.cuda.synchronize()
+    assert np.array_equal(recv2.cpu().numpy(), oracle_brute(small))
+
+
 def test_negative_device_counts_are_refused_and_the_plan_recovers():
     wl = W.make_random(9, 300, seed=71, zero_frac=0.2)
     plan = B.plan_for(wl, 3, explicit_layout=False)
