@@ -522,6 +522,10 @@ struct tuna_plan {
   int64_t *d_sz[2] = {nullptr, nullptr}, *d_loc[2] = {nullptr, nullptr};
   int64_t *d_seg_total = nullptr, *d_seg_raw = nullptr, *d_seg_base = nullptr;
   int64_t *d_tmp = nullptr;      // P*P scratch (transpose)
+  // The small tables an update reads back are slices of one allocation, so that one
+  // copy into one pinned host buffer fetches them all.
+  int64_t *d_readback = nullptr, *h_readback = nullptr;
+  int64_t readback_words = 0;
   int64_t *d_scal = nullptr;     // per list: stream bytes, bytes moved
   int64_t *d_wbase = nullptr;    // phases + 1 workspace offsets
   int64_t *d_extents = nullptr;  // send extent, receive extent (bytes), total of the counts (elements),
@@ -541,6 +545,12 @@ struct tuna_plan {
   int64_t launch_count = 0;  // kernels launched by this plan since creation
   cudaEvent_t in_flight = nullptr;  // end of the last exchange this plan enqueued (outside graph capture)
   bool in_flight_set = false;
+  // The plan kernels of an update from device counts, captured once as a CUDA graph
+  // (their arguments do not change from update to update) and replayed afterwards.
+  cudaStream_t capture_stream = nullptr;
+  cudaGraphExec_t tables_graph = nullptr;
+  const int64_t *tables_graph_counts = nullptr;  // the count buffer the captured kernels read
+  int64_t tables_graph_launches = 0;
 
   // optional per-launch timing (CUDA events on the caller's stream)
   bool timing = false;
@@ -987,6 +997,52 @@ int host_layout(int P, const int64_t *counts, const int64_t *sdispls, const int6
   return TUNA_OK;
 }
 
+// Updates from device counts enqueue the same kernels with the same arguments every
+// time (the plan's tables never move), a few dozen short launches: they are captured
+// once, on a stream of the plan's own, and replayed as one graph launch on the
+// caller's stream.  TUNA_PLAN_GRAPH=0 turns this off; so does any failure to capture.
+template <class F>
+int replay_tables_graph(tuna_plan *pl, F &enqueue, cudaStream_t st) {
+  static const bool enabled = env_i64("TUNA_PLAN_GRAPH", 1) != 0;
+  if (!enabled) return enqueue(st);
+  if (pl->tables_graph && pl->tables_graph_counts != pl->d_counts) {
+    cudaGraphExecDestroy(pl->tables_graph);
+    pl->tables_graph = nullptr;
+  }
+  if (!pl->tables_graph) {
+    if (!pl->capture_stream &&
+        cudaStreamCreateWithFlags(&pl->capture_stream, cudaStreamNonBlocking) != cudaSuccess) {
+      (void)cudaGetLastError();
+      pl->capture_stream = nullptr;
+      return enqueue(st);
+    }
+    if (cudaStreamBeginCapture(pl->capture_stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
+      (void)cudaGetLastError();
+      return enqueue(st);
+    }
+    const int64_t before = pl->launch_count;
+    const int rc = enqueue(pl->capture_stream);
+    cudaGraph_t g = nullptr;
+    const cudaError_t ce = cudaStreamEndCapture(pl->capture_stream, &g);
+    pl->tables_graph_launches = pl->launch_count - before;
+    pl->launch_count = before;  // nothing has run yet
+    cudaGraphExec_t ex = nullptr;
+    if (rc == TUNA_OK && ce == cudaSuccess && g && cudaGraphInstantiate(&ex, g, 0) == cudaSuccess) {
+      pl->tables_graph = ex;
+      pl->tables_graph_counts = pl->d_counts;
+    }
+    if (g) cudaGraphDestroy(g);
+    if (!pl->tables_graph) {
+      (void)cudaGetLastError();
+      pl->cuda_err = 0;
+      return enqueue(st);
+    }
+  }
+  TUNA_CUDA(pl, cudaGraphLaunch(pl->tables_graph, st));
+  pl->launch_count += pl->tables_graph_launches;
+  return TUNA_OK;
+}
+
 // Uploads the layout, runs every plan kernel, reads the totals back.  Without a
 // host layout (`hl` null) the counts are already in pl->d_counts and the layout
 // is packed: region bases, extents and the payload are worked out on the device.
@@ -1009,148 +1065,171 @@ int build_tables(tuna_plan *pl, const HostLayout *hl, const int64_t *sdispls, co
   if (rdispls) pl->h_rdispls.assign(rdispls, rdispls + PP); else pl->h_rdispls.clear();
   pl->h_counts_valid = hl != nullptr;
 
-  Timed plan_timer(pl, TUNA_TIMER_PLAN, 0, st);
-  if (hl) {
-    pl->payload = hl->payload * t.elem;
-    pl->send_extent = hl->send_extent * t.elem;
-    pl->recv_extent = hl->recv_extent * t.elem;
-    if (!pl->counts_uploaded)
-      TUNA_CUDA(pl, cudaMemcpyAsync(pl->d_counts, counts, PP * 8, cudaMemcpyHostToDevice, st));
-    TUNA_CUDA(pl, cudaMemcpyAsync(pl->d_sendbase, hl->sendbase.data(), P * 8, cudaMemcpyHostToDevice, st));
-    TUNA_CUDA(pl, cudaMemcpyAsync(pl->d_recvbase, hl->recvbase.data(), P * 8, cudaMemcpyHostToDevice, st));
-    const int64_t ext[4] = {pl->send_extent, pl->recv_extent, hl->payload, 0};
-    TUNA_CUDA(pl, cudaMemcpyAsync(pl->d_extents, ext, sizeof(ext), cudaMemcpyHostToDevice, st));
-    // (pageable sources: the runtime stages these copies before it returns)
-  } else {
-    TUNA_CUDA(pl, cudaMemsetAsync(pl->d_extents, 0, 4 * 8, st));
-  }
-  pl->counts_uploaded = false;
   const int th = 256;
   const unsigned gPP = (unsigned)((PP + th - 1) / th);
   const unsigned gseg = (unsigned)(((int64_t)P * 32 + th - 1) / th);
-  if (sdispls) {
-    TUNA_CUDA(pl, cudaMemcpyAsync(pl->d_sdispls, sdispls, PP * 8, cudaMemcpyHostToDevice, st));
-  } else {  // packed: exclusive scan of every rank's row of counts
-    tuna_segscan_kernel<0><<<gseg, th, 0, st>>>(pl->d_counts, pl->d_sdispls, pl->d_seg_total,
-                                                 nullptr, P, P);
-    TUNA_LAUNCHED(pl);
-    if (!hl) {  // send regions laid end to end: bases = scan of the row sums
-      tuna_segbase_kernel<<<1, 1024, 0, st>>>(pl->d_seg_total, nullptr, pl->d_sendbase, P, pl->d_scal, nullptr, 0,
-                                              nullptr);
-      TUNA_LAUNCHED(pl);
-      tuna_packed_extents_kernel<<<1, 32, 0, st>>>(pl->d_scal, t.elem, pl->d_extents);
-      TUNA_LAUNCHED(pl);
-    }
-  }
-  if (rdispls) {
-    TUNA_CUDA(pl, cudaMemcpyAsync(pl->d_rdispls, rdispls, PP * 8, cudaMemcpyHostToDevice, st));
-  } else {  // packed: scan of the receive counts = rows of the transposed matrix
-    tuna_transpose_kernel<<<gPP, th, 0, st>>>(pl->d_counts, pl->d_tmp, P, hl ? nullptr : pl->d_extents + 3);
-    TUNA_LAUNCHED(pl);
-    tuna_segscan_kernel<0><<<gseg, th, 0, st>>>(pl->d_tmp, pl->d_rdispls, pl->d_seg_total,
-                                                 nullptr, P, P);
-    TUNA_LAUNCHED(pl);
-    if (!hl) {  // receive regions likewise: scan of the column sums
-      tuna_segbase_kernel<<<1, 1024, 0, st>>>(pl->d_seg_total, nullptr, pl->d_recvbase, P, pl->d_scal, nullptr, 0,
-                                              nullptr);
-      TUNA_LAUNCHED(pl);
-    }
-  }
-
   const int nph = (int)pl->phases.size();
-  TUNA_CUDA(pl, cudaMemsetAsync(pl->d_round_bytes, 0, (size_t)std::max<int64_t>(pl->stats_n, 1) * 8, st));
-  TUNA_CUDA(pl, cudaMemsetAsync(pl->d_wbase, 0, (size_t)(nph + 1) * 8, st));
-  if (pl->classic) {
-    TUNA_CUDA(pl, cudaMemsetAsync(pl->rot.len, 0, (size_t)PP * 8, st));
-    TUNA_CUDA(pl, cudaMemsetAsync(pl->rot.src, 0, (size_t)PP * 8, st));
-    TUNA_CUDA(pl, cudaMemsetAsync(pl->rot.dst, 0, (size_t)PP * 8, st));
-  }
-  tuna_init_tables_kernel<<<gPP, th, 0, st>>>(t, pl->d_counts, pl->d_sdispls, pl->d_rdispls,
-                                              pl->d_sendbase, pl->d_recvbase, pl->d_sz[0],
-                                              pl->d_loc[0], pl->dir.len, pl->dir.src, pl->dir.dst,
-                                              pl->rot.len, pl->rot.src, pl->rot.dst,
-                                              pl->classic ? 1 : 0);
-  TUNA_LAUNCHED(pl);
-
-  int cur = 0;
-  for (int f = 0; f < nph; f++) {
-    const TunaPhase &ph = pl->phases[f];
-    TunaList &k = pl->keep[f];
-    TunaList &d = pl->deliver[f];
-    if (ph.stag_hi > 0) {  // a batch of the staggered exchange: every block arrives
-      const int64_t nd = (int64_t)P * (ph.stag_hi - ph.stag_lo);
-      tuna_stagger_batch_kernel<<<(unsigned)((nd + th - 1) / th), th, 0, st>>>(
-          t, ph.stag_lo, ph.stag_hi, pl->d_sz[cur], pl->d_loc[cur], pl->d_rdispls, pl->d_recvbase,
-          d.len, d.src, d.dst, pl->d_round_bytes + ph.stats_off);
-      TUNA_LAUNCHED(pl);
-      rc = scan_list(pl, k, 0, P, f, pl->d_wbase + f, 1, false, st, 0);
-      if (rc) return rc;
-      rc = scan_list(pl, d, ph.finals, P, nph + f, nullptr, 0, true, st, 1);
-      if (rc) return rc;
-      continue;
-    }
-    PhaseDev pd{ph.level, ph.radix, ph.count, ph.stride, ph.moving, ph.per_rank, ph.finals};
-    const size_t smem = ph.radix <= 4096 ? (size_t)ph.radix * 8 : 0;
-    tuna_meta_exchange_kernel<<<gPP, th, smem, st>>>(t, pd, pl->d_sz[cur], pl->d_loc[cur],
-                                                     pl->d_sz[cur ^ 1], k.len, k.src, d.len, d.src,
-                                                     pl->d_round_bytes + ph.stats_off);
-    TUNA_LAUNCHED(pl);
-    // per-rank prefix sums of both lists; the KEEP stream is this phase's workspace region
-    rc = scan_list(pl, k, ph.per_rank - ph.finals, P, f, pl->d_wbase + f, 1, false, st, 0);
-    if (rc) return rc;
-    rc = scan_list(pl, d, ph.finals, P, nph + f, nullptr, 0, false, st, 1);
-    if (rc) return rc;
-    tuna_place_kernel<<<gPP, th, 0, st>>>(t, pd, pl->d_loc[cur], pl->d_loc[cur ^ 1], k.pos,
-                                          pl->d_seg_base, k.len, d.pos, pl->d_seg_base + P, d.dst,
-                                          pl->d_wbase + f, pl->d_rdispls, pl->d_recvbase,
-                                          pl->classic ? 1 : 0, pl->rot.len, pl->rot.src, pl->rot.dst);
-    TUNA_LAUNCHED(pl);
-    cur ^= 1;
-  }
-  // work partitions of the rotation and direct lists
-  rc = scan_list(pl, pl->rot, pl->classic ? P : 1, P, 2 * nph, nullptr, 0, true, st);
-  if (rc) return rc;
-  rc = scan_list(pl, pl->dir, P, P, 2 * nph + 1, nullptr, 0, true, st);
-  if (rc) return rc;
-
-  // self-check: every descriptor of every list stays inside its buffers
-  // (the same pass sums, per list, the bytes of the blocks whose source and
-  // destination differ modulo 16: they pick the kernel build)
   const int nlists = 2 * nph + 2;
-  TUNA_CUDA(pl, cudaMemsetAsync(pl->d_violations, 0, sizeof(unsigned long long) * (1 + nlists), st));
-  auto check = [&](const TunaList &l, int keep_phase, int id) -> int {
-    if (l.n <= 0) return TUNA_OK;
-    tuna_check_list_kernel<<<(unsigned)std::min<int64_t>((l.n + th - 1) / th, 148 * 8), th, 0, st>>>(
-        l.len, l.pos, l.src, l.kind == TUNA_LIST_DELIVER ? l.dst : nullptr, l.n, pl->d_extents,
-        pl->d_wbase + nph, keep_phase, pl->d_wbase, pl->d_violations,
-        pl->d_violations + 1 + id);
-    TUNA_LAUNCHED(pl);
-    return TUNA_OK;
-  };
-  for (int f = 0; f < nph; f++) {
-    rc = check(pl->keep[f], f, f);
-    if (rc) return rc;
-    rc = check(pl->deliver[f], 0, nph + f);
-    if (rc) return rc;
-  }
-  rc = check(pl->rot, 0, 2 * nph);
-  if (rc) return rc;
-  rc = check(pl->dir, 0, 2 * nph + 1);
-  if (rc) return rc;
+  // Everything from the layout to the self-check only enqueues work on one stream
+  // and reads nothing back, so it can run directly or be captured as a graph.
+  auto enqueue_tables = [&](cudaStream_t st) -> int {
+    int rc = TUNA_OK;
+    if (hl) {
+      pl->payload = hl->payload * t.elem;
+      pl->send_extent = hl->send_extent * t.elem;
+      pl->recv_extent = hl->recv_extent * t.elem;
+      if (!pl->counts_uploaded)
+        TUNA_CUDA(pl, cudaMemcpyAsync(pl->d_counts, counts, PP * 8, cudaMemcpyHostToDevice, st));
+      TUNA_CUDA(pl, cudaMemcpyAsync(pl->d_sendbase, hl->sendbase.data(), P * 8, cudaMemcpyHostToDevice, st));
+      TUNA_CUDA(pl, cudaMemcpyAsync(pl->d_recvbase, hl->recvbase.data(), P * 8, cudaMemcpyHostToDevice, st));
+      const int64_t ext[4] = {pl->send_extent, pl->recv_extent, hl->payload, 0};
+      TUNA_CUDA(pl, cudaMemcpyAsync(pl->d_extents, ext, sizeof(ext), cudaMemcpyHostToDevice, st));
+      // (pageable sources: the runtime stages these copies before it returns)
+    } else {
+      TUNA_CUDA(pl, cudaMemsetAsync(pl->d_extents, 0, 4 * 8, st));
+    }
+    pl->counts_uploaded = false;
+    if (sdispls) {
+      TUNA_CUDA(pl, cudaMemcpyAsync(pl->d_sdispls, sdispls, PP * 8, cudaMemcpyHostToDevice, st));
+    } else {  // packed: exclusive scan of every rank's row of counts
+      tuna_segscan_kernel<0><<<gseg, th, 0, st>>>(pl->d_counts, pl->d_sdispls, pl->d_seg_total,
+                                                   nullptr, P, P);
+      TUNA_LAUNCHED(pl);
+      if (!hl) {  // send regions laid end to end: bases = scan of the row sums
+        tuna_segbase_kernel<<<1, 1024, 0, st>>>(pl->d_seg_total, nullptr, pl->d_sendbase, P, pl->d_scal, nullptr, 0,
+                                                nullptr);
+        TUNA_LAUNCHED(pl);
+        tuna_packed_extents_kernel<<<1, 32, 0, st>>>(pl->d_scal, t.elem, pl->d_extents);
+        TUNA_LAUNCHED(pl);
+      }
+    }
+    if (rdispls) {
+      TUNA_CUDA(pl, cudaMemcpyAsync(pl->d_rdispls, rdispls, PP * 8, cudaMemcpyHostToDevice, st));
+    } else {  // packed: scan of the receive counts = rows of the transposed matrix
+      tuna_transpose_kernel<<<gPP, th, 0, st>>>(pl->d_counts, pl->d_tmp, P, hl ? nullptr : pl->d_extents + 3);
+      TUNA_LAUNCHED(pl);
+      tuna_segscan_kernel<0><<<gseg, th, 0, st>>>(pl->d_tmp, pl->d_rdispls, pl->d_seg_total,
+                                                   nullptr, P, P);
+      TUNA_LAUNCHED(pl);
+      if (!hl) {  // receive regions likewise: scan of the column sums
+        tuna_segbase_kernel<<<1, 1024, 0, st>>>(pl->d_seg_total, nullptr, pl->d_recvbase, P, pl->d_scal, nullptr, 0,
+                                                nullptr);
+        TUNA_LAUNCHED(pl);
+      }
+    }
 
+    TUNA_CUDA(pl, cudaMemsetAsync(pl->d_round_bytes, 0, (size_t)std::max<int64_t>(pl->stats_n, 1) * 8, st));
+    TUNA_CUDA(pl, cudaMemsetAsync(pl->d_wbase, 0, (size_t)(nph + 1) * 8, st));
+    if (pl->classic) {
+      TUNA_CUDA(pl, cudaMemsetAsync(pl->rot.len, 0, (size_t)PP * 8, st));
+      TUNA_CUDA(pl, cudaMemsetAsync(pl->rot.src, 0, (size_t)PP * 8, st));
+      TUNA_CUDA(pl, cudaMemsetAsync(pl->rot.dst, 0, (size_t)PP * 8, st));
+    }
+    tuna_init_tables_kernel<<<gPP, th, 0, st>>>(t, pl->d_counts, pl->d_sdispls, pl->d_rdispls,
+                                                pl->d_sendbase, pl->d_recvbase, pl->d_sz[0],
+                                                pl->d_loc[0], pl->dir.len, pl->dir.src, pl->dir.dst,
+                                                pl->rot.len, pl->rot.src, pl->rot.dst,
+                                                pl->classic ? 1 : 0);
+    TUNA_LAUNCHED(pl);
+
+    int cur = 0;
+    for (int f = 0; f < nph; f++) {
+      const TunaPhase &ph = pl->phases[f];
+      TunaList &k = pl->keep[f];
+      TunaList &d = pl->deliver[f];
+      if (ph.stag_hi > 0) {  // a batch of the staggered exchange: every block arrives
+        const int64_t nd = (int64_t)P * (ph.stag_hi - ph.stag_lo);
+        tuna_stagger_batch_kernel<<<(unsigned)((nd + th - 1) / th), th, 0, st>>>(
+            t, ph.stag_lo, ph.stag_hi, pl->d_sz[cur], pl->d_loc[cur], pl->d_rdispls, pl->d_recvbase,
+            d.len, d.src, d.dst, pl->d_round_bytes + ph.stats_off);
+        TUNA_LAUNCHED(pl);
+        rc = scan_list(pl, k, 0, P, f, pl->d_wbase + f, 1, false, st, 0);
+        if (rc) return rc;
+        rc = scan_list(pl, d, ph.finals, P, nph + f, nullptr, 0, true, st, 1);
+        if (rc) return rc;
+        continue;
+      }
+      PhaseDev pd{ph.level, ph.radix, ph.count, ph.stride, ph.moving, ph.per_rank, ph.finals};
+      const size_t smem = ph.radix <= 4096 ? (size_t)ph.radix * 8 : 0;
+      tuna_meta_exchange_kernel<<<gPP, th, smem, st>>>(t, pd, pl->d_sz[cur], pl->d_loc[cur],
+                                                       pl->d_sz[cur ^ 1], k.len, k.src, d.len, d.src,
+                                                       pl->d_round_bytes + ph.stats_off);
+      TUNA_LAUNCHED(pl);
+      // per-rank prefix sums of both lists; the KEEP stream is this phase's workspace region
+      rc = scan_list(pl, k, ph.per_rank - ph.finals, P, f, pl->d_wbase + f, 1, false, st, 0);
+      if (rc) return rc;
+      rc = scan_list(pl, d, ph.finals, P, nph + f, nullptr, 0, false, st, 1);
+      if (rc) return rc;
+      tuna_place_kernel<<<gPP, th, 0, st>>>(t, pd, pl->d_loc[cur], pl->d_loc[cur ^ 1], k.pos,
+                                            pl->d_seg_base, k.len, d.pos, pl->d_seg_base + P, d.dst,
+                                            pl->d_wbase + f, pl->d_rdispls, pl->d_recvbase,
+                                            pl->classic ? 1 : 0, pl->rot.len, pl->rot.src, pl->rot.dst);
+      TUNA_LAUNCHED(pl);
+      cur ^= 1;
+    }
+    // work partitions of the rotation and direct lists
+    rc = scan_list(pl, pl->rot, pl->classic ? P : 1, P, 2 * nph, nullptr, 0, true, st);
+    if (rc) return rc;
+    rc = scan_list(pl, pl->dir, P, P, 2 * nph + 1, nullptr, 0, true, st);
+    if (rc) return rc;
+
+    // self-check: every descriptor of every list stays inside its buffers
+    // (the same pass sums, per list, the bytes of the blocks whose source and
+    // destination differ modulo 16: they pick the kernel build)
+    TUNA_CUDA(pl, cudaMemsetAsync(pl->d_violations, 0, sizeof(unsigned long long) * (1 + nlists), st));
+    auto check = [&](const TunaList &l, int keep_phase, int id) -> int {
+      if (l.n <= 0) return TUNA_OK;
+      tuna_check_list_kernel<<<(unsigned)std::min<int64_t>((l.n + th - 1) / th, 148 * 8), th, 0, st>>>(
+          l.len, l.pos, l.src, l.kind == TUNA_LIST_DELIVER ? l.dst : nullptr, l.n, pl->d_extents,
+          pl->d_wbase + nph, keep_phase, pl->d_wbase, pl->d_violations,
+          pl->d_violations + 1 + id);
+      TUNA_LAUNCHED(pl);
+      return TUNA_OK;
+    };
+    for (int f = 0; f < nph; f++) {
+      rc = check(pl->keep[f], f, f);
+      if (rc) return rc;
+      rc = check(pl->deliver[f], 0, nph + f);
+      if (rc) return rc;
+    }
+    rc = check(pl->rot, 0, 2 * nph);
+    if (rc) return rc;
+    rc = check(pl->dir, 0, 2 * nph + 1);
+    if (rc) return rc;
+
+    return rc;
+  };
+  Timed plan_timer(pl, TUNA_TIMER_PLAN, 0, st);
+  rc = hl ? enqueue_tables(st) : replay_tables_graph(pl, enqueue_tables, st);
+  if (rc) return rc;
   plan_timer.stop();  // the chunk tables below are timed separately, after the read-back
   // one read-back: stream totals, workspace offsets, per-round bytes
   std::vector<int64_t> scal(2 * (2 * nph + 2)), wbase(nph + 1);
   std::vector<unsigned long long> rbytes(std::max<int64_t>(pl->stats_n, 1));
-  TUNA_CUDA(pl, cudaMemcpyAsync(scal.data(), pl->d_scal, scal.size() * 8, cudaMemcpyDeviceToHost, st));
-  TUNA_CUDA(pl, cudaMemcpyAsync(wbase.data(), pl->d_wbase, wbase.size() * 8, cudaMemcpyDeviceToHost, st));
-  TUNA_CUDA(pl, cudaMemcpyAsync(rbytes.data(), pl->d_round_bytes, rbytes.size() * 8,
-                                cudaMemcpyDeviceToHost, st));
   std::vector<unsigned long long> checked(1 + nlists);
-  TUNA_CUDA(pl, cudaMemcpyAsync(checked.data(), pl->d_violations, checked.size() * 8, cudaMemcpyDeviceToHost, st));
   int64_t ext[4] = {0, 0, 0, 0};
-  if (!hl) TUNA_CUDA(pl, cudaMemcpyAsync(ext, pl->d_extents, sizeof(ext), cudaMemcpyDeviceToHost, st));
-  TUNA_CUDA(pl, cudaStreamSynchronize(st));
+  if (pl->h_readback) {  // one copy of the whole block into pinned memory
+    TUNA_CUDA(pl, cudaMemcpyAsync(pl->h_readback, pl->d_readback, (size_t)pl->readback_words * 8,
+                                  cudaMemcpyDeviceToHost, st));
+    TUNA_CUDA(pl, cudaStreamSynchronize(st));
+    const int64_t *h = pl->h_readback;
+    std::copy(h + (pl->d_scal - pl->d_readback), h + (pl->d_scal - pl->d_readback) + scal.size(), scal.begin());
+    std::copy(h + (pl->d_wbase - pl->d_readback), h + (pl->d_wbase - pl->d_readback) + wbase.size(), wbase.begin());
+    std::copy(h + (pl->d_extents - pl->d_readback), h + (pl->d_extents - pl->d_readback) + 4, ext);
+    const unsigned long long *hu = reinterpret_cast<const unsigned long long *>(h);
+    const int64_t o_rb = reinterpret_cast<int64_t *>(pl->d_round_bytes) - pl->d_readback;
+    const int64_t o_vi = reinterpret_cast<int64_t *>(pl->d_violations) - pl->d_readback;
+    std::copy(hu + o_rb, hu + o_rb + rbytes.size(), rbytes.begin());
+    std::copy(hu + o_vi, hu + o_vi + checked.size(), checked.begin());
+  } else {
+    TUNA_CUDA(pl, cudaMemcpyAsync(scal.data(), pl->d_scal, scal.size() * 8, cudaMemcpyDeviceToHost, st));
+    TUNA_CUDA(pl, cudaMemcpyAsync(wbase.data(), pl->d_wbase, wbase.size() * 8, cudaMemcpyDeviceToHost, st));
+    TUNA_CUDA(pl, cudaMemcpyAsync(rbytes.data(), pl->d_round_bytes, rbytes.size() * 8,
+                                  cudaMemcpyDeviceToHost, st));
+    TUNA_CUDA(pl, cudaMemcpyAsync(checked.data(), pl->d_violations, checked.size() * 8, cudaMemcpyDeviceToHost, st));
+    TUNA_CUDA(pl, cudaMemcpyAsync(ext, pl->d_extents, sizeof(ext), cudaMemcpyDeviceToHost, st));
+    TUNA_CUDA(pl, cudaStreamSynchronize(st));
+  }
   if (!hl) {
     if (ext[3] != 0) return TUNA_ERR_INVALID_ARG;  // negative counts
     pl->send_extent = ext[0];
@@ -1430,6 +1509,8 @@ int tuna_plan_destroy(tuna_plan_t *pl) {
     if (pl->in_flight_set) (void)cudaEventSynchronize(pl->in_flight);  // the tables are freed below
     cudaEventDestroy(pl->in_flight);
   }
+  if (pl->tables_graph) cudaGraphExecDestroy(pl->tables_graph);
+  if (pl->capture_stream) cudaStreamDestroy(pl->capture_stream);
   for (auto &l : pl->keep) free_list(l);
   for (auto &l : pl->deliver) free_list(l);
   free_list(pl->rot);
@@ -1456,12 +1537,9 @@ int tuna_plan_destroy(tuna_plan_t *pl) {
   cudaFree(pl->d_seg_raw);
   cudaFree(pl->d_seg_base);
   cudaFree(pl->d_tmp);
-  cudaFree(pl->d_scal);
-  cudaFree(pl->d_wbase);
-  cudaFree(pl->d_extents);
-  cudaFree(pl->d_round_bytes);
+  cudaFree(pl->d_readback);  // (d_scal, d_wbase, d_extents, d_round_bytes, d_violations are slices of it)
+  if (pl->h_readback) cudaFreeHost(pl->h_readback);
   cudaFree(pl->d_error);
-  cudaFree(pl->d_violations);
   for (auto &s : pl->stamps) {
     cudaEventDestroy(s.a);
     cudaEventDestroy(s.b);
@@ -1558,12 +1636,23 @@ static int plan_create(tuna_plan_t **out, int P, int radix, int radix_global, in
   TUNA_TRY(dev_alloc(&pl->d_seg_raw, P));
   TUNA_TRY(dev_alloc(&pl->d_seg_base, 2 * P));
   TUNA_TRY(dev_alloc(&pl->d_tmp, PP));
-  TUNA_TRY(dev_alloc(&pl->d_scal, 2 * (2 * nph + 3)));
-  TUNA_TRY(dev_alloc(&pl->d_wbase, nph + 1));
-  TUNA_TRY(dev_alloc(&pl->d_extents, 6));  // [4], [5]: extents of the row exchange's buffers
-  TUNA_TRY(dev_alloc(&pl->d_round_bytes, pl->stats_n));
+  {
+    const int64_t n_scal = 2 * (2 * nph + 3), n_wbase = nph + 1, n_ext = 6;  // ext [4], [5]: the row exchange's buffers
+    const int64_t n_rb = std::max<int64_t>(pl->stats_n, 1), n_viol = 1 + 2 * nph + 3;
+    pl->readback_words = n_scal + n_wbase + n_ext + n_rb + n_viol;
+    TUNA_TRY(dev_alloc(&pl->d_readback, pl->readback_words));
+    TUNA_TRY(cudaMemset(pl->d_readback, 0, (size_t)pl->readback_words * 8));
+    if (cudaHostAlloc((void **)&pl->h_readback, (size_t)pl->readback_words * 8, cudaHostAllocDefault) != cudaSuccess) {
+      (void)cudaGetLastError();
+      pl->h_readback = nullptr;  // (the copies then go to pageable memory, one by one)
+    }
+    pl->d_scal = pl->d_readback;
+    pl->d_wbase = pl->d_scal + n_scal;
+    pl->d_extents = pl->d_wbase + n_wbase;
+    pl->d_round_bytes = reinterpret_cast<unsigned long long *>(pl->d_extents + n_ext);
+    pl->d_violations = pl->d_round_bytes + n_rb;
+  }
   TUNA_TRY(dev_alloc(&pl->d_error, 1));
-  TUNA_TRY(dev_alloc(&pl->d_violations, 1 + 2 * nph + 3));
   TUNA_TRY(cudaMemset(pl->d_error, 0, sizeof(int)));
   pl->keep.resize(nph);
   pl->deliver.resize(nph);
@@ -1636,13 +1725,14 @@ int tuna_plan_update_counts_device(tuna_plan_t *pl, const int64_t *d_sendcounts,
   if (!pl || !d_sendcounts) return TUNA_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;
   const int64_t PP = (int64_t)pl->topo.P * pl->topo.P;
-  // the plan keeps its own copy (the caller may reuse its array at once); it goes
-  // into the spare buffer, like an upload from the host
-  int64_t *spare = pl->d_counts == pl->d_counts_buf[0] ? pl->d_counts_buf[1] : pl->d_counts_buf[0];
-  if (d_sendcounts != spare)
-    TUNA_CUDA(pl, cudaMemcpyAsync(spare, d_sendcounts, (size_t)PP * 8, cudaMemcpyDeviceToDevice, st));
-  pl->d_counts = spare;
-  pl->counts_uploaded = true;
+  // the plan keeps its own copy (the caller may reuse its array at once), in the
+  // buffer its tables were last built from: the kernels that read it stay the same
+  {
+    const int wrc = wait_in_flight(pl);
+    if (wrc) return wrc;
+  }
+  pl->tables_valid = false;
+  TUNA_CUDA(pl, cudaMemcpyAsync(pl->d_counts, d_sendcounts, (size_t)PP * 8, cudaMemcpyDeviceToDevice, st));
   return build_tables(pl, nullptr, nullptr, nullptr, st);
 }
 
