@@ -323,6 +323,9 @@ int tuna_rows_alltoallv(tuna_plan_t *plan, const void *rows_in, void *rows_out, 
  * blocks that have arrived and land in the receive buffer (empty in
  * TUNA_FLAG_CLASSIC_ROTATE mode); the two lists of a phase share one kernel launch.
  * phase -1 selects the rotation list and -2 the direct list (`part` ignored).
+ * A flat plan whose radix is at least P (one digit phase that delivers every
+ * block) keeps no separate direct list: tuna_direct_alltoallv then runs that
+ * phase's DELIVER list and the self blocks, and phase -2 reports no entries.
  * `entries` descriptor rows, `bytes` moved, `stream_bytes` the padded length of the
  * list's stream (for a KEEP list: the size of its workspace region).
  */

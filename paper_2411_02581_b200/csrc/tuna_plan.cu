@@ -81,7 +81,7 @@ __global__ void tuna_init_tables_kernel(TunaTopo t, const int64_t *__restrict__ 
   sz[idx] = bytes;
   loc[idx] = sloc;
   // direct list entry (d = p as receiver, s = sigma as source index)
-  {
+  if (dir_len) {
     const int d = p, s = sigma;
     dir_len[idx] = counts[(int64_t)s * t.P + d] * t.elem;
     dir_src[idx] = TUNA_LOC(TUNA_BUF_SEND, (sendbase[s] + sdispls[(int64_t)s * t.P + d]) * t.elem);
@@ -411,22 +411,22 @@ __global__ void tuna_check_list_kernel(const int64_t *__restrict__ len, const in
   bool bad = false;
   int64_t skewed = 0;  // bytes of blocks whose source and destination differ modulo 16
   const int64_t send_extent = extents[0], recv_extent = extents[1];
+  const int64_t wext = *work_extent, wb = wbase[keep_base_index];
   for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < n; e += (int64_t)gridDim.x * blockDim.x) {
-    const int64_t L = len[e];
-    bad = bad || L < 0 || pos[e + 1] < pos[e];
+    // all of a descriptor's fields at once: one round trip to memory per descriptor
+    const int64_t L = len[e], p0 = pos[e], p1 = pos[e + 1], s = src[e], d = dst ? dst[e] : 0;
+    bad = bad || L < 0 || p1 < p0;
     if (L > 0) {
-      const int64_t s = src[e];
       const int sb = TUNA_LOC_BUF(s);
       const int64_t so = TUNA_LOC_OFF(s);
-      const int64_t sext = sb == TUNA_BUF_SEND ? send_extent : (sb == TUNA_BUF_WORK ? *work_extent : -1);
+      const int64_t sext = sb == TUNA_BUF_SEND ? send_extent : (sb == TUNA_BUF_WORK ? wext : -1);
       bad = bad || so < 0 || so + L > sext;
       if (dst) {  // DELIVER: into the receive buffer
-        const int64_t d = dst[e];
         bad = bad || TUNA_LOC_BUF(d) != TUNA_BUF_RECV || TUNA_LOC_OFF(d) + L > recv_extent;
         if (((so - TUNA_LOC_OFF(d)) & 15) != 0) skewed += L;
       } else {    // KEEP: at its stream position in the phase's workspace region
-        const int64_t o = wbase[keep_base_index] + pos[e];
-        bad = bad || (o & (TUNA_ALIGN - 1)) != 0 || o + pad16(L) > *work_extent || pos[e + 1] - pos[e] != pad16(L);
+        const int64_t o = wb + p0;
+        bad = bad || (o & (TUNA_ALIGN - 1)) != 0 || o + pad16(L) > wext || p1 - p0 != pad16(L);
         if ((so & 15) != 0) skewed += L;
       }
     }
@@ -485,6 +485,10 @@ struct tuna_plan {
   std::vector<TunaList> keep;     // per phase: blocks that travel on (workspace)
   std::vector<TunaList> deliver;  // per phase: blocks that have arrived (receive buffer)
   TunaList rot, dir;
+  // A flat direct-to-R plan with a single digit phase (radix >= P) delivers every
+  // block in that phase: its DELIVER list and the self blocks together are the
+  // direct exchange, so no separate direct list is built.
+  bool dir_shared = false;
   // exchange of rows through a gather and a scatter map (tuna_plan_set_row_maps)
   TunaList rowsl;
   int64_t rows_cap = 0;          // descriptors allocated in rowsl
@@ -1170,7 +1174,7 @@ int build_tables(tuna_plan *pl, const HostLayout *hl, const int64_t *sdispls, co
     // work partitions of the rotation and direct lists
     rc = scan_list(pl, pl->rot, pl->classic ? P : 1, P, 2 * nph, nullptr, 0, true, st);
     if (rc) return rc;
-    rc = scan_list(pl, pl->dir, P, P, 2 * nph + 1, nullptr, 0, true, st);
+    if (!pl->dir_shared) rc = scan_list(pl, pl->dir, P, P, 2 * nph + 1, nullptr, 0, true, st);
     if (rc) return rc;
 
     // self-check: every descriptor of every list stays inside its buffers
@@ -1194,7 +1198,7 @@ int build_tables(tuna_plan *pl, const HostLayout *hl, const int64_t *sdispls, co
     }
     rc = check(pl->rot, 0, 2 * nph);
     if (rc) return rc;
-    rc = check(pl->dir, 0, 2 * nph + 1);
+    if (!pl->dir_shared) rc = check(pl->dir, 0, 2 * nph + 1);
     if (rc) return rc;
 
     return rc;
@@ -1248,7 +1252,7 @@ int build_tables(tuna_plan *pl, const HostLayout *hl, const int64_t *sdispls, co
     take(pl->deliver[f], nph + f);
   }
   take(pl->rot, 2 * nph);
-  take(pl->dir, 2 * nph + 1);
+  if (!pl->dir_shared) take(pl->dir, 2 * nph + 1);
   pl->workspace_need = wbase[nph];
   for (auto &r : pl->rounds) r.bytes = (int64_t)rbytes[r.stat];
 
@@ -1261,7 +1265,7 @@ int build_tables(tuna_plan *pl, const HostLayout *hl, const int64_t *sdispls, co
   }
   rc = build_chunks(pl, pl->rot, st);
   if (rc) return rc;
-  rc = build_chunks(pl, pl->dir, st);
+  if (!pl->dir_shared) rc = build_chunks(pl, pl->dir, st);
   if (rc) return rc;
   TUNA_CUDA(pl, cudaStreamSynchronize(st));
   pl->tables_valid = true;
@@ -1464,7 +1468,19 @@ int run_tuna(tuna_plan *pl, const void *send, void *recv, cudaStream_t st) {
 
 int run_direct(tuna_plan *pl, const void *send, void *recv, cudaStream_t st) {
   int launches = 0;
-  if (pl->dir.nchunks > 0) {
+  if (pl->dir_shared) {  // the single phase's DELIVER list and the self blocks: every block, once
+    const TunaList &d = pl->deliver[0];
+    if (d.nchunks > 0 || pl->rot.nchunks > 0) {
+      const int64_t bytes = d.bytes + pl->rot.bytes;
+      const int64_t small_bytes = (d.small_blocks ? d.bytes : 0) + (pl->rot.small_blocks ? pl->rot.bytes : 0);
+      Timed tm(pl, TUNA_TIMER_DIRECT, bytes, st);
+      TunaMoveArgs a = move_args(pl, send, recv, nullptr);
+      a.del = list_args(d);
+      a.rot = list_args(pl->rot);
+      TUNA_CUDA(pl, tuna_launch_move(TUNA_K_DIRECT, a, 2 * small_bytes >= bytes, st));
+      launches++;
+    }
+  } else if (pl->dir.nchunks > 0) {
     Timed tm(pl, TUNA_TIMER_DIRECT, pl->dir.bytes, st);
     TunaMoveArgs a = move_args(pl, send, recv, nullptr);
     a.del = list_args(pl->dir);
@@ -1668,8 +1684,12 @@ static int plan_create(tuna_plan_t **out, int P, int radix, int radix_global, in
   }
   rc = alloc_list(pl, pl->rot, TUNA_LIST_DELIVER, pl->classic ? PP : P);
   if (rc) return nomem(rc);
-  rc = alloc_list(pl, pl->dir, TUNA_LIST_DELIVER, PP);
-  if (rc) return nomem(rc);
+  pl->dir_shared = !pl->classic && g == 1 && block_count == 0 && nph == 1 &&
+                   pl->phases[0].finals == pl->phases[0].per_rank;
+  if (!pl->dir_shared) {
+    rc = alloc_list(pl, pl->dir, TUNA_LIST_DELIVER, PP);
+    if (rc) return nomem(rc);
+  }
 #undef TUNA_TRY
   rc = build_tables(pl, &hl, sdispls, rdispls, st);
   if (rc) return fail(rc);
