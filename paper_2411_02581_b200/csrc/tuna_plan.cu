@@ -150,6 +150,56 @@ __global__ void tuna_meta_exchange_kernel(TunaTopo t, PhaseDev ph, const int64_t
   }
 }
 
+// The same exchange for the one phase of a flat plan whose radix is at least P
+// (every slot o >= 1 moves once, from rank p - o to rank p): the general kernel
+// would read the two tables along anti-diagonals, one 32-byte sector per value,
+// and add one byte counter per slot to global memory.  Here a CTA reads a
+// 32 x 32 tile (sender, slot) along rows, and writes it out by receiver, where
+// each receiver's slots are again consecutive; a round's bytes are summed per tile
+// column first.  Grid: ceil(P/32) x ceil(P/32) CTAs of 32 x 8 threads.
+__global__ void tuna_meta_exchange_diag_kernel(TunaTopo t, PhaseDev ph, const int64_t *__restrict__ sz_cur,
+                                               const int64_t *__restrict__ loc_cur, int64_t *sz_next,
+                                               int64_t *keep_len, int64_t *keep_src, int64_t *del_len,
+                                               int64_t *del_src, unsigned long long *round_bytes) {
+  __shared__ int64_t s_sz[32][32], s_loc[32][32];
+  const int P = t.P, tx = threadIdx.x, ty = threadIdx.y;
+  const int g0 = blockIdx.x * 32, s0 = blockIdx.y * 32;  // first slot and first sender of the tile
+  for (int j = ty; j < 32; j += 8) {
+    const int sd = s0 + j, g = g0 + tx;
+    const bool in = sd < P && g < P;
+    s_sz[j][tx] = in ? sz_cur[(int64_t)sd * P + g] : 0;
+    s_loc[j][tx] = in ? loc_cur[(int64_t)sd * P + g] : 0;
+  }
+  __syncthreads();
+  if (ty == 0 && g0 + tx >= 1 && g0 + tx < P) {  // round z = slot: bytes sent by this tile's senders
+    int64_t sum = 0;
+#pragma unroll 8
+    for (int j = 0; j < 32; j++) sum += s_sz[j][tx];
+    if (sum > 0) atomicAdd(&round_bytes[g0 + tx], (unsigned long long)sum);
+  }
+  for (int pr = ty; pr < 63; pr += 8) {  // receivers s0 + g0 + pr (mod P): a diagonal of the tile each
+    const int sr = pr - tx;
+    if (sr < 0 || sr >= 32) continue;
+    const int sd = s0 + sr, g = g0 + tx;
+    if (sd >= P || g >= P) continue;
+    int p = sd + g;
+    if (p >= P) p -= P;
+    const int64_t bytes = s_sz[sr][tx], where = s_loc[sr][tx];
+    sz_next[(int64_t)p * P + g] = bytes;  // (slot 0 never moves: sender and receiver are the same rank)
+    if (g == 0) continue;
+    const int64_t c = g - 1;  // position among the P - 1 blocks the rank receives, in slot order
+    if (c < ph.finals) {
+      const int64_t e = (int64_t)p * ph.finals + c;
+      del_len[e] = bytes;
+      del_src[e] = where;
+    } else {
+      const int64_t e = (int64_t)p * (ph.per_rank - ph.finals) + (c - ph.finals);
+      keep_len[e] = bytes;
+      keep_src[e] = where;
+    }
+  }
+}
+
 // Staggered inter-group exchange (Sec. IV-B, Algorithm 2), one batch: the steps
 // ii in [lo, hi) of the index ii = gi*Q + gr, gi >= 1.  In step (gi, gr) rank
 // (n, q) receives, from rank ((n + gi) mod N, q), the one block whose original
@@ -447,15 +497,26 @@ __global__ void tuna_check_list_kernel(const int64_t *__restrict__ len, const in
   }
 }
 
-// out = in^T.  With `negatives`, entries below zero are counted there (counts that
-// arrive in device memory are validated in this pass).
+// out = in^T, in 32 x 32 tiles through shared memory so that both the reads and the
+// writes run along rows (grid: ceil(P/32) x ceil(P/32) CTAs of 32 x 8 threads).
+// With `negatives`, entries below zero are counted there (counts that arrive in
+// device memory are validated in this pass).
 __global__ void tuna_transpose_kernel(const int64_t *__restrict__ in, int64_t *out, int P, int64_t *negatives) {
-  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (idx >= (int64_t)P * P) return;
-  const int r = (int)((unsigned)idx / (unsigned)P), c = (int)((unsigned)idx % (unsigned)P);
-  const int64_t v = in[(int64_t)c * P + r];
-  out[idx] = v;
-  if (negatives && v < 0) atomicAdd(reinterpret_cast<unsigned long long *>(negatives), 1ULL);
+  __shared__ int64_t tile[32][33];
+  const int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32;  // the tile in[r0.., c0..]
+  for (int j = threadIdx.y; j < 32; j += 8) {
+    const int r = r0 + j, c = c0 + threadIdx.x;
+    if (r < P && c < P) {
+      const int64_t v = in[(int64_t)r * P + c];
+      tile[j][threadIdx.x] = v;
+      if (negatives && v < 0) atomicAdd(reinterpret_cast<unsigned long long *>(negatives), 1ULL);
+    }
+  }
+  __syncthreads();
+  for (int j = threadIdx.y; j < 32; j += 8) {
+    const int r = c0 + j, c = r0 + threadIdx.x;  // out[r][c] = in[c][r]
+    if (r < P && c < P) out[(int64_t)r * P + c] = tile[threadIdx.x][j];
+  }
 }
 
 // Packed layout worked out on the device: both buffers extend over the sum of all
@@ -1110,7 +1171,7 @@ int build_tables(tuna_plan *pl, const HostLayout *hl, const int64_t *sdispls, co
     if (rdispls) {
       TUNA_CUDA(pl, cudaMemcpyAsync(pl->d_rdispls, rdispls, PP * 8, cudaMemcpyHostToDevice, st));
     } else {  // packed: scan of the receive counts = rows of the transposed matrix
-      tuna_transpose_kernel<<<gPP, th, 0, st>>>(pl->d_counts, pl->d_tmp, P, hl ? nullptr : pl->d_extents + 3);
+      tuna_transpose_kernel<<<dim3((P + 31) / 32, (P + 31) / 32), dim3(32, 8), 0, st>>>(pl->d_counts, pl->d_tmp, P, hl ? nullptr : pl->d_extents + 3);
       TUNA_LAUNCHED(pl);
       tuna_segscan_kernel<0><<<gseg, th, 0, st>>>(pl->d_tmp, pl->d_rdispls, pl->d_seg_total,
                                                    nullptr, P, P);
@@ -1154,10 +1215,16 @@ int build_tables(tuna_plan *pl, const HostLayout *hl, const int64_t *sdispls, co
         continue;
       }
       PhaseDev pd{ph.level, ph.radix, ph.count, ph.stride, ph.moving, ph.per_rank, ph.finals};
-      const size_t smem = ph.radix <= 4096 ? (size_t)ph.radix * 8 : 0;
-      tuna_meta_exchange_kernel<<<gPP, th, smem, st>>>(t, pd, pl->d_sz[cur], pl->d_loc[cur],
-                                                       pl->d_sz[cur ^ 1], k.len, k.src, d.len, d.src,
-                                                       pl->d_round_bytes + ph.stats_off);
+      if (ph.level == 0 && t.N == 1 && ph.stride == 1 && ph.radix >= P) {
+        tuna_meta_exchange_diag_kernel<<<dim3((P + 31) / 32, (P + 31) / 32), dim3(32, 8), 0, st>>>(
+            t, pd, pl->d_sz[cur], pl->d_loc[cur], pl->d_sz[cur ^ 1], k.len, k.src, d.len, d.src,
+            pl->d_round_bytes + ph.stats_off);
+      } else {
+        const size_t smem = ph.radix <= 4096 ? (size_t)ph.radix * 8 : 0;
+        tuna_meta_exchange_kernel<<<gPP, th, smem, st>>>(t, pd, pl->d_sz[cur], pl->d_loc[cur],
+                                                         pl->d_sz[cur ^ 1], k.len, k.src, d.len, d.src,
+                                                         pl->d_round_bytes + ph.stats_off);
+      }
       TUNA_LAUNCHED(pl);
       // per-rank prefix sums of both lists; the KEEP stream is this phase's workspace region
       rc = scan_list(pl, k, ph.per_rank - ph.finals, P, f, pl->d_wbase + f, 1, false, st, 0);
@@ -1894,7 +1961,7 @@ int tuna_plan_set_row_maps(tuna_plan_t *pl, const int64_t *gather_rows, const in
   const int nph = (int)pl->phases.size();
   Timed plan_timer(pl, TUNA_TIMER_PLAN, 0, st);
   // rows before every block in receive-side order: scan of the transposed counts
-  tuna_transpose_kernel<<<gPP, th, 0, st>>>(pl->d_counts, pl->d_tmp, P, nullptr);
+  tuna_transpose_kernel<<<dim3((P + 31) / 32, (P + 31) / 32), dim3(32, 8), 0, st>>>(pl->d_counts, pl->d_tmp, P, nullptr);
   TUNA_LAUNCHED(pl);
   tuna_segscan_kernel<0><<<gseg, th, 0, st>>>(pl->d_tmp, pl->d_row_start, pl->d_seg_total, nullptr, P, P);
   TUNA_LAUNCHED(pl);
@@ -2235,7 +2302,7 @@ int tuna_direct_alltoallv_static(int P, int elem_size, const int64_t *sendcounts
   if (rdispls) {
     TUNA_STATIC_CUDA(cudaMemcpyAsync(t.rdispls, rdispls, PP * 8, cudaMemcpyHostToDevice, st));
   } else {
-    tuna_transpose_kernel<<<gPP, th, 0, st>>>(t.counts, t.tmp, P, nullptr);
+    tuna_transpose_kernel<<<dim3((P + 31) / 32, (P + 31) / 32), dim3(32, 8), 0, st>>>(t.counts, t.tmp, P, nullptr);
     TUNA_STATIC_CUDA(cudaGetLastError());
     tuna_segscan_kernel<0><<<gseg, th, 0, st>>>(t.tmp, t.rdispls, t.seg_total, nullptr, P, P);
     TUNA_STATIC_CUDA(cudaGetLastError());
