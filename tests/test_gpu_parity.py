@@ -148,7 +148,7 @@ def test_hier_small(Q, N, rl, rg):
         check_rounds(plan, rounds)
 
 
-@pytest.mark.parametrize("P,r", [(8, 2), (9, 3), (16, 4), (20, 5), (64, 8)])
+@pytest.mark.parametrize("P,r", [(8, 2), (9, 3), (16, 4), (20, 5), (64, 8), (5, 5), (33, 33), (70, 70), (64, 64)])
 def test_metadata_and_prefix_sums(P, r):
     """Descriptor tables of every digit phase: sizes equal the oracle's
     message-passed metadata, positions equal its running sums."""
@@ -189,6 +189,8 @@ def test_metadata_and_prefix_sums(P, r):
                 s = (p - o) % P
                 assert dst[p, j] == (1 << 56) | int(wl.recvbase[p] + wl.rdispls[p, s]) * wl.elem_size
     assert plan.workspace_bytes() == work_off
+    # one phase that delivers everything: it doubles as the direct exchange's list
+    assert plan.phase_info(-2)["entries"] == (0 if r >= P else P * P)
     # classic mode keeps every block in the workspace and rotates at the end
     classic = B.plan_for(wl, r, flags=B.FLAG_CLASSIC_ROTATE)
     for x in range(classic.num_phases()):
