@@ -236,6 +236,61 @@ __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wa
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
+// ------------------------------------------------------------------ one skewed block
+//
+// A run of m whole vectors inside one block whose source is not 16-byte aligned
+// (dst is).  Every output vector needs two neighbouring aligned source vectors;
+// instead of loading both, a lane loads one and takes the other from the next lane
+// by shuffle, so the loads are those of a plain copy.  A warp therefore turns 32
+// loaded vectors into 31 stored ones; consecutive warp tiles overlap by one vector.
+// The source's offset in its vector is the same for the whole run, so which words
+// to merge is decided once (Q = offset / 4), outside the loop.
+// Reads [src - (src & 15), src + 16 m + 16 - (src & 15)).
+template <int kUnroll, int Q>
+__device__ __forceinline__ void skewed_run_q(const uint4 *a0, unsigned bits, char *dst, int m) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  constexpr int kWarps = kThreads / 32;
+  for (int g0 = warp; g0 * 31 < m; g0 += kUnroll * kWarps) {  // (warp-uniform: the shuffles need every lane)
+    uint4 A[kUnroll];
+#pragma unroll
+    for (int k = 0; k < kUnroll; k++) {
+      const int i = (g0 + k * kWarps) * 31 + lane;
+      A[k] = i <= m ? a0[i] : make_uint4(0, 0, 0, 0);
+    }
+#pragma unroll
+    for (int k = 0; k < kUnroll; k++) {
+      const int i = (g0 + k * kWarps) * 31 + lane;
+      // words Q .. Q + 4 of the eight this lane and the next one hold
+      uint32_t w[8];
+      w[0] = A[k].x, w[1] = A[k].y, w[2] = A[k].z, w[3] = A[k].w;
+#pragma unroll
+      for (int j = 0; j <= Q; j++) {
+        const uint32_t mine = j == 0 ? A[k].x : j == 1 ? A[k].y : j == 2 ? A[k].z : A[k].w;
+        w[4 + j] = __shfl_down_sync(0xffffffffu, mine, 1);
+      }
+      uint4 x;
+      x.x = __funnelshift_r(w[Q], w[Q + 1], bits);
+      x.y = __funnelshift_r(w[Q + 1], w[Q + 2], bits);
+      x.z = __funnelshift_r(w[Q + 2], w[Q + 3], bits);
+      x.w = __funnelshift_r(w[Q + 3], w[Q + 4], bits);
+      if (lane < 31 && i < m) st16(dst + ((int64_t)i << 4), x);
+    }
+  }
+}
+
+template <int kUnroll>
+__device__ __forceinline__ void skewed_run(const char *src, char *dst, int m) {
+  const unsigned sh = (unsigned)(reinterpret_cast<uintptr_t>(src) & 15);
+  const uint4 *a0 = reinterpret_cast<const uint4 *>(src - sh);
+  const unsigned bits = (sh & 3) * 8;
+  switch (sh >> 2) {
+    case 0: skewed_run_q<kUnroll, 0>(a0, bits, dst, m); break;
+    case 1: skewed_run_q<kUnroll, 1>(a0, bits, dst, m); break;
+    case 2: skewed_run_q<kUnroll, 2>(a0, bits, dst, m); break;
+    default: skewed_run_q<kUnroll, 3>(a0, bits, dst, m); break;
+  }
+}
+
 // ------------------------------------------------------------------ the mover
 
 template <bool DELIVER, int kUnroll, bool kBulk>  // kUnroll: vectors a thread has in flight
@@ -377,6 +432,16 @@ __device__ __forceinline__ void move_body(const TunaListArgs &l, const TunaMoveA
         }
         for (; i < m; i += kThreads) st16(dst + ((int64_t)i << 4), ld16(src + ((int64_t)i << 4)));
         continue;
+      }
+      // The same range with a skewed source: still one block, every vector whole.
+      // (Only in the build with registers to spare; lists of large blocks run it.)
+      if constexpr (kUnroll >= 4) {
+        bool whole = s_careful[0] == 0 && (reinterpret_cast<uintptr_t>(src) & 15) != 0;
+        if (DELIVER) whole = whole && s_org[0] <= (vlo << 4) && s_end[0] >= (vhi << 4);
+        if (whole) {
+          skewed_run<kUnroll>(src, dst, vhi - vlo);
+          continue;
+        }
       }
     }
     if (!single) {

@@ -774,6 +774,12 @@ int64_t env_i64(const char *name, int64_t dflt) {
 // their block size; the large build otherwise.  Lists small enough to live in L2
 // are latency-bound rather than DRAM-bound and also do better with the small
 // build's higher occupancy (c3, 16 x 16 ranks, radix 16/2: 0.144 ms against 0.169 ms).
+// Skewed lists of large blocks go back to the large build: a chunk inside one
+// skewed block takes its own path there (one aligned load per vector, the
+// neighbour's words by shuffle).  Measured, small / large build: 5.27 / 4.95 TB/s
+// at 128 KiB mean block size, 5.29 / 5.36 at 256 KiB, 5.36 / 5.78 at 1 MiB,
+// 5.53 / 6.22 at 4 MiB.
+constexpr int64_t kSkewedLargeBlockBytes = 256 << 10;
 constexpr int64_t kSmallBlockBytes = 256;
 constexpr int64_t kSmallListBytes = 64 << 20;
 constexpr int64_t kStaticSmallBlockBytes = 65536;  // the table-free entry point decides by size alone
@@ -798,7 +804,8 @@ int64_t pick_chunk(const TunaList &l) {
 int build_chunks(tuna_plan *pl, TunaList &l, cudaStream_t st) {
   l.small_blocks = l.n > 0 && (l.bytes / l.n < env_i64("TUNA_SMALL_BLOCK_BYTES", kSmallBlockBytes) ||
                                l.bytes < env_i64("TUNA_SMALL_LIST_BYTES", kSmallListBytes) ||
-                               (2 * l.unaligned_bytes > l.bytes && env_i64("TUNA_SKEWED_SMALL", 1) != 0));
+                               (2 * l.unaligned_bytes > l.bytes && l.bytes / l.n < kSkewedLargeBlockBytes &&
+                                env_i64("TUNA_SKEWED_SMALL", 1) != 0));
   l.chunk = pick_chunk(l);
   l.nchunks = l.total > 0 ? (l.total + l.chunk - 1) / l.chunk : 0;
   if (l.nchunks > l.chunk_cap) {

@@ -116,6 +116,27 @@ def test_large_blocks_span_many_chunks():
     assert np.array_equal(got, ref)
 
 
+@pytest.mark.parametrize("misalign", [0, 5])
+def test_large_skewed_blocks(misalign):
+    """Megabyte blocks of odd byte counts in lists large enough for the large-block
+    build: chunks inside one block whose source is skewed against its destination
+    (one aligned load per vector, the neighbour's words by shuffle)."""
+    wl = W.make_random(12, 2_100_000, elem_size=1, seed=91, zero_frac=0.1, gaps=True)
+    assert wl.payload_bytes_total > 96 << 20
+    ref, rounds, _, _ = oracle_flat(wl, 3)
+    for flags in (0, B.FLAG_CLASSIC_ROTATE):
+        got, plan = gpu_run(wl, 3, flags=flags, misalign=misalign)
+        assert np.array_equal(got, ref)
+    check_rounds(plan, rounds)
+    got, _ = gpu_run(wl, 12, misalign=misalign)
+    assert np.array_equal(got, ref)
+    got, _ = gpu_run(wl, 2, direct=True, misalign=misalign)
+    assert np.array_equal(got, ref)
+    wl8 = W.make_random(12, 260_000, elem_size=8, seed=92)            # skew of 0 or 8 bytes only
+    got, _ = gpu_run(wl8, 12, misalign=misalign)
+    assert np.array_equal(got, oracle_brute(wl8))
+
+
 def test_bulk_copy_route():
     """TUNA_FLAG_BULK_COPY: chunks inside large aligned blocks go through
     cp.async.bulk; same bytes, and no kernel gives up a wait."""
