@@ -369,7 +369,35 @@ __device__ __forceinline__ void move_body(const TunaListArgs &l, const TunaMoveA
     const int vlo = first_rel > 0 ? (int)(first_rel >> 4) : 0;
     const int vhi = (next_rel >> 4) < nv ? (int)(next_rel >> 4) : nv;
     __syncthreads();
-    if (vhi <= vlo) continue;
+    if (vhi <= vlo) {
+      // Nothing of this batch lies in the chunk.  If its blocks are all empty, the run
+      // of empty blocks may go on for millions of descriptors (ranks that send or
+      // receive nothing): stream positions do not move along it, so its end is found
+      // by doubling steps and a bisection instead of batch by batch.  Every thread
+      // reads the same entries and takes the same steps.
+      if (next_rel == first_rel && b + cnt <= e_hi) {
+        const int64_t p0 = first_rel + cA;
+        int64_t lo = b + cnt, hi = lo, step = kBatch;  // pos[lo] == p0
+        bool more = true;
+        for (;;) {
+          hi = lo + step < e_hi + 1 ? lo + step : e_hi + 1;  // (pos has an entry behind the last descriptor)
+          if (l.pos[hi] > p0) break;
+          if (hi == e_hi + 1) {
+            more = false;  // empty to the end of this chunk's descriptors
+            break;
+          }
+          lo = hi;
+          step <<= 1;
+        }
+        if (!more) break;
+        while (hi - lo > 1) {  // pos[lo] == p0 < pos[hi]
+          const int64_t mid = lo + ((hi - lo) >> 1);
+          if (l.pos[mid] > p0) hi = mid; else lo = mid;
+        }
+        b = lo - kBatch;  // descriptor lo is the first one with bytes: the next batch starts there
+      }
+      continue;
+    }
     if (!waited) {  // everything above read only the plan's tables; the data may still be in the making
       grid_dependency_wait();
       waited = true;
@@ -547,9 +575,9 @@ __device__ __forceinline__ void launch_body(const TunaMoveArgs &a) {
 // of its set-up (chunk table, descriptors, then data), so eight resident CTAs per
 // SM with two vectors in flight each do better (measured: 1.15-1.4x on 180-byte
 // blocks, 1.02x on 16 KiB blocks, 0.98x on 128 KiB blocks).
-__global__ void __launch_bounds__(kThreads) tuna_round_kernel(const TunaMoveArgs a) { launch_body<4, true>(a); }
-__global__ void __launch_bounds__(kThreads) tuna_rotate_kernel(const TunaMoveArgs a) { launch_body<4, true>(a); }
-__global__ void __launch_bounds__(kThreads) tuna_direct_kernel(const TunaMoveArgs a) { launch_body<4, true>(a); }
+__global__ void __launch_bounds__(kThreads, 4) tuna_round_kernel(const TunaMoveArgs a) { launch_body<4, true>(a); }
+__global__ void __launch_bounds__(kThreads, 4) tuna_rotate_kernel(const TunaMoveArgs a) { launch_body<4, true>(a); }
+__global__ void __launch_bounds__(kThreads, 4) tuna_direct_kernel(const TunaMoveArgs a) { launch_body<4, true>(a); }
 __global__ void __launch_bounds__(kThreads, 8) tuna_round_small_kernel(const TunaMoveArgs a) { launch_body<2, false>(a); }
 __global__ void __launch_bounds__(kThreads, 8) tuna_rotate_small_kernel(const TunaMoveArgs a) { launch_body<2, false>(a); }
 __global__ void __launch_bounds__(kThreads, 8) tuna_direct_small_kernel(const TunaMoveArgs a) { launch_body<2, false>(a); }

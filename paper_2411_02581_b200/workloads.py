@@ -354,6 +354,16 @@ def make_random(P: int, max_count: int, elem_size: int = 1, seed: int = 11,
     return _finish("random", P, elem_size, seed, c.reshape(P, P), gaps=gaps)
 
 
+def make_silent_ranks(P: int, max_count: int, silent_from: int, silent_to: int, deaf_from: int,
+                      deaf_to: int, elem_size: int = 1, seed: int = 13, gaps: bool = False) -> Workload:
+    """Random counts in which the ranks [silent_from, silent_to) send nothing and the ranks
+    [deaf_from, deaf_to) receive nothing: long runs of empty blocks in every list."""
+    c = uniform_int(seed, S_COUNTS, P * P, 0, max_count).numpy().reshape(P, P).copy()
+    c[silent_from:silent_to, :] = 0
+    c[:, deaf_from:deaf_to] = 0
+    return _finish("silent_ranks", P, elem_size, seed, c, gaps=gaps)
+
+
 # ---- the paper's other count patterns (Sec. VI-A and VI-C), all closed-form or seeded ----
 
 def make_normal(seed: int | None = None, P: int = 4096, mean: float = 1000.0, sd: float = 240.0,

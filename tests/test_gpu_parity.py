@@ -137,6 +137,18 @@ def test_large_skewed_blocks(misalign):
     assert np.array_equal(got, oracle_brute(wl8))
 
 
+@pytest.mark.parametrize("kw", [dict(radix=2), dict(radix=8), dict(radix=600), dict(radix=2, flags=B.FLAG_CLASSIC_ROTATE),
+                                dict(radix=5, l=20, g=30, rg=6), dict(radix=600, direct=True)])
+def test_ranks_that_send_or_receive_nothing(kw):
+    """Runs of tens of thousands of empty blocks inside a chunk's descriptors (the mover
+    finds their end by doubling steps and bisection, not batch by batch)."""
+    wl = W.make_silent_ranks(600, 90, 150, 520, 80, 410, gaps=True)
+    assert (wl.sendcounts == 0).mean() > 0.8
+    kw = dict(kw)
+    got, _ = gpu_run(wl, kw.pop("radix"), **kw)
+    assert np.array_equal(got, oracle_brute(wl))
+
+
 def test_bulk_copy_route():
     """TUNA_FLAG_BULK_COPY: chunks inside large aligned blocks go through
     cp.async.bulk; same bytes, and no kernel gives up a wait."""
