@@ -522,6 +522,36 @@ def test_degenerate_inputs():
             assert np.array_equal(got, oracle_brute(wl))
 
 
+def test_degenerate_inputs_from_device_counts():
+    """The same corner cases through the device-count update (captured plan kernels):
+    one rank, two ranks, nothing to move, a single block, then real counts again."""
+    for P in (1, 2, 7):
+        for radix in (2, max(2, P)):
+            plan = B.plan_for(W.make_uniform(P, 3), radix, explicit_layout=False)
+            zeros = torch.zeros((P, P), dtype=torch.int64, device="cuda")
+            for _ in range(2):                                   # the second update replays the graph
+                plan.update_counts_device(zeros)
+                assert plan.extents() == (0, 0, 0)
+                empty = torch.empty(0, dtype=torch.uint8, device="cuda")
+                plan.alltoallv(empty, empty)
+                assert plan.last_launches() == 0
+            one = np.zeros((P, P), dtype=np.int64)
+            one[P - 1, 0] = 54321
+            for counts in (one, W.make_random(P, 70, seed=3 + P).sendcounts):
+                wl = W._finish("dev", P, 1, 5, counts)
+                plan.update_counts_device(torch.from_numpy(wl.sendcounts).cuda())
+                plan.alloc_workspace()
+                send, recv = wl.make_send("cuda"), wl.make_recv("cuda", fill=CANARY)
+                plan.alltoallv(send, recv)
+                torch.cuda.synchronize()
+                assert np.array_equal(recv.cpu().numpy(), oracle_brute(wl))
+                recv.fill_(CANARY)
+                plan.direct_alltoallv(send, recv)
+                torch.cuda.synchronize()
+                assert np.array_equal(recv.cpu().numpy(), oracle_brute(wl))
+            plan.destroy()
+
+
 # ---------------------------------------------------------------- the five workloads
 
 def test_c1_full():
