@@ -293,13 +293,20 @@ __device__ __forceinline__ void skewed_run(const char *src, char *dst, int m) {
 
 // ------------------------------------------------------------------ the mover
 
+struct __align__(16) BlockPtrs {
+  const char *sadj;
+  char *dadj;
+};
+
 template <bool DELIVER, int kUnroll, bool kBulk>  // kUnroll: vectors a thread has in flight
 __device__ __forceinline__ void move_body(const TunaListArgs &l, const TunaMoveArgs &a, int64_t c) {
   __shared__ int s_vs[kBatch];             // first vector of the block, relative to the chunk
-  __shared__ int s_org[kBatch];            // DELIVER: chunk-relative position of the block's first byte
-  __shared__ int s_end[kBatch];            // DELIVER: ... and one past its last byte (clamped when far)
-  __shared__ const char *s_sadj[kBatch];   // source address of chunk vector v is s_sadj + 16 v
-  __shared__ char *s_dadj[kBatch];         // DELIVER: destination address likewise (16-byte aligned)
+  // per block of the batch: (DELIVER) the chunk-relative position of its first byte and
+  // one past its last byte (clamped when far); the source address of chunk vector v
+  // minus 16 v and (DELIVER) the destination address likewise (16-byte aligned).
+  // Paired up so that a vector's look-up is one 8-byte and one 16-byte shared load.
+  __shared__ int2 s_oe[DELIVER ? kBatch : 1];
+  __shared__ BlockPtrs s_sd[kBatch];
   __shared__ unsigned char s_careful[kBatch];
   __shared__ __align__(16) unsigned char s_edge[DELIVER ? kBatch * 32 : 16];  // two parking slots per block: its partial first and last vector
   extern __shared__ __align__(16) unsigned char s_who[];  // owner of every vector of the chunk (chunk / 16 bytes)
@@ -350,17 +357,21 @@ __device__ __forceinline__ void move_body(const TunaListArgs &l, const TunaMoveA
         if (end > ((int64_t)kClampVec << 4)) end = (int64_t)kClampVec << 4;
         my_org = (int)(vs << 4) + ad;
         my_end = (int)end;
-        s_org[tid] = my_org;
-        s_end[tid] = my_end;
-        s_sadj[tid] = sp - org;
-        s_dadj[tid] = dp - org;
+        s_oe[tid] = make_int2(my_org, my_end);
+        BlockPtrs ptrs;
+        ptrs.sadj = sp - org;
+        ptrs.dadj = dp - org;
+        s_sd[tid] = ptrs;
         s_careful[tid] = (L > 0 && (sp - 31 < sbase || sp + L + 31 > sbase + extent_of(a, sb))) ? 1 : 0;
         my_edges = L > 0 && (ad != 0 || (L & 15) != 0);
         if (L > 0 && tid > 0 && vs < nv) mark_at = (int)vs;
       } else {
         const int64_t pn = l.pos[e + 1];
         if (pn > p && tid > 0 && vs < nv) mark_at = (int)vs;
-        s_sadj[tid] = sp - rel;
+        BlockPtrs ptrs;
+        ptrs.sadj = sp - rel;
+        ptrs.dadj = nullptr;
+        s_sd[tid] = ptrs;
         s_careful[tid] = (sp - 15 < sbase || sp + (pn - p) + 16 > sbase + extent_of(a, sb)) ? 1 : 0;
       }
     }
@@ -407,10 +418,10 @@ __device__ __forceinline__ void move_body(const TunaListArgs &l, const TunaMoveA
       // One block covers the whole range (a chunk inside a large block).  If both
       // ends are 16-byte aligned and no vector of the range is partial, this is a
       // plain strided copy: no table look-ups in the loop.
-      const char *src = s_sadj[0] + ((int64_t)vlo << 4);
-      char *dst = (DELIVER ? s_dadj[0] : keep_out) + ((int64_t)vlo << 4);
+      const char *src = s_sd[0].sadj + ((int64_t)vlo << 4);
+      char *dst = (DELIVER ? s_sd[0].dadj : keep_out) + ((int64_t)vlo << 4);
       bool plain = (reinterpret_cast<uintptr_t>(src) & 15) == 0 && s_careful[0] == 0;
-      if (DELIVER) plain = plain && s_org[0] <= (vlo << 4) && s_end[0] >= (vhi << 4);
+      if (DELIVER) plain = plain && s_oe[0].x <= (vlo << 4) && s_oe[0].y >= (vhi << 4);
       if (kBulk && a.bulk_off > 0 && plain && ((vhi - vlo) << 4) >= kBulkMin && ((vhi - vlo) << 4) <= kBulkBytes) {
         if (tid == 0) {
           const unsigned bytes = (unsigned)(vhi - vlo) << 4;
@@ -465,7 +476,7 @@ __device__ __forceinline__ void move_body(const TunaListArgs &l, const TunaMoveA
       // (Only in the build with registers to spare; lists of large blocks run it.)
       if constexpr (kUnroll >= 4) {
         bool whole = s_careful[0] == 0 && (reinterpret_cast<uintptr_t>(src) & 15) != 0;
-        if (DELIVER) whole = whole && s_org[0] <= (vlo << 4) && s_end[0] >= (vhi << 4);
+        if (DELIVER) whole = whole && s_oe[0].x <= (vlo << 4) && s_oe[0].y >= (vhi << 4);
         if (whole) {
           skewed_run<kUnroll>(src, dst, vhi - vlo);
           continue;
@@ -493,22 +504,24 @@ __device__ __forceinline__ void move_body(const TunaListArgs &l, const TunaMoveA
         if (on) {
           if (!single) t = s_who[vv];
           const int64_t vb = (int64_t)vv << 4;
+          const BlockPtrs ptrs = s_sd[t];
           if (DELIVER) {
             // A vector that lies wholly inside the block goes straight to its place.
             // The block's partial first and last vector are loaded here too, beside
             // their neighbours (the same cache lines), and parked in the block's two
             // slots of shared memory; the block's own thread stores their bytes later.
-            const int org = s_org[t], end = s_end[t];
+            const int2 oe = s_oe[t];
+            const int org = oe.x, end = oe.y;
             b0 = org - (int)vb;
             b1 = end - (int)vb;
             const bool full = b0 <= 0 && b1 >= 16;
             on = b0 < 16 && b1 > 0;
-            out[k] = full ? s_dadj[t] + vb
-                          : reinterpret_cast<char *>(s_edge) + t * 32 + (vv == (org >> 4) ? 0 : 16);
+            out[k] = full ? ptrs.dadj + vb
+                          : reinterpret_cast<char *>(s_edge) + t * 32 + (b0 >= 0 ? 0 : 16);  // (b0 >= 0: the vector that holds the block's first byte)
           } else {
             out[k] = keep_out + vb;
           }
-          sa = s_sadj[t] + vb;
+          sa = ptrs.sadj + vb;
           careful = s_careful[t] != 0;
           if (!on) out[k] = nullptr;
         }
@@ -540,10 +553,10 @@ __device__ __forceinline__ void move_body(const TunaListArgs &l, const TunaMoveA
         if (vh >= vlo && vh < vhi && ((my_org & 15) != 0 || my_end < (vh << 4) + 16)) {
           const int b0 = my_org - (vh << 4);
           const int b1 = my_end - (vh << 4) < 16 ? my_end - (vh << 4) : 16;
-          store_pieces(s_dadj[tid] + ((int64_t)vh << 4), s_edge + tid * 32, b0, b1);
+          store_pieces(s_sd[tid].dadj + ((int64_t)vh << 4), s_edge + tid * 32, b0, b1);
         }
         if (vt > vh && vt >= vlo && vt < vhi && (my_end & 15) != 0)
-          store_pieces(s_dadj[tid] + ((int64_t)vt << 4), s_edge + tid * 32 + 16, 0, my_end - (vt << 4));
+          store_pieces(s_sd[tid].dadj + ((int64_t)vt << 4), s_edge + tid * 32 + 16, 0, my_end - (vt << 4));
       }
     }
   }
