@@ -39,7 +39,7 @@ UNIT = "GB/s"
 # reported as null.  Captures: profiles/round_kernel_c4_reduced.md (c4, reduced to
 # 2 GiB) and profiles/round_small_kernel_c5.md (c5 at full size).
 NCU_TRAFFIC_PER_PAYLOAD_BYTE: dict[str, dict[str, float]] = {
-    "966e01440768d4d9ef938d28dae3bd74901c64af47b6332821f699f84d6166e1": {"c4": 1.990, "c5": 2.177},
+    "40d1ef79ac5a7db5d7f95e0971c78d65d8717af48a8ce3359f2843065c9199a2": {"c4": 1.995, "c5": 2.151},
 }
 
 
