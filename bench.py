@@ -37,9 +37,10 @@ UNIT = "GB/s"
 # proportion to the bytes moved, so the full-size figure is this ratio times the
 # launch's bytes.  A changed source makes the figures stale: the traffic is then
 # reported as null.  Captures: profiles/round_kernel_c4_reduced.md (c4, reduced to
-# 2 GiB) and profiles/round_small_kernel_c5.md (c5 at full size).
+# 2 GiB), profiles/round_small_kernel_c5.md (c5 at full size) and
+# profiles/round_small_kernel_c3.md (c3 at full size, both launches of an exchange).
 NCU_TRAFFIC_PER_PAYLOAD_BYTE: dict[str, dict[str, float]] = {
-    "40d1ef79ac5a7db5d7f95e0971c78d65d8717af48a8ce3359f2843065c9199a2": {"c4": 1.995, "c5": 2.151},
+    "40d1ef79ac5a7db5d7f95e0971c78d65d8717af48a8ce3359f2843065c9199a2": {"c4": 1.995, "c5": 2.151, "c3": 1.543},
 }
 
 
