@@ -75,7 +75,7 @@ __global__ void tuna_init_tables_kernel(TunaTopo t, const int64_t *__restrict__ 
   if (idx >= PP) return;
   const int p = (int)((unsigned)idx / (unsigned)t.P), sigma = (int)((unsigned)idx % (unsigned)t.P);  // (P * P < 2^31)
   const int n = p / t.Q, q = p % t.Q, io = sigma / t.Q, jo = sigma % t.Q;
-  const int dest = ((n + io) % t.N) * t.Q + (q + jo) % t.Q;
+  const int dest = (n + io - (n + io >= t.N ? t.N : 0)) * t.Q + (q + jo - (q + jo >= t.Q ? t.Q : 0));
   const int64_t bytes = counts[(int64_t)p * t.P + dest] * t.elem;
   const int64_t sloc = TUNA_LOC(TUNA_BUF_SEND, (sendbase[p] + sdispls[(int64_t)p * t.P + dest]) * t.elem);
   sz[idx] = bytes;
@@ -111,6 +111,8 @@ __global__ void tuna_meta_exchange_kernel(TunaTopo t, PhaseDev ph, const int64_t
   }
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   const int64_t PP = (int64_t)t.P * t.P;
+  unsigned long long add = 0;  // bytes this thread's slot moves in round add_to (0: none)
+  int add_to = 0;
   if (idx < PP) {
     const int p = (int)((unsigned)idx / (unsigned)t.P), sigma = (int)((unsigned)idx % (unsigned)t.P);  // (P * P < 2^31)
     const int n = p / t.Q, q = p % t.Q, io = sigma / t.Q, jo = sigma % t.Q;
@@ -119,9 +121,16 @@ __global__ void tuna_meta_exchange_kernel(TunaTopo t, PhaseDev ph, const int64_t
     if (dig == 0) {
       sz_next[idx] = sz_cur[idx];
     } else {
-      const int64_t dist = dig * ph.stride;
-      const int sender = ph.level == 0 ? n * t.Q + (int)(((q - dist) % t.Q + t.Q) % t.Q)
-                                       : (int)(((n - dist) % t.N + t.N) % t.N) * t.Q + q;
+      const int dist = dig * (int)ph.stride;  // below Q (level 0) or N (level 1): a wrap is one addition
+      int qs = q, ns = n;
+      if (ph.level == 0) {
+        qs -= dist;
+        if (qs < 0) qs += t.Q;
+      } else {
+        ns -= dist;
+        if (ns < 0) ns += t.N;
+      }
+      const int sender = ns * t.Q + qs;
       const int64_t c = row_position(t, ph, io, jo);
       const int64_t bytes = sz_cur[(int64_t)sender * t.P + sigma];
       const int64_t where = loc_cur[(int64_t)sender * t.P + sigma];
@@ -135,12 +144,24 @@ __global__ void tuna_meta_exchange_kernel(TunaTopo t, PhaseDev ph, const int64_t
         keep_len[e] = bytes;
         keep_src[e] = where;
       }
-      if (bytes > 0) {
-        if (use_smem)
-          atomicAdd(&s_hist[dig], (unsigned long long)bytes);
-        else
-          atomicAdd(&round_bytes[dig], (unsigned long long)bytes);
-      }
+      add = (unsigned long long)bytes;
+      add_to = dig;
+    }
+  }
+  // per-round byte counters.  The lanes of a warp often share the digit (slots of one
+  // group, or a run of `stride` slots): they then add once, not 32 times to one address.
+  {
+    const int first = __shfl_sync(0xffffffffu, add_to, 0);
+    if (__all_sync(0xffffffffu, add_to == first)) {
+#pragma unroll
+      for (int d = 16; d > 0; d >>= 1) add += __shfl_xor_sync(0xffffffffu, add, d);
+      if ((threadIdx.x & 31) != 0) add = 0;
+    }
+    if (add > 0 && add_to > 0) {
+      if (use_smem)
+        atomicAdd(&s_hist[add_to], add);
+      else
+        atomicAdd(&round_bytes[add_to], add);
     }
   }
   if (use_smem) {
@@ -150,50 +171,56 @@ __global__ void tuna_meta_exchange_kernel(TunaTopo t, PhaseDev ph, const int64_t
   }
 }
 
-// The same exchange for the one phase of a flat plan whose radix is at least P
-// (every slot o >= 1 moves once, from rank p - o to rank p): the general kernel
-// would read the two tables along anti-diagonals, one 32-byte sector per value,
-// and add one byte counter per slot to global memory.  Here a CTA reads a
-// 32 x 32 tile (sender, slot) along rows, and writes it out by receiver, where
-// each receiver's slots are again consecutive; a round's bytes are summed per tile
-// column first.  Grid: ceil(P/32) x ceil(P/32) CTAs of 32 x 8 threads.
+// The same exchange for a level-0 phase whose radix is at least Q (one phase moves
+// every local offset jo >= 1 once, from rank (n, q - jo) to rank (n, q); a flat plan
+// with radix >= P is the case N = 1).  The general kernel would read the two tables
+// along anti-diagonals, one 32-byte sector per value.  Here a CTA takes, for one
+// group n and one destination group offset io, a 32 x 32 tile (sender's local id,
+// jo): it reads the tile along rows and writes it out by receiver, where each
+// receiver's slots are again consecutive; a round's bytes are summed per tile
+// column first.  Grid: (tiles of a Q x Q square, N, N), CTAs of 32 x 8 threads.
 __global__ void tuna_meta_exchange_diag_kernel(TunaTopo t, PhaseDev ph, const int64_t *__restrict__ sz_cur,
                                                const int64_t *__restrict__ loc_cur, int64_t *sz_next,
                                                int64_t *keep_len, int64_t *keep_src, int64_t *del_len,
                                                int64_t *del_src, unsigned long long *round_bytes) {
   __shared__ int64_t s_sz[32][32], s_loc[32][32];
-  const int P = t.P, tx = threadIdx.x, ty = threadIdx.y;
-  const int g0 = blockIdx.x * 32, s0 = blockIdx.y * 32;  // first slot and first sender of the tile
+  const int P = t.P, Q = t.Q, tx = threadIdx.x, ty = threadIdx.y;
+  const int tiles = (Q + 31) / 32;
+  const int g0 = ((int)blockIdx.x % tiles) * 32, s0 = ((int)blockIdx.x / tiles) * 32;  // first jo, first sender id
+  const int io = blockIdx.y, n = blockIdx.z;
+  const int64_t row0 = (int64_t)n * Q;       // first rank of the group
+  const int col0 = io * Q;                   // first slot of the destination group offset
   for (int j = ty; j < 32; j += 8) {
     const int sd = s0 + j, g = g0 + tx;
-    const bool in = sd < P && g < P;
-    s_sz[j][tx] = in ? sz_cur[(int64_t)sd * P + g] : 0;
-    s_loc[j][tx] = in ? loc_cur[(int64_t)sd * P + g] : 0;
+    const bool in = sd < Q && g < Q;
+    s_sz[j][tx] = in ? sz_cur[(row0 + sd) * P + col0 + g] : 0;
+    s_loc[j][tx] = in ? loc_cur[(row0 + sd) * P + col0 + g] : 0;
   }
   __syncthreads();
-  if (ty == 0 && g0 + tx >= 1 && g0 + tx < P) {  // round z = slot: bytes sent by this tile's senders
+  if (ty == 0 && g0 + tx >= 1 && g0 + tx < Q) {  // round z = jo: bytes sent by this tile's senders
     int64_t sum = 0;
 #pragma unroll 8
     for (int j = 0; j < 32; j++) sum += s_sz[j][tx];
     if (sum > 0) atomicAdd(&round_bytes[g0 + tx], (unsigned long long)sum);
   }
-  for (int pr = ty; pr < 63; pr += 8) {  // receivers s0 + g0 + pr (mod P): a diagonal of the tile each
+  for (int pr = ty; pr < 63; pr += 8) {  // receivers s0 + g0 + pr (mod Q): a diagonal of the tile each
     const int sr = pr - tx;
     if (sr < 0 || sr >= 32) continue;
     const int sd = s0 + sr, g = g0 + tx;
-    if (sd >= P || g >= P) continue;
-    int p = sd + g;
-    if (p >= P) p -= P;
+    if (sd >= Q || g >= Q) continue;
+    int q = sd + g;
+    if (q >= Q) q -= Q;
+    const int64_t p = row0 + q;
     const int64_t bytes = s_sz[sr][tx], where = s_loc[sr][tx];
-    sz_next[(int64_t)p * P + g] = bytes;  // (slot 0 never moves: sender and receiver are the same rank)
+    sz_next[p * P + col0 + g] = bytes;  // (jo = 0 never moves in this phase: sender and receiver are the same rank)
     if (g == 0) continue;
-    const int64_t c = g - 1;  // position among the P - 1 blocks the rank receives, in slot order
+    const int64_t c = (int64_t)io * ph.moving + (g - 1);  // position among the blocks the rank receives, in slot order
     if (c < ph.finals) {
-      const int64_t e = (int64_t)p * ph.finals + c;
+      const int64_t e = p * ph.finals + c;
       del_len[e] = bytes;
       del_src[e] = where;
     } else {
-      const int64_t e = (int64_t)p * (ph.per_rank - ph.finals) + (c - ph.finals);
+      const int64_t e = p * (ph.per_rank - ph.finals) + (c - ph.finals);
       keep_len[e] = bytes;
       keep_src[e] = where;
     }
@@ -407,7 +434,7 @@ __global__ void tuna_place_kernel(TunaTopo t, PhaseDev ph, const int64_t *__rest
   const int64_t c = row_position(t, ph, io, jo);
   const unsigned sr = (unsigned)ph.stride * (unsigned)ph.radix;
   const bool fin = ph.level == 0 ? (io == 0 && (unsigned)jo < sr) : (unsigned)io < sr;
-  const int origin = ((n - io + t.N) % t.N) * t.Q + (q - jo + t.Q) % t.Q;
+  const int origin = (n - io + (n < io ? t.N : 0)) * t.Q + (q - jo + (q < jo ? t.Q : 0));
   const int64_t rloc =
       TUNA_LOC(TUNA_BUF_RECV, (recvbase[p] + rdispls[(int64_t)p * t.P + origin]) * t.elem);
   if (c < ph.finals) {  // DELIVER list (only in direct-to-R mode; these blocks have arrived)
@@ -1222,8 +1249,9 @@ int build_tables(tuna_plan *pl, const HostLayout *hl, const int64_t *sdispls, co
         continue;
       }
       PhaseDev pd{ph.level, ph.radix, ph.count, ph.stride, ph.moving, ph.per_rank, ph.finals};
-      if (ph.level == 0 && t.N == 1 && ph.stride == 1 && ph.radix >= P) {
-        tuna_meta_exchange_diag_kernel<<<dim3((P + 31) / 32, (P + 31) / 32), dim3(32, 8), 0, st>>>(
+      if (ph.level == 0 && ph.stride == 1 && ph.radix >= t.Q && t.N <= 65535) {
+        const unsigned tiles = (unsigned)((t.Q + 31) / 32);
+        tuna_meta_exchange_diag_kernel<<<dim3(tiles * tiles, t.N, t.N), dim3(32, 8), 0, st>>>(
             t, pd, pl->d_sz[cur], pl->d_loc[cur], pl->d_sz[cur ^ 1], k.len, k.src, d.len, d.src,
             pl->d_round_bytes + ph.stats_off);
       } else {
