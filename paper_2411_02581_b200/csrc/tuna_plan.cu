@@ -479,12 +479,12 @@ __global__ void tuna_chunk_index_kernel(const int64_t *__restrict__ pos, int64_t
 // buffer and write inside its destination.  The movers touch no other bytes than
 // these ranges (plus the documented aligned over-read inside the source buffer),
 // so a clean check bounds every access of the exchange.  Violations are counted.
-__global__ void tuna_check_list_kernel(const int64_t *__restrict__ len, const int64_t *__restrict__ pos,
-                                       const int64_t *__restrict__ src, const int64_t *__restrict__ dst,
-                                       int64_t n, const int64_t *__restrict__ extents,
-                                       const int64_t *__restrict__ work_extent, int64_t keep_base_index,
-                                       const int64_t *__restrict__ wbase, unsigned long long *violations,
-                                       unsigned long long *unaligned_bytes) {
+__device__ __forceinline__ void check_list_body(const int64_t *__restrict__ len, const int64_t *__restrict__ pos,
+                                                const int64_t *__restrict__ src, const int64_t *__restrict__ dst,
+                                                int64_t n, const int64_t *__restrict__ extents,
+                                                const int64_t *__restrict__ work_extent, int64_t keep_base_index,
+                                                const int64_t *__restrict__ wbase, unsigned long long *violations,
+                                                unsigned long long *unaligned_bytes) {
   bool bad = false;
   int64_t skewed = 0;  // bytes of blocks whose source and destination differ modulo 16
   const int64_t send_extent = extents[0], recv_extent = extents[1];
@@ -522,6 +522,32 @@ __global__ void tuna_check_list_kernel(const int64_t *__restrict__ len, const in
     for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(0xffffffffu, v, d);
     if (threadIdx.x == 0 && v > 0) atomicAdd(unaligned_bytes, (unsigned long long)v);
   }
+}
+
+__global__ void tuna_check_list_kernel(const int64_t *__restrict__ len, const int64_t *__restrict__ pos,
+                                       const int64_t *__restrict__ src, const int64_t *__restrict__ dst,
+                                       int64_t n, const int64_t *__restrict__ extents,
+                                       const int64_t *__restrict__ work_extent, int64_t keep_base_index,
+                                       const int64_t *__restrict__ wbase, unsigned long long *violations,
+                                       unsigned long long *unaligned_bytes) {
+  check_list_body(len, pos, src, dst, n, extents, work_extent, keep_base_index, wbase, violations, unaligned_bytes);
+}
+
+// All lists of a plan in one launch: blockIdx.y picks the list.
+struct TunaCheckItem {
+  const int64_t *len, *pos, *src, *dst;  // dst null: a KEEP list
+  int64_t n;
+  int64_t keep_base_index;  // KEEP lists: the phase, whose workspace offset is wbase[phase]
+  int64_t id;               // slot of the list's skewed-byte counter behind violations[0]
+};
+
+__global__ void tuna_check_lists_kernel(const TunaCheckItem *__restrict__ items, const int64_t *__restrict__ extents,
+                                        const int64_t *__restrict__ work_extent,
+                                        const int64_t *__restrict__ wbase, unsigned long long *violations) {
+  const TunaCheckItem it = items[blockIdx.y];
+  if ((int64_t)blockIdx.x * blockDim.x >= it.n) return;  // (whole CTA: short lists need few of them)
+  check_list_body(it.len, it.pos, it.src, it.dst, it.n, extents, work_extent, it.keep_base_index, wbase,
+                  violations, violations + 1 + it.id);
 }
 
 // out = in^T, in 32 x 32 tiles through shared memory so that both the reads and the
@@ -635,6 +661,9 @@ struct tuna_plan {
   size_t workspace_bytes = 0;
 
   int64_t launch_count = 0;  // kernels launched by this plan since creation
+  void *d_check_items = nullptr;    // the plan's lists as the self-check kernel takes them (fixed at creation)
+  int n_check_items = 0;
+  int64_t check_max_n = 0;
   cudaEvent_t in_flight = nullptr;  // end of the last exchange this plan enqueued (outside graph capture)
   bool in_flight_set = false;
   // The plan kernels of an update from device counts, captured once as a CUDA graph
@@ -1173,6 +1202,9 @@ int build_tables(tuna_plan *pl, const HostLayout *hl, const int64_t *sdispls, co
   // and reads nothing back, so it can run directly or be captured as a graph.
   auto enqueue_tables = [&](cudaStream_t st) -> int {
     int rc = TUNA_OK;
+    // list totals, workspace offsets, extents, per-round bytes and self-check counters
+    // all start from zero: they are slices of one block
+    TUNA_CUDA(pl, cudaMemsetAsync(pl->d_readback, 0, (size_t)pl->readback_words * 8, st));
     if (hl) {
       pl->payload = hl->payload * t.elem;
       pl->send_extent = hl->send_extent * t.elem;
@@ -1184,8 +1216,6 @@ int build_tables(tuna_plan *pl, const HostLayout *hl, const int64_t *sdispls, co
       const int64_t ext[4] = {pl->send_extent, pl->recv_extent, hl->payload, 0};
       TUNA_CUDA(pl, cudaMemcpyAsync(pl->d_extents, ext, sizeof(ext), cudaMemcpyHostToDevice, st));
       // (pageable sources: the runtime stages these copies before it returns)
-    } else {
-      TUNA_CUDA(pl, cudaMemsetAsync(pl->d_extents, 0, 4 * 8, st));
     }
     pl->counts_uploaded = false;
     if (sdispls) {
@@ -1217,8 +1247,6 @@ int build_tables(tuna_plan *pl, const HostLayout *hl, const int64_t *sdispls, co
       }
     }
 
-    TUNA_CUDA(pl, cudaMemsetAsync(pl->d_round_bytes, 0, (size_t)std::max<int64_t>(pl->stats_n, 1) * 8, st));
-    TUNA_CUDA(pl, cudaMemsetAsync(pl->d_wbase, 0, (size_t)(nph + 1) * 8, st));
     if (pl->classic) {
       TUNA_CUDA(pl, cudaMemsetAsync(pl->rot.len, 0, (size_t)PP * 8, st));
       TUNA_CUDA(pl, cudaMemsetAsync(pl->rot.src, 0, (size_t)PP * 8, st));
@@ -1282,26 +1310,13 @@ int build_tables(tuna_plan *pl, const HostLayout *hl, const int64_t *sdispls, co
     // self-check: every descriptor of every list stays inside its buffers
     // (the same pass sums, per list, the bytes of the blocks whose source and
     // destination differ modulo 16: they pick the kernel build)
-    TUNA_CUDA(pl, cudaMemsetAsync(pl->d_violations, 0, sizeof(unsigned long long) * (1 + nlists), st));
-    auto check = [&](const TunaList &l, int keep_phase, int id) -> int {
-      if (l.n <= 0) return TUNA_OK;
-      tuna_check_list_kernel<<<(unsigned)std::min<int64_t>((l.n + th - 1) / th, 148 * 8), th, 0, st>>>(
-          l.len, l.pos, l.src, l.kind == TUNA_LIST_DELIVER ? l.dst : nullptr, l.n, pl->d_extents,
-          pl->d_wbase + nph, keep_phase, pl->d_wbase, pl->d_violations,
-          pl->d_violations + 1 + id);
+    if (pl->n_check_items > 0) {
+      const unsigned gx = (unsigned)std::min<int64_t>((pl->check_max_n + th - 1) / th, 148 * 8);
+      tuna_check_lists_kernel<<<dim3(gx, pl->n_check_items), th, 0, st>>>(
+          static_cast<const TunaCheckItem *>(pl->d_check_items), pl->d_extents, pl->d_wbase + nph, pl->d_wbase,
+          pl->d_violations);
       TUNA_LAUNCHED(pl);
-      return TUNA_OK;
-    };
-    for (int f = 0; f < nph; f++) {
-      rc = check(pl->keep[f], f, f);
-      if (rc) return rc;
-      rc = check(pl->deliver[f], 0, nph + f);
-      if (rc) return rc;
     }
-    rc = check(pl->rot, 0, 2 * nph);
-    if (rc) return rc;
-    if (!pl->dir_shared) rc = check(pl->dir, 0, 2 * nph + 1);
-    if (rc) return rc;
 
     return rc;
   };
@@ -1655,6 +1670,7 @@ int tuna_plan_destroy(tuna_plan_t *pl) {
   cudaFree(pl->d_seg_raw);
   cudaFree(pl->d_seg_base);
   cudaFree(pl->d_tmp);
+  cudaFree(pl->d_check_items);
   cudaFree(pl->d_readback);  // (d_scal, d_wbase, d_extents, d_round_bytes, d_violations are slices of it)
   if (pl->h_readback) cudaFreeHost(pl->h_readback);
   cudaFree(pl->d_error);
@@ -1791,6 +1807,26 @@ static int plan_create(tuna_plan_t **out, int P, int radix, int radix_global, in
   if (!pl->dir_shared) {
     rc = alloc_list(pl, pl->dir, TUNA_LIST_DELIVER, PP);
     if (rc) return nomem(rc);
+  }
+  {  // the self-check's view of the lists: their arrays never move
+    std::vector<TunaCheckItem> items;
+    auto add = [&](const TunaList &l, int keep_phase, int id) {
+      if (l.n <= 0) return;
+      items.push_back(TunaCheckItem{l.len, l.pos, l.src, l.kind == TUNA_LIST_DELIVER ? l.dst : nullptr, l.n,
+                                    keep_phase, id});
+      pl->check_max_n = std::max(pl->check_max_n, l.n);
+    };
+    for (int f = 0; f < nph; f++) {
+      add(pl->keep[f], f, f);
+      add(pl->deliver[f], 0, nph + f);
+    }
+    add(pl->rot, 0, 2 * nph);
+    if (!pl->dir_shared) add(pl->dir, 0, 2 * nph + 1);
+    pl->n_check_items = (int)items.size();
+    if (!items.empty()) {
+      TUNA_TRY(cudaMalloc(&pl->d_check_items, items.size() * sizeof(TunaCheckItem)));
+      TUNA_TRY(cudaMemcpy(pl->d_check_items, items.data(), items.size() * sizeof(TunaCheckItem), cudaMemcpyHostToDevice));
+    }
   }
 #undef TUNA_TRY
   rc = build_tables(pl, &hl, sdispls, rdispls, st);
