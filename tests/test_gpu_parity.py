@@ -366,6 +366,16 @@ def test_update_counts_from_device_memory(kw):
     (plan.direct_alltoallv if direct else plan.alltoallv)(send, recv)
     torch.cuda.synchronize()
     assert np.array_equal(recv.cpu().numpy(), oracle_brute(wl))
+    # device counts once more: the host update moved the plan's count buffer, so the
+    # captured plan kernels are captured afresh
+    wl = W.make_random(12, 333, seed=66, zero_frac=0.2)
+    for _ in range(2):
+        plan.update_counts_device(torch.from_numpy(wl.sendcounts).cuda())
+        plan.alloc_workspace()
+        send, recv = wl.make_send("cuda"), wl.make_recv("cuda", fill=CANARY)
+        (plan.direct_alltoallv if direct else plan.alltoallv)(send, recv)
+        torch.cuda.synchronize()
+        assert np.array_equal(recv.cpu().numpy(), oracle_brute(wl))
 
 
 def test_update_waits_for_the_plans_own_exchange_in_flight():
