@@ -134,8 +134,11 @@ int tuna_plan_create_staggered(tuna_plan_t **out, int P, int radix, int block_co
 /*
  * tuna_plan_update_counts - same plan shape, new counts (e.g. routing that changes
  * every step): re-runs the metadata exchange and the prefix sums on the device.
- * Arguments as in tuna_plan_create.  Synchronises `stream` once.  The required
- * workspace size may change; query it again.  The tables are rewritten in place,
+ * Arguments as in tuna_plan_create.  Synchronises `stream` once (for the list
+ * totals); when the call returns, the sizes the plan reports are final, while its
+ * last kernels (the work partition) may still be running on `stream`: exchange
+ * calls order themselves behind them, on whatever stream they are given.  The
+ * required workspace size may change; query it again.  The tables are rewritten in place,
  * so the update first waits (on the host) for the exchanges this plan has
  * enqueued, whatever their stream; replays of an exchange captured into a CUDA
  * graph are not tracked and must have finished before the call.  To overlap the

@@ -666,6 +666,11 @@ struct tuna_plan {
   int64_t check_max_n = 0;
   cudaEvent_t in_flight = nullptr;  // end of the last exchange this plan enqueued (outside graph capture)
   bool in_flight_set = false;
+  // An update's last kernels (the chunk tables) are not waited for on the host: an
+  // event marks their end, and an exchange on another stream waits for it there.
+  cudaEvent_t tables_ready = nullptr;
+  bool tables_ready_set = false;
+  cudaStream_t ready_waited = nullptr;  // the stream that is known to be ordered behind the event
   // The plan kernels of an update from device counts, captured once as a CUDA graph
   // (their arguments do not change from update to update) and replayed afterwards.
   cudaStream_t capture_stream = nullptr;
@@ -727,6 +732,36 @@ int wait_in_flight(tuna_plan *pl) {
     TUNA_CUDA(pl, cudaEventSynchronize(pl->in_flight));
     pl->in_flight_set = false;
   }
+  if (pl->tables_ready_set) {  // (the previous update's chunk tables, possibly on another stream)
+    TUNA_CUDA(pl, cudaEventSynchronize(pl->tables_ready));
+    pl->tables_ready_set = false;
+  }
+  return TUNA_OK;
+}
+
+// End of an update: the tables are complete once everything enqueued on `st` so far has run.
+int mark_tables_ready(tuna_plan *pl, cudaStream_t st) {
+  if (!pl->tables_ready) TUNA_CUDA(pl, cudaEventCreateWithFlags(&pl->tables_ready, cudaEventDisableTiming));
+  TUNA_CUDA(pl, cudaEventRecord(pl->tables_ready, st));
+  pl->tables_ready_set = true;
+  pl->ready_waited = st;  // work enqueued on the same stream is behind it already
+  return TUNA_OK;
+}
+
+// Start of an exchange on `st`: order it behind the last update's kernels.
+int await_tables(tuna_plan *pl, cudaStream_t st) {
+  if (!pl->tables_ready_set || st == pl->ready_waited) return TUNA_OK;
+  cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+  if (cudaStreamIsCapturing(st, &cap) != cudaSuccess) {
+    (void)cudaGetLastError();
+    cap = cudaStreamCaptureStatusNone;
+  }
+  if (cap != cudaStreamCaptureStatusNone) {  // a capture cannot wait for an event from outside: wait here
+    TUNA_CUDA(pl, cudaEventSynchronize(pl->tables_ready));
+    return TUNA_OK;
+  }
+  TUNA_CUDA(pl, cudaStreamWaitEvent(st, pl->tables_ready, 0));
+  pl->ready_waited = st;
   return TUNA_OK;
 }
 
@@ -1384,7 +1419,8 @@ int build_tables(tuna_plan *pl, const HostLayout *hl, const int64_t *sdispls, co
   if (rc) return rc;
   if (!pl->dir_shared) rc = build_chunks(pl, pl->dir, st);
   if (rc) return rc;
-  TUNA_CUDA(pl, cudaStreamSynchronize(st));
+  rc = mark_tables_ready(pl, st);  // (no second wait on the host: exchanges order themselves behind this)
+  if (rc) return rc;
   pl->tables_valid = true;
   return TUNA_OK;
 }
@@ -1542,6 +1578,10 @@ TunaMoveArgs move_args(const tuna_plan *pl, const void *send, void *recv, char *
 // the first launch, the self blocks (they depend on nothing).  In classic mode
 // the rotation list needs every phase finished and gets a launch of its own.
 int run_tuna(tuna_plan *pl, const void *send, void *recv, cudaStream_t st) {
+  {
+    const int arc = await_tables(pl, st);
+    if (arc) return arc;
+  }
   if (pl->workspace_need > 0 &&
       (!pl->workspace || pl->workspace_bytes < (size_t)pl->workspace_need))
     return TUNA_ERR_WORKSPACE;
@@ -1584,6 +1624,10 @@ int run_tuna(tuna_plan *pl, const void *send, void *recv, cudaStream_t st) {
 }
 
 int run_direct(tuna_plan *pl, const void *send, void *recv, cudaStream_t st) {
+  {
+    const int arc = await_tables(pl, st);
+    if (arc) return arc;
+  }
   int launches = 0;
   if (pl->dir_shared) {  // the single phase's DELIVER list and the self blocks: every block, once
     const TunaList &d = pl->deliver[0];
@@ -1641,6 +1685,10 @@ int tuna_plan_destroy(tuna_plan_t *pl) {
   if (pl->in_flight) {
     if (pl->in_flight_set) (void)cudaEventSynchronize(pl->in_flight);  // the tables are freed below
     cudaEventDestroy(pl->in_flight);
+  }
+  if (pl->tables_ready) {
+    if (pl->tables_ready_set) (void)cudaEventSynchronize(pl->tables_ready);
+    cudaEventDestroy(pl->tables_ready);
   }
   if (pl->tables_graph) cudaGraphExecDestroy(pl->tables_graph);
   if (pl->capture_stream) cudaStreamDestroy(pl->capture_stream);
@@ -2065,9 +2113,10 @@ int tuna_plan_set_row_maps(tuna_plan_t *pl, const int64_t *gather_rows, const in
   TUNA_CUDA(pl, cudaStreamSynchronize(st));
   if (checked[0] != 0) return TUNA_ERR_RANGE;
   l.unaligned_bytes = (int64_t)checked[1];
-  const int rc = build_chunks(pl, l, st);
+  int rc = build_chunks(pl, l, st);
   if (rc) return rc;
-  TUNA_CUDA(pl, cudaStreamSynchronize(st));
+  rc = mark_tables_ready(pl, st);
+  if (rc) return rc;
   pl->rows_valid = true;
   return TUNA_OK;
 }
@@ -2081,6 +2130,10 @@ int tuna_rows_alltoallv(tuna_plan_t *pl, const void *rows_in, void *rows_out, vo
     return TUNA_ERR_OVERLAP;
   int launches = 0;
   cudaStream_t st = (cudaStream_t)stream;
+  {
+    const int arc = await_tables(pl, st);
+    if (arc) return arc;
+  }
   if (l.nchunks > 0) {
     Timed tm(pl, TUNA_TIMER_DIRECT, l.bytes, st);
     TunaMoveArgs a = move_args(pl, rows_in, rows_out, nullptr);
