@@ -303,9 +303,9 @@ __global__ void tuna_rows_list_kernel(int P, int64_t row_bytes, const int64_t *_
 // adds 16 spare bytes behind every non-zero value.  seg_total[s] receives the
 // segment's sum, seg_raw[s] (optional) the sum of the unmodified values.
 template <int MODE>
-__global__ void tuna_segscan_kernel(const int64_t *__restrict__ val, int64_t *out,
-                                    int64_t *seg_total, int64_t *seg_raw, int64_t seglen,
-                                    int64_t nseg) {
+__device__ __forceinline__ void segscan_body(const int64_t *__restrict__ val, int64_t *out,
+                                             int64_t *seg_total, int64_t *seg_raw, int64_t seglen,
+                                             int64_t nseg) {
   const int64_t w = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int lane = threadIdx.x & 31;
   if (w >= nseg) return;
@@ -349,14 +349,41 @@ __global__ void tuna_segscan_kernel(const int64_t *__restrict__ val, int64_t *ou
   }
 }
 
+template <int MODE>
+__global__ void tuna_segscan_kernel(const int64_t *__restrict__ val, int64_t *out,
+                                    int64_t *seg_total, int64_t *seg_raw, int64_t seglen,
+                                    int64_t nseg) {
+  segscan_body<MODE>(val, out, seg_total, seg_raw, seglen, nseg);
+}
+
+// One list's scan as the kernels below take it.
+struct TunaScanArgs {
+  const int64_t *val;
+  int64_t *out, *seg_total, *seg_raw, *seg_base;
+  int64_t seglen, nseg;
+  int64_t *scal, *wbase;
+  int uses_work;
+  int64_t *pos_end;
+};
+
+// The two lists of a digit phase in one launch: blockIdx.y = 0 scans the KEEP list
+// (lengths rounded up to 16), blockIdx.y = 1 the DELIVER list (16 spare bytes more).
+__global__ void tuna_segscan_pair_kernel(TunaScanArgs keep, TunaScanArgs del) {
+  if (blockIdx.y == 0) {
+    if (keep.seglen > 0) segscan_body<1>(keep.val, keep.out, keep.seg_total, keep.seg_raw, keep.seglen, keep.nseg);
+  } else {
+    if (del.seglen > 0) segscan_body<2>(del.val, del.out, del.seg_total, del.seg_raw, del.seglen, del.nseg);
+  }
+}
+
 // Exclusive scan of the nseg segment totals (one CTA), giving every segment's
 // base in the list's stream.  scal[0] = stream bytes, scal[1] = bytes moved.
 // If wbase is given, wbase[1] = wbase[0] + (stream bytes rounded up to 256),
 // or wbase[0] when the phase keeps nothing in the workspace.
-__global__ void tuna_segbase_kernel(const int64_t *__restrict__ seg_total,
-                                    const int64_t *__restrict__ seg_raw, int64_t *seg_base,
-                                    int64_t nseg, int64_t *scal, int64_t *wbase, int uses_work,
-                                    int64_t *pos_end) {
+__device__ __forceinline__ void segbase_body(const int64_t *__restrict__ seg_total,
+                                             const int64_t *__restrict__ seg_raw, int64_t *seg_base,
+                                             int64_t nseg, int64_t *scal, int64_t *wbase, int uses_work,
+                                             int64_t *pos_end) {
   __shared__ int64_t s_warp[32];
   __shared__ int64_t s_carry;
   __shared__ int64_t s_raw[32];
@@ -396,6 +423,23 @@ __global__ void tuna_segbase_kernel(const int64_t *__restrict__ seg_total,
     if (pos_end) *pos_end = s_carry;  // pos[n]: one past the last block
     if (wbase) wbase[1] = wbase[0] + (uses_work ? ((s_carry + 255) & ~(int64_t)255) : 0);
   }
+}
+
+__global__ void tuna_segbase_kernel(const int64_t *__restrict__ seg_total,
+                                    const int64_t *__restrict__ seg_raw, int64_t *seg_base,
+                                    int64_t nseg, int64_t *scal, int64_t *wbase, int uses_work,
+                                    int64_t *pos_end) {
+  segbase_body(seg_total, seg_raw, seg_base, nseg, scal, wbase, uses_work, pos_end);
+}
+
+// The same for the two lists of a digit phase: CTA 0 the KEEP list, CTA 1 the DELIVER list.
+__global__ void tuna_segbase_pair_kernel(TunaScanArgs keep, TunaScanArgs del) {
+  if (blockIdx.x == 0)
+    segbase_body(keep.seg_total, keep.seg_raw, keep.seg_base, keep.seglen > 0 ? keep.nseg : 0, keep.scal,
+                 keep.wbase, keep.uses_work, keep.pos_end);
+  else
+    segbase_body(del.seg_total, del.seg_raw, del.seg_base, del.seglen > 0 ? del.nseg : 0, del.scal, del.wbase,
+                 del.uses_work, del.pos_end);
 }
 
 // pos[e] += base of its segment (turns per-rank scans into one stream position).
@@ -473,6 +517,34 @@ __global__ void tuna_chunk_index_kernel(const int64_t *__restrict__ pos, int64_t
       hi = mid;
   }
   first[c] = (int32_t)(lo > 0 ? lo - 1 : 0);
+}
+
+// The same for several lists in one launch (blockIdx.y picks the list; the lists'
+// parameters travel in the kernel's arguments).
+struct TunaChunkItem {
+  const int64_t *pos;
+  int32_t *first;
+  int64_t n, chunk, nchunks, total;
+};
+constexpr int kChunkBatch = 32;
+struct TunaChunkBatch {
+  TunaChunkItem it[kChunkBatch];
+};
+
+__global__ void tuna_chunk_index_batch_kernel(const __grid_constant__ TunaChunkBatch b) {
+  const TunaChunkItem &it = b.it[blockIdx.y];
+  const int64_t c = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (c > it.nchunks) return;
+  const int64_t target = c < it.nchunks ? c * it.chunk : it.total - 1;
+  int64_t lo = 0, hi = it.n;  // first index with pos > target
+  while (lo < hi) {
+    const int64_t mid = (lo + hi) >> 1;
+    if (it.pos[mid] <= target)
+      lo = mid + 1;
+    else
+      hi = mid;
+  }
+  it.first[c] = (int32_t)(lo > 0 ? lo - 1 : 0);
 }
 
 // Self-check of a finished list: every descriptor must read inside its source
@@ -892,7 +964,25 @@ int64_t pick_chunk(const TunaList &l) {
   return c;
 }
 
-int build_chunks(tuna_plan *pl, TunaList &l, cudaStream_t st) {
+// With `batch`, the list's table is not computed here: its parameters are collected
+// and launch_chunk_batch computes the tables of all collected lists in one launch.
+struct ChunkCollector {
+  TunaChunkBatch b;
+  int n = 0;
+  int64_t max_chunks = 0;
+};
+
+int launch_chunk_batch(tuna_plan *pl, ChunkCollector &cc, cudaStream_t st) {
+  if (cc.n == 0) return TUNA_OK;
+  const int th = 128;
+  tuna_chunk_index_batch_kernel<<<dim3((unsigned)((cc.max_chunks + th) / th), cc.n), th, 0, st>>>(cc.b);
+  TUNA_LAUNCHED(pl);
+  cc.n = 0;
+  cc.max_chunks = 0;
+  return TUNA_OK;
+}
+
+int build_chunks(tuna_plan *pl, TunaList &l, cudaStream_t st, ChunkCollector *batch = nullptr) {
   l.small_blocks = l.n > 0 && (l.bytes / l.n < env_i64("TUNA_SMALL_BLOCK_BYTES", kSmallBlockBytes) ||
                                l.bytes < env_i64("TUNA_SMALL_LIST_BYTES", kSmallListBytes) ||
                                (2 * l.unaligned_bytes > l.bytes && l.bytes / l.n < kSkewedLargeBlockBytes &&
@@ -906,7 +996,14 @@ int build_chunks(tuna_plan *pl, TunaList &l, cudaStream_t st) {
     TUNA_CUDA(pl, dev_alloc(&l.chunk_first, l.nchunks + 1));
     l.chunk_cap = l.nchunks;
   }
-  if (l.nchunks > 0) {
+  if (l.nchunks > 0 && batch) {
+    if (batch->n == kChunkBatch) {
+      const int rc = launch_chunk_batch(pl, *batch, st);
+      if (rc) return rc;
+    }
+    batch->b.it[batch->n++] = TunaChunkItem{l.pos, l.chunk_first, l.n, l.chunk, l.nchunks, l.total};
+    batch->max_chunks = std::max(batch->max_chunks, l.nchunks);
+  } else if (l.nchunks > 0) {
     const int th = 128;
     tuna_chunk_index_kernel<<<(unsigned)((l.nchunks + th) / th), th, 0, st>>>(
         l.pos, l.n, l.chunk, l.nchunks, l.total, l.chunk_first);
@@ -941,6 +1038,25 @@ int scan_list(tuna_plan *pl, TunaList &l, int64_t seglen, int64_t nseg, int list
     tuna_add_base_kernel<<<(unsigned)((l.n + th - 1) / th), th, 0, st>>>(l.pos, seg_base, seglen, l.n);
     TUNA_LAUNCHED(pl);
   }
+  return TUNA_OK;
+}
+
+// The KEEP and the DELIVER list of a digit phase, scanned together: two launches
+// instead of four.
+int scan_phase_lists(tuna_plan *pl, TunaList &k, int64_t keep_seglen, int keep_id, int64_t *wbase_slot,
+                     TunaList &d, int64_t del_seglen, int del_id, cudaStream_t st) {
+  const int P = pl->topo.P;
+  TunaScanArgs a{k.len, k.pos, pl->d_seg_total, pl->d_seg_raw, pl->d_seg_base, keep_seglen, P,
+                 pl->d_scal + 2 * keep_id, wbase_slot, 1, k.pos + k.n};
+  TunaScanArgs b{d.len, d.pos, pl->d_seg_total + P, pl->d_seg_raw + P, pl->d_seg_base + P, del_seglen, P,
+                 pl->d_scal + 2 * del_id, nullptr, 0, d.pos + d.n};
+  if (keep_seglen > 0 || del_seglen > 0) {
+    const int th = 256;
+    tuna_segscan_pair_kernel<<<dim3((unsigned)(((int64_t)P * 32 + th - 1) / th), 2), th, 0, st>>>(a, b);
+    TUNA_LAUNCHED(pl);
+  }
+  tuna_segbase_pair_kernel<<<2, 1024, 0, st>>>(a, b);
+  TUNA_LAUNCHED(pl);
   return TUNA_OK;
 }
 
@@ -1325,9 +1441,7 @@ int build_tables(tuna_plan *pl, const HostLayout *hl, const int64_t *sdispls, co
       }
       TUNA_LAUNCHED(pl);
       // per-rank prefix sums of both lists; the KEEP stream is this phase's workspace region
-      rc = scan_list(pl, k, ph.per_rank - ph.finals, P, f, pl->d_wbase + f, 1, false, st, 0);
-      if (rc) return rc;
-      rc = scan_list(pl, d, ph.finals, P, nph + f, nullptr, 0, false, st, 1);
+      rc = scan_phase_lists(pl, k, ph.per_rank - ph.finals, f, pl->d_wbase + f, d, ph.finals, nph + f, st);
       if (rc) return rc;
       tuna_place_kernel<<<gPP, th, 0, st>>>(t, pd, pl->d_loc[cur], pl->d_loc[cur ^ 1], k.pos,
                                             pl->d_seg_base, k.len, d.pos, pl->d_seg_base + P, d.dst,
@@ -1409,15 +1523,18 @@ int build_tables(tuna_plan *pl, const HostLayout *hl, const int64_t *sdispls, co
   for (auto &r : pl->rounds) r.bytes = (int64_t)rbytes[r.stat];
 
   Timed chunk_timer(pl, TUNA_TIMER_PLAN, 0, st);
+  ChunkCollector cc;  // the chunk tables of all lists: one launch (per 32 lists)
   for (int f = 0; f < nph; f++) {
-    rc = build_chunks(pl, pl->keep[f], st);
+    rc = build_chunks(pl, pl->keep[f], st, &cc);
     if (rc) return rc;
-    rc = build_chunks(pl, pl->deliver[f], st);
+    rc = build_chunks(pl, pl->deliver[f], st, &cc);
     if (rc) return rc;
   }
-  rc = build_chunks(pl, pl->rot, st);
+  rc = build_chunks(pl, pl->rot, st, &cc);
   if (rc) return rc;
-  if (!pl->dir_shared) rc = build_chunks(pl, pl->dir, st);
+  if (!pl->dir_shared) rc = build_chunks(pl, pl->dir, st, &cc);
+  if (rc) return rc;
+  rc = launch_chunk_batch(pl, cc, st);
   if (rc) return rc;
   rc = mark_tables_ready(pl, st);  // (no second wait on the host: exchanges order themselves behind this)
   if (rc) return rc;
@@ -1815,7 +1932,7 @@ static int plan_create(tuna_plan_t **out, int P, int radix, int radix_global, in
     TUNA_TRY(dev_alloc(&pl->d_loc[i], PP));
   }
   TUNA_TRY(dev_alloc(&pl->d_seg_total, 2 * P));
-  TUNA_TRY(dev_alloc(&pl->d_seg_raw, P));
+  TUNA_TRY(dev_alloc(&pl->d_seg_raw, 2 * P));
   TUNA_TRY(dev_alloc(&pl->d_seg_base, 2 * P));
   TUNA_TRY(dev_alloc(&pl->d_tmp, PP));
   {
