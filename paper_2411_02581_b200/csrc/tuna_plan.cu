@@ -383,7 +383,9 @@ __global__ void tuna_segscan_pair_kernel(TunaScanArgs keep, TunaScanArgs del) {
 __device__ __forceinline__ void segbase_body(const int64_t *__restrict__ seg_total,
                                              const int64_t *__restrict__ seg_raw, int64_t *seg_base,
                                              int64_t nseg, int64_t *scal, int64_t *wbase, int uses_work,
-                                             int64_t *pos_end) {
+                                             int64_t *pos_end, int spaced = 0) {
+  // (spaced: the values are block lengths, one block per segment: each is rounded up
+  // to 16 and given 16 spare bytes here, and seg_base is the list's position array)
   __shared__ int64_t s_warp[32];
   __shared__ int64_t s_carry;
   __shared__ int64_t s_raw[32];
@@ -393,8 +395,13 @@ __device__ __forceinline__ void segbase_body(const int64_t *__restrict__ seg_tot
   __syncthreads();
   for (int64_t base = 0; base < nseg; base += blockDim.x) {
     const int64_t i = base + threadIdx.x;
-    const int64_t x = i < nseg ? seg_total[i] : 0;
-    if (seg_raw && i < nseg) raw += seg_raw[i];
+    int64_t x = i < nseg ? seg_total[i] : 0;
+    if (spaced) {
+      raw += x;
+      x = x > 0 ? pad16(x) + 16 : 0;
+    } else if (seg_raw && i < nseg) {
+      raw += seg_raw[i];
+    }
     int64_t incl = x;
 #pragma unroll
     for (int d = 1; d < 32; d <<= 1) {
@@ -428,8 +435,8 @@ __device__ __forceinline__ void segbase_body(const int64_t *__restrict__ seg_tot
 __global__ void tuna_segbase_kernel(const int64_t *__restrict__ seg_total,
                                     const int64_t *__restrict__ seg_raw, int64_t *seg_base,
                                     int64_t nseg, int64_t *scal, int64_t *wbase, int uses_work,
-                                    int64_t *pos_end) {
-  segbase_body(seg_total, seg_raw, seg_base, nseg, scal, wbase, uses_work, pos_end);
+                                    int64_t *pos_end, int spaced) {
+  segbase_body(seg_total, seg_raw, seg_base, nseg, scal, wbase, uses_work, pos_end, spaced);
 }
 
 // The same for the two lists of a digit phase: CTA 0 the KEEP list, CTA 1 the DELIVER list.
@@ -1017,6 +1024,13 @@ int scan_list(tuna_plan *pl, TunaList &l, int64_t seglen, int64_t nseg, int list
               int64_t *wbase_slot, int uses_work, bool add_base, cudaStream_t st, int slot = 0) {
   int64_t *seg_total = pl->d_seg_total + (int64_t)slot * pl->topo.P;
   int64_t *seg_base = pl->d_seg_base + (int64_t)slot * pl->topo.P;
+  if (seglen == 1 && add_base && l.kind == TUNA_LIST_DELIVER && l.n == nseg && nseg > 0) {
+    // one block per segment (the self blocks): the positions are one scan of the spaced lengths
+    tuna_segbase_kernel<<<1, 1024, 0, st>>>(l.len, nullptr, l.pos, nseg, pl->d_scal + 2 * list_id, wbase_slot,
+                                            uses_work, l.pos + l.n, 1);
+    TUNA_LAUNCHED(pl);
+    return TUNA_OK;
+  }
   if (nseg > 0 && seglen > 0) {
     const int th = 256;
     const int64_t blocks = (nseg * 32 + th - 1) / th;
@@ -1031,7 +1045,7 @@ int scan_list(tuna_plan *pl, TunaList &l, int64_t seglen, int64_t nseg, int list
   tuna_segbase_kernel<<<1, 1024, 0, st>>>(seg_total, pl->d_seg_raw, seg_base,
                                           (nseg > 0 && seglen > 0) ? nseg : 0,
                                           pl->d_scal + 2 * list_id, wbase_slot, uses_work,
-                                          l.pos + l.n);
+                                          l.pos + l.n, 0);
   TUNA_LAUNCHED(pl);
   if (add_base && l.n > 0) {
     const int th = 256;
@@ -1377,7 +1391,7 @@ int build_tables(tuna_plan *pl, const HostLayout *hl, const int64_t *sdispls, co
       TUNA_LAUNCHED(pl);
       if (!hl) {  // send regions laid end to end: bases = scan of the row sums
         tuna_segbase_kernel<<<1, 1024, 0, st>>>(pl->d_seg_total, nullptr, pl->d_sendbase, P, pl->d_scal, nullptr, 0,
-                                                nullptr);
+                                                nullptr, 0);
         TUNA_LAUNCHED(pl);
         tuna_packed_extents_kernel<<<1, 32, 0, st>>>(pl->d_scal, t.elem, pl->d_extents);
         TUNA_LAUNCHED(pl);
@@ -1393,7 +1407,7 @@ int build_tables(tuna_plan *pl, const HostLayout *hl, const int64_t *sdispls, co
       TUNA_LAUNCHED(pl);
       if (!hl) {  // receive regions likewise: scan of the column sums
         tuna_segbase_kernel<<<1, 1024, 0, st>>>(pl->d_seg_total, nullptr, pl->d_recvbase, P, pl->d_scal, nullptr, 0,
-                                                nullptr);
+                                                nullptr, 0);
         TUNA_LAUNCHED(pl);
       }
     }
@@ -2202,7 +2216,7 @@ int tuna_plan_set_row_maps(tuna_plan_t *pl, const int64_t *gather_rows, const in
   tuna_segscan_kernel<0><<<gseg, th, 0, st>>>(pl->d_tmp, pl->d_row_start, pl->d_seg_total, nullptr, P, P);
   TUNA_LAUNCHED(pl);
   tuna_segbase_kernel<<<1, 1024, 0, st>>>(pl->d_seg_total, nullptr, pl->d_seg_base, P,
-                                          pl->d_scal + 2 * (2 * nph + 2), nullptr, 0, nullptr);
+                                          pl->d_scal + 2 * (2 * nph + 2), nullptr, 0, nullptr, 0);
   TUNA_LAUNCHED(pl);
   tuna_add_base_kernel<<<gPP, th, 0, st>>>(pl->d_row_start, pl->d_seg_base, P, PP);
   TUNA_LAUNCHED(pl);
@@ -2554,7 +2568,7 @@ int tuna_direct_alltoallv_static(int P, int elem_size, const int64_t *sendcounts
   tuna_segscan_kernel<2><<<gseg, th, 0, st>>>(t.len, t.pos, t.seg_total, t.seg_raw, P, P);
   TUNA_STATIC_CUDA(cudaGetLastError());
   tuna_segbase_kernel<<<1, 1024, 0, st>>>(t.seg_total, t.seg_raw, t.seg_base, P, t.scal, nullptr, 0,
-                                          t.pos + PP);
+                                          t.pos + PP, 0);
   TUNA_STATIC_CUDA(cudaGetLastError());
   tuna_add_base_kernel<<<gPP, th, 0, st>>>(t.pos, t.seg_base, P, PP);
   TUNA_STATIC_CUDA(cudaGetLastError());
