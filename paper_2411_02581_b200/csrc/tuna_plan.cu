@@ -1064,9 +1064,16 @@ int scan_phase_lists(tuna_plan *pl, TunaList &k, int64_t keep_seglen, int keep_i
                  pl->d_scal + 2 * keep_id, wbase_slot, 1, k.pos + k.n};
   TunaScanArgs b{d.len, d.pos, pl->d_seg_total + P, pl->d_seg_raw + P, pl->d_seg_base + P, del_seglen, P,
                  pl->d_scal + 2 * del_id, nullptr, 0, d.pos + d.n};
-  if (keep_seglen > 0 || del_seglen > 0) {
-    const int th = 256;
-    tuna_segscan_pair_kernel<<<dim3((unsigned)(((int64_t)P * 32 + th - 1) / th), 2), th, 0, st>>>(a, b);
+  const int th = 256;
+  const unsigned gx = (unsigned)(((int64_t)P * 32 + th - 1) / th);
+  if (keep_seglen > 0 && del_seglen > 0) {
+    tuna_segscan_pair_kernel<<<dim3(gx, 2), th, 0, st>>>(a, b);
+    TUNA_LAUNCHED(pl);
+  } else if (keep_seglen > 0) {  // (a phase with one list only runs the leaner single-list kernel)
+    tuna_segscan_kernel<1><<<gx, th, 0, st>>>(a.val, a.out, a.seg_total, a.seg_raw, a.seglen, a.nseg);
+    TUNA_LAUNCHED(pl);
+  } else if (del_seglen > 0) {
+    tuna_segscan_kernel<2><<<gx, th, 0, st>>>(b.val, b.out, b.seg_total, b.seg_raw, b.seglen, b.nseg);
     TUNA_LAUNCHED(pl);
   }
   tuna_segbase_pair_kernel<<<2, 1024, 0, st>>>(a, b);
