@@ -362,7 +362,11 @@ def ours_arm(args):
     recv = wl.make_recv(dev)
     payload = wl.payload_bytes_total
 
-    def make_plan(r, l=None, g=1, rg=2, flags=0, block_count=0):
+    def make_plan(r, l=None, g=1, rg=2, flags=0, block_count=0, direct=False):
+        # plans that only run their own schedule are told so: multi-phase plans then keep
+        # no direct list, which shortens every re-plan
+        if not direct:
+            flags |= B.FLAG_NO_DIRECT
         return B.plan_for(wl, r, l=l, g=g, radix_global=rg, flags=flags, explicit_layout=False,
                           block_count=block_count)
 
@@ -520,7 +524,7 @@ def ours_arm(args):
 
         plan.set_workspace(None)
         torch.cuda.empty_cache()
-        entry("direct", make_plan(wl.P), direct=True)
+        entry("direct", make_plan(wl.P, direct=True), direct=True)
         for r in wl.radices:
             entry(f"flat r={r}", make_plan(r))
         if wl.radices:

@@ -58,6 +58,9 @@ typedef enum tuna_status {
 #define TUNA_FLAG_BULK_COPY 2u      /* chunks inside one large 16-byte aligned block go through the SM's bulk
                                        copy engine (cp.async.bulk through shared memory) instead of vector loads
                                        and stores; same result, measured about 1 % slower, hence optional */
+#define TUNA_FLAG_NO_DIRECT 4u      /* the plan will not be used for tuna_direct_alltoallv (nor the direct schedule
+                                       of tuna_alltoallv_host): no separate direct list is built, which shortens
+                                       every update of a multi-phase plan; those calls return TUNA_ERR_INVALID_ARG */
 
 /* schedules for the host-buffer entry point */
 #define TUNA_SCHEDULE_TUNA 0

@@ -21,6 +21,7 @@ _VP = ctypes.c_void_p
 FLAG_DIRECT_TO_R = 0
 FLAG_CLASSIC_ROTATE = 1
 FLAG_BULK_COPY = 2
+FLAG_NO_DIRECT = 4
 PART_KEEP = 0
 PART_DELIVER = 1
 SCHEDULE_TUNA = 0

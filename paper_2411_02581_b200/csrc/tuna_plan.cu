@@ -682,6 +682,7 @@ struct tuna_plan {
   // block in that phase: its DELIVER list and the self blocks together are the
   // direct exchange, so no separate direct list is built.
   bool dir_shared = false;
+  bool no_direct = false;  // TUNA_FLAG_NO_DIRECT: no direct list at all (unless the phase's lists serve as one)
   // exchange of rows through a gather and a scatter map (tuna_plan_set_row_maps)
   TunaList rowsl;
   int64_t rows_cap = 0;          // descriptors allocated in rowsl
@@ -1474,7 +1475,7 @@ int build_tables(tuna_plan *pl, const HostLayout *hl, const int64_t *sdispls, co
     // work partitions of the rotation and direct lists
     rc = scan_list(pl, pl->rot, pl->classic ? P : 1, P, 2 * nph, nullptr, 0, true, st);
     if (rc) return rc;
-    if (!pl->dir_shared) rc = scan_list(pl, pl->dir, P, P, 2 * nph + 1, nullptr, 0, true, st);
+    if (!pl->dir_shared && !pl->no_direct) rc = scan_list(pl, pl->dir, P, P, 2 * nph + 1, nullptr, 0, true, st);
     if (rc) return rc;
 
     // self-check: every descriptor of every list stays inside its buffers
@@ -1539,7 +1540,7 @@ int build_tables(tuna_plan *pl, const HostLayout *hl, const int64_t *sdispls, co
     take(pl->deliver[f], nph + f);
   }
   take(pl->rot, 2 * nph);
-  if (!pl->dir_shared) take(pl->dir, 2 * nph + 1);
+  if (!pl->dir_shared && !pl->no_direct) take(pl->dir, 2 * nph + 1);
   pl->workspace_need = wbase[nph];
   for (auto &r : pl->rounds) r.bytes = (int64_t)rbytes[r.stat];
 
@@ -1553,7 +1554,7 @@ int build_tables(tuna_plan *pl, const HostLayout *hl, const int64_t *sdispls, co
   }
   rc = build_chunks(pl, pl->rot, st, &cc);
   if (rc) return rc;
-  if (!pl->dir_shared) rc = build_chunks(pl, pl->dir, st, &cc);
+  if (!pl->dir_shared && !pl->no_direct) rc = build_chunks(pl, pl->dir, st, &cc);
   if (rc) return rc;
   rc = launch_chunk_batch(pl, cc, st);
   if (rc) return rc;
@@ -1762,6 +1763,7 @@ int run_tuna(tuna_plan *pl, const void *send, void *recv, cudaStream_t st) {
 }
 
 int run_direct(tuna_plan *pl, const void *send, void *recv, cudaStream_t st) {
+  if (pl->no_direct) return TUNA_ERR_INVALID_ARG;  // the plan was created without a direct list
   {
     const int arc = await_tables(pl, st);
     if (arc) return arc;
@@ -1990,7 +1992,8 @@ static int plan_create(tuna_plan_t **out, int P, int radix, int radix_global, in
   if (rc) return nomem(rc);
   pl->dir_shared = !pl->classic && g == 1 && block_count == 0 && nph == 1 &&
                    pl->phases[0].finals == pl->phases[0].per_rank;
-  if (!pl->dir_shared) {
+  pl->no_direct = (flags & TUNA_FLAG_NO_DIRECT) != 0 && !pl->dir_shared;
+  if (!pl->dir_shared && !pl->no_direct) {
     rc = alloc_list(pl, pl->dir, TUNA_LIST_DELIVER, PP);
     if (rc) return nomem(rc);
   }
@@ -2007,7 +2010,7 @@ static int plan_create(tuna_plan_t **out, int P, int radix, int radix_global, in
       add(pl->deliver[f], 0, nph + f);
     }
     add(pl->rot, 0, 2 * nph);
-    if (!pl->dir_shared) add(pl->dir, 0, 2 * nph + 1);
+    if (!pl->dir_shared && !pl->no_direct) add(pl->dir, 0, 2 * nph + 1);
     pl->n_check_items = (int)items.size();
     if (!items.empty()) {
       TUNA_TRY(cudaMalloc(&pl->d_check_items, items.size() * sizeof(TunaCheckItem)));

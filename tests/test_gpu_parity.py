@@ -409,6 +409,44 @@ def test_update_waits_for_the_plans_own_exchange_in_flight():
     assert np.array_equal(recv2.cpu().numpy(), oracle_brute(small))
 
 
+def test_plans_without_a_direct_list():
+    """TUNA_FLAG_NO_DIRECT: the plan's own schedule works as ever, the direct exchange is
+    refused, except where the single phase's lists are the direct exchange anyway."""
+    wl = W.make_random(12, 300, seed=73, zero_frac=0.2, gaps=True)
+    ref = oracle_brute(wl)
+    send = wl.make_send("cuda")
+    for kw in (dict(radix=2), dict(radix=3, l=4, g=3, radix_global=3), dict(radix=2, flags=B.FLAG_CLASSIC_ROTATE)):
+        kw = dict(kw)
+        kw["flags"] = kw.get("flags", 0) | B.FLAG_NO_DIRECT
+        plan = B.plan_for(wl, **kw)
+        plan.alloc_workspace()
+        assert plan.phase_info(-2)["entries"] == 0
+        recv = wl.make_recv("cuda", fill=CANARY)
+        plan.alltoallv(send, recv)
+        torch.cuda.synchronize()
+        assert np.array_equal(recv.cpu().numpy(), ref)
+        recv = wl.make_recv("cuda", fill=CANARY)
+        with pytest.raises(B.TunaError, match="INVALID_ARG"):
+            plan.direct_alltoallv(send, recv)
+        torch.cuda.synchronize()
+        assert bool((recv == CANARY).all())
+    plan = B.plan_for(wl, 12, flags=B.FLAG_NO_DIRECT)   # radix >= P: the phase's lists serve
+    recv = wl.make_recv("cuda", fill=CANARY)
+    plan.direct_alltoallv(send, recv)
+    torch.cuda.synchronize()
+    assert np.array_equal(recv.cpu().numpy(), ref)
+    # packed counts from device memory on a hierarchical plan without a direct list
+    wp = W.make_random(12, 500, seed=74, zero_frac=0.3)
+    plan = B.plan_for(W.make_uniform(12, 2), 4, l=4, g=3, radix_global=3, flags=B.FLAG_NO_DIRECT, explicit_layout=False)
+    for _ in range(2):
+        plan.update_counts_device(torch.from_numpy(wp.sendcounts).cuda())
+        plan.alloc_workspace()
+        recv = wp.make_recv("cuda", fill=CANARY)
+        plan.alltoallv(wp.make_send("cuda"), recv)
+        torch.cuda.synchronize()
+        assert np.array_equal(recv.cpu().numpy(), oracle_brute(wp))
+
+
 def test_negative_device_counts_are_refused_and_the_plan_recovers():
     wl = W.make_random(9, 300, seed=71, zero_frac=0.2)
     plan = B.plan_for(wl, 3, explicit_layout=False)
