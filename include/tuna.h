@@ -332,6 +332,7 @@ int tuna_rows_alltoallv(tuna_plan_t *plan, const void *rows_in, void *rows_out, 
  * A flat plan whose radix is at least P (one digit phase that delivers every
  * block) keeps no separate direct list: tuna_direct_alltoallv then runs that
  * phase's DELIVER list and the self blocks, and phase -2 reports no entries.
+ * Plans created with TUNA_FLAG_NO_DIRECT report none either.
  * `entries` descriptor rows, `bytes` moved, `stream_bytes` the padded length of the
  * list's stream (for a KEEP list: the size of its workspace region).
  */
