@@ -37,6 +37,8 @@ extern "C" {
 
 typedef struct tuna_plan tuna_plan_t;
 
+#define TUNA_MAX_P 32768 /* ranks of one plan, at most */
+
 typedef enum tuna_status {
   TUNA_OK = 0,
   TUNA_ERR_INVALID_ARG = -1,    /* null pointer, P < 1, elem_size < 1, negative count or offset */
@@ -81,9 +83,17 @@ typedef enum tuna_status {
  * ranks with equal local id; radix_global == g is the paper's coalesced exchange).
  *
  *   out           host; receives the plan.
- *   P             number of ranks, >= 1.
- *   radix         flat radix (g == 1) or local radix, in [2, max(2, l)].
- *   radix_global  global radix in [2, max(2, g)]; ignored when g == 1.
+ *   P             number of ranks, 1 <= P <= TUNA_MAX_P (TUNA_ERR_RANGE above: the
+ *                 tables index P * P blocks with 32-bit arithmetic).
+ *   radix         flat radix (g == 1) or local radix, in [2, max(2, l)], or 0 = choose.
+ *   radix_global  global radix in [2, max(2, g)], or 0 = choose; ignored when g == 1.
+ *                 The choice is the largest radix, l and g: one hop per level.  The
+ *                 paper's Sec. V-A finds small radices best for small blocks, where
+ *                 per-message latency dominates, and large ones for large blocks,
+ *                 where the bytes forwarded dominate; with every rank in one memory
+ *                 there is no per-message latency to save, only the forwarding cost
+ *                 (each hop reads and writes the block once more), and every measured
+ *                 workload ran fastest with the fewest hops.
  *   l, g          ranks per group and number of groups, l*g == P; g == 1 is flat TuNA.
  *   elem_size     bytes per element, >= 1.
  *   flags         TUNA_FLAG_*.
@@ -250,6 +260,11 @@ int tuna_direct_alltoallv(tuna_plan_t *plan, const void *sendbuf, const int64_t 
  *   limit        the work stream (every non-empty block rounded up to 16 bytes plus
  *                16) may not exceed TUNA_STATIC_MAX_CHUNKS * 256 KiB = 4 GiB, else
  *                TUNA_ERR_RANGE; nothing is launched in that case.
+ * Errors: besides the limits above, an entry (count, displacement or base) above
+ * 2^47 bytes gives TUNA_ERR_RANGE; every size check comes before the buffers are
+ * looked at and before anything is enqueued.  The call hands the host arrays to
+ * asynchronous copies, which only an eager call may do: on a stream that is being
+ * captured it returns TUNA_ERR_INVALID_ARG and records nothing.
  * The first call on a device looks up the array's device address; make that call
  * before starting a stream capture on that device.  All calls share the one array
  * and it keeps the previous call's tables; every table a call reads it first

@@ -10,8 +10,9 @@ ROOT = os.path.dirname(_HERE)
 CSRC = os.path.join(_HERE, "csrc")
 LIB_DIR = os.path.join(_HERE, "_lib")
 LIB_PATH = os.path.join(LIB_DIR, "libtuna.so")
-SOURCES = ["tuna_plan.cu", "tuna_move.cu"]
-HEADERS = [os.path.join(CSRC, "tuna_internal.h"), os.path.join(ROOT, "include", "tuna.h")]
+SOURCES = ["tuna_plan.cu", "tuna_api.cu", "tuna_static.cu", "tuna_move.cu"]
+HEADERS = [os.path.join(CSRC, h) for h in ("tuna_internal.h", "tuna_plan.h", "tuna_plan_kernels.cuh")] + [
+    os.path.join(ROOT, "include", "tuna.h")]
 
 
 def _nvcc() -> str:

@@ -99,7 +99,12 @@ enum TunaMoveKernel {
 };
 
 // Launches one mover kernel (tuna_move.cu).  `small_blocks` picks the build tuned
-// for lists whose blocks are far smaller than a chunk.
-cudaError_t tuna_launch_move(int kernel, const TunaMoveArgs &a, bool small_blocks, cudaStream_t stream);
+// for lists whose blocks are far smaller than a chunk.  `early_start` lets the
+// kernel's CTAs begin their set-up while the previous kernel of the stream drains
+// (they read the plan's tables before they wait for it): only for a launch whose
+// predecessor on the stream is an earlier launch of the same exchange, never for
+// the first one, which may follow the kernels that write those tables.
+cudaError_t tuna_launch_move(int kernel, const TunaMoveArgs &a, bool small_blocks, bool early_start,
+                             cudaStream_t stream);
 
 #endif

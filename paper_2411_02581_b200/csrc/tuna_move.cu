@@ -227,11 +227,15 @@ __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wa
 
 // ------------------------------------------------------------------ dependent launches
 //
-// The launches of one exchange form a chain on a stream.  Each is launched with
-// programmatic stream serialization: its CTAs may start while the previous launch
-// is still draining, do their set-up (which reads only the plan's tables), and
-// then block in hardware until the previous launch has completed and its writes
-// are visible.  Every launch lets its successor start early right away.
+// The launches of one exchange form a chain on a stream.  From the second one on,
+// each is launched with programmatic stream serialization: its CTAs may start
+// while the previous launch is still draining, do their set-up (which reads only
+// the plan's tables), and then block in hardware until the previous launch has
+// completed and its writes are visible.  Every launch lets its successor start
+// early right away.  The first launch of an exchange starts the ordinary way:
+// what precedes it on the stream may be the plan kernels that write the very
+// tables its set-up reads, and their stores are only guaranteed visible to a
+// launch that waits for them in full.
 
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
@@ -597,7 +601,8 @@ __global__ void __launch_bounds__(kThreads, 8) tuna_direct_small_kernel(const Tu
 
 }  // namespace
 
-cudaError_t tuna_launch_move(int kernel, const TunaMoveArgs &a_in, bool small_blocks, cudaStream_t stream) {
+cudaError_t tuna_launch_move(int kernel, const TunaMoveArgs &a_in, bool small_blocks, bool early_start,
+                             cudaStream_t stream) {
   TunaMoveArgs a = a_in;
   const TunaListArgs *ls[3] = {&a.keep, &a.del, &a.rot};
   int64_t nchunks = 0, max_chunk = 0;
@@ -653,7 +658,7 @@ cudaError_t tuna_launch_move(int kernel, const TunaMoveArgs &a_in, bool small_bl
     return !(e && e[0] == '0');
   }();
   cfg.attrs = attr;
-  cfg.numAttrs = chain ? 1 : 0;
+  cfg.numAttrs = (chain && early_start) ? 1 : 0;
   const cudaError_t le = cudaLaunchKernelEx(&cfg, fn, a);
   if (le != cudaSuccess) return le;
   return cudaGetLastError();

@@ -75,6 +75,51 @@ def test_host_validation_rejects_before_any_gpu_work(lib):
     assert lib.tuna_alltoallv(None, None, None, None, None, None, None, None) == -1
 
 
+def test_radix_zero_means_choose_and_rank_limit(lib):
+    z = np.zeros((4, 4), dtype=np.int64)
+    # radix 0 passes validation (what follows needs a GPU: without one the first CUDA
+    # call fails, with one the plan is built); it is not a radix error either way
+    assert _create(lib, 4, 0, 0, 2, 2, 1, z) in (0, -7, -8)
+    assert _create(lib, 4, 0, 2, 4, 1, 1, z) in (0, -7, -8)
+    big = np.zeros((1, 1), dtype=np.int64)
+    assert _create(lib, 32769, 2, 2, 32769, 1, 1, big) == -9   # above TUNA_MAX_P: refused before the counts are read
+
+
+def _static(lib, P, elem, counts, sdispls=None, sendbase=None):
+    def arr(a):
+        if a is None:
+            return None, None
+        a = np.ascontiguousarray(a, dtype=np.int64)
+        return a, a.ctypes.data_as(ctypes.POINTER(ctypes.c_int64))
+    c, cp = arr(counts)
+    s, sp = arr(sdispls)
+    b, bp = arr(sendbase)
+    return lib.tuna_direct_alltoallv_static(P, elem, cp, sp, None, bp, None, None, None, None)
+
+
+def test_static_entry_refuses_sizes_before_it_looks_at_buffers(lib):
+    """Limits of the allocation-free entry point, with NULL buffers and no GPU: a size
+    over a limit must come back as TUNA_ERR_RANGE, never reach a launch."""
+    huge = np.zeros((2, 2), dtype=np.int64)
+    huge[0, 1] = 5 << 30                                       # 5 GiB of blocks: work stream over 4 GiB
+    assert _static(lib, 2, 1, huge) == -9
+    many = np.full((2, 2), 1 << 30, dtype=np.int64)            # 4 x 1 Gi elements of 8 bytes
+    assert _static(lib, 2, 8, many) == -9
+    wrap = np.zeros((2, 2), dtype=np.int64)
+    wrap[1, 0] = (1 << 62) // 3                                # bytes = count * 12 would wrap
+    assert _static(lib, 2, 12, wrap) == -9
+    small = np.ones((2, 2), dtype=np.int64)
+    far = np.zeros((2, 2), dtype=np.int64)
+    far[0, 0] = 1 << 60                                        # displacement + count beyond any buffer
+    assert _static(lib, 2, 1, small, sdispls=far) == -9
+    assert _static(lib, 2, 1, small, sendbase=[0, 1 << 61]) == -9
+    assert _static(lib, 129, 1, np.zeros((129, 129), dtype=np.int64)) == -9     # above TUNA_STATIC_MAX_P
+    assert _static(lib, 2, 1, small) == -1                     # fine sizes, NULL buffers
+    neg = small.copy()
+    neg[0, 1] = -1
+    assert _static(lib, 2, 1, neg) == -1
+
+
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(B, "_lib", None)
     monkeypatch.setattr(build_mod, "LIB_PATH", str(tmp_path / "nope.so"))
