@@ -23,8 +23,11 @@ if os.environ.get("TUNA_ORACLE_SOURCE"):
     _SRC = os.environ["TUNA_ORACLE_SOURCE"]
     _OUT_DIR = os.path.dirname(_SRC)
     _LIB = os.path.splitext(_SRC)[0] + ".so"
+_SRC_MT = os.path.join(_HERE, "tuna_oracle_mt.c")       # threaded timing variant (not the checker)
+_LIB_MT = os.path.join(_HERE, "_build", "libtuna_oracle_mt.so")
 _lock = threading.Lock()
 _lib = None
+_lib_mt = None
 
 RS_COLS = 6
 RS_LEVEL, RS_X, RS_Z, RS_UNITS, RS_BYTES_SENT, RS_BYTES_RECV = range(6)
@@ -41,6 +44,17 @@ def build(force: bool = False) -> str:
                                "-o", tmp, _SRC])
         os.replace(tmp, _LIB)
     return _LIB
+
+
+def build_mt(force: bool = False) -> str:
+    """Compile the threaded timing variant of the flat oracle."""
+    os.makedirs(os.path.dirname(_LIB_MT), exist_ok=True)
+    if force or not os.path.exists(_LIB_MT) or os.path.getmtime(_LIB_MT) < os.path.getmtime(_SRC_MT):
+        tmp = _LIB_MT + ".tmp.%d" % os.getpid()
+        subprocess.check_call(["gcc", "-O2", "-std=gnu11", "-Wall", "-Wextra", "-shared", "-fPIC", "-pthread",
+                               "-o", tmp, _SRC_MT])
+        os.replace(tmp, _LIB_MT)
+    return _LIB_MT
 
 
 _I64P = ctypes.POINTER(ctypes.c_int64)
@@ -66,6 +80,9 @@ def _load():
             lib.oracle_tuna_hier.argtypes = (
                 [ctypes.c_int] * 5 + [_I64P] * 5 + [_U8P, _U8P, ctypes.c_int64, _U8P, _I64P,
                                                     ctypes.c_int, _IP])
+            lib.oracle_tuna_hier_tables.argtypes = (
+                [ctypes.c_int] * 5 + [_I64P] * 5 + [_U8P, _U8P, ctypes.c_int64, _U8P, _I64P, _I64P,
+                                                    _I64P])
             lib.oracle_tuna_hier_staggered.argtypes = (
                 [ctypes.c_int] * 5 + [_I64P] * 5 + [_U8P, _U8P, ctypes.c_int64, _U8P, _I64P,
                                                     ctypes.c_int, _IP, _IP])
@@ -169,6 +186,30 @@ def tuna_flat(wl, r: int, send: np.ndarray, recv: np.ndarray, trace_rank: int = 
     return recv, rounds[:K], Bc.value, trace
 
 
+def tuna_flat_mt(wl, r: int, send: np.ndarray, recv: np.ndarray, threads: int):
+    """Algorithm 1 with the ranks of every round shared out over ``threads`` plain threads:
+    a TIMING variant for the CPU baseline, checked against :func:`tuna_flat` by a test; never
+    used to check anything itself.  Returns (recv, rounds[K, RS_COLS])."""
+    global _lib_mt
+    with _lock:
+        if _lib_mt is None:
+            lib = ctypes.CDLL(build_mt())
+            lib.oracle_tuna_flat_mt.argtypes = ([ctypes.c_int] * 3 + [_I64P] * 5
+                                                + [_U8P, _U8P, _I64P, ctypes.c_int, ctypes.c_int])
+            _lib_mt = lib
+    c, cp = _i64(wl.sendcounts)
+    sd, sdp = _i64(wl.sdispls)
+    rd, rdp = _i64(wl.rdispls)
+    sb, sbp = _i64(wl.sendbase)
+    rb, rbp = _i64(wl.recvbase)
+    K = _load().oracle_round_list(wl.P, r, None, None, 0)
+    rounds = np.zeros((max(K, 1), RS_COLS), dtype=np.int64)
+    _check(_lib_mt.oracle_tuna_flat_mt(wl.P, r, wl.elem_size, cp, sdp, rdp, sbp, rbp, _u8(send),
+                                       _u8(recv), rounds.ctypes.data_as(_I64P), K, int(threads)),
+           "oracle_tuna_flat_mt")
+    return recv, rounds[:K]
+
+
 def tuna_hier(wl, Q: int, N: int, rl: int, rg: int, send: np.ndarray, recv: np.ndarray,
               want_after_local: bool = False):
     """Hierarchical exchange.  Returns (recv, rounds, (K_local, K_global), recv_after_local)."""
@@ -188,6 +229,33 @@ def tuna_hier(wl, Q: int, N: int, rl: int, rg: int, send: np.ndarray, recv: np.n
                                 rounds.ctypes.data_as(_I64P), K, Ks), "oracle_tuna_hier")
     assert Ks[0] + Ks[1] == K
     return recv, rounds[:K], (Ks[0], Ks[1]), after
+
+
+def tuna_hier_tables(wl, Q: int, N: int, rl: int, rg: int, send: np.ndarray, recv: np.ndarray):
+    """The hierarchical exchange with the metadata the ranks hold copied out.  Returns
+    (recv, recv_after_local, sz_local[wl, P, N, Q], usz_compact[P, N, Q],
+    usz_global[wg, P, N, Q]): block sizes by (rank, destination group, local offset) after
+    every local digit phase; sub-block sizes by (rank, group offset, source local id) after
+    the compaction and after every global digit phase."""
+    lib = _load()
+    assert Q * N == wl.P
+    P = wl.P
+    c, cp = _i64(wl.sendcounts)
+    sd, sdp = _i64(wl.sdispls)
+    rd, rdp = _i64(wl.rdispls)
+    sb, sbp = _i64(wl.sendbase)
+    rb, rbp = _i64(wl.recvbase)
+    wloc, wglo = lib.oracle_num_digits(Q, rl), lib.oracle_num_digits(N, rg)
+    sz_local = np.zeros((max(wloc, 1), P, N, Q), dtype=np.int64)
+    usz_compact = np.zeros((P, N, Q), dtype=np.int64)
+    usz_global = np.zeros((max(wglo, 1), P, N, Q), dtype=np.int64)
+    after = np.empty_like(recv)
+    _check(lib.oracle_tuna_hier_tables(Q, N, rl, rg, wl.elem_size, cp, sdp, rdp, sbp, rbp, _u8(send),
+                                       _u8(recv), recv.nbytes, _u8(after),
+                                       sz_local.ctypes.data_as(_I64P),
+                                       usz_compact.ctypes.data_as(_I64P),
+                                       usz_global.ctypes.data_as(_I64P)), "oracle_tuna_hier_tables")
+    return recv, after, sz_local[:wloc], usz_compact, usz_global[:wglo]
 
 
 def tuna_hier_staggered(wl, Q: int, N: int, rl: int, block_count: int, send: np.ndarray,

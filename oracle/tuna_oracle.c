@@ -403,12 +403,23 @@ done:
  *
  * `recv_after_local` (may be NULL) receives a copy of the receive buffer as it
  * stands after the local phase.  K_out[0] = local rounds, K_out[1] = global.
+ * Three more optional outputs copy out the metadata the ranks hold (Sec. III-B:
+ * sizes travel ahead of the data), without touching it:
+ *   sz_local     wl*P*P values: after all rounds of local digit position x,
+ *                sz_local[x][p][i*Q + jo] = bytes of the block rank p = (n, q) holds
+ *                for rank (i, (q + jo) % Q);
+ *   usz_compact  P*N*Q values: after the compaction (Sec. IV-B),
+ *                usz_compact[p][io][q'] = bytes of the part that came from rank
+ *                (n, q') in the super-block rank p holds for group (n + io) % N;
+ *   usz_global   wg*P*N*Q values: the same table after all rounds of global digit
+ *                position x.
  */
 static int hier_impl(int Q, int N, int rl, int rg, int block_count, int elem,
                      const int64_t *counts, const int64_t *sdispls, const int64_t *rdispls,
                      const int64_t *sendbase, const int64_t *recvbase, const uint8_t *send,
                      uint8_t *recv, int64_t recv_bytes, uint8_t *recv_after_local,
-                     int64_t *rounds, int rounds_cap, int *K_out, int *batches_out) {
+                     int64_t *rounds, int rounds_cap, int *K_out, int *batches_out,
+                     int64_t *sz_local, int64_t *usz_compact, int64_t *usz_global) {
   if (Q < 1 || N < 1 || rl < 2 || rg < 2 || elem < 1 || block_count < 0) return ORACLE_EARG;
   const int P = Q * N;
   int rc = ORACLE_OK;
@@ -529,6 +540,7 @@ static int hier_impl(int Q, int N, int rl, int rg, int block_count, int elem,
       }
       k++;
     }
+    if (sz_local) memcpy(sz_local + (int64_t)x * P * P, sz, sizeof(int64_t) * (size_t)P * P);
   }
   if (k != Kl) {
     rc = ORACLE_ESCHED;
@@ -647,6 +659,8 @@ static int hier_impl(int Q, int N, int rl, int rg, int block_count, int elem,
     }
   }
 
+  if (usz_compact) memcpy(usz_compact, usz, sizeof(int64_t) * (size_t)P * N * Q);
+
   /* global phase: Algorithm 1 over the N ranks with the same q; the unit is a
      super-block, its metadata the Q sizes of its parts */
   for (int x = 0; x < wg; x++) {
@@ -747,6 +761,8 @@ static int hier_impl(int Q, int N, int rl, int rg, int block_count, int elem,
       }
       k++;
     }
+    if (usz_global)
+      memcpy(usz_global + (int64_t)x * P * N * Q, usz, sizeof(int64_t) * (size_t)P * N * Q);
   }
   if (k != Kl + Kg) rc = ORACLE_ESCHED;
 
@@ -779,7 +795,19 @@ int oracle_tuna_hier(int Q, int N, int rl, int rg, int elem, const int64_t *coun
                      int64_t recv_bytes, uint8_t *recv_after_local, int64_t *rounds,
                      int rounds_cap, int *K_out) {
   return hier_impl(Q, N, rl, rg, 0, elem, counts, sdispls, rdispls, sendbase, recvbase, send, recv,
-                   recv_bytes, recv_after_local, rounds, rounds_cap, K_out, NULL);
+                   recv_bytes, recv_after_local, rounds, rounds_cap, K_out, NULL, NULL, NULL, NULL);
+}
+
+/* oracle_tuna_hier with the metadata tables of hier_impl copied out as well. */
+int oracle_tuna_hier_tables(int Q, int N, int rl, int rg, int elem, const int64_t *counts,
+                            const int64_t *sdispls, const int64_t *rdispls,
+                            const int64_t *sendbase, const int64_t *recvbase,
+                            const uint8_t *send, uint8_t *recv, int64_t recv_bytes,
+                            uint8_t *recv_after_local, int64_t *sz_local, int64_t *usz_compact,
+                            int64_t *usz_global) {
+  return hier_impl(Q, N, rl, rg, 0, elem, counts, sdispls, rdispls, sendbase, recvbase, send, recv,
+                   recv_bytes, recv_after_local, NULL, 0, NULL, NULL, sz_local, usz_compact,
+                   usz_global);
 }
 
 /*
@@ -797,7 +825,7 @@ int oracle_tuna_hier_staggered(int Q, int N, int rl, int block_count, int elem,
   if (block_count < 1) return ORACLE_EARG;
   return hier_impl(Q, N, rl, 2, block_count, elem, counts, sdispls, rdispls, sendbase, recvbase,
                    send, recv, recv_bytes, recv_after_local, rounds, rounds_cap, K_out,
-                   batches_out);
+                   batches_out, NULL, NULL, NULL);
 }
 
 /*

@@ -234,6 +234,107 @@ def test_metadata_and_prefix_sums(P, r):
     rot = classic.phase_tables(-1)
     assert np.array_equal(rot["len"].reshape(P, P), sizes[-1])   # every block, in slot order
 
+def _digit(v, r, x):
+    return (v // r ** x) % r
+
+
+@pytest.mark.parametrize("Q,N,rl,rg", [(5, 3, 2, 3), (4, 4, 2, 2), (3, 4, 3, 2), (6, 5, 2, 3), (8, 4, 8, 4),
+                                       (16, 16, 4, 4), (32, 8, 32, 8)])
+def test_hier_metadata_and_prefix_sums(Q, N, rl, rg):
+    """Descriptor tables of every local and global digit phase of a hierarchical plan:
+    sizes equal the oracle's message-passed metadata (the global phases' against the
+    sub-block sizes of its compacted super-blocks), positions equal its running sums,
+    and every block is read from where the previous phase put it."""
+    P = Q * N
+    wl = W.make_random(P, 300, elem_size=3, seed=17 * P + rl + rg, zero_frac=0.3, gaps=True)
+    send = wl.make_send().numpy()
+    recv = wl.make_recv(fill=CANARY).numpy().copy()
+    _, _, sz_local, usz_compact, usz_global = oracle.tuna_hier_tables(wl, Q, N, rl, rg, send, recv)
+    plan = B.plan_for(wl, rl, l=Q, g=N, radix_global=rg)
+    wloc, wglo = sz_local.shape[0], usz_global.shape[0]
+    assert plan.num_phases() == wloc + wglo
+    E = wl.elem_size
+    ranks = np.arange(P)
+    n_of, q_of = ranks // Q, ranks % Q
+
+    def recv_loc(p, origin):
+        return (1 << 56) | int(wl.recvbase[p] + wl.rdispls[p, origin]) * E
+
+    # where every rank keeps the block of slot (io, jo): at first in its send region
+    loc = {}
+    for p in range(P):
+        for io in range(N):
+            for jo in range(Q):
+                dest = ((n_of[p] + io) % N) * Q + (q_of[p] + jo) % Q
+                loc[p, io, jo] = int(wl.sendbase[p] + wl.sdispls[p, dest]) * E
+    work_off = 0
+    for f in range(wloc + wglo):
+        level, x = (0, f) if f < wloc else (1, f - wloc)
+        if level == 0:
+            moving = [jo for jo in range(Q) if _digit(jo, rl, x) != 0]
+            row = [(io, jo) for io in range(N) for jo in moving]
+            arrived = [(0, jo) for jo in moving if jo < rl ** (x + 1)]       # own group, no digit above x
+            # the oracle's table is by destination group; a slot names the group offset
+            size = lambda p, io, jo: sz_local[x, p, (n_of[p] + io) % N, jo]
+            sender = lambda p, io, jo: n_of[p] * Q + (q_of[p] - _digit(jo, rl, x) * rl ** x) % Q
+        else:
+            moving = [io for io in range(N) if _digit(io, rg, x) != 0]
+            row = [(io, jo) for io in moving for jo in range(Q)]
+            arrived = [(io, jo) for io in moving if io < rg ** (x + 1) for jo in range(Q)]
+            # a super-block's parts are listed by source local id q' = q - jo
+            size = lambda p, io, jo: usz_global[x, p, io, (q_of[p] - jo) % Q]
+            sender = lambda p, io, jo: ((n_of[p] - _digit(io, rg, x) * rg ** x) % N) * Q + q_of[p]
+        assert row[:len(arrived)] == arrived                                # the arrived ones come first
+        onward = row[len(arrived):]
+        new_loc = {}
+        for part, slots in ((B.PART_KEEP, onward), (B.PART_DELIVER, arrived)):
+            t = plan.phase_tables(f, part)
+            m = len(slots)
+            exp_len = np.array([[size(p, io, jo) for io, jo in slots] for p in range(P)], dtype=np.int64).reshape(P, m)
+            assert np.array_equal(t["len"].reshape(P, m), exp_len)
+            if level == 1 and x == 0:
+                # what the first global phase gathers is what the compaction laid out at the sender
+                comp = np.array([[usz_compact[sender(p, io, jo), io, (q_of[p] - jo) % Q] for io, jo in slots]
+                                 for p in range(P)], dtype=np.int64).reshape(P, m)
+                assert np.array_equal(exp_len, comp)
+            spaced = (exp_len + 15) // 16 * 16 + (16 * (exp_len > 0) if part == B.PART_DELIVER else 0)
+            scan, tot = oracle.segmented_exclusive_scan(spaced, 1)
+            base, _ = oracle.segmented_exclusive_scan(tot.reshape(1, P), 1)
+            exp_pos = scan + base.reshape(P, 1)
+            assert np.array_equal(t["pos"].reshape(P, m), exp_pos)
+            info = plan.phase_info(f, part)
+            assert info["bytes"] == exp_len.sum() and info["level"] == level and info["x"] == x
+            src, dst = t["src"].reshape(P, m), t["dst"].reshape(P, m)
+            for p in range(P):
+                for j, (io, jo) in enumerate(slots):
+                    assert src[p, j] == loc[sender(p, io, jo), io, jo]
+                    if part == B.PART_KEEP:
+                        assert dst[p, j] == (2 << 56) | (work_off + int(exp_pos[p, j]))
+                    else:
+                        origin = ((n_of[p] - io) % N) * Q + (q_of[p] - jo) % Q
+                        assert dst[p, j] == recv_loc(p, origin)
+                    new_loc[p, io, jo] = int(dst[p, j])
+            if part == B.PART_KEEP:
+                assert info["stream_bytes"] == tot.sum()
+                work_off += (int(tot.sum()) + 255) // 256 * 256
+        loc.update(new_loc)
+    assert plan.workspace_bytes() == work_off
+    # at the end every block but the self blocks sits at its place in the receive buffer
+    for p in range(P):
+        for io in range(N):
+            for jo in range(Q):
+                if io or jo:
+                    assert loc[p, io, jo] == recv_loc(p, ((n_of[p] - io) % N) * Q + (q_of[p] - jo) % Q)
+
+
+def test_radix_zero_chooses_one_hop_per_level():
+    wl = W.make_random(12, 100, elem_size=2, seed=5, zero_frac=0.2, gaps=True)
+    ref = oracle_brute(wl)
+    got, plan = gpu_run(wl, 0)
+    assert np.array_equal(got, ref) and plan.num_phases() == 1 and plan.num_rounds() == 11
+    got, plan = gpu_run(wl, 0, l=4, g=3, rg=0)
+    assert np.array_equal(got, ref) and plan.num_phases() == 2 and plan.num_rounds() == 3 + 2
+
 
 def test_packed_layout_defaults_match_explicit():
     """NULL displacement arrays mean 'packed'; the device-side scans must give
@@ -635,10 +736,15 @@ def test_c3_full(rl, rg):
     check_rounds(plan, rounds)
 
 
-def test_c4_scaled_down():
+@pytest.mark.parametrize("skew", [False, True])
+def test_c4_scaled_down(skew):
     """The token-dispatch shape with fewer tokens and a narrower hidden size, so
-    that the oracle finishes in seconds; blocks still span many chunks."""
-    wl = W.make_c4(P=64, tokens=256, hidden=512)
+    that the oracle finishes in seconds; blocks still span many chunks.  ``skew``:
+    one bias per destination shared by all ranks, so a few experts draw most tokens."""
+    wl = W.make_c4(P=64, tokens=256, hidden=512, skew=skew)
+    if skew:
+        col = wl.sendcounts.sum(axis=0)
+        assert col.max() > 4 * np.median(col)                 # the hot experts really are hot
     for r in (2, 8, 64):
         ref, rounds, _, _ = oracle_flat(wl, r)
         got, plan = gpu_run(wl, r)
@@ -676,22 +782,81 @@ def _block_sums(buf_words, base, displs, counts, elem_words):
     return cs[end] - cs[start]
 
 
-@pytest.mark.parametrize("schedule", ["r64", "r2", "r8_classic", "direct"])
+def _host_memory_available():
+    """Bytes of host memory this process may still take (the smaller of what the
+    machine has free and what its control group allows)."""
+    import psutil
+    avail = psutil.virtual_memory().available
+    for limit, used in (("/sys/fs/cgroup/memory.max", "/sys/fs/cgroup/memory.current"),
+                        ("/sys/fs/cgroup/memory/memory.limit_in_bytes",
+                         "/sys/fs/cgroup/memory/memory.usage_in_bytes")):
+        try:
+            lim = open(limit).read().strip()
+            if lim != "max":
+                avail = min(avail, int(lim) - int(open(used).read().strip()))
+        except (OSError, ValueError):
+            pass
+    return avail
+
+
+def _equal_in_slices(dev, host, step=1 << 28):
+    """Device tensor against a host array of the same bytes, a slice at a time."""
+    for a in range(0, dev.numel(), step):
+        b = min(a + step, dev.numel())
+        if not np.array_equal(dev[a:b].cpu().numpy(), host[a:b]):
+            return False
+    return True
+
+
+def test_c4_full_size_against_the_oracle():
+    """The 8 GiB token-dispatch shape, every byte: the receive buffer of the radix-64
+    schedule (the configuration the benchmark times) and of the direct exchange against
+    the oracle's definition of the exchange on the same send buffer, and the schedule's
+    per-round table against the oracle's radix-64 run."""
+    free, _ = torch.cuda.mem_get_info()
+    if free < 20 * 2**30:
+        pytest.skip("needs about 20 GiB of free device memory")
+    if _host_memory_available() < 30 * 2**30:
+        pytest.skip("needs about 30 GiB of host memory for the oracle's buffers")
+    wl = W.make_c4()
+    assert wl.payload_bytes_total == 8 * 2**30
+    send = wl.make_send("cuda")
+    send_h = send.cpu().numpy()
+    ref = np.full(wl.recv_bytes, CANARY, dtype=np.uint8)
+    oracle.bruteforce(wl, send_h, ref)
+    plan = B.plan_for(wl, 64)
+    plan.alloc_workspace()
+    recv = wl.make_recv("cuda", fill=CANARY)
+    plan.alltoallv(send, recv)
+    torch.cuda.synchronize()
+    assert _equal_in_slices(recv, ref)
+    recv.fill_(CANARY)
+    plan.direct_alltoallv(send, recv)
+    torch.cuda.synchronize()
+    assert _equal_in_slices(recv, ref)
+    del recv
+    flat = np.full(wl.recv_bytes, CANARY, dtype=np.uint8)
+    _, rounds, _, _ = oracle.tuna_flat(wl, 64, send_h, flat)
+    assert np.array_equal(flat, ref)
+    check_rounds(plan, rounds)
+
+
+@pytest.mark.parametrize("schedule", ["r64", "r2", "r8_classic", "direct", "skew_r64", "skew_r2"])
 def test_c4_full_size(schedule):
     """The 8 GiB token-dispatch shape in the configuration the benchmark times.
-    The oracle cannot run it in seconds, so the check is (a) sampled received bytes
+    The oracle runs this size once, in a test of its own, so here the check is (a) sampled received bytes
     against the definition of the exchange applied to the generator, and (b) a
     property that holds at any size: every one of the P^2 received blocks has the
     same 64-bit word sum as the block that was sent."""
     free, _ = torch.cuda.mem_get_info()
     if free < 70 * 2**30:
         pytest.skip("needs about 70 GiB of free device memory")
-    wl = W.make_c4()
+    wl = W.make_c4(skew=schedule.startswith("skew"))
     assert wl.payload_bytes_total == 8 * 2**30
     send = wl.make_send("cuda")
     recv = wl.make_recv("cuda", fill=CANARY)
     kw = dict(r64=dict(radix=64), r2=dict(radix=2), r8_classic=dict(radix=8, flags=B.FLAG_CLASSIC_ROTATE),
-              direct=dict(radix=64))[schedule]
+              direct=dict(radix=64), skew_r64=dict(radix=64), skew_r2=dict(radix=2))[schedule]
     plan = B.plan_for(wl, **kw)
     plan.alloc_workspace()
     if schedule == "direct":
@@ -702,8 +867,9 @@ def test_c4_full_size(schedule):
     # (a) samples
     rng = np.random.default_rng(2024)
     n = 1 << 20
-    s = rng.integers(0, wl.P, n)
-    d = rng.integers(0, wl.P, n)
+    pairs = np.argwhere(wl.sendcounts > 0)                    # (the skewed routing leaves some pairs empty)
+    pick = pairs[rng.integers(0, len(pairs), n)]
+    s, d = pick[:, 0], pick[:, 1]
     k = (rng.random(n) * (wl.sendcounts[s, d] * wl.elem_size)).astype(np.int64)
     src = torch.from_numpy((wl.sendbase[s] + wl.sdispls[s, d]) * wl.elem_size + k).cuda()
     dst = torch.from_numpy((wl.recvbase[d] + wl.rdispls[d, s]) * wl.elem_size + k).cuda()

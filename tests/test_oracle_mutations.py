@@ -34,6 +34,9 @@ MUTATIONS = [
      "int from = (int)(((n - dist) % N + N) % N) * Q + q;", "int from = (int)((n + dist) % N) * Q + q;"),
     ("hier_own_group_blocks_kept_in_T",
      "if (local_final && i == n) {", "if (0) {"),
+    ("compaction_lists_parts_by_local_offset",   # Sec. IV-B: parts in ascending source local id
+     "        int64_t nb = sz[(int64_t)p * P + i * Q + jo];\n        usz[((int64_t)p * N + io) * Q + qs] = nb;",
+     "        int64_t nb = sz[(int64_t)p * P + i * Q + jo];\n        usz[((int64_t)p * N + io) * Q + jo] = nb;"),
     ("staggered_sends_the_wrong_way",
      "          int ndst = ((n - gi) % N + N) % N;\n          if (ndst == n) continue;\n          active = 1;",
      "          int ndst = (n + gi) % N;\n          if (ndst == n) continue;\n          active = 1;"),

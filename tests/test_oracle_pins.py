@@ -452,6 +452,65 @@ def test_size_tables_follow_the_blocks(P, r):
                 assert sizes[x, p, o] == C[s, (s + o) % P]
 
 
+@pytest.mark.parametrize("Q,N,rl,rg", [(5, 3, 2, 3), (4, 4, 2, 2), (3, 4, 3, 2), (6, 5, 2, 3), (8, 4, 8, 4), (1, 5, 2, 2), (5, 1, 2, 2)])
+def test_hier_size_tables_follow_the_blocks(Q, N, rl, rg):
+    """The metadata the hierarchical schedule holds, by closed form.  After the local
+    rounds of digit x the block rank (n, q) holds for rank (i, q + jo) has come from the
+    rank (jo mod rl^(x+1)) local places below; the compaction (Sec. IV-B) lists, for every
+    group offset, the parts in ascending source local id; after the global rounds of digit
+    x a super-block has come (io mod rg^(x+1)) groups; and after the local phase R holds
+    the own group's blocks and nothing else (Fig. 5)."""
+    P = Q * N
+    wl = W.make_random(P, 23, elem_size=3, seed=11 * P + rl + rg, zero_frac=0.25, gaps=True)
+    send = wl.make_send().numpy()
+    recv = wl.make_recv(fill=CANARY).numpy().copy()
+    recv, after, sz_local, usz_compact, usz_global = oracle.tuna_hier_tables(wl, Q, N, rl, rg, send, recv)
+    ref = brute(wl)
+    assert np.array_equal(recv, ref)
+    C = wl.sendcounts * wl.elem_size
+    assert sz_local.shape[0] == oracle.num_digits(Q, rl) and usz_global.shape[0] == oracle.num_digits(N, rg)
+    for x in range(sz_local.shape[0]):
+        for p in range(P):
+            n, q = divmod(p, Q)
+            for i in range(N):
+                for jo in range(Q):
+                    qs = (q - jo % rl ** (x + 1)) % Q
+                    assert sz_local[x, p, i, jo] == C[n * Q + qs, i * Q + (qs + jo) % Q]
+    for p in range(P):
+        n, q = divmod(p, Q)
+        assert not usz_compact[p, 0].any()                      # the own group's blocks are not compacted
+        for io in range(1, N):
+            for qs in range(Q):
+                assert usz_compact[p, io, qs] == C[n * Q + qs, ((n + io) % N) * Q + q]
+    for x in range(usz_global.shape[0]):
+        for p in range(P):
+            n, q = divmod(p, Q)
+            for io in range(1, N):
+                n0 = (n - io % rg ** (x + 1)) % N
+                for qs in range(Q):
+                    assert usz_global[x, p, io, qs] == C[n0 * Q + qs, ((n0 + io) % N) * Q + q]
+    own = np.zeros(wl.recv_bytes, dtype=bool)
+    for d in range(P):
+        for s_ in range(P):
+            if s_ // Q == d // Q:
+                o = int(wl.recvbase[d] + wl.rdispls[d, s_]) * wl.elem_size
+                own[o:o + int(C[s_, d])] = True
+    assert np.array_equal(after[own], ref[own]) and np.all(after[~own] == CANARY)
+
+
+@pytest.mark.parametrize("P,r,threads", [(1, 2, 1), (2, 2, 2), (8, 2, 3), (9, 3, 4), (13, 2, 13), (20, 5, 7), (12, 12, 5),
+                                         (33, 6, 8), (64, 64, 16)])
+def test_threaded_timing_variant_matches_the_checker(P, r, threads):
+    """The threaded variant of the flat schedule exists only to be timed; it must write the
+    same bytes (canary gaps included) and count the same rounds as the single-threaded oracle."""
+    wl = W.make_random(P, 700, elem_size=3, seed=3 * P + r, zero_frac=0.25, gaps=True)
+    send, recv, rounds, _, _ = run_flat(wl, r)
+    got = wl.make_recv(fill=CANARY).numpy().copy()
+    got, rounds_mt = oracle.tuna_flat_mt(wl, r, send, got, threads)
+    assert np.array_equal(got, recv)
+    assert np.array_equal(rounds_mt, rounds)
+
+
 def test_segmented_scan_against_numpy():
     rng = np.random.default_rng(5)
     for nseg, seglen, align in [(1, 1, 1), (3, 7, 1), (5, 33, 16), (64, 64, 16), (2, 100, 4)]:
