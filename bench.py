@@ -30,17 +30,13 @@ if ROOT not in sys.path:
 METRIC = "alltoallv_payload_throughput"
 UNIT = "GB/s"
 
-# DRAM traffic of the dominant kernel from ncu captures
+# DRAM traffic of the dominant kernel from ncu captures of it
 # (dram__bytes_read.sum + dram__bytes_write.sum per launch) divided by the payload
 # bytes that launch moved, keyed by the SHA-256 of the kernel source the capture
-# was taken with, then by workload (at its default radix).  Traffic grows in
-# proportion to the bytes moved, so the full-size figure is this ratio times the
-# launch's bytes.  A changed source makes the figures stale: the traffic is then
-# reported as null.  Captures: profiles/round_kernel_c4_reduced.md (c4, reduced to
-# 2 GiB), profiles/round_small_kernel_c5.md (c5 at full size) and
-# profiles/round_small_kernel_c3.md (c3 at full size, both launches of an exchange).
+# was taken with, then by "workload/schedule".  Traffic grows in proportion to the
+# bytes moved, so the full-size figure is this ratio times the launch's bytes.  A
+# changed source makes the figures stale: the traffic is then reported as null.
 NCU_TRAFFIC_PER_PAYLOAD_BYTE: dict[str, dict[str, float]] = {
-    "40d1ef79ac5a7db5d7f95e0971c78d65d8717af48a8ce3359f2843065c9199a2": {"c4": 1.995, "c5": 2.151, "c3": 1.543},
 }
 
 
@@ -55,6 +51,8 @@ def parse_args():
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-small-blocks", action="store_true",
+                    help="skip the secondary entries that time the small-block build (c5, c3)")
     ap.add_argument("--sweep-steps", type=int, default=10)
     ap.add_argument("--tokens", type=int, default=0,
                     help="c4 only: tokens per rank (default 8192); smaller values give the "
@@ -192,16 +190,133 @@ def default_radix(wl, radix):
     return max(wl.radices) if wl.radices else 0
 
 
-def run_oracle_once(wl, radix, send, recv):
+def configure_host_allocator():
+    """Pins down glibc's allocator for the oracle's timing (harness only; the oracle's
+    arithmetic is untouched).  The oracle mallocs and frees every message of every
+    round.  Left alone, glibc serves requests above a threshold by mmap (fresh,
+    page-faulting memory every time) and moves that threshold whenever a large chunk
+    is freed, so the same run measured 2.2 GB/s in a fresh process and 5.3 GB/s in one
+    that had freed large arrays before.  With the threshold at its maximum and the heap
+    never trimmed, messages up to 32 MiB reuse warm heap memory in every process."""
+    import ctypes
+    try:
+        libc = ctypes.CDLL("libc.so.6")
+        M_TRIM_THRESHOLD, M_MMAP_THRESHOLD = -1, -3
+        ok1 = libc.mallopt(M_MMAP_THRESHOLD, 32 << 20)
+        ok2 = libc.mallopt(M_TRIM_THRESHOLD, 1 << 30)
+        return bool(ok1 and ok2)
+    except Exception:
+        return False
+
+
+def cpu_model():
+    try:
+        with open("/proc/cpuinfo") as f:
+            for line in f:
+                if line.lower().startswith("model name"):
+                    return line.split(":", 1)[1].strip()
+    except OSError:
+        pass
+    import platform
+    return platform.processor() or platform.machine()
+
+
+def usable_cores():
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:
+        return os.cpu_count() or 1
+
+
+def host_memory_available():
+    import psutil
+    avail = psutil.virtual_memory().available
+    for limit, used in (("/sys/fs/cgroup/memory.max", "/sys/fs/cgroup/memory.current"),
+                        ("/sys/fs/cgroup/memory/memory.limit_in_bytes",
+                         "/sys/fs/cgroup/memory/memory.usage_in_bytes")):
+        try:
+            lim = open(limit).read().strip()
+            if lim != "max":
+                avail = min(avail, int(lim) - int(open(used).read().strip()))
+        except (OSError, ValueError):
+            pass
+    return avail
+
+
+def run_oracle_once(wl, radix, send, recv, threads=1):
+    """One run of the oracle's schedule (the workload's headline one); seconds."""
     import oracle
     t0 = time.perf_counter()
     if wl.hier and not wl.radices:
         l, g = wl.hier
         rl, rg = wl.hier_radices[-1]
         oracle.tuna_hier(wl, l, g, rl, rg, send, recv)
+    elif threads > 1:
+        oracle.tuna_flat_mt(wl, radix, send, recv, threads)   # timing variant, checked against the oracle by a test
     else:
         oracle.tuna_flat(wl, radix, send, recv)
     return time.perf_counter() - t0
+
+
+def run_bruteforce_once(wl, send, recv):
+    import oracle
+    t0 = time.perf_counter()
+    oracle.bruteforce(wl, send, recv)
+    return time.perf_counter() - t0
+
+
+def cpu_baseline_block(wl_name, radix_arg, full_send=None, full_wl=None, runs=5):
+    """The oracle, as it stands, on the host cores: the definition of the exchange (the
+    CPU's own direct exchange), the headline schedule on one thread and, for flat
+    schedules, the same steps with the ranks shared out over all cores; on a bounded
+    sample of the workload, and once at full size when the host has the memory."""
+    import numpy as np
+    pinned = configure_host_allocator()
+    cores = usable_cores()
+    wls, sample = oracle_sample_workload(wl_name, 8.0)
+    hs = wls.make_send().numpy()
+    hr = np.empty(max(wls.recv_bytes, 1), dtype=np.uint8)[:wls.recv_bytes]
+    r = default_radix(wls, radix_arg)
+    pay = wls.payload_bytes_total
+    flat = not (wls.hier and not wls.radices)
+    first = run_oracle_once(wls, r, hs, hr)                       # first touch of every buffer
+    one = [run_oracle_once(wls, r, hs, hr) for _ in range(runs)]
+    brute = [run_bruteforce_once(wls, hs, hr) for _ in range(runs)]
+    block = {"value": pay / statistics.median(one) / 1e9, "unit": UNIT, "cores": 1, "threads": 1,
+             "kind": "oracle", "sample": sample + f", median of {runs} runs after one warm-up run",
+             "first_run_GBps": pay / first / 1e9,
+             "bruteforce_GBps": pay / statistics.median(brute) / 1e9,
+             "cpu_model": cpu_model(), "host_cores_available": cores,
+             "allocator_pinned": pinned}
+    if flat and cores > 1:
+        run_oracle_once(wls, r, hs, hr, threads=cores)
+        many = [run_oracle_once(wls, r, hs, hr, threads=cores) for _ in range(runs)]
+        block["all_cores"] = {"value": pay / statistics.median(many) / 1e9, "unit": UNIT, "threads": min(cores, wls.P),
+                              "kind": "threaded timing variant of the oracle's flat schedule "
+                                      "(ranks of a round shared out over plain threads)"}
+    else:
+        block["all_cores"] = None
+    del hs, hr
+    # once at full size (the oracle's buffers need twice the payload in host memory)
+    if full_wl is not None and full_wl.payload_bytes_total > pay:
+        need = 2 * full_wl.payload_bytes_total + (4 << 30)
+        if host_memory_available() < need:
+            block["full_size"] = {"skipped": f"needs {need >> 30} GiB of host memory"}
+        else:
+            fs = full_send.cpu().numpy() if full_send is not None else full_wl.make_send().numpy()
+            fr = np.empty(full_wl.recv_bytes, dtype=np.uint8)
+            fpay = full_wl.payload_bytes_total
+            rf = default_radix(full_wl, radix_arg)
+            tb = run_bruteforce_once(full_wl, fs, fr)
+            t1 = run_oracle_once(full_wl, rf, fs, fr)
+            full = {"payload_bytes": fpay, "runs": 1, "bruteforce_GBps": fpay / tb / 1e9,
+                    "oracle_GBps": fpay / t1 / 1e9, "threads": 1}
+            if flat and cores > 1:
+                tm = run_oracle_once(full_wl, rf, fs, fr, threads=cores)
+                full["oracle_all_cores_GBps"] = fpay / tm / 1e9
+            block["full_size"] = full
+            del fs, fr
+    return block
 
 
 def reference_arm(args):
@@ -209,23 +324,28 @@ def reference_arm(args):
     if int(os.environ.get("RANK", "0")) != 0:
         return
     import numpy as np
-    budget = max(0.5, min(10.0, 150.0 / max(1, args.steps + args.warmup)))
-    wl, sample = oracle_sample_workload(args.workload, budget)
+    configure_host_allocator()
+    wl, sample = oracle_sample_workload(args.workload, 8.0)
     radix = default_radix(wl, args.radix)
     send = wl.make_send().numpy()
     recv = np.empty(max(wl.recv_bytes, 1), dtype=np.uint8)[:wl.recv_bytes]
-    for _ in range(args.warmup):
+    for _ in range(max(1, args.warmup)):
         run_oracle_once(wl, radix, send, recv)
     t = [run_oracle_once(wl, radix, send, recv) for _ in range(args.steps)]
     total = sum(t)
     value = wl.payload_bytes_total * args.steps / total / 1e9
+    sched = (f"hierarchical {wl.hier[0]}x{wl.hier[1]} radix {wl.hier_radices[-1][0]}/{wl.hier_radices[-1][1]}"
+             if wl.hier and not wl.radices else f"flat radix {radix}")
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u8",
         "data": "synthetic",
-        "config": {"workload": f"{wl.name} P={wl.P} flat radix {radix}", "sample": sample},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "config": {"workload": f"{wl.name} P={wl.P} {sched}", "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "threads": 1, "kind": "oracle",
+                         "sample": sample, "cpu_model": cpu_model(),
+                         "host_cores_available": usable_cores(),
+                         "median_GBps": wl.payload_bytes_total / statistics.median(t) / 1e9},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
     print(json.dumps(line), flush=True)
@@ -307,7 +427,8 @@ def token_dispatch_entry(wl, args, send, recv, payload):
     return {"schedule": "token dispatch in one pass: gather + exchange + scatter (rows)",
             "ms_per_step": ms, "payload_GBps": payload / ms / 1e6, "exchange_only_ms": ms_x,
             "rounds": 1, "launches": 1, "moved_over_payload": 1.0,
-            "effective_hbm_GBps": 2 * payload / ms_x / 1e6, "workspace_bytes": 0,
+            "effective_hbm_GBps": 2 * payload / ms_x / 1e6, "frac": 2 * payload / ms_x / 1e6 / measured_peaks()[0],
+            "workspace_bytes": 0,
             "three_passes_exchange_only_ms": ms_3, "matches_three_passes": same}
 
 
@@ -330,6 +451,62 @@ def verify_samples(wl, recv, n=4096):
     want = W.payload_byte_at(wl.seed, torch.from_numpy(src))
     got = recv[torch.from_numpy(dst).to(recv.device)].cpu()
     return bool(torch.equal(want, got))
+
+
+def small_block_entries(dev, peak, peak_kind, steps=20, warmup=3):
+    """Exchange-only timing of the schedules whose launches run the small-block build:
+    c5 (P = 2048, 179-byte unaligned blocks) in one hop and at radix 2, c3 (16 x 16
+    ranks, Zipf-sized blocks) at radix 16/16.  Per entry a roofline of its own: 2 x bytes
+    moved by the timed launches over their CUDA-event time (events inside the library,
+    around every launch)."""
+    import torch
+    from paper_2411_02581_b200 import binding as B, workloads as W
+    out = []
+    sha = kernel_source_sha()
+    for name, make, kw, label in (
+            ("c5", W.make_c5, dict(radix=2048), "flat radix 2048"),
+            ("c5", W.make_c5, dict(radix=2), "flat radix 2"),
+            ("c3", W.make_c3, dict(radix=16, l=16, g=16, radix_global=16), "hierarchical l=16 g=16 radix 16/16")):
+        wl = make()
+        send = wl.make_send(dev)
+        recv = wl.make_recv(dev)
+        plan = B.plan_for(wl, explicit_layout=False, flags=B.FLAG_NO_DIRECT, **kw)
+        plan.alloc_workspace(device=dev)
+        for _ in range(warmup):
+            plan.alltoallv(send, recv)
+        torch.cuda.synchronize()
+        ok = verify_samples(wl, recv)
+        plan.enable_timing(True)
+        plan.get_timing(reset=True)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(steps):
+            plan.alltoallv(send, recv)
+        b.record()
+        torch.cuda.synchronize()
+        t = plan.get_timing(reset=True)
+        plan.enable_timing(False)
+        ms = t["round_local"]["ms"] + t["round_global"]["ms"]
+        ln = t["round_local"]["launches"] + t["round_global"]["launches"]
+        by = t["round_local"]["bytes"] + t["round_global"]["bytes"]
+        ach = 2.0 * by / (ms * 1e-3) / 1e9 if ms > 0 else 0.0
+        n_small, n_all = plan.last_small_launches(), plan.last_launches()
+        per_byte = NCU_TRAFFIC_PER_PAYLOAD_BYTE.get(sha, {}).get(f"{name}/{label}")
+        out.append({"workload": f"{name} P={wl.P} {label}", "payload_bytes": wl.payload_bytes_total,
+                    "exchange_ms": a.elapsed_time(b) / steps, "steps": steps, "parity_samples_ok": ok,
+                    "roofline": {"bound": "hbm",
+                                 "kernel": "tuna_round_small_kernel" if n_small == n_all else
+                                           "tuna_round_kernel" if n_small == 0 else "both builds",
+                                 "achieved": ach, "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
+                                 "frac": ach / peak, "frac_of_nominal_8000": ach / 8000.0,
+                                 "traffic": per_byte * by / ln if per_byte and ln else None,
+                                 "algorithmic_bytes_per_launch": 2.0 * by / ln if ln else 0,
+                                 "avg_launch_ms": ms / ln if ln else None, "launches": ln}})
+        plan.set_workspace(None)
+        plan.destroy()
+        del send, recv
+        torch.cuda.empty_cache()
+    return out
 
 
 def ours_arm(args):
@@ -425,13 +602,14 @@ def ours_arm(args):
     # roofline of the dominant kernel: the fused pack-move-unpack kernel, one launch
     # per digit phase
     peak, peak_kind = measured_peaks()
-    kname = "tuna_round_kernel"
+    n_small, n_all = plan.last_small_launches(), plan.last_launches()
+    kname = ("tuna_round_small_kernel" if n_small == n_all else "tuna_round_kernel" if n_small == 0
+             else f"tuna_round_kernel ({n_all - n_small} launches) + tuna_round_small_kernel ({n_small})")
     rk_ms = timing["round_local"]["ms"] + timing["round_global"]["ms"]
     rk_launches = timing["round_local"]["launches"] + timing["round_global"]["launches"]
     rk_bytes = timing["round_local"]["bytes"] + timing["round_global"]["bytes"]
     achieved = 2.0 * rk_bytes / (rk_ms * 1e-3) / 1e9 if rk_ms > 0 else 0.0
-    per_byte = NCU_TRAFFIC_PER_PAYLOAD_BYTE.get(kernel_source_sha(), {}).get(wl.name) \
-        if not args.radix else None
+    per_byte = NCU_TRAFFIC_PER_PAYLOAD_BYTE.get(kernel_source_sha(), {}).get(f"{wl.name}/{sched}")
     roofline = {
         "bound": "hbm", "kernel": kname, "achieved": achieved, "peak": peak,
         "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,
@@ -517,6 +695,8 @@ def ours_arm(args):
                           "launches": p.last_launches(),
                           "moved_over_payload": moved / max(payload, 1),
                           "effective_hbm_GBps": 2 * moved / ms_x / 1e6,
+                          "frac": 2 * moved / ms_x / 1e6 / peak,
+                          "small_build_launches": p.last_small_launches(),
                           "workspace_bytes": 0 if direct else p.workspace_bytes()})
             p.set_workspace(None)
             p.destroy()
@@ -569,6 +749,7 @@ def ours_arm(args):
             sweep.append({"schedule": f"flat r={radix}, two plans taking turns (re-plan of the next batch "
                                       "beside the exchange; wall clock)",
                           "ms_per_step": ms, "payload_GBps": payload / ms / 1e6,
+                          "frac": None,
                           "launches": pair[0].last_launches()})
             for p in pair:
                 p.set_workspace(None)
@@ -578,17 +759,18 @@ def ours_arm(args):
         if args.workload in ("c4", "c4_skew"):
             sweep.append(token_dispatch_entry(wl, args, send, recv, payload))
 
+    # the small-block build of the mover under the same clock: the all-unaligned single
+    # hop and the radix-2 schedule on c5-sized blocks, and the short launches of c3
+    small = None
+    if rank == 0 and not args.no_small_blocks and args.workload == "c4":
+        small = small_block_entries(dev, peak, peak_kind)
+
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         import oracle  # noqa: F401  (the CPU-baseline leg is the one place bench.py runs the oracle)
-        wls, sample = oracle_sample_workload(args.workload, 8.0)
-        hs = wls.make_send().numpy()
-        hr = np.empty(max(wls.recv_bytes, 1), dtype=np.uint8)[:wls.recv_bytes]
-        r = default_radix(wls, args.radix)
-        times = [run_oracle_once(wls, r, hs, hr) for _ in range(3)]
-        cpu = {"value": wls.payload_bytes_total / statistics.median(times) / 1e9, "unit": UNIT,
-               "cores": 1, "kind": "oracle", "sample": sample + ", median of 3 runs",
-               "host_cores_available": os.cpu_count()}
+        full = None if args.tokens else wl
+        cpu = cpu_baseline_block(args.workload, args.radix, full_send=send if full is not None else None,
+                                 full_wl=full)
 
     if rank == 0:
         line = {
@@ -602,7 +784,7 @@ def ours_arm(args):
                        "replicas": "one independent exchange per GPU" if world > 1 else "single GPU"},
             "gpu_launches": int(launches), "parity_samples_ok": ok,
             "clocks": clocks.summary(), "e2e": e2e, "roofline": roofline,
-            "cpu_baseline": cpu, "step_ms": step_ms, "replan_ms": replan, "sweep": sweep,
+            "cpu_baseline": cpu, "small_blocks": small, "step_ms": step_ms, "replan_ms": replan, "sweep": sweep,
         }
         print(json.dumps(line), flush=True)
     if dist:

@@ -373,9 +373,13 @@ int tuna_plan_phase_info(const tuna_plan_t *plan, int phase, int part, int *leve
 int tuna_plan_phase_tables(const tuna_plan_t *plan, int phase, int part, int64_t cap, int64_t *len,
                            int64_t *pos, int64_t *src, int64_t *dst, int64_t *rows);
 
-/* Kernels launched by the last exchange call on this plan (host counter), and by
- * every call on this plan since its creation, plan kernels included. */
+/* Kernels launched by the last exchange call on this plan (host counter); how many
+ * of them ran the small-block build of the mover (kernel names ending in
+ * _small_kernel: the build for lists of tiny, mostly skewed or cache-resident
+ * blocks) rather than the large-block build; and the kernels launched by every call
+ * on this plan since its creation, plan kernels included. */
 int tuna_plan_last_launches(const tuna_plan_t *plan, int *launches);
+int tuna_plan_last_small_launches(const tuna_plan_t *plan, int *launches);
 int tuna_plan_launch_count(const tuna_plan_t *plan, int64_t *launches);
 
 /*

@@ -62,6 +62,7 @@ SIGNATURES = {
     "tuna_plan_phase_info": (ctypes.c_int, [_VP, ctypes.c_int, ctypes.c_int, _INTP, _INTP, _I64P, _I64P, _I64P]),
     "tuna_plan_phase_tables": (ctypes.c_int, [_VP, ctypes.c_int, ctypes.c_int, ctypes.c_int64] + [_I64P] * 5),
     "tuna_plan_last_launches": (ctypes.c_int, [_VP, _INTP]),
+    "tuna_plan_last_small_launches": (ctypes.c_int, [_VP, _INTP]),
     "tuna_plan_launch_count": (ctypes.c_int, [_VP, _I64P]),
     "tuna_plan_enable_timing": (ctypes.c_int, [_VP, ctypes.c_int]),
     "tuna_plan_get_timing": (ctypes.c_int, [_VP, ctypes.c_int, ctypes.POINTER(ctypes.c_double), _I64P, _I64P]),
@@ -283,7 +284,11 @@ class Plan:
         n = ctypes.c_int()
         self._check(lib().tuna_plan_last_launches(self._h, ctypes.byref(n)), "tuna_plan_last_launches")
         return n.value
-
+    def last_small_launches(self) -> int:
+        n = ctypes.c_int()
+        self._check(lib().tuna_plan_last_small_launches(self._h, ctypes.byref(n)),
+                    "tuna_plan_last_small_launches")
+        return n.value
 
     def device_status(self) -> int:
         """0, or 1 if a kernel of this plan gave up a bounded wait (synchronises the device)."""

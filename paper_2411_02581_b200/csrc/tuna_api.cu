@@ -92,7 +92,7 @@ int run_tuna(tuna_plan *pl, const void *send, void *recv, cudaStream_t st) {
   if (pl->workspace_need > 0 &&
       (!pl->workspace || pl->workspace_bytes < (size_t)pl->workspace_need))
     return TUNA_ERR_WORKSPACE;
-  int launches = 0;
+  int launches = 0, smalls = 0;
   bool rot_done = pl->rot.nchunks == 0;
   for (size_t f = 0; f < pl->phases.size(); f++) {
     const int kind = pl->phases[f].level == 0 ? TUNA_TIMER_ROUND_LOCAL : TUNA_TIMER_ROUND_GLOBAL;
@@ -117,6 +117,7 @@ int run_tuna(tuna_plan *pl, const void *send, void *recv, cudaStream_t st) {
     Timed tm(pl, kind, bytes, st);
     TUNA_CUDA(pl, tuna_launch_move(TUNA_K_ROUND, a, small, launches > 0, st));
     launches++;
+    smalls += small ? 1 : 0;
   }
   if (!rot_done) {
     Timed tm(pl, TUNA_TIMER_ROTATE, pl->rot.bytes, st);
@@ -124,7 +125,9 @@ int run_tuna(tuna_plan *pl, const void *send, void *recv, cudaStream_t st) {
     a.rot = list_args(pl->rot);
     TUNA_CUDA(pl, tuna_launch_move(TUNA_K_ROTATE, a, pl->rot.small_blocks, launches > 0, st));
     launches++;
+    smalls += pl->rot.small_blocks ? 1 : 0;
   }
+  pl->last_small = smalls;
   pl->last_launches = launches;
   pl->launch_count += launches;
   return launches > 0 ? mark_in_flight(pl, st) : TUNA_OK;
@@ -137,6 +140,7 @@ int run_direct(tuna_plan *pl, const void *send, void *recv, cudaStream_t st) {
     if (arc) return arc;
   }
   int launches = 0;
+  pl->last_small = 0;
   if (pl->dir_shared) {  // the single phase's DELIVER list and the self blocks: every block, once
     const TunaList &d = pl->deliver[0];
     if (d.nchunks > 0 || pl->rot.nchunks > 0) {
@@ -148,6 +152,7 @@ int run_direct(tuna_plan *pl, const void *send, void *recv, cudaStream_t st) {
       a.rot = list_args(pl->rot);
       TUNA_CUDA(pl, tuna_launch_move(TUNA_K_DIRECT, a, 2 * small_bytes >= bytes, false, st));
       launches++;
+      pl->last_small = 2 * small_bytes >= bytes ? 1 : 0;
     }
   } else if (pl->dir.nchunks > 0) {
     Timed tm(pl, TUNA_TIMER_DIRECT, pl->dir.bytes, st);
@@ -155,6 +160,7 @@ int run_direct(tuna_plan *pl, const void *send, void *recv, cudaStream_t st) {
     a.del = list_args(pl->dir);
     TUNA_CUDA(pl, tuna_launch_move(TUNA_K_DIRECT, a, pl->dir.small_blocks, false, st));
     launches++;
+    pl->last_small = pl->dir.small_blocks ? 1 : 0;
   }
   pl->last_launches = launches;
   pl->launch_count += launches;
@@ -299,6 +305,7 @@ int tuna_rows_alltoallv(tuna_plan_t *pl, const void *rows_in, void *rows_out, vo
   if (ranges_overlap(rows_in, (size_t)pl->rows_in_bytes, rows_out, (size_t)pl->rows_out_bytes))
     return TUNA_ERR_OVERLAP;
   int launches = 0;
+  pl->last_small = 0;
   cudaStream_t st = (cudaStream_t)stream;
   {
     const int arc = await_tables(pl, st);
@@ -312,6 +319,7 @@ int tuna_rows_alltoallv(tuna_plan_t *pl, const void *rows_in, void *rows_out, vo
     a.del = list_args(l);
     TUNA_CUDA(pl, tuna_launch_move(TUNA_K_DIRECT, a, l.small_blocks, false, st));
     launches++;
+    pl->last_small = l.small_blocks ? 1 : 0;
   }
   pl->last_launches = launches;
   pl->launch_count += launches;
@@ -393,6 +401,12 @@ int tuna_plan_phase_tables(const tuna_plan_t *pl, int phase, int part, int64_t c
 int tuna_plan_last_launches(const tuna_plan_t *pl, int *launches) {
   if (!pl || !launches) return TUNA_ERR_INVALID_ARG;
   *launches = pl->last_launches;
+  return TUNA_OK;
+}
+
+int tuna_plan_last_small_launches(const tuna_plan_t *pl, int *launches) {
+  if (!pl || !launches) return TUNA_ERR_INVALID_ARG;
+  *launches = pl->last_small;
   return TUNA_OK;
 }
 

@@ -18,6 +18,7 @@ struct tuna_plan {
   bool classic = false;
   int cuda_err = 0;
   int last_launches = 0;
+  int last_small = 0;  // ... of which ran the small-block build of the mover
 
   std::vector<TunaPhase> phases;
   std::vector<TunaList> keep;     // per phase: blocks that travel on (workspace)
