@@ -54,6 +54,12 @@ def parse_args():
     ap.add_argument("--no-small-blocks", action="store_true",
                     help="skip the secondary entries that time the small-block build (c5, c3)")
     ap.add_argument("--sweep-steps", type=int, default=10)
+    ap.add_argument("--replicas", action="store_true",
+                    help="N > 1: N independent exchanges, one per GPU, instead of one exchange "
+                         "whose ranks are spread over the N GPUs")
+    ap.add_argument("--same-device", action="store_true",
+                    help="N > 1: every process uses GPU 0 and the gloo backend (a check of the "
+                         "sharded orchestration on a one-GPU machine, not a measurement)")
     ap.add_argument("--tokens", type=int, default=0,
                     help="c4 only: tokens per rank (default 8192); smaller values give the "
                          "reduced case used for profiler captures")
@@ -509,6 +515,127 @@ def small_block_entries(dev, peak, peak_kind, steps=20, warmup=3):
     return out
 
 
+def sharded_arm(args):
+    """N > 1: ONE exchange whose P ranks are spread over the N GPUs, P / N per GPU (the
+    hierarchical schedule with one group per GPU: local phases in each GPU's memory, the
+    inter-group phase as stores into the other GPUs' receive buffers).  The total payload
+    is the workload's whatever N is: strong scaling.  A step is, on every GPU, the re-plan
+    for the batch's counts (all-gather of the count matrix, count-metadata exchange and
+    prefix sums of this GPU's plan) and its share of the exchange between two barriers."""
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+    from paper_2411_02581_b200 import binding as B
+    from paper_2411_02581_b200 import build as build_mod
+    from paper_2411_02581_b200 import sharded as S
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = 0 if args.same_device else int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if args.same_device:
+        dist.init_process_group("gloo")
+    else:
+        dist.init_process_group("nccl", device_id=dev)
+    if rank == 0:
+        build_mod.build()
+    dist.barrier()
+    B.lib()
+    wl = make_workload(args.workload, args.tokens)
+    if wl.P % world:
+        raise SystemExit(f"{wl.name}: P = {wl.P} ranks do not divide over {world} GPUs")
+    l, E = wl.P // world, wl.elem_size
+    mine = S.ranks_of_gpu(wl.P, world, rank)
+    my_rows = np.ascontiguousarray(wl.sendcounts[mine.start:mine.stop])
+    radix = args.radix if args.radix else 0
+    ex = S.ShardedExchange(wl.P, E, my_rows, radix=radix, dist=dist)
+    # this GPU's part of the workload's send buffer: the regions of its own ranks
+    lo = int(wl.sendbase[mine.start]) * E
+    full = wl.make_send(dev) if wl.send_bytes <= (24 << 30) else None
+    if full is not None:
+        send = full[lo:lo + ex.send_bytes].clone()
+        del full
+    else:
+        send = torch.empty(ex.send_bytes, dtype=torch.uint8, device=dev)
+        send.view(torch.int64)[:ex.send_bytes // 8].random_()
+    torch.cuda.empty_cache()
+
+    def step():
+        ex.update_counts(my_rows)
+        ex.exchange(send)
+
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    # sampled parity: bytes this GPU received against the generator at their source position
+    rng = np.random.default_rng(777 + rank)
+    C = wl.sendcounts
+    nz = np.argwhere(C[:, mine.start:mine.stop] > 0)
+    ok = None
+    if len(nz):
+        pick = nz[rng.integers(0, len(nz), 4096)]
+        s, d = pick[:, 0], pick[:, 1] + mine.start
+        k = (rng.random(len(s)) * (C[s, d] * E)).astype(np.int64)
+        src = (wl.sendbase[s] + wl.sdispls[s, d]) * E + k
+        dst = (wl.recvbase[d] - wl.recvbase[mine.start] + wl.rdispls[d, s]) * E + k
+        from paper_2411_02581_b200 import workloads as W
+        want = W.payload_byte_at(wl.seed, torch.from_numpy(src))
+        ok = bool(torch.equal(want, ex.recv[torch.from_numpy(dst).to(dev)].cpu())) if wl.send_bytes <= (24 << 30) else None
+    ex.plan.enable_timing(True)
+    ex.plan.get_timing(reset=True)
+    launches0 = ex.plan.launch_count()
+    dist.barrier()
+    torch.cuda.synchronize()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local) as clocks:
+        ev0.record()
+        for _ in range(args.steps):
+            step()
+        ev1.record()
+        torch.cuda.synchronize()
+    dist.barrier()
+    ms_per_step = max_over_ranks(ev0.elapsed_time(ev1), dist, dev if not args.same_device else "cpu") / args.steps
+    timing = ex.plan.get_timing(reset=True)
+    launches = ex.plan.launch_count() - launches0
+    payload = wl.payload_bytes_total
+    g_ms, g_by = timing["round_global"]["ms"], timing["round_global"]["bytes"]
+    l_ms, l_by = timing["round_local"]["ms"], timing["round_local"]["bytes"]
+    peak, peak_kind = measured_peaks()
+    # the push crosses NVLink: bytes this GPU stores into other GPUs over its device time,
+    # against the measured 770 GB/s per direction of a peer copy on this kind of machine
+    link_peak = 770.0
+    ach_link = g_by / (g_ms * 1e-3) / 1e9 if g_ms > 0 else 0.0
+    ach_local = 2.0 * l_by / (l_ms * 1e-3) / 1e9 if l_ms > 0 else 0.0
+    flags = torch.tensor([1.0 if ok in (True, None) else 0.0], dtype=torch.float64,
+                         device="cpu" if args.same_device else dev)
+    dist.all_reduce(flags, op=dist.ReduceOp.MIN)
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": payload / (ms_per_step * 1e-3) / 1e9, "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "strong", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+            "config": {"workload": f"{wl.name} P={wl.P}, {l} ranks per GPU: local radix {radix or max(2, l)}, "
+                                   f"inter-GPU phase pushed into the peers' receive buffers, payload {payload} bytes "
+                                   f"in total, elem {E} B, re-plan every step from all-gathered counts",
+                       "l2": "inputs larger than L2" if payload / world > 256e6 else "inputs fit in L2",
+                       "sharding": "one group of the hierarchical schedule per GPU",
+                       "emulated_on_one_gpu": bool(args.same_device)},
+            "gpu_launches": int(launches) * world, "parity_samples_ok": bool(flags.item() == 1.0),
+            "clocks": clocks.summary(),
+            "roofline": {"bound": "nvlink", "kernel": "tuna_round_kernel (inter-GPU push of rank 0)",
+                         "achieved": ach_link, "peak": link_peak, "peak_kind": "of the measured peer-copy rate",
+                         "unit": "GB/s", "frac": ach_link / link_peak, "traffic": None,
+                         "local_phases_GBps": ach_local, "local_frac_of_hbm": ach_local / peak,
+                         "hbm_peak_kind": f"of {peak_kind}"},
+            "e2e": None, "cpu_baseline": None,
+        }
+        print(json.dumps(line), flush=True)
+    dist.barrier()
+    ex.destroy()
+    dist.destroy_process_group()
+
+
 def ours_arm(args):
     import numpy as np
     import torch
@@ -796,6 +923,8 @@ def main():
     args = parse_args()
     if args.impl == "reference":
         reference_arm(args)
+    elif int(os.environ.get("WORLD_SIZE", "1")) > 1 and not args.replicas:
+        sharded_arm(args)
     else:
         ours_arm(args)
 

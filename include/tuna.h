@@ -280,6 +280,93 @@ int tuna_direct_alltoallv_static(int P, int elem_size, const int64_t *sendcounts
                                  const void *sendbuf, void *recvbuf, void *stream);
 
 /*
+ * Sharded plans: the ranks spread over several GPUs of one node, one process per GPU.
+ *
+ * Defines: Sec. IV of the paper with one group per GPU.  The paper's hierarchy exists
+ * because links inside a node are faster than links between nodes; here the "node" is
+ * one GPU's memory and the slower link is NVLink between GPUs.  Group n (ranks n*l ..
+ * n*l + l - 1, l = P / n_gpus) lives on GPU n: its send regions in that GPU's send buffer,
+ * its receive regions in that GPU's receive buffer.  The local phases (Sec. IV-A,
+ * radix `radix` on the local offset, for all destination groups at once) run inside each
+ * GPU; the inter-group phase is the coalesced exchange of Sec. IV-B / Algorithm 3 (one
+ * hop, n_gpus - 1 rounds of one super-block of l blocks each) executed as a push: the
+ * sending GPU stores every block straight into its place in the receiving GPU's receive
+ * buffer.  An inter-group radix below n_gpus would forward super-blocks through third
+ * GPUs' memory for no gain (every GPU pair is one hop apart) and is not offered.
+ *
+ * tuna_shard_plan_create - the plan of GPU `my_gpu`.  Every GPU calls it with the SAME
+ * P x P count matrix (all-gather the rows first) and the same displacement arrays.
+ *   sendbase[p], recvbase[p]   element offset of rank p's region inside the buffer of
+ *                 THE GPU THAT HOLDS RANK p; NULL = that GPU's l regions packed in rank
+ *                 order from offset 0.  sdispls / rdispls as in tuna_plan_create.
+ *   flags         TUNA_FLAG_CLASSIC_ROTATE and TUNA_FLAG_BULK_COPY are refused
+ *                 (TUNA_ERR_INVALID_ARG); TUNA_FLAG_NO_DIRECT is implied.
+ *   errors        P not a multiple of n_gpus: TUNA_ERR_BAD_HIERARCHY; n_gpus above 240 or
+ *                 my_gpu outside [0, n_gpus): TUNA_ERR_INVALID_ARG; otherwise as
+ *                 tuna_plan_create.
+ * The plan holds the tables of all P ranks (the metadata work is replicated on every
+ * GPU, the data movement is not): its descriptor lists carry a length only where this
+ * GPU moves the block.  Introspection reports this GPU's share: a round's `bytes` are the
+ * bytes this GPU moves in it, so the sum over the n_gpus plans is the round's volume.
+ * tuna_plan_workspace_bytes / tuna_plan_set_workspace: this GPU's workspace (local
+ * phases only; the inter-group phase needs none).  tuna_plan_update_counts works
+ * (same rule for NULL bases); tuna_plan_update_counts_device, tuna_alltoallv,
+ * tuna_direct_alltoallv, tuna_alltoallv_host and the row exchange return
+ * TUNA_ERR_INVALID_ARG for a sharded plan.
+ *
+ * tuna_shard_extents - bytes of GPU `gpu`'s send and receive buffer that the layout covers.
+ *
+ * tuna_shard_alltoallv - run this GPU's share.
+ *   sendbuf     device, this GPU's send buffer.
+ *   recvbufs    HOST array of n_gpus DEVICE pointers: the receive buffer of every GPU as
+ *               this process can address it (its own, and the others' mapped through peer
+ *               access or an inter-process memory handle).  The caller owns the mappings.
+ *   phases      TUNA_SHARD_LOCAL, TUNA_SHARD_GLOBAL or both: the local phases (with the
+ *               self blocks) and the inter-group push.  Both in one call is the normal
+ *               use; separately they let a caller overlap or inspect the two parts.  The
+ *               push reads what the local phases left in the workspace: same stream, or
+ *               ordered by the caller.
+ * Asynchronous on `stream`; only enqueues kernels.  No kernel waits for another GPU, so
+ * the call cannot deadlock whatever the other GPUs do.  It does NOT tell when the other
+ * GPUs' stores into this GPU's receive buffer have landed: the caller closes the exchange
+ * with a barrier across the GPUs that is ordered behind this call on every GPU's stream
+ * (e.g. an NCCL all-reduce on the same stream), and must not reuse a receive buffer
+ * before every GPU has passed the previous exchange's barrier.
+ *
+ * Host-only helpers (no GPU is touched, so they can run before any buffer exists):
+ * tuna_shard_layout - the layout rule above, worked out for all GPUs: region bases of
+ *   every rank inside its GPU's buffers (sendbase_out, recvbase_out: P values, elements)
+ *   and every GPU's buffer sizes (send_bytes, recv_bytes: n_gpus values, bytes); any
+ *   output may be NULL.  Use it to size and allocate the buffers whose addresses the
+ *   GPUs then exchange.
+ * tuna_shard_round_table - the rounds of the sharded schedule in execution order with
+ *   what GPU my_gpu sends in each: `level`, `x`, `z` as tuna_plan_round_info; `units` =
+ *   blocks (level 0) or super-blocks (level 1) its ranks send, `bytes` their volume.  Up
+ *   to `cap` rows are written, *rounds receives the number of rounds.  Level-1 bytes are
+ *   this GPU's traffic onto the inter-GPU links.
+ * tuna_shard_enable_peer_access - lets kernels of the current device store into
+ *   peer_device's memory (cudaDeviceEnablePeerAccess; already enabled counts as success;
+ *   TUNA_ERR_INVALID_ARG if the two GPUs have no peer path).
+ */
+#define TUNA_SHARD_LOCAL 1
+#define TUNA_SHARD_GLOBAL 2
+int tuna_shard_layout(int P, int n_gpus, int elem_size, const int64_t *sendcounts, const int64_t *sdispls,
+                      const int64_t *rdispls, const int64_t *sendbase, const int64_t *recvbase,
+                      int64_t *sendbase_out, int64_t *recvbase_out, int64_t *send_bytes,
+                      int64_t *recv_bytes);
+int tuna_shard_round_table(int P, int n_gpus, int my_gpu, int radix, int elem_size,
+                           const int64_t *sendcounts, int cap, int *level, int *x, int *z,
+                           int64_t *units, int64_t *bytes, int *rounds);
+int tuna_shard_enable_peer_access(int peer_device);
+int tuna_shard_plan_create(tuna_plan_t **out, int P, int radix, int n_gpus, int my_gpu, int elem_size,
+                           unsigned flags, const int64_t *sendcounts, const int64_t *sdispls,
+                           const int64_t *rdispls, const int64_t *sendbase, const int64_t *recvbase,
+                           void *stream);
+int tuna_shard_extents(const tuna_plan_t *plan, int gpu, size_t *send_bytes, size_t *recv_bytes);
+int tuna_shard_alltoallv(tuna_plan_t *plan, const void *sendbuf, void *const *recvbufs, int phases,
+                         void *stream);
+
+/*
  * tuna_alltoallv_host - the same exchange on HOST buffers, all on `stream`,
  * returning without synchronising.  `schedule` is TUNA_SCHEDULE_TUNA or
  * TUNA_SCHEDULE_DIRECT, optionally OR-ed with TUNA_HOST_STAGED.

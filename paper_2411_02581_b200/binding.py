@@ -24,6 +24,8 @@ FLAG_BULK_COPY = 2
 FLAG_NO_DIRECT = 4
 PART_KEEP = 0
 PART_DELIVER = 1
+SHARD_LOCAL = 1
+SHARD_GLOBAL = 2
 SCHEDULE_TUNA = 0
 SCHEDULE_DIRECT = 1
 HOST_STAGED = 0x100
@@ -56,6 +58,14 @@ SIGNATURES = {
     "tuna_direct_alltoallv": (ctypes.c_int, [_VP, _VP, _I64P, _I64P, _VP, _I64P, _I64P, _VP]),
     "tuna_alltoallv_host": (ctypes.c_int, [_VP, _VP, _VP, ctypes.c_int, _VP]),
     "tuna_direct_alltoallv_static": (ctypes.c_int, [ctypes.c_int, ctypes.c_int] + [_I64P] * 5 + [_VP, _VP, _VP]),
+    "tuna_shard_plan_create": (ctypes.c_int, [ctypes.POINTER(_VP)] + [ctypes.c_int] * 5 + [ctypes.c_uint]
+                               + [_I64P] * 5 + [_VP]),
+    "tuna_shard_extents": (ctypes.c_int, [_VP, ctypes.c_int, _SZP, _SZP]),
+    "tuna_shard_layout": (ctypes.c_int, [ctypes.c_int] * 3 + [_I64P] * 9),
+    "tuna_shard_round_table": (ctypes.c_int, [ctypes.c_int] * 5 + [_I64P, ctypes.c_int, _INTP, _INTP, _INTP,
+                                                                _I64P, _I64P, _INTP]),
+    "tuna_shard_enable_peer_access": (ctypes.c_int, [ctypes.c_int]),
+    "tuna_shard_alltoallv": (ctypes.c_int, [_VP, _VP, ctypes.POINTER(_VP), ctypes.c_int, _VP]),
     "tuna_plan_num_rounds": (ctypes.c_int, [_VP, _INTP]),
     "tuna_plan_round_info": (ctypes.c_int, [_VP, ctypes.c_int, _INTP, _INTP, _INTP, _I64P, _I64P]),
     "tuna_plan_num_phases": (ctypes.c_int, [_VP, _INTP]),
@@ -134,13 +144,18 @@ class Plan:
 
     def __init__(self, P, radix, l=None, g=1, radix_global=2, elem_size=1, flags=0,
                  sendcounts=None, sdispls=None, rdispls=None, sendbase=None, recvbase=None,
-                 stream=None, block_count=0):
-        """``block_count`` > 0 selects ``tuna_plan_create_staggered`` (``radix_global`` unused)."""
+                 stream=None, block_count=0, shard=None):
+        """``block_count`` > 0 selects ``tuna_plan_create_staggered`` (``radix_global`` unused);
+        ``shard`` = (n_gpus, my_gpu) selects ``tuna_shard_plan_create`` (``l``, ``g`` unused)."""
         self._h = _VP()
         self._ws = None
         l = P if l is None else l
         keep = [_h(x) for x in (sendcounts, sdispls, rdispls, sendbase, recvbase)]
-        if block_count:
+        if shard is not None:
+            what = "tuna_shard_plan_create"
+            rc = lib().tuna_shard_plan_create(ctypes.byref(self._h), P, radix, shard[0], shard[1],
+                                              elem_size, flags, *[k[1] for k in keep], _stream(stream))
+        elif block_count:
             what = "tuna_plan_create_staggered"
             rc = lib().tuna_plan_create_staggered(ctypes.byref(self._h), P, radix, block_count, l, g,
                                                   elem_size, flags, *[k[1] for k in keep],
@@ -237,6 +252,18 @@ class Plan:
         self._check(lib().tuna_rows_alltoallv(self._h, _ptr(rows_in), _ptr(rows_out), _stream(stream)),
                     "tuna_rows_alltoallv")
 
+    def shard_extents(self, gpu):
+        a, b = ctypes.c_size_t(), ctypes.c_size_t()
+        self._check(lib().tuna_shard_extents(self._h, gpu, ctypes.byref(a), ctypes.byref(b)),
+                    "tuna_shard_extents")
+        return a.value, b.value
+
+    def shard_alltoallv(self, sendbuf, recvbufs, phases=SHARD_LOCAL | SHARD_GLOBAL, stream=None):
+        """``recvbufs``: one tensor (or address) per GPU, as this process addresses them."""
+        ptrs = (_VP * len(recvbufs))(*[_ptr(r) for r in recvbufs])
+        self._check(lib().tuna_shard_alltoallv(self._h, _ptr(sendbuf), ptrs, phases, _stream(stream)),
+                    "tuna_shard_alltoallv")
+
     def alltoallv_host(self, host_send, host_recv, schedule=SCHEDULE_TUNA, stream=None):
         self._check(lib().tuna_alltoallv_host(self._h, _ptr(host_send), _ptr(host_recv), schedule,
                                               _stream(stream)), "tuna_alltoallv_host")
@@ -327,6 +354,39 @@ def direct_alltoallv_static(P, elem_size, sendcounts, sendbuf, recvbuf, sdispls=
                                             _ptr(recvbuf), _stream(stream))
     if rc != 0:
         raise TunaError(rc, "tuna_direct_alltoallv_static")
+
+
+def shard_layout(P, n_gpus, elem_size, sendcounts, sdispls=None, rdispls=None, sendbase=None,
+                 recvbase=None):
+    """Host only: (sendbase[P], recvbase[P], send_bytes[n_gpus], recv_bytes[n_gpus]) of a sharded
+    layout (``tuna_shard_layout``)."""
+    keep = [_h(x) for x in (sendcounts, sdispls, rdispls, sendbase, recvbase)]
+    sb, rb = np.zeros(P, dtype=np.int64), np.zeros(P, dtype=np.int64)
+    se, re = np.zeros(n_gpus, dtype=np.int64), np.zeros(n_gpus, dtype=np.int64)
+    rc = lib().tuna_shard_layout(P, n_gpus, elem_size, *[k[1] for k in keep],
+                                 *[a.ctypes.data_as(_I64P) for a in (sb, rb, se, re)])
+    if rc != 0:
+        raise TunaError(rc, "tuna_shard_layout")
+    return sb, rb, se, re
+
+
+def shard_round_table(P, n_gpus, my_gpu, radix, elem_size, sendcounts):
+    """Host only: the rounds of the sharded schedule with what GPU ``my_gpu`` sends in each,
+    as a list of dicts like :meth:`Plan.rounds` (``tuna_shard_round_table``)."""
+    c, cp = _h(sendcounts)
+    n = ctypes.c_int()
+    rc = lib().tuna_shard_round_table(P, n_gpus, my_gpu, radix, elem_size, cp, 0, None, None, None, None,
+                                      None, ctypes.byref(n))
+    if rc != 0:
+        raise TunaError(rc, "tuna_shard_round_table")
+    K = n.value
+    lv, x, z = [(ctypes.c_int * max(K, 1))() for _ in range(3)]
+    u, b = np.zeros(max(K, 1), dtype=np.int64), np.zeros(max(K, 1), dtype=np.int64)
+    rc = lib().tuna_shard_round_table(P, n_gpus, my_gpu, radix, elem_size, cp, K, lv, x, z,
+                                      u.ctypes.data_as(_I64P), b.ctypes.data_as(_I64P), ctypes.byref(n))
+    if rc != 0:
+        raise TunaError(rc, "tuna_shard_round_table")
+    return [dict(level=lv[k], x=x[k], z=z[k], units=int(u[k]), bytes=int(b[k])) for k in range(K)]
 
 
 def plan_for(wl, radix, l=None, g=1, radix_global=2, flags=0, explicit_layout=True, stream=None,

@@ -10,7 +10,7 @@ ROOT = os.path.dirname(_HERE)
 CSRC = os.path.join(_HERE, "csrc")
 LIB_DIR = os.path.join(_HERE, "_lib")
 LIB_PATH = os.path.join(LIB_DIR, "libtuna.so")
-SOURCES = ["tuna_plan.cu", "tuna_api.cu", "tuna_static.cu", "tuna_move.cu"]
+SOURCES = ["tuna_plan.cu", "tuna_api.cu", "tuna_static.cu", "tuna_shard.cu", "tuna_move.cu"]
 HEADERS = [os.path.join(CSRC, h) for h in ("tuna_internal.h", "tuna_plan.h", "tuna_plan_kernels.cuh")] + [
     os.path.join(ROOT, "include", "tuna.h")]
 

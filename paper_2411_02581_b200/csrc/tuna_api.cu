@@ -3,6 +3,39 @@
 
 #include "tuna_plan.h"
 
+namespace tuna_host {
+
+TunaListArgs list_args(const TunaList &l) {
+  TunaListArgs a{};
+  a.len = l.len;
+  a.pos = l.pos;
+  a.src = l.src;
+  a.dst = l.dst;
+  a.chunk_first = l.chunk_first;
+  a.n = l.n;
+  a.total = l.total;
+  a.chunk = l.chunk;
+  a.nchunks = l.n > 0 ? l.nchunks : 0;
+  return a;
+}
+
+TunaMoveArgs move_args(const tuna_plan *pl, const void *send, void *recv, char *work) {
+  TunaMoveArgs a{};
+  a.base[TUNA_BUF_SEND] = (char *)const_cast<void *>(send);
+  a.base[TUNA_BUF_RECV] = (char *)recv;
+  a.base[TUNA_BUF_WORK] = work;
+  a.extent[TUNA_BUF_SEND] = pl->send_extent;
+  a.extent[TUNA_BUF_RECV] = pl->recv_extent;
+  a.extent[TUNA_BUF_WORK] = work ? pl->workspace_need : 0;
+  a.keep_base = 0;
+  a.peer = pl->d_peer_ptrs;
+  a.error = pl->d_error;
+  a.bulk_off = (pl->flags & TUNA_FLAG_BULK_COPY) ? 1 : 0;
+  return a;
+}
+
+}  // namespace tuna_host
+
 using namespace tuna_host;
 
 namespace {
@@ -51,34 +84,6 @@ int check_call_args(tuna_plan *pl, const int64_t *sendcounts, const int64_t *sdi
     }
   }
   return TUNA_OK;
-}
-
-TunaListArgs list_args(const TunaList &l) {
-  TunaListArgs a{};
-  a.len = l.len;
-  a.pos = l.pos;
-  a.src = l.src;
-  a.dst = l.dst;
-  a.chunk_first = l.chunk_first;
-  a.n = l.n;
-  a.total = l.total;
-  a.chunk = l.chunk;
-  a.nchunks = l.n > 0 ? l.nchunks : 0;
-  return a;
-}
-
-TunaMoveArgs move_args(const tuna_plan *pl, const void *send, void *recv, char *work) {
-  TunaMoveArgs a{};
-  a.base[TUNA_BUF_SEND] = (char *)const_cast<void *>(send);
-  a.base[TUNA_BUF_RECV] = (char *)recv;
-  a.base[TUNA_BUF_WORK] = work;
-  a.extent[TUNA_BUF_SEND] = pl->send_extent;
-  a.extent[TUNA_BUF_RECV] = pl->recv_extent;
-  a.extent[TUNA_BUF_WORK] = work ? pl->workspace_need : 0;
-  a.keep_base = 0;
-  a.error = pl->d_error;
-  a.bulk_off = (pl->flags & TUNA_FLAG_BULK_COPY) ? 1 : 0;
-  return a;
 }
 
 // One launch per digit phase: its KEEP list, its DELIVER list and, riding along in
@@ -223,6 +228,7 @@ int tuna_alltoallv(tuna_plan_t *pl, const void *sendbuf, const int64_t *sendcoun
                    const int64_t *sdispls, void *recvbuf, const int64_t *recvcounts,
                    const int64_t *rdispls, void *stream) {
   if (!pl) return TUNA_ERR_INVALID_ARG;
+  if (pl->topo.shard_n > 0) return TUNA_ERR_INVALID_ARG;  // a sharded plan runs through tuna_shard_alltoallv
   if ((!sendbuf && pl->send_extent > 0) || (!recvbuf && pl->recv_extent > 0)) return TUNA_ERR_INVALID_ARG;
   int rc = check_call_args(pl, sendcounts, sdispls, recvcounts, rdispls);
   if (rc) return rc;
@@ -235,6 +241,7 @@ int tuna_direct_alltoallv(tuna_plan_t *pl, const void *sendbuf, const int64_t *s
                           const int64_t *sdispls, void *recvbuf, const int64_t *recvcounts,
                           const int64_t *rdispls, void *stream) {
   if (!pl) return TUNA_ERR_INVALID_ARG;
+  if (pl->topo.shard_n > 0) return TUNA_ERR_INVALID_ARG;  // a sharded plan runs through tuna_shard_alltoallv
   if ((!sendbuf && pl->send_extent > 0) || (!recvbuf && pl->recv_extent > 0)) return TUNA_ERR_INVALID_ARG;
   int rc = check_call_args(pl, sendcounts, sdispls, recvcounts, rdispls);
   if (rc) return rc;
@@ -259,6 +266,7 @@ static void *mapped_alias(const void *host) {
 int tuna_alltoallv_host(tuna_plan_t *pl, const void *host_send, void *host_recv, int schedule,
                         void *stream) {
   if (!pl) return TUNA_ERR_INVALID_ARG;
+  if (pl->topo.shard_n > 0) return TUNA_ERR_INVALID_ARG;  // a sharded plan runs through tuna_shard_alltoallv
   if ((!host_send && pl->send_extent > 0) || (!host_recv && pl->recv_extent > 0)) return TUNA_ERR_INVALID_ARG;
   const bool force_staging = (schedule & TUNA_HOST_STAGED) != 0;
   schedule &= ~TUNA_HOST_STAGED;
@@ -299,6 +307,7 @@ int tuna_alltoallv_host(tuna_plan_t *pl, const void *host_send, void *host_recv,
 
 int tuna_rows_alltoallv(tuna_plan_t *pl, const void *rows_in, void *rows_out, void *stream) {
   if (!pl) return TUNA_ERR_INVALID_ARG;
+  if (pl->topo.shard_n > 0) return TUNA_ERR_INVALID_ARG;  // a sharded plan runs through tuna_shard_alltoallv
   if (!pl->rows_valid) return TUNA_ERR_COUNT_MISMATCH;
   const TunaList &l = pl->rowsl;
   if (l.n > 0 && (!rows_in || !rows_out)) return TUNA_ERR_INVALID_ARG;

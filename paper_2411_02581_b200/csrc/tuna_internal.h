@@ -13,6 +13,8 @@
 #define TUNA_BUF_SEND 0
 #define TUNA_BUF_RECV 1
 #define TUNA_BUF_WORK 2
+// Sharded plans (ranks spread over several GPUs): the receive buffer of GPU n.
+#define TUNA_BUF_PEER0 16
 #define TUNA_LOC(buf, off) ((((int64_t)(buf)) << 56) | (int64_t)(off))
 #define TUNA_LOC_BUF(loc) ((int)((loc) >> 56))
 #define TUNA_LOC_OFF(loc) ((loc) & ((((int64_t)1) << 56) - 1))
@@ -26,6 +28,13 @@
 struct TunaTopo {
   int P, Q, N;
   int elem;
+  // Sharded plan: group n lives on GPU n, and this plan describes the work of GPU
+  // shard_me only (shard_n == N GPUs).  Every GPU builds the tables of all P ranks, so
+  // that sizes and locations flow through the phases as in a plan for one GPU, but a
+  // descriptor is given its length only where this GPU executes it: in a local phase the
+  // blocks its own ranks receive, in the global phase the blocks its own ranks send
+  // (they are stored straight into the receiving GPU's buffer).  shard_n == 0: one GPU.
+  int shard_n, shard_me;
 };
 
 // One digit phase: all rounds (x, z), z = 1..radix-1, of one digit position.
@@ -85,6 +94,7 @@ struct TunaMoveArgs {
   TunaListArgs del;   // blocks of a digit phase that have arrived, or the direct list
   TunaListArgs rot;   // rotation list (self blocks, or every block in classic mode)
   char *base[3];
+  char *const *peer;  // sharded plans: device array of the GPUs' receive buffers (null otherwise)
   int64_t extent[3];  // bytes of each buffer that may be accessed, from its base
   int64_t keep_base;  // workspace offset of stream position 0 of the KEEP list
   int *error;         // device flag raised when a bounded wait inside a kernel gave up (may be null)

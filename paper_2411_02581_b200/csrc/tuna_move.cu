@@ -58,6 +58,7 @@ __device__ __forceinline__ void st16(char *p, uint4 v) { *reinterpret_cast<uint4
 
 // (a select, not an index: indexing a kernel parameter array spills it to local memory)
 __device__ __forceinline__ char *base_of(const TunaMoveArgs &a, int buf) {
+  if (buf >= TUNA_BUF_PEER0) return a.peer[buf - TUNA_BUF_PEER0];  // another GPU's receive buffer (sharded plans)
   return buf == TUNA_BUF_SEND ? a.base[0] : (buf == TUNA_BUF_RECV ? a.base[1] : a.base[2]);
 }
 __device__ __forceinline__ int64_t extent_of(const TunaMoveArgs &a, int buf) {

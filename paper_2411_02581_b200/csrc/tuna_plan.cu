@@ -116,6 +116,36 @@ int validate_layout(int P, const int64_t *counts, const int64_t *sdispls, const 
   return TUNA_OK;
 }
 
+void shard_layout(int P, int l, const int64_t *counts, const int64_t *sdispls, const int64_t *rdispls,
+                  const int64_t *sendbase, const int64_t *recvbase, std::vector<int64_t> *sb,
+                  std::vector<int64_t> *rb, std::vector<int64_t> *send_extent,
+                  std::vector<int64_t> *recv_extent) {
+  const int g = P / l;
+  std::vector<int64_t> sreg(P, 0), rreg(P, 0);  // elements every rank's regions span
+  for (int s = 0; s < P; s++)
+    for (int d = 0; d < P; d++) {
+      const int64_t c = counts[(int64_t)s * P + d];
+      if (sdispls) sreg[s] = std::max(sreg[s], sdispls[(int64_t)s * P + d] + c); else sreg[s] += c;
+      if (rdispls) rreg[d] = std::max(rreg[d], rdispls[(int64_t)d * P + s] + c); else rreg[d] += c;
+    }
+  sb->assign(P, 0);
+  rb->assign(P, 0);
+  send_extent->assign(g, 0);
+  recv_extent->assign(g, 0);
+  for (int n = 0; n < g; n++) {
+    int64_t acc_s = 0, acc_r = 0;  // packed: a GPU's regions back to back, from 0
+    for (int q = 0; q < l; q++) {
+      const int p = n * l + q;
+      (*sb)[p] = sendbase ? sendbase[p] : acc_s;
+      (*rb)[p] = recvbase ? recvbase[p] : acc_r;
+      acc_s += sreg[p];
+      acc_r += rreg[p];
+      (*send_extent)[n] = std::max((*send_extent)[n], (*sb)[p] + sreg[p]);
+      (*recv_extent)[n] = std::max((*recv_extent)[n], (*rb)[p] + rreg[p]);
+    }
+  }
+}
+
 int sm_count() {
   static int cached[64] = {};
   int dev = 0, n = 0;
@@ -614,6 +644,12 @@ int build_tables(tuna_plan *pl, const HostLayout *hl, const int64_t *sdispls, co
       pl->payload = hl->payload * t.elem;
       pl->send_extent = hl->send_extent * t.elem;
       pl->recv_extent = hl->recv_extent * t.elem;
+      if (t.shard_n > 0) {  // this GPU's buffers; the self-check needs every GPU's receive extent
+        pl->send_extent = pl->shard_send_extent[t.shard_me];
+        pl->recv_extent = pl->shard_recv_extent[t.shard_me];
+        TUNA_CUDA(pl, cudaMemcpyAsync(pl->d_peer_extent, pl->shard_recv_extent.data(), (size_t)t.shard_n * 8,
+                                      cudaMemcpyHostToDevice, st));
+      }
       if (!pl->counts_uploaded)
         TUNA_CUDA(pl, cudaMemcpyAsync(pl->d_counts, counts, PP * 8, cudaMemcpyHostToDevice, st));
       TUNA_CUDA(pl, cudaMemcpyAsync(pl->d_sendbase, hl->sendbase.data(), P * 8, cudaMemcpyHostToDevice, st));
@@ -717,7 +753,7 @@ int build_tables(tuna_plan *pl, const HostLayout *hl, const int64_t *sdispls, co
       const unsigned gx = (unsigned)std::min<int64_t>((pl->check_max_n + th - 1) / th, (int64_t)sm_count() * 8);
       tuna_check_lists_kernel<<<dim3(gx, pl->n_check_items), th, 0, st>>>(
           static_cast<const TunaCheckItem *>(pl->d_check_items), pl->d_extents, pl->d_wbase + nph, pl->d_wbase,
-          pl->d_violations);
+          pl->d_violations, pl->d_peer_extent);
       TUNA_LAUNCHED(pl);
     }
 
@@ -912,6 +948,8 @@ int tuna_plan_destroy(tuna_plan_t *pl) {
   cudaFree(pl->d_readback);  // (d_scal, d_wbase, d_extents, d_round_bytes, d_violations are slices of it)
   if (pl->h_readback) cudaFreeHost(pl->h_readback);
   cudaFree(pl->d_error);
+  cudaFree(pl->d_peer_extent);
+  cudaFree(pl->d_peer_ptrs);
   for (auto &s : pl->stamps) {
     cudaEventDestroy(s.a);
     cudaEventDestroy(s.b);
@@ -921,15 +959,26 @@ int tuna_plan_destroy(tuna_plan_t *pl) {
   return TUNA_OK;
 }
 
-static int plan_create(tuna_plan_t **out, int P, int radix, int radix_global, int block_count,
-                       int l, int g, int elem_size, unsigned flags, const int64_t *sendcounts,
-                       const int64_t *sdispls, const int64_t *rdispls, const int64_t *sendbase,
-                       const int64_t *recvbase, void *stream) {
+}  // extern "C"
+
+int tuna_host::plan_create(tuna_plan_t **out, int P, int radix, int radix_global, int block_count,
+                           int l, int g, int elem_size, unsigned flags, const int64_t *sendcounts,
+                           const int64_t *sdispls, const int64_t *rdispls, const int64_t *sendbase,
+                           const int64_t *recvbase, void *stream, int shard_n, int shard_me) {
   if (!out) return TUNA_ERR_INVALID_ARG;
   *out = nullptr;
   if (P < 1 || elem_size < 1 || !sendcounts || l < 1 || g < 1) return TUNA_ERR_INVALID_ARG;
   if (P > TUNA_MAX_P) return TUNA_ERR_RANGE;
   if ((int64_t)l * g != P) return TUNA_ERR_BAD_HIERARCHY;
+  if (shard_n > 0) {
+    // one group per GPU, one hop between GPUs, blocks delivered straight into the receive
+    // buffers, no direct list (a GPU reaches only its own send buffer)
+    if (shard_n != g || shard_me < 0 || shard_me >= shard_n || block_count != 0 ||
+        shard_n > 256 - TUNA_BUF_PEER0 || (flags & (TUNA_FLAG_CLASSIC_ROTATE | TUNA_FLAG_BULK_COPY)))
+      return TUNA_ERR_INVALID_ARG;
+    radix_global = std::max(2, g);
+    flags |= TUNA_FLAG_NO_DIRECT;
+  }
   // radix 0 = choose: one hop per level (with all ranks in one memory every further
   // hop only adds a read and a write of the block; there is no message latency to save)
   if (radix == 0) radix = std::max(2, l);
@@ -963,6 +1012,20 @@ static int plan_create(tuna_plan_t **out, int P, int radix, int radix_global, in
     }
   }
   HostLayout hl;
+  std::vector<int64_t> shard_sb, shard_rb;
+  if (shard_n > 0) {  // region bases are per GPU: worked out here, explicit from here on
+    int vrc = validate_layout(P, sendcounts, sdispls, rdispls, sendbase, recvbase);
+    if (vrc) {
+      tuna_plan_destroy(pl);
+      return vrc;
+    }
+    shard_layout(P, l, sendcounts, sdispls, rdispls, sendbase, recvbase, &shard_sb, &shard_rb,
+                 &pl->shard_send_extent, &pl->shard_recv_extent);
+    for (auto &v : pl->shard_send_extent) v *= elem_size;
+    for (auto &v : pl->shard_recv_extent) v *= elem_size;
+    sendbase = shard_sb.data();
+    recvbase = shard_rb.data();
+  }
   int rc = host_layout(P, sendcounts, sdispls, rdispls, sendbase, recvbase, &hl, pl->h_buf[0]);
   if (rc) {
     tuna_plan_destroy(pl);
@@ -970,7 +1033,7 @@ static int plan_create(tuna_plan_t **out, int P, int radix, int radix_global, in
   }
   pl->h_cur = 0;
   pl->h_counts = pl->h_buf[0];
-  pl->topo = TunaTopo{P, l, g, elem_size};
+  pl->topo = TunaTopo{P, l, g, elem_size, shard_n, shard_me};
   pl->radix_l = radix;
   pl->radix_g = (g > 1 && block_count == 0) ? radix_global : 2;
   pl->block_count = block_count;
@@ -1030,6 +1093,11 @@ static int plan_create(tuna_plan_t **out, int P, int radix, int radix_global, in
     pl->d_violations = pl->d_round_bytes + n_rb;
   }
   TUNA_TRY(dev_alloc(&pl->d_error, 1));
+  if (shard_n > 0) {
+    TUNA_TRY(dev_alloc(&pl->d_peer_extent, shard_n));
+    TUNA_TRY(dev_alloc(&pl->d_peer_ptrs, shard_n));
+    TUNA_TRY(cudaMemset(pl->d_peer_ptrs, 0, (size_t)shard_n * sizeof(char *)));
+  }
   TUNA_TRY(cudaMemset(pl->d_error, 0, sizeof(int)));
   pl->keep.resize(nph);
   pl->deliver.resize(nph);
@@ -1079,6 +1147,8 @@ static int plan_create(tuna_plan_t **out, int P, int radix, int radix_global, in
   return TUNA_OK;
 }
 
+extern "C" {
+
 int tuna_plan_create(tuna_plan_t **out, int P, int radix, int radix_global, int l, int g,
                      int elem_size, unsigned flags, const int64_t *sendcounts,
                      const int64_t *sdispls, const int64_t *rdispls, const int64_t *sendbase,
@@ -1104,6 +1174,15 @@ int tuna_plan_update_counts(tuna_plan_t *pl, const int64_t *sendcounts, const in
                             const int64_t *recvbase, void *stream) {
   if (!pl || !sendcounts) return TUNA_ERR_INVALID_ARG;
   HostLayout hl;
+  std::vector<int64_t> shard_sb, shard_rb, shard_se, shard_re;
+  if (pl->topo.shard_n > 0) {  // a sharded plan's region bases are per GPU
+    const int vrc = validate_layout(pl->topo.P, sendcounts, sdispls, rdispls, sendbase, recvbase);
+    if (vrc) return vrc;
+    shard_layout(pl->topo.P, pl->topo.Q, sendcounts, sdispls, rdispls, sendbase, recvbase, &shard_sb, &shard_rb,
+                 &shard_se, &shard_re);
+    sendbase = shard_sb.data();
+    recvbase = shard_rb.data();
+  }
   const int spare = pl->h_cur ^ 1;
   CountUpload up;  // the spare device buffer takes the new counts while the pass is running
   up.d_dst = pl->d_counts == pl->d_counts_buf[0] ? pl->d_counts_buf[1] : pl->d_counts_buf[0];
@@ -1116,6 +1195,12 @@ int tuna_plan_update_counts(tuna_plan_t *pl, const int64_t *sendcounts, const in
   }
   pl->h_cur = spare;
   pl->h_counts = pl->h_buf[spare];
+  if (pl->topo.shard_n > 0) {
+    for (int n = 0; n < pl->topo.shard_n; n++) {
+      pl->shard_send_extent[n] = shard_se[n] * pl->topo.elem;
+      pl->shard_recv_extent[n] = shard_re[n] * pl->topo.elem;
+    }
+  }
   if (up.done) {
     pl->d_counts = up.d_dst;
     pl->counts_uploaded = true;
@@ -1125,6 +1210,7 @@ int tuna_plan_update_counts(tuna_plan_t *pl, const int64_t *sendcounts, const in
 
 int tuna_plan_update_counts_device(tuna_plan_t *pl, const int64_t *d_sendcounts, void *stream) {
   if (!pl || !d_sendcounts) return TUNA_ERR_INVALID_ARG;
+  if (pl->topo.shard_n > 0) return TUNA_ERR_INVALID_ARG;  // (the device-side packed layout is for one GPU)
   cudaStream_t st = (cudaStream_t)stream;
   const int64_t PP = (int64_t)pl->topo.P * pl->topo.P;
   // the plan keeps its own copy (the caller may reuse its array at once), in the
@@ -1140,7 +1226,7 @@ int tuna_plan_update_counts_device(tuna_plan_t *pl, const int64_t *d_sendcounts,
 
 int tuna_plan_set_row_maps(tuna_plan_t *pl, const int64_t *gather_rows, const int64_t *scatter_rows,
                            int64_t in_rows, int64_t out_rows, void *stream) {
-  if (!pl || in_rows < 0 || out_rows < 0) return TUNA_ERR_INVALID_ARG;
+  if (!pl || in_rows < 0 || out_rows < 0 || pl->topo.shard_n > 0) return TUNA_ERR_INVALID_ARG;
   if (!pl->tables_valid) return TUNA_ERR_INTERNAL;
   cudaStream_t st = (cudaStream_t)stream;
   const TunaTopo &t = pl->topo;

@@ -81,6 +81,14 @@ struct tuna_plan {
                                                // [1 + list id]: bytes of that list's blocks whose source
                                                // and destination differ modulo 16
 
+  // Sharded plan (topo.shard_n > 0): per GPU, the bytes of its send and receive buffer
+  // the layout covers; on the device the receive extents (for the self-check) and the
+  // GPUs' receive buffer addresses (for the mover), the latter set by every exchange call.
+  std::vector<int64_t> shard_send_extent, shard_recv_extent;
+  int64_t *d_peer_extent = nullptr;
+  char **d_peer_ptrs = nullptr;
+  std::vector<char *> h_peer_ptrs;  // what d_peer_ptrs was last given
+
   std::vector<int64_t> h_wbase;  // workspace offset of every phase's KEEP stream
   int64_t workspace_need = 0;
   char *workspace = nullptr;
@@ -146,6 +154,21 @@ int await_tables(tuna_plan *pl, cudaStream_t st);
 cudaEvent_t take_event(tuna_plan *pl);
 int validate_layout(int P, const int64_t *counts, const int64_t *sdispls, const int64_t *rdispls,
                     const int64_t *sendbase, const int64_t *recvbase);
+// Creates a plan; shard_n > 0 makes it the plan of GPU shard_me among shard_n (then
+// g == shard_n, the global radix is g, and sendbase / recvbase are per GPU).
+int plan_create(tuna_plan_t **out, int P, int radix, int radix_global, int block_count, int l, int g,
+                int elem_size, unsigned flags, const int64_t *sendcounts, const int64_t *sdispls,
+                const int64_t *rdispls, const int64_t *sendbase, const int64_t *recvbase, void *stream,
+                int shard_n = 0, int shard_me = 0);
+// Region bases of a sharded layout: every GPU's buffers hold the regions of its own l
+// ranks; a NULL base array means they are packed in rank order from offset 0 of that
+// GPU's buffer.  Also every GPU's buffer extents, in elements.
+void shard_layout(int P, int l, const int64_t *counts, const int64_t *sdispls, const int64_t *rdispls,
+                  const int64_t *sendbase, const int64_t *recvbase, std::vector<int64_t> *sb,
+                  std::vector<int64_t> *rb, std::vector<int64_t> *send_extent,
+                  std::vector<int64_t> *recv_extent);
+TunaListArgs list_args(const TunaList &l);
+TunaMoveArgs move_args(const tuna_plan *pl, const void *send, void *recv, char *work);
 // Multiprocessors of the current device (read once per device; 148 on a B200).
 int sm_count();
 

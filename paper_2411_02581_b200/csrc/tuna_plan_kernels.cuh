@@ -22,6 +22,14 @@ __device__ __forceinline__ int64_t compact_of(int64_t v, int64_t stride, int rad
   return (int64_t)hi * (radix - 1) * stride + (rem - stride);
 }
 
+// Sharded plans: does this GPU hold rank p, and where does rank p receive.
+__device__ __forceinline__ bool resident(const TunaTopo &t, int p) {
+  return t.shard_n == 0 || p / t.Q == t.shard_me;
+}
+__device__ __forceinline__ int64_t recv_loc(const TunaTopo &t, int p, int64_t off) {
+  return TUNA_LOC(t.shard_n ? TUNA_BUF_PEER0 + p / t.Q : TUNA_BUF_RECV, off);
+}
+
 struct PhaseDev {
   int level, radix, count;
   int64_t stride, moving, per_rank, finals;
@@ -66,9 +74,9 @@ __global__ void tuna_init_tables_kernel(TunaTopo t, const int64_t *__restrict__ 
   }
   if (sigma == 0) {
     const int64_t r = rot_dense ? idx : p;
-    rot_len[r] = bytes;
+    rot_len[r] = resident(t, p) ? bytes : 0;  // (a sharded plan copies its own ranks' self blocks only)
     rot_src[r] = sloc;
-    rot_dst[r] = TUNA_LOC(TUNA_BUF_RECV, (recvbase[p] + rdispls[(int64_t)p * t.P + p]) * t.elem);
+    rot_dst[r] = recv_loc(t, p, (recvbase[p] + rdispls[(int64_t)p * t.P + p]) * t.elem);
   }
 }
 
@@ -109,9 +117,12 @@ __global__ void tuna_meta_exchange_kernel(TunaTopo t, PhaseDev ph, const int64_t
       }
       const int sender = ns * t.Q + qs;
       const int64_t c = row_position(t, ph, io, jo);
-      const int64_t bytes = sz_cur[(int64_t)sender * t.P + sigma];
+      const int64_t size = sz_cur[(int64_t)sender * t.P + sigma];
       const int64_t where = loc_cur[(int64_t)sender * t.P + sigma];
-      sz_next[idx] = bytes;
+      sz_next[idx] = size;
+      // sharded plans list a block only on the GPU that moves it: the receiver's in a
+      // local phase (both ranks are there), the sender's in the global phase (a push)
+      const int64_t bytes = resident(t, ph.level == 0 ? p : sender) ? size : 0;
       if (c < ph.finals) {
         const int64_t e = (int64_t)p * ph.finals + c;
         del_len[e] = bytes;
@@ -165,6 +176,7 @@ __global__ void tuna_meta_exchange_diag_kernel(TunaTopo t, PhaseDev ph, const in
   const int tiles = (Q + 31) / 32;
   const int g0 = ((int)blockIdx.x % tiles) * 32, s0 = ((int)blockIdx.x / tiles) * 32;  // first jo, first sender id
   const int io = blockIdx.y, n = blockIdx.z;
+  const bool listed = t.shard_n == 0 || n == t.shard_me;  // (sharded plans: only the own group's blocks get a length)
   const int64_t row0 = (int64_t)n * Q;       // first rank of the group
   const int col0 = io * Q;                   // first slot of the destination group offset
   for (int j = ty; j < 32; j += 8) {
@@ -178,7 +190,7 @@ __global__ void tuna_meta_exchange_diag_kernel(TunaTopo t, PhaseDev ph, const in
     int64_t sum = 0;
 #pragma unroll 8
     for (int j = 0; j < 32; j++) sum += s_sz[j][tx];
-    if (sum > 0) atomicAdd(&round_bytes[g0 + tx], (unsigned long long)sum);
+    if (sum > 0 && listed) atomicAdd(&round_bytes[g0 + tx], (unsigned long long)sum);
   }
   for (int pr = ty; pr < 63; pr += 8) {  // receivers s0 + g0 + pr (mod Q): a diagonal of the tile each
     const int sr = pr - tx;
@@ -188,9 +200,11 @@ __global__ void tuna_meta_exchange_diag_kernel(TunaTopo t, PhaseDev ph, const in
     int q = sd + g;
     if (q >= Q) q -= Q;
     const int64_t p = row0 + q;
-    const int64_t bytes = s_sz[sr][tx], where = s_loc[sr][tx];
+    int64_t bytes = s_sz[sr][tx];
+    const int64_t where = s_loc[sr][tx];
     sz_next[p * P + col0 + g] = bytes;  // (jo = 0 never moves in this phase: sender and receiver are the same rank)
     if (g == 0) continue;
+    if (!listed) bytes = 0;
     const int64_t c = (int64_t)io * ph.moving + (g - 1);  // position among the blocks the rank receives, in slot order
     if (c < ph.finals) {
       const int64_t e = p * ph.finals + c;
@@ -463,8 +477,7 @@ __global__ void tuna_place_kernel(TunaTopo t, PhaseDev ph, const int64_t *__rest
   const unsigned sr = (unsigned)ph.stride * (unsigned)ph.radix;
   const bool fin = ph.level == 0 ? (io == 0 && (unsigned)jo < sr) : (unsigned)io < sr;
   const int origin = (n - io + (n < io ? t.N : 0)) * t.Q + (q - jo + (q < jo ? t.Q : 0));
-  const int64_t rloc =
-      TUNA_LOC(TUNA_BUF_RECV, (recvbase[p] + rdispls[(int64_t)p * t.P + origin]) * t.elem);
+  const int64_t rloc = recv_loc(t, p, (recvbase[p] + rdispls[(int64_t)p * t.P + origin]) * t.elem);
   if (c < ph.finals) {  // DELIVER list (only in direct-to-R mode; these blocks have arrived)
     const int64_t e = (int64_t)p * ph.finals + c;
     del_pos[e] += del_base[p];
@@ -540,7 +553,8 @@ __device__ __forceinline__ void check_list_body(const int64_t *__restrict__ len,
                                                 int64_t n, const int64_t *__restrict__ extents,
                                                 const int64_t *__restrict__ work_extent, int64_t keep_base_index,
                                                 const int64_t *__restrict__ wbase, unsigned long long *violations,
-                                                unsigned long long *unaligned_bytes) {
+                                                unsigned long long *unaligned_bytes,
+                                                const int64_t *__restrict__ peer_extents = nullptr) {
   bool bad = false;
   int64_t skewed = 0;  // bytes of blocks whose source and destination differ modulo 16
   const int64_t send_extent = extents[0], recv_extent = extents[1];
@@ -554,8 +568,11 @@ __device__ __forceinline__ void check_list_body(const int64_t *__restrict__ len,
       const int64_t so = TUNA_LOC_OFF(s);
       const int64_t sext = sb == TUNA_BUF_SEND ? send_extent : (sb == TUNA_BUF_WORK ? wext : -1);
       bad = bad || so < 0 || so + L > sext;
-      if (dst) {  // DELIVER: into the receive buffer
-        bad = bad || TUNA_LOC_BUF(d) != TUNA_BUF_RECV || TUNA_LOC_OFF(d) + L > recv_extent;
+      if (dst) {  // DELIVER: into the receive buffer (sharded plans: the receiving GPU's)
+        const int db = TUNA_LOC_BUF(d);
+        const int64_t dext = db == TUNA_BUF_RECV ? recv_extent
+                                                 : (db >= TUNA_BUF_PEER0 && peer_extents ? peer_extents[db - TUNA_BUF_PEER0] : -1);
+        bad = bad || TUNA_LOC_OFF(d) + L > dext;
         if (((so - TUNA_LOC_OFF(d)) & 15) != 0) skewed += L;
       } else {    // KEEP: at its stream position in the phase's workspace region
         const int64_t o = wb + p0;
@@ -599,11 +616,12 @@ struct TunaCheckItem {
 
 __global__ void tuna_check_lists_kernel(const TunaCheckItem *__restrict__ items, const int64_t *__restrict__ extents,
                                         const int64_t *__restrict__ work_extent,
-                                        const int64_t *__restrict__ wbase, unsigned long long *violations) {
+                                        const int64_t *__restrict__ wbase, unsigned long long *violations,
+                                        const int64_t *__restrict__ peer_extents) {
   const TunaCheckItem it = items[blockIdx.y];
   if ((int64_t)blockIdx.x * blockDim.x >= it.n) return;  // (whole CTA: short lists need few of them)
   check_list_body(it.len, it.pos, it.src, it.dst, it.n, extents, work_extent, it.keep_base_index, wbase,
-                  violations, violations + 1 + it.id);
+                  violations, violations + 1 + it.id, peer_extents);
 }
 
 // out = in^T, in 32 x 32 tiles through shared memory so that both the reads and the
