@@ -16,6 +16,7 @@ TunaListArgs list_args(const TunaList &l) {
   a.total = l.total;
   a.chunk = l.chunk;
   a.nchunks = l.n > 0 ? l.nchunks : 0;
+  a.skewed = 2 * l.unaligned_bytes > l.bytes ? 1 : 0;
   return a;
 }
 

@@ -85,6 +85,7 @@ struct TunaListArgs {
   const int64_t *len, *pos, *src, *dst;
   const int32_t *chunk_first;
   int64_t n, total, chunk, nchunks;  // nchunks == 0: the list takes no part in the launch
+  int skewed;  // most of the list's bytes sit in blocks whose source and destination differ modulo 16
 };
 
 // One launch moves up to three independent lists: the CTAs [0, keep.nchunks) take
@@ -100,6 +101,8 @@ struct TunaMoveArgs {
   int *error;         // device flag raised when a bounded wait inside a kernel gave up (may be null)
   int bulk_off;       // in: non-zero asks for the bulk-copy route; the launcher turns it into the offset
                       // of the staging area in dynamic shared memory (0 = route off)
+  int wait_first;     // set by the launcher: wait for the previous kernel of the stream before the first
+                      // table read (the first launch of an exchange, which may follow the plan kernels)
 };
 
 enum TunaMoveKernel {
@@ -109,11 +112,12 @@ enum TunaMoveKernel {
 };
 
 // Launches one mover kernel (tuna_move.cu).  `small_blocks` picks the build tuned
-// for lists whose blocks are far smaller than a chunk.  `early_start` lets the
-// kernel's CTAs begin their set-up while the previous kernel of the stream drains
-// (they read the plan's tables before they wait for it): only for a launch whose
+// for lists whose blocks are far smaller than a chunk.  Every launch may be scheduled
+// while the previous kernel of the stream drains; `early_start` also lets its CTAs
+// read the plan's tables before they wait for that kernel: only for a launch whose
 // predecessor on the stream is an earlier launch of the same exchange, never for
-// the first one, which may follow the kernels that write those tables.
+// the first one, which may follow the kernels that write those tables (it waits
+// before its first table read instead).
 cudaError_t tuna_launch_move(int kernel, const TunaMoveArgs &a, bool small_blocks, bool early_start,
                              cudaStream_t stream);
 

@@ -233,10 +233,11 @@ __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wa
 // while the previous launch is still draining, do their set-up (which reads only
 // the plan's tables), and then block in hardware until the previous launch has
 // completed and its writes are visible.  Every launch lets its successor start
-// early right away.  The first launch of an exchange starts the ordinary way:
-// what precedes it on the stream may be the plan kernels that write the very
-// tables its set-up reads, and their stores are only guaranteed visible to a
-// launch that waits for them in full.
+// early right away.  The first launch of an exchange waits before it reads
+// anything: what precedes it on the stream may be the plan kernels that write the
+// very tables its set-up reads, and their stores are only guaranteed visible
+// behind the wait (its CTAs are still scheduled early, which hides the launch
+// latency).
 
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
@@ -531,7 +532,7 @@ __device__ __forceinline__ void move_body(const TunaListArgs &l, const TunaMoveA
           if (!on) out[k] = nullptr;
         }
         const bool aligned = (reinterpret_cast<uintptr_t>(sa) & 15) == 0;
-        if (__all_sync(0xffffffffu, !on || (aligned && !careful))) {
+        if (!l.skewed && __all_sync(0xffffffffu, !on || (aligned && !careful))) {
           if (on) x[k] = ld16(sa);
         } else if (on) {
           if (!careful) {
@@ -571,6 +572,7 @@ __device__ __forceinline__ void move_body(const TunaListArgs &l, const TunaMoveA
 template <int kUnroll, bool kBulk>
 __device__ __forceinline__ void launch_body(const TunaMoveArgs &a) {
   grid_launch_dependents();
+  if (a.wait_first) grid_dependency_wait();  // the tables read below may be the previous kernel's output
   int64_t c = blockIdx.x;
   if (c < a.keep.nchunks) {
     move_body<false, kUnroll, kBulk>(a.keep, a, c);
@@ -659,7 +661,8 @@ cudaError_t tuna_launch_move(int kernel, const TunaMoveArgs &a_in, bool small_bl
     return !(e && e[0] == '0');
   }();
   cfg.attrs = attr;
-  cfg.numAttrs = (chain && early_start) ? 1 : 0;
+  cfg.numAttrs = chain ? 1 : 0;
+  a.wait_first = early_start ? 0 : 1;
   const cudaError_t le = cudaLaunchKernelEx(&cfg, fn, a);
   if (le != cudaSuccess) return le;
   return cudaGetLastError();
