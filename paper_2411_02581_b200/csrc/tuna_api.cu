@@ -121,7 +121,7 @@ int run_tuna(tuna_plan *pl, const void *send, void *recv, cudaStream_t st) {
     }
     const bool small = 2 * small_bytes >= bytes;
     Timed tm(pl, kind, bytes, st);
-    TUNA_CUDA(pl, tuna_launch_move(TUNA_K_ROUND, a, small, launches > 0, st));
+    TUNA_CUDA(pl, tuna_launch_move(TUNA_K_ROUND, a, small, launches > 0 || !pl->tables_fresh, st));
     launches++;
     smalls += small ? 1 : 0;
   }
@@ -129,13 +129,14 @@ int run_tuna(tuna_plan *pl, const void *send, void *recv, cudaStream_t st) {
     Timed tm(pl, TUNA_TIMER_ROTATE, pl->rot.bytes, st);
     TunaMoveArgs a = move_args(pl, send, recv, pl->workspace);
     a.rot = list_args(pl->rot);
-    TUNA_CUDA(pl, tuna_launch_move(TUNA_K_ROTATE, a, pl->rot.small_blocks, launches > 0, st));
+    TUNA_CUDA(pl, tuna_launch_move(TUNA_K_ROTATE, a, pl->rot.small_blocks, launches > 0 || !pl->tables_fresh, st));
     launches++;
     smalls += pl->rot.small_blocks ? 1 : 0;
   }
   pl->last_small = smalls;
   pl->last_launches = launches;
   pl->launch_count += launches;
+  if (launches > 0) pl->tables_fresh = false;  // (a launch that waited in full has run behind the plan kernels)
   return launches > 0 ? mark_in_flight(pl, st) : TUNA_OK;
 }
 
@@ -156,7 +157,7 @@ int run_direct(tuna_plan *pl, const void *send, void *recv, cudaStream_t st) {
       TunaMoveArgs a = move_args(pl, send, recv, nullptr);
       a.del = list_args(d);
       a.rot = list_args(pl->rot);
-      TUNA_CUDA(pl, tuna_launch_move(TUNA_K_DIRECT, a, 2 * small_bytes >= bytes, false, st));
+      TUNA_CUDA(pl, tuna_launch_move(TUNA_K_DIRECT, a, 2 * small_bytes >= bytes, !pl->tables_fresh, st));
       launches++;
       pl->last_small = 2 * small_bytes >= bytes ? 1 : 0;
     }
@@ -164,12 +165,13 @@ int run_direct(tuna_plan *pl, const void *send, void *recv, cudaStream_t st) {
     Timed tm(pl, TUNA_TIMER_DIRECT, pl->dir.bytes, st);
     TunaMoveArgs a = move_args(pl, send, recv, nullptr);
     a.del = list_args(pl->dir);
-    TUNA_CUDA(pl, tuna_launch_move(TUNA_K_DIRECT, a, pl->dir.small_blocks, false, st));
+    TUNA_CUDA(pl, tuna_launch_move(TUNA_K_DIRECT, a, pl->dir.small_blocks, !pl->tables_fresh, st));
     launches++;
     pl->last_small = pl->dir.small_blocks ? 1 : 0;
   }
   pl->last_launches = launches;
   pl->launch_count += launches;
+  if (launches > 0) pl->tables_fresh = false;  // (a launch that waited in full has run behind the plan kernels)
   return launches > 0 ? mark_in_flight(pl, st) : TUNA_OK;
 }
 
@@ -327,12 +329,13 @@ int tuna_rows_alltoallv(tuna_plan_t *pl, const void *rows_in, void *rows_out, vo
     a.extent[TUNA_BUF_SEND] = pl->rows_in_bytes;
     a.extent[TUNA_BUF_RECV] = pl->rows_out_bytes;
     a.del = list_args(l);
-    TUNA_CUDA(pl, tuna_launch_move(TUNA_K_DIRECT, a, l.small_blocks, false, st));
+    TUNA_CUDA(pl, tuna_launch_move(TUNA_K_DIRECT, a, l.small_blocks, !pl->tables_fresh, st));
     launches++;
     pl->last_small = l.small_blocks ? 1 : 0;
   }
   pl->last_launches = launches;
   pl->launch_count += launches;
+  if (launches > 0) pl->tables_fresh = false;  // (a launch that waited in full has run behind the plan kernels)
   return launches > 0 ? mark_in_flight(pl, st) : TUNA_OK;
 }
 

@@ -114,10 +114,10 @@ enum TunaMoveKernel {
 // Launches one mover kernel (tuna_move.cu).  `small_blocks` picks the build tuned
 // for lists whose blocks are far smaller than a chunk.  Every launch may be scheduled
 // while the previous kernel of the stream drains; `early_start` also lets its CTAs
-// read the plan's tables before they wait for that kernel: only for a launch whose
-// predecessor on the stream is an earlier launch of the same exchange, never for
-// the first one, which may follow the kernels that write those tables (it waits
-// before its first table read instead).
+// read the plan's tables before they wait for that kernel: only for a launch that
+// cannot follow the kernels that write those tables directly (a later launch of an
+// exchange, or the first one when an earlier exchange has already run behind the
+// last update); otherwise it waits before its first table read.
 cudaError_t tuna_launch_move(int kernel, const TunaMoveArgs &a, bool small_blocks, bool early_start,
                              cudaStream_t stream);
 

@@ -233,11 +233,12 @@ __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wa
 // while the previous launch is still draining, do their set-up (which reads only
 // the plan's tables), and then block in hardware until the previous launch has
 // completed and its writes are visible.  Every launch lets its successor start
-// early right away.  The first launch of an exchange waits before it reads
-// anything: what precedes it on the stream may be the plan kernels that write the
-// very tables its set-up reads, and their stores are only guaranteed visible
-// behind the wait (its CTAs are still scheduled early, which hides the launch
-// latency).
+// early right away.  The first launch after the plan's tables have been rewritten
+// waits before it reads anything: what precedes it on the stream may be the plan
+// kernels that write the very tables its set-up reads, and their stores are only
+// guaranteed visible behind the wait (its CTAs are still scheduled early, which
+// hides the launch latency).  Once one launch has run behind those kernels in
+// full, the tables are settled and later exchanges start early again.
 
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }

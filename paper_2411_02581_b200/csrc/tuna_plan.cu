@@ -829,6 +829,7 @@ int build_tables(tuna_plan *pl, const HostLayout *hl, const int64_t *sdispls, co
   rc = mark_tables_ready(pl, st);  // (no second wait on the host: exchanges order themselves behind this)
   if (rc) return rc;
   pl->tables_valid = true;
+  pl->tables_fresh = true;
   return TUNA_OK;
 }
 
@@ -1293,6 +1294,7 @@ int tuna_plan_set_row_maps(tuna_plan_t *pl, const int64_t *gather_rows, const in
   rc = mark_tables_ready(pl, st);
   if (rc) return rc;
   pl->rows_valid = true;
+  pl->tables_fresh = true;
   return TUNA_OK;
 }
 

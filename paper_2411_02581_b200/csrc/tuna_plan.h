@@ -56,6 +56,9 @@ struct tuna_plan {
   bool have_sdispls = false, have_rdispls = false;
   bool h_counts_valid = true;   // false after an update from device counts, until they are read back
   bool tables_valid = false;    // false while an update is under way and after one that failed
+  // The tables have been rewritten since the last exchange was enqueued: the next exchange's first
+  // launch must not read them before the kernels that wrote them are known to be complete.
+  bool tables_fresh = true;
   int64_t send_extent = 0, recv_extent = 0, payload = 0;  // bytes
 
   // device tables

@@ -165,6 +165,7 @@ int tuna_shard_alltoallv(tuna_plan_t *pl, const void *sendbuf, void *const *recv
       const int wrc = wait_in_flight(pl);  // an exchange still running reads the table rewritten below
       if (wrc) return wrc;
     }
+    pl->tables_fresh = true;  // (the launch that follows reads the table uploaded here)
     pl->h_peer_ptrs.assign(N, nullptr);
     for (int n = 0; n < N; n++) pl->h_peer_ptrs[n] = (char *)recvbufs[n];
     TUNA_CUDA(pl, cudaMemcpyAsync(pl->d_peer_ptrs, pl->h_peer_ptrs.data(), (size_t)N * sizeof(char *),
@@ -194,7 +195,7 @@ int tuna_shard_alltoallv(tuna_plan_t *pl, const void *sendbuf, void *const *recv
     }
     const bool small = 2 * small_bytes >= bytes;
     Timed tm(pl, level == 0 ? TUNA_TIMER_ROUND_LOCAL : TUNA_TIMER_ROUND_GLOBAL, bytes, st);
-    TUNA_CUDA(pl, tuna_launch_move(TUNA_K_ROUND, a, small, launches > 0, st));
+    TUNA_CUDA(pl, tuna_launch_move(TUNA_K_ROUND, a, small, launches > 0 || !pl->tables_fresh, st));
     launches++;
     smalls += small ? 1 : 0;
   }
@@ -203,13 +204,14 @@ int tuna_shard_alltoallv(tuna_plan_t *pl, const void *sendbuf, void *const *recv
     TunaMoveArgs a = move_args(pl, sendbuf, recvbufs[me], pl->workspace);
     a.bulk_off = 0;
     a.rot = list_args(pl->rot);
-    TUNA_CUDA(pl, tuna_launch_move(TUNA_K_ROTATE, a, pl->rot.small_blocks, launches > 0, st));
+    TUNA_CUDA(pl, tuna_launch_move(TUNA_K_ROTATE, a, pl->rot.small_blocks, launches > 0 || !pl->tables_fresh, st));
     launches++;
     smalls += pl->rot.small_blocks ? 1 : 0;
   }
   pl->last_launches = launches;
   pl->last_small = smalls;
   pl->launch_count += launches;
+  if (launches > 0) pl->tables_fresh = false;
   return launches > 0 ? mark_in_flight(pl, st) : TUNA_OK;
 }
 
