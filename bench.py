@@ -37,6 +37,11 @@ UNIT = "GB/s"
 # bytes moved, so the full-size figure is this ratio times the launch's bytes.  A
 # changed source makes the figures stale: the traffic is then reported as null.
 NCU_TRAFFIC_PER_PAYLOAD_BYTE: dict[str, dict[str, float]] = {
+    "3caae7ab91d126f8fdb8d1198d3337598395d5529248d37da030b3ef7b8b2b48": {
+        "c4/flat radix 64": 1.997,                                  # reduced to 2 GiB for the capture
+        "c5/flat radix 2048": 2.166, "c5/flat radix 2": 2.256,      # at full size (0.75 GB)
+        "c3/hierarchical l=16 g=16 radix 16/16": 1.539,             # at full size, both launches
+    },
 }
 
 
