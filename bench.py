@@ -566,8 +566,10 @@ def sharded_arm(args):
         send.view(torch.int64)[:ex.send_bytes // 8].random_()
     torch.cuda.empty_cache()
 
+    d_rows = torch.from_numpy(my_rows).to(dev)   # the batch's counts are in device memory, like its payload
+
     def step():
-        ex.update_counts(my_rows)
+        ex.update_counts_device(d_rows)
         ex.exchange(send)
 
     for _ in range(args.warmup):
@@ -622,7 +624,7 @@ def sharded_arm(args):
             "scaling": "strong", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
             "config": {"workload": f"{wl.name} P={wl.P}, {l} ranks per GPU: local radix {radix or max(2, l)}, "
                                    f"inter-GPU phase pushed into the peers' receive buffers, payload {payload} bytes "
-                                   f"in total, elem {E} B, re-plan every step from all-gathered counts",
+                                   f"in total, elem {E} B, re-plan every step from counts in device memory (all-gathered there)",
                        "l2": "inputs larger than L2" if payload / world > 256e6 else "inputs fit in L2",
                        "sharding": "one group of the hierarchical schedule per GPU",
                        "emulated_on_one_gpu": bool(args.same_device)},

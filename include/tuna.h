@@ -309,10 +309,11 @@ int tuna_direct_alltoallv_static(int P, int elem_size, const int64_t *sendcounts
  * GPU moves the block.  Introspection reports this GPU's share: a round's `bytes` are the
  * bytes this GPU moves in it, so the sum over the n_gpus plans is the round's volume.
  * tuna_plan_workspace_bytes / tuna_plan_set_workspace: this GPU's workspace (local
- * phases only; the inter-group phase needs none).  tuna_plan_update_counts works
- * (same rule for NULL bases); tuna_plan_update_counts_device, tuna_alltoallv,
- * tuna_direct_alltoallv, tuna_alltoallv_host and the row exchange return
- * TUNA_ERR_INVALID_ARG for a sharded plan.
+ * phases only; the inter-group phase needs none).  tuna_plan_update_counts and
+ * tuna_plan_update_counts_device work (the whole P x P matrix, all-gathered; packed
+ * bases per GPU; the buffer sizes may change: query tuna_shard_extents again);
+ * tuna_alltoallv, tuna_direct_alltoallv, tuna_alltoallv_host and the row exchange
+ * return TUNA_ERR_INVALID_ARG for a sharded plan.
  *
  * tuna_shard_extents - bytes of GPU `gpu`'s send and receive buffer that the layout covers.
  *

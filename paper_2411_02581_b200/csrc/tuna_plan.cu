@@ -665,7 +665,11 @@ int build_tables(tuna_plan *pl, const HostLayout *hl, const int64_t *sdispls, co
       tuna_segscan_kernel<0><<<gseg, th, 0, st>>>(pl->d_counts, pl->d_sdispls, pl->d_seg_total,
                                                    nullptr, P, P);
       TUNA_LAUNCHED(pl);
-      if (!hl) {  // send regions laid end to end: bases = scan of the row sums
+      if (!hl && t.shard_n > 0) {  // every GPU's send regions laid end to end from 0 of its own buffer
+        tuna_shard_bases_kernel<<<(unsigned)((P + th - 1) / th), th, 0, st>>>(pl->d_seg_total, P, t.Q, pl->d_sendbase,
+                                                                              pl->d_shard_send_total);
+        TUNA_LAUNCHED(pl);
+      } else if (!hl) {  // send regions laid end to end: bases = scan of the row sums
         tuna_segbase_kernel<<<1, 1024, 0, st>>>(pl->d_seg_total, nullptr, pl->d_sendbase, P, pl->d_scal, nullptr, 0,
                                                 nullptr, 0);
         TUNA_LAUNCHED(pl);
@@ -681,7 +685,15 @@ int build_tables(tuna_plan *pl, const HostLayout *hl, const int64_t *sdispls, co
       tuna_segscan_kernel<0><<<gseg, th, 0, st>>>(pl->d_tmp, pl->d_rdispls, pl->d_seg_total,
                                                    nullptr, P, P);
       TUNA_LAUNCHED(pl);
-      if (!hl) {  // receive regions likewise: scan of the column sums
+      if (!hl && t.shard_n > 0) {
+        tuna_shard_bases_kernel<<<(unsigned)((P + th - 1) / th), th, 0, st>>>(pl->d_seg_total, P, t.Q, pl->d_recvbase,
+                                                                              pl->d_shard_recv_total);
+        TUNA_LAUNCHED(pl);
+        tuna_shard_extents_kernel<<<1, 32, 0, st>>>(pl->d_shard_send_total, pl->d_shard_recv_total, t.shard_n,
+                                                    t.shard_me, t.elem, pl->d_extents, pl->d_peer_extent,
+                                                    pl->d_shard_send_extent);
+        TUNA_LAUNCHED(pl);
+      } else if (!hl) {  // receive regions likewise: scan of the column sums
         tuna_segbase_kernel<<<1, 1024, 0, st>>>(pl->d_seg_total, nullptr, pl->d_recvbase, P, pl->d_scal, nullptr, 0,
                                                 nullptr, 0);
         TUNA_LAUNCHED(pl);
@@ -795,6 +807,19 @@ int build_tables(tuna_plan *pl, const HostLayout *hl, const int64_t *sdispls, co
     pl->send_extent = ext[0];
     pl->recv_extent = ext[1];
     pl->payload = ext[2] * t.elem;
+    if (t.shard_n > 0) {  // every GPU's buffer sizes, worked out on the device
+      std::vector<int64_t> both(2 * (size_t)t.shard_n);
+      if (pl->h_readback) {
+        const int64_t *h = pl->h_readback + (pl->d_shard_send_extent - pl->d_readback);
+        std::copy(h, h + 2 * t.shard_n, both.begin());
+      } else {
+        TUNA_CUDA(pl, cudaMemcpy(both.data(), pl->d_shard_send_extent, both.size() * 8, cudaMemcpyDeviceToHost));
+      }
+      for (int n = 0; n < t.shard_n; n++) {
+        pl->shard_send_extent[n] = both[n];
+        pl->shard_recv_extent[n] = both[t.shard_n + n];
+      }
+    }
   }
   if (checked[0] != 0) return TUNA_ERR_INTERNAL;
   pl->h_wbase = wbase;
@@ -949,7 +974,6 @@ int tuna_plan_destroy(tuna_plan_t *pl) {
   cudaFree(pl->d_readback);  // (d_scal, d_wbase, d_extents, d_round_bytes, d_violations are slices of it)
   if (pl->h_readback) cudaFreeHost(pl->h_readback);
   cudaFree(pl->d_error);
-  cudaFree(pl->d_peer_extent);
   cudaFree(pl->d_peer_ptrs);
   for (auto &s : pl->stamps) {
     cudaEventDestroy(s.a);
@@ -1080,7 +1104,8 @@ int tuna_host::plan_create(tuna_plan_t **out, int P, int radix, int radix_global
   {
     const int64_t n_scal = 2 * (2 * nph + 3), n_wbase = nph + 1, n_ext = 6;  // ext [4], [5]: the row exchange's buffers
     const int64_t n_rb = std::max<int64_t>(pl->stats_n, 1), n_viol = 1 + 2 * nph + 3;
-    pl->readback_words = n_scal + n_wbase + n_ext + n_rb + n_viol;
+    const int64_t n_shard = 4 * (int64_t)shard_n;  // the GPUs' send and receive totals and extents
+    pl->readback_words = n_scal + n_wbase + n_ext + n_rb + n_viol + n_shard;
     TUNA_TRY(dev_alloc(&pl->d_readback, pl->readback_words));
     TUNA_TRY(cudaMemset(pl->d_readback, 0, (size_t)pl->readback_words * 8));
     if (cudaHostAlloc((void **)&pl->h_readback, (size_t)pl->readback_words * 8, cudaHostAllocDefault) != cudaSuccess) {
@@ -1092,10 +1117,15 @@ int tuna_host::plan_create(tuna_plan_t **out, int P, int radix, int radix_global
     pl->d_extents = pl->d_wbase + n_wbase;
     pl->d_round_bytes = reinterpret_cast<unsigned long long *>(pl->d_extents + n_ext);
     pl->d_violations = pl->d_round_bytes + n_rb;
+    if (shard_n > 0) {
+      pl->d_shard_send_total = reinterpret_cast<int64_t *>(pl->d_violations + n_viol);
+      pl->d_shard_recv_total = pl->d_shard_send_total + shard_n;
+      pl->d_shard_send_extent = pl->d_shard_recv_total + shard_n;
+      pl->d_peer_extent = pl->d_shard_send_extent + shard_n;
+    }
   }
   TUNA_TRY(dev_alloc(&pl->d_error, 1));
   if (shard_n > 0) {
-    TUNA_TRY(dev_alloc(&pl->d_peer_extent, shard_n));
     TUNA_TRY(dev_alloc(&pl->d_peer_ptrs, shard_n));
     TUNA_TRY(cudaMemset(pl->d_peer_ptrs, 0, (size_t)shard_n * sizeof(char *)));
   }
@@ -1211,7 +1241,6 @@ int tuna_plan_update_counts(tuna_plan_t *pl, const int64_t *sendcounts, const in
 
 int tuna_plan_update_counts_device(tuna_plan_t *pl, const int64_t *d_sendcounts, void *stream) {
   if (!pl || !d_sendcounts) return TUNA_ERR_INVALID_ARG;
-  if (pl->topo.shard_n > 0) return TUNA_ERR_INVALID_ARG;  // (the device-side packed layout is for one GPU)
   cudaStream_t st = (cudaStream_t)stream;
   const int64_t PP = (int64_t)pl->topo.P * pl->topo.P;
   // the plan keeps its own copy (the caller may reuse its array at once), in the

@@ -88,7 +88,8 @@ struct tuna_plan {
   // the layout covers; on the device the receive extents (for the self-check) and the
   // GPUs' receive buffer addresses (for the mover), the latter set by every exchange call.
   std::vector<int64_t> shard_send_extent, shard_recv_extent;
-  int64_t *d_peer_extent = nullptr;
+  int64_t *d_peer_extent = nullptr;   // (a slice of d_readback, like the three below)
+  int64_t *d_shard_send_total = nullptr, *d_shard_recv_total = nullptr, *d_shard_send_extent = nullptr;
   char **d_peer_ptrs = nullptr;
   std::vector<char *> h_peer_ptrs;  // what d_peer_ptrs was last given
 

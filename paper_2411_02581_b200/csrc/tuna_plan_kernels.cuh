@@ -656,6 +656,39 @@ __global__ void tuna_packed_extents_kernel(const int64_t *__restrict__ tot, int 
   }
 }
 
+// Sharded plans whose counts arrive in device memory: a GPU's regions are packed in
+// rank order from offset 0 of ITS buffer, so the bases are running sums that start
+// anew with every group of Q ranks.  base[p] = elements of the regions before rank p's
+// on its GPU; group_total[n] = elements of GPU n's buffer.
+__global__ void tuna_shard_bases_kernel(const int64_t *__restrict__ seg_total, int P, int Q, int64_t *base,
+                                        int64_t *group_total) {
+  const int p = blockIdx.x * blockDim.x + threadIdx.x;
+  if (p >= P) return;
+  const int n = p / Q;
+  int64_t sum = 0;
+  for (int i = n * Q; i < p; i++) sum += seg_total[i];
+  base[p] = sum;
+  if (p == n * Q + Q - 1) group_total[n] = sum + seg_total[p];
+}
+
+// ... and the extents that follow from the GPUs' totals: this GPU's two buffers and the
+// payload (extents[0..2], as for a plan on one GPU), every GPU's receive buffer for the
+// self-check (peer_extent) and every GPU's send buffer for the host (send_extent), in bytes.
+__global__ void tuna_shard_extents_kernel(const int64_t *__restrict__ send_total,
+                                          const int64_t *__restrict__ recv_total, int N, int me, int elem,
+                                          int64_t *extents, int64_t *peer_extent, int64_t *send_extent) {
+  if (blockIdx.x != 0 || threadIdx.x != 0) return;
+  int64_t all = 0;
+  for (int n = 0; n < N; n++) {
+    all += send_total[n];
+    peer_extent[n] = recv_total[n] * elem;
+    send_extent[n] = send_total[n] * elem;
+  }
+  extents[0] = send_total[me] * elem;
+  extents[1] = recv_total[me] * elem;
+  extents[2] = all;
+}
+
 }  // namespace
 
 #endif

@@ -106,6 +106,33 @@ class ShardedExchange:
         if self.plan.workspace_bytes() > self.workspace.numel():
             self.workspace = self.plan.alloc_workspace(device=self.device)
 
+    def update_counts_device(self, my_rows_dev, stream=None):
+        """The same from counts in device memory (routing decided on the GPU): ``my_rows_dev``
+        is an int64 CUDA tensor ``[l, P]``; the matrix is all-gathered on the device (NCCL;
+        with gloo through the host) and the plan re-built from it there.  Only a few totals
+        cross back to the host."""
+        import torch
+        multi = self.world > 1
+        if not multi:
+            full = my_rows_dev.contiguous()
+        elif self.dist.get_backend(self.group) == "nccl":
+            full = torch.empty((self.P, self.P), dtype=torch.int64, device=self.device)
+            if stream is None:
+                self.dist.all_gather_into_tensor(full, my_rows_dev.contiguous(), group=self.group)
+            else:
+                with torch.cuda.stream(stream):
+                    self.dist.all_gather_into_tensor(full, my_rows_dev.contiguous(), group=self.group)
+        else:
+            full = torch.from_numpy(gather_counts(my_rows_dev.cpu().numpy(), self.dist, self.group)).to(self.device)
+        self.plan.update_counts_device(full, stream=stream)
+        se, re = self.plan.shard_extents(self.me)
+        if re > self.recv.numel():
+            raise ValueError("the receive buffer is too small for the new counts")
+        self.send_bytes, self.recv_bytes = se, re
+        self.counts = None            # (the host copy is stale now)
+        if self.plan.workspace_bytes() > self.workspace.numel():
+            self.workspace = self.plan.alloc_workspace(device=self.device)
+
     def _barrier(self, stream):
         import torch
         if self.dist.get_backend(self.group) == "nccl":

@@ -70,9 +70,14 @@ def main():
         ex = S.ShardedExchange(P, E, wl.sendcounts[mine.start:mine.stop], radix=radix, dist=dist)
         assert (ex.send_bytes, ex.recv_bytes) == (cut_s[rank + 1] - cut_s[rank], cut_r[rank + 1] - cut_r[rank])
         my_send = torch.from_numpy(send[cut_s[rank]:cut_s[rank + 1]]).cuda()
-        for _ in range(2):                                                   # twice: the buffers are reused
+        d_rows = torch.from_numpy(np.ascontiguousarray(wl.sendcounts[mine.start:mine.stop])).cuda()
+        for it in range(3):                                                  # again and again: the buffers are reused
             ex.recv.fill_(CANARY)
             torch.cuda.synchronize()
+            if it == 1:
+                ex.update_counts(wl.sendcounts[mine.start:mine.stop])        # re-plan from host rows ...
+            if it == 2:
+                ex.update_counts_device(d_rows)                              # ... and from rows in device memory
             ex.exchange(my_send)
             got = ex.recv[:ex.recv_bytes].cpu().numpy()
             assert np.array_equal(got, ref[cut_r[rank]:cut_r[rank + 1]])

@@ -120,6 +120,73 @@ def test_local_part_alone_leaves_the_own_groups_blocks(P, G, radix):
     assert np.array_equal(got, ref)
 
 
+def oracle_brute(wl):
+    return oracle.bruteforce(wl, wl.make_send().numpy(), wl.make_recv(fill=CANARY).numpy().copy())
+
+
+def test_large_blocks_cross_between_shards():
+    """Megabyte blocks: the pushes run the large-block build of the mover (chunks inside one
+    block, plain and skewed) with destinations in the other shards' buffers."""
+    wl = W.make_random(8, 2_100_000, elem_size=1, seed=5, zero_frac=0.1, gaps=True)      # odd byte counts: skewed
+    assert wl.payload_bytes_total > 48 << 20
+    ref = oracle_brute(wl)
+    for G in (2, 4):
+        got, plans = run_sharded(wl, G, 2)
+        assert np.array_equal(got, ref)
+        assert any(p.last_launches() > p.last_small_launches() for p in plans)            # the large build did run
+    aligned = W.make_c4(P=16, tokens=256, hidden=2048)                                  # 4 KiB rows, aligned
+    got, _ = run_sharded(aligned, 4, 0)
+    assert np.array_equal(got, oracle_brute(aligned))
+
+
+@pytest.mark.parametrize("elem", [1, 3, 8, 48])
+def test_element_sizes(elem):
+    wl = W.make_random(12, 300, elem_size=elem, seed=elem, zero_frac=0.2, gaps=True)
+    ref = oracle_brute(wl)
+    for G, r in ((3, 2), (6, 0), (12, 2)):
+        got, _ = run_sharded(wl, G, r)
+        assert np.array_equal(got, ref)
+
+
+def test_c5_over_eight_shards():
+    """The 2048-rank workload of tiny unaligned blocks, 256 ranks per shard: every byte
+    against the definition of the exchange, the shards' rounds against the oracle's."""
+    wl = W.make_c5()
+    l, G = wl.P // 8, 8
+    ref, rounds, _, _ = oracle_hier(wl, l, G, l)
+    got, plans = run_sharded(wl, G, 0, explicit_bases=False)
+    assert np.array_equal(got, ref)
+    total = np.zeros(len(rounds), dtype=np.int64)
+    for plan in plans:
+        total += np.array([r["bytes"] for r in plan.rounds()])
+    assert np.array_equal(total, rounds[:, oracle.RS_BYTES_SENT])
+    # every shard's launches: one local phase (with the self blocks) and the push
+    assert all(p.last_launches() == 2 for p in plans)
+
+
+def test_timing_kinds_and_self_blocks_only():
+    wl = W.make_random(8, 200, elem_size=2, seed=21)
+    plans = None
+    got, plans = run_sharded(wl, 8, 2)                       # one rank per shard: no local phase at all
+    assert np.array_equal(got, oracle_brute(wl))
+    diag = W._finish("diag", 8, 2, 1, np.diag(np.arange(1, 9)).astype(np.int64))    # nothing but self blocks
+    got, plans = run_sharded(diag, 4, 2)
+    assert np.array_equal(got, oracle_brute(diag))
+    wl2 = W.make_random(16, 200, elem_size=2, seed=22)
+    cut_s, cut_r, sb, rb = shard_buffers(wl2, 2)
+    plan = B.Plan(16, 4, elem_size=2, sendcounts=wl2.sendcounts, sdispls=wl2.sdispls, rdispls=wl2.rdispls,
+                  sendbase=sb, recvbase=rb, shard=(2, 0))
+    plan.alloc_workspace()
+    plan.enable_timing(True)
+    send = wl2.make_send("cuda")[cut_s[0]:cut_s[1]].clone()
+    recvs = [torch.zeros(max(cut_r[n + 1] - cut_r[n], 16), dtype=torch.uint8, device="cuda") for n in range(2)]
+    plan.shard_alltoallv(send, recvs)
+    t = plan.get_timing()
+    assert t["round_local"]["launches"] == 2 and t["round_global"]["launches"] == 1     # radix 4 over 8 ranks: 2 local phases
+    mine = plan.rounds()
+    assert t["round_global"]["bytes"] == sum(r["bytes"] for r in mine if r["level"] == 1)
+
+
 def test_packed_bases_and_recount():
     """NULL bases = every GPU's regions packed from offset 0 of its own buffers; an update
     with new counts re-plans the shard."""
@@ -146,6 +213,32 @@ def test_packed_bases_and_recount():
     torch.cuda.synchronize()
     got2 = torch.cat([recvs[n][:cut_r[n + 1] - cut_r[n]] for n in range(G)]).cpu().numpy()
     assert np.array_equal(got2, ref2)
+    # and from a count matrix in device memory: bases and buffer sizes worked out on the device
+    wl3 = W.make_random(P, 700, elem_size=4, seed=6, zero_frac=0.4)
+    ref3, rounds3, _, _ = oracle_hier(wl3, P // G, G, 2)
+    cut_s, cut_r, _, _ = shard_buffers(wl3, G)
+    d_counts = torch.from_numpy(wl3.sendcounts).cuda()
+    send = wl3.make_send("cuda")
+    recvs = [torch.full((max(cut_r[n + 1] - cut_r[n], 16),), CANARY, dtype=torch.uint8, device="cuda")
+             for n in range(G)]
+    total = np.zeros(len(rounds3), dtype=np.int64)
+    for n, plan in enumerate(plans):
+        plan.update_counts_device(d_counts)
+        for m in range(G):
+            assert plan.shard_extents(m) == (cut_s[m + 1] - cut_s[m], cut_r[m + 1] - cut_r[m])
+        assert plan.extents() == (cut_s[n + 1] - cut_s[n], cut_r[n + 1] - cut_r[n], wl3.payload_bytes_total)
+        plan.alloc_workspace()
+        plan.shard_alltoallv(send[cut_s[n]:cut_s[n + 1]].clone(), recvs)
+        total += np.array([r["bytes"] for r in plan.rounds()])
+    torch.cuda.synchronize()
+    got3 = torch.cat([recvs[n][:cut_r[n + 1] - cut_r[n]] for n in range(G)]).cpu().numpy()
+    assert np.array_equal(got3, ref3)
+    assert np.array_equal(total, rounds3[:, oracle.RS_BYTES_SENT])
+    neg = d_counts.clone()
+    neg[3, 5] = -2
+    with pytest.raises(B.TunaError, match="INVALID_ARG"):
+        plans[0].update_counts_device(neg)
+    plans[0].update_counts_device(d_counts)                  # and the plan recovers
 
 
 def test_sharded_plan_argument_checks():
@@ -165,9 +258,6 @@ def test_sharded_plan_argument_checks():
     plan.alloc_workspace()
     with pytest.raises(B.TunaError, match="OVERLAP"):
         plan.shard_alltoallv(buf, [buf, buf[32768:]])
-    d_counts = torch.from_numpy(wl.sendcounts).cuda()
-    with pytest.raises(B.TunaError, match="INVALID_ARG"):
-        plan.update_counts_device(d_counts)
 
 
 def test_two_processes_share_one_gpu():
