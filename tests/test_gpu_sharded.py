@@ -124,9 +124,10 @@ def oracle_brute(wl):
     return oracle.bruteforce(wl, wl.make_send().numpy(), wl.make_recv(fill=CANARY).numpy().copy())
 
 
-def test_large_blocks_cross_between_shards():
+def test_large_blocks_cross_between_shards(monkeypatch):
     """Megabyte blocks: the pushes run the large-block build of the mover (chunks inside one
     block, plain and skewed) with destinations in the other shards' buffers."""
+    monkeypatch.setenv("TUNA_SMALL_LIST_BYTES", "0")      # (lists this short would otherwise take the other build)
     wl = W.make_random(8, 2_100_000, elem_size=1, seed=5, zero_frac=0.1, gaps=True)      # odd byte counts: skewed
     assert wl.payload_bytes_total > 48 << 20
     ref = oracle_brute(wl)
