@@ -276,7 +276,7 @@ def run_bruteforce_once(wl, send, recv):
     return time.perf_counter() - t0
 
 
-def cpu_baseline_block(wl_name, radix_arg, full_send=None, full_wl=None, runs=5):
+def cpu_baseline_block(wl_name, radix_arg, full_send=None, full_wl=None, runs=7):
     """The oracle, as it stands, on the host cores: the definition of the exchange (the
     CPU's own direct exchange), the headline schedule on one thread and, for flat
     schedules, the same steps with the ranks shared out over all cores; on a bounded
@@ -291,11 +291,13 @@ def cpu_baseline_block(wl_name, radix_arg, full_send=None, full_wl=None, runs=5)
     pay = wls.payload_bytes_total
     flat = not (wls.hier and not wls.radices)
     first = run_oracle_once(wls, r, hs, hr)                       # first touch of every buffer
+    run_oracle_once(wls, r, hs, hr)                               # (one more: the allocator's pools settle)
     one = [run_oracle_once(wls, r, hs, hr) for _ in range(runs)]
     brute = [run_bruteforce_once(wls, hs, hr) for _ in range(runs)]
     block = {"value": pay / statistics.median(one) / 1e9, "unit": UNIT, "cores": 1, "threads": 1,
-             "kind": "oracle", "sample": sample + f", median of {runs} runs after one warm-up run",
+             "kind": "oracle", "sample": sample + f", median of {runs} runs after two warm-up runs",
              "first_run_GBps": pay / first / 1e9,
+             "min_max_GBps": [pay / max(one) / 1e9, pay / min(one) / 1e9],
              "bruteforce_GBps": pay / statistics.median(brute) / 1e9,
              "cpu_model": cpu_model(), "host_cores_available": cores,
              "allocator_pinned": pinned}
