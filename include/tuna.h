@@ -301,7 +301,7 @@ int tuna_direct_alltoallv_static(int P, int elem_size, const int64_t *sendcounts
  *                 order from offset 0.  sdispls / rdispls as in tuna_plan_create.
  *   flags         TUNA_FLAG_CLASSIC_ROTATE and TUNA_FLAG_BULK_COPY are refused
  *                 (TUNA_ERR_INVALID_ARG); TUNA_FLAG_NO_DIRECT is implied.
- *   errors        P not a multiple of n_gpus: TUNA_ERR_BAD_HIERARCHY; n_gpus above 240 or
+ *   errors        P not a multiple of n_gpus: TUNA_ERR_BAD_HIERARCHY; n_gpus above 111 or
  *                 my_gpu outside [0, n_gpus): TUNA_ERR_INVALID_ARG; otherwise as
  *                 tuna_plan_create.
  * The plan holds the tables of all P ranks (the metadata work is replicated on every

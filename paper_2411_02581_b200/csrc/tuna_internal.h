@@ -15,6 +15,7 @@
 #define TUNA_BUF_WORK 2
 // Sharded plans (ranks spread over several GPUs): the receive buffer of GPU n.
 #define TUNA_BUF_PEER0 16
+#define TUNA_MAX_SHARDS (127 - TUNA_BUF_PEER0)  // (a buffer id sits in the top byte of a location and stays positive)
 #define TUNA_LOC(buf, off) ((((int64_t)(buf)) << 56) | (int64_t)(off))
 #define TUNA_LOC_BUF(loc) ((int)((loc) >> 56))
 #define TUNA_LOC_OFF(loc) ((loc) & ((((int64_t)1) << 56) - 1))

@@ -999,7 +999,7 @@ int tuna_host::plan_create(tuna_plan_t **out, int P, int radix, int radix_global
     // one group per GPU, one hop between GPUs, blocks delivered straight into the receive
     // buffers, no direct list (a GPU reaches only its own send buffer)
     if (shard_n != g || shard_me < 0 || shard_me >= shard_n || block_count != 0 ||
-        shard_n > 256 - TUNA_BUF_PEER0 || (flags & (TUNA_FLAG_CLASSIC_ROTATE | TUNA_FLAG_BULK_COPY)))
+        shard_n > TUNA_MAX_SHARDS || (flags & (TUNA_FLAG_CLASSIC_ROTATE | TUNA_FLAG_BULK_COPY)))
       return TUNA_ERR_INVALID_ARG;
     radix_global = std::max(2, g);
     flags |= TUNA_FLAG_NO_DIRECT;
