@@ -327,8 +327,10 @@ int tuna_direct_alltoallv_static(int P, int elem_size, const int64_t *sendcounts
  *               use; separately they let a caller overlap or inspect the two parts.  The
  *               push reads what the local phases left in the workspace: same stream, or
  *               ordered by the caller.
- * Asynchronous on `stream`; only enqueues kernels.  No kernel waits for another GPU, so
- * the call cannot deadlock whatever the other GPUs do.  It does NOT tell when the other
+ * Asynchronous on `stream`; enqueues kernels and, when the addresses in `recvbufs` differ
+ * from the previous call's, one small copy of them from a host array the plan keeps (so
+ * a call whose addresses changed is not for stream capture).  No kernel waits for another
+ * GPU, so the call cannot deadlock whatever the other GPUs do.  It does NOT tell when the other
  * GPUs' stores into this GPU's receive buffer have landed: the caller closes the exchange
  * with a barrier across the GPUs that is ordered behind this call on every GPU's stream
  * (e.g. an NCCL all-reduce on the same stream), and must not reuse a receive buffer

@@ -266,7 +266,11 @@ def test_two_processes_share_one_gpu():
     counts all-gathered, receive buffers exported and mapped through memory handles, the
     push into the other process's buffer, host-level barriers (the NCCL backend needs one
     GPU per process, so this run uses gloo)."""
-    env = dict(os.environ, MASTER_ADDR="127.0.0.1", MASTER_PORT="29631", PYTHONPATH=ROOT)
+    import socket
+    with socket.socket() as sock:                      # a port that is free right now
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    env = dict(os.environ, MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), PYTHONPATH=ROOT)
     procs = [subprocess.Popen([sys.executable, os.path.join(ROOT, "tests", "sharded_worker.py"), str(r), "2"],
                               env=env, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)
              for r in range(2)]

@@ -20,7 +20,11 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 @pytest.mark.parametrize("world", [2, 3])
 def test_gloo_processes_agree_with_the_oracle(world):
     build_mod.build()
-    env = dict(os.environ, MASTER_ADDR="127.0.0.1", MASTER_PORT=str(29640 + world), PYTHONPATH=ROOT,
+    import socket
+    with socket.socket() as sock:                      # a port that is free right now
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    env = dict(os.environ, MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), PYTHONPATH=ROOT,
                CUDA_VISIBLE_DEVICES="")
     procs = [subprocess.Popen([sys.executable, os.path.join(ROOT, "tests", "sharded_worker.py"), str(r),
                                str(world), "cpu"], env=env, stdout=subprocess.PIPE, stderr=subprocess.STDOUT,
