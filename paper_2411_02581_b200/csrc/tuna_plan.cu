@@ -730,22 +730,25 @@ int build_tables(tuna_plan *pl, const HostLayout *hl, const int64_t *sdispls, co
         continue;
       }
       PhaseDev pd{ph.level, ph.radix, ph.count, ph.stride, ph.moving, ph.per_rank, ph.finals};
+      // (the tables that follow the blocks have no reader behind the last phase)
+      int64_t *const sz_next = f + 1 < nph ? pl->d_sz[cur ^ 1] : nullptr;
+      int64_t *const loc_next = f + 1 < nph ? pl->d_loc[cur ^ 1] : nullptr;
       if (ph.level == 0 && ph.stride == 1 && ph.radix >= t.Q && t.N <= 65535) {
         const unsigned tiles = (unsigned)((t.Q + 31) / 32);
         tuna_meta_exchange_diag_kernel<<<dim3(tiles * tiles, t.N, t.N), dim3(32, 8), 0, st>>>(
-            t, pd, pl->d_sz[cur], pl->d_loc[cur], pl->d_sz[cur ^ 1], k.len, k.src, d.len, d.src,
+            t, pd, pl->d_sz[cur], pl->d_loc[cur], sz_next, k.len, k.src, d.len, d.src,
             pl->d_round_bytes + ph.stats_off);
       } else {
         const size_t smem = ph.radix <= 4096 ? (size_t)ph.radix * 8 : 0;
         tuna_meta_exchange_kernel<<<gPP, th, smem, st>>>(t, pd, pl->d_sz[cur], pl->d_loc[cur],
-                                                         pl->d_sz[cur ^ 1], k.len, k.src, d.len, d.src,
+                                                         sz_next, k.len, k.src, d.len, d.src,
                                                          pl->d_round_bytes + ph.stats_off);
       }
       TUNA_LAUNCHED(pl);
       // per-rank prefix sums of both lists; the KEEP stream is this phase's workspace region
       rc = scan_phase_lists(pl, k, ph.per_rank - ph.finals, f, pl->d_wbase + f, d, ph.finals, nph + f, st);
       if (rc) return rc;
-      tuna_place_kernel<<<gPP, th, 0, st>>>(t, pd, pl->d_loc[cur], pl->d_loc[cur ^ 1], k.pos,
+      tuna_place_kernel<<<gPP, th, 0, st>>>(t, pd, pl->d_loc[cur], loc_next, k.pos,
                                             pl->d_seg_base, k.len, d.pos, pl->d_seg_base + P, d.dst,
                                             pl->d_wbase + f, pl->d_rdispls, pl->d_recvbase,
                                             pl->classic ? 1 : 0, pl->rot.len, pl->rot.src, pl->rot.dst);

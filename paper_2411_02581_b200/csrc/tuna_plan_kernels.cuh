@@ -83,7 +83,8 @@ __global__ void tuna_init_tables_kernel(TunaTopo t, const int64_t *__restrict__ 
 // Count-metadata exchange of one digit phase: the receiver (p', sigma) of every
 // moving slot learns the size of the block its partner holds, and where the
 // partner keeps it.  Non-moving slots keep their size.  Also accumulates the
-// per-round byte totals (round z = the slots whose digit equals z).
+// per-round byte totals (round z = the slots whose digit equals z).  sz_next is
+// null in a plan's last phase: nothing reads the size table after it.
 __global__ void tuna_meta_exchange_kernel(TunaTopo t, PhaseDev ph, const int64_t *__restrict__ sz_cur,
                                           const int64_t *__restrict__ loc_cur, int64_t *sz_next,
                                           int64_t *keep_len, int64_t *keep_src, int64_t *del_len,
@@ -104,7 +105,7 @@ __global__ void tuna_meta_exchange_kernel(TunaTopo t, PhaseDev ph, const int64_t
     const int v = ph.level == 0 ? jo : io;
     const int dig = (int)(((unsigned)v / (unsigned)ph.stride) % (unsigned)ph.radix);
     if (dig == 0) {
-      sz_next[idx] = sz_cur[idx];
+      if (sz_next) sz_next[idx] = sz_cur[idx];
     } else {
       const int dist = dig * (int)ph.stride;  // below Q (level 0) or N (level 1): a wrap is one addition
       int qs = q, ns = n;
@@ -119,7 +120,7 @@ __global__ void tuna_meta_exchange_kernel(TunaTopo t, PhaseDev ph, const int64_t
       const int64_t c = row_position(t, ph, io, jo);
       const int64_t size = sz_cur[(int64_t)sender * t.P + sigma];
       const int64_t where = loc_cur[(int64_t)sender * t.P + sigma];
-      sz_next[idx] = size;
+      if (sz_next) sz_next[idx] = size;
       // sharded plans list a block only on the GPU that moves it: the receiver's in a
       // local phase (both ranks are there), the sender's in the global phase (a push)
       const int64_t bytes = resident(t, ph.level == 0 ? p : sender) ? size : 0;
@@ -202,7 +203,7 @@ __global__ void tuna_meta_exchange_diag_kernel(TunaTopo t, PhaseDev ph, const in
     const int64_t p = row0 + q;
     int64_t bytes = s_sz[sr][tx];
     const int64_t where = s_loc[sr][tx];
-    sz_next[p * P + col0 + g] = bytes;  // (jo = 0 never moves in this phase: sender and receiver are the same rank)
+    if (sz_next) sz_next[p * P + col0 + g] = bytes;  // (jo = 0 never moves in this phase: sender and receiver are the same rank)
     if (g == 0) continue;
     if (!listed) bytes = 0;
     const int64_t c = (int64_t)io * ph.moving + (g - 1);  // position among the blocks the rank receives, in slot order
@@ -470,7 +471,7 @@ __global__ void tuna_place_kernel(TunaTopo t, PhaseDev ph, const int64_t *__rest
   const int v = ph.level == 0 ? jo : io;
   const int dig = (int)(((unsigned)v / (unsigned)ph.stride) % (unsigned)ph.radix);
   if (dig == 0) {
-    loc_next[idx] = loc_cur[idx];
+    if (loc_next) loc_next[idx] = loc_cur[idx];
     return;
   }
   const int64_t c = row_position(t, ph, io, jo);
@@ -482,13 +483,13 @@ __global__ void tuna_place_kernel(TunaTopo t, PhaseDev ph, const int64_t *__rest
     const int64_t e = (int64_t)p * ph.finals + c;
     del_pos[e] += del_base[p];
     del_dst[e] = rloc;
-    loc_next[idx] = rloc;
+    if (loc_next) loc_next[idx] = rloc;
   } else {
     const int64_t e = (int64_t)p * (ph.per_rank - ph.finals) + (c - ph.finals);
     const int64_t w = keep_pos[e] + keep_base[p];
     keep_pos[e] = w;
     const int64_t wloc = TUNA_LOC(TUNA_BUF_WORK, wbase[0] + w);
-    loc_next[idx] = wloc;
+    if (loc_next) loc_next[idx] = wloc;
     if (fin && classic) {
       rot_len[idx] = keep_len[e];
       rot_src[idx] = wloc;
