@@ -705,9 +705,11 @@ int build_tables(tuna_plan *pl, const HostLayout *hl, const int64_t *sdispls, co
       TUNA_CUDA(pl, cudaMemsetAsync(pl->rot.src, 0, (size_t)PP * 8, st));
       TUNA_CUDA(pl, cudaMemsetAsync(pl->rot.dst, 0, (size_t)PP * 8, st));
     }
+    // (a plan that starts with a digit phase reads sizes and locations off the layout there)
+    const bool init_tables = nph == 0 || pl->phases[0].stag_hi > 0;
     tuna_init_tables_kernel<<<gPP, th, 0, st>>>(t, pl->d_counts, pl->d_sdispls, pl->d_rdispls,
-                                                pl->d_sendbase, pl->d_recvbase, pl->d_sz[0],
-                                                pl->d_loc[0], pl->dir.len, pl->dir.src, pl->dir.dst,
+                                                pl->d_sendbase, pl->d_recvbase, init_tables ? pl->d_sz[0] : nullptr,
+                                                init_tables ? pl->d_loc[0] : nullptr, pl->dir.len, pl->dir.src, pl->dir.dst,
                                                 pl->rot.len, pl->rot.src, pl->rot.dst,
                                                 pl->classic ? 1 : 0);
     TUNA_LAUNCHED(pl);
@@ -733,14 +735,16 @@ int build_tables(tuna_plan *pl, const HostLayout *hl, const int64_t *sdispls, co
       // (the tables that follow the blocks have no reader behind the last phase)
       int64_t *const sz_next = f + 1 < nph ? pl->d_sz[cur ^ 1] : nullptr;
       int64_t *const loc_next = f + 1 < nph ? pl->d_loc[cur ^ 1] : nullptr;
+      const TunaFirst first = f == 0 ? TunaFirst{pl->d_counts, pl->d_sdispls, pl->d_sendbase}
+                                     : TunaFirst{nullptr, nullptr, nullptr};
       if (ph.level == 0 && ph.stride == 1 && ph.radix >= t.Q && t.N <= 65535) {
         const unsigned tiles = (unsigned)((t.Q + 31) / 32);
         tuna_meta_exchange_diag_kernel<<<dim3(tiles * tiles, t.N, t.N), dim3(32, 8), 0, st>>>(
-            t, pd, pl->d_sz[cur], pl->d_loc[cur], sz_next, k.len, k.src, d.len, d.src,
+            t, pd, first, pl->d_sz[cur], pl->d_loc[cur], sz_next, k.len, k.src, d.len, d.src,
             pl->d_round_bytes + ph.stats_off);
       } else {
         const size_t smem = ph.radix <= 4096 ? (size_t)ph.radix * 8 : 0;
-        tuna_meta_exchange_kernel<<<gPP, th, smem, st>>>(t, pd, pl->d_sz[cur], pl->d_loc[cur],
+        tuna_meta_exchange_kernel<<<gPP, th, smem, st>>>(t, pd, first, pl->d_sz[cur], pl->d_loc[cur],
                                                          sz_next, k.len, k.src, d.len, d.src,
                                                          pl->d_round_bytes + ph.stats_off);
       }
@@ -748,7 +752,7 @@ int build_tables(tuna_plan *pl, const HostLayout *hl, const int64_t *sdispls, co
       // per-rank prefix sums of both lists; the KEEP stream is this phase's workspace region
       rc = scan_phase_lists(pl, k, ph.per_rank - ph.finals, f, pl->d_wbase + f, d, ph.finals, nph + f, st);
       if (rc) return rc;
-      tuna_place_kernel<<<gPP, th, 0, st>>>(t, pd, pl->d_loc[cur], loc_next, k.pos,
+      tuna_place_kernel<<<gPP, th, 0, st>>>(t, pd, first, pl->d_loc[cur], loc_next, k.pos,
                                             pl->d_seg_base, k.len, d.pos, pl->d_seg_base + P, d.dst,
                                             pl->d_wbase + f, pl->d_rdispls, pl->d_recvbase,
                                             pl->classic ? 1 : 0, pl->rot.len, pl->rot.src, pl->rot.dst);

@@ -44,7 +44,24 @@ __device__ __forceinline__ int64_t row_position(const TunaTopo &t, const PhaseDe
                        : compact_of(io, ph.stride, ph.radix) * t.Q + jo;
 }
 
-// Initial tables (before any phase): every block is in its owner's send region.
+// A plan's first phase finds every block where its owner put it: sizes and locations
+// then follow from the layout itself, and the two tables need not exist yet.
+struct TunaFirst {
+  const int64_t *counts, *sdispls, *sendbase;  // all null from the second phase on
+};
+__device__ __forceinline__ int dest_of(const TunaTopo &t, int p, int sigma) {
+  const int n = p / t.Q, q = p % t.Q, io = sigma / t.Q, jo = sigma % t.Q;
+  return (n + io - (n + io >= t.N ? t.N : 0)) * t.Q + (q + jo - (q + jo >= t.Q ? t.Q : 0));
+}
+__device__ __forceinline__ int64_t first_size(const TunaTopo &t, const TunaFirst &f, int p, int sigma) {
+  return f.counts[(int64_t)p * t.P + dest_of(t, p, sigma)] * t.elem;
+}
+__device__ __forceinline__ int64_t first_loc(const TunaTopo &t, const TunaFirst &f, int p, int sigma) {
+  return TUNA_LOC(TUNA_BUF_SEND, (f.sendbase[p] + f.sdispls[(int64_t)p * t.P + dest_of(t, p, sigma)]) * t.elem);
+}
+
+// Initial tables (before any phase): every block is in its owner's send region
+// (sz and loc may be null: a plan whose first phase is a digit phase works them out itself).
 // Also fills the direct list (receive-side order (d, s)) and the self entries of
 // the rotation list.
 __global__ void tuna_init_tables_kernel(TunaTopo t, const int64_t *__restrict__ counts,
@@ -59,12 +76,15 @@ __global__ void tuna_init_tables_kernel(TunaTopo t, const int64_t *__restrict__ 
   const int64_t PP = (int64_t)t.P * t.P;
   if (idx >= PP) return;
   const int p = (int)((unsigned)idx / (unsigned)t.P), sigma = (int)((unsigned)idx % (unsigned)t.P);  // (P * P < 2^31)
+  if (!sz && !dir_len && sigma != 0) return;  // only the self blocks are left to describe
   const int n = p / t.Q, q = p % t.Q, io = sigma / t.Q, jo = sigma % t.Q;
   const int dest = (n + io - (n + io >= t.N ? t.N : 0)) * t.Q + (q + jo - (q + jo >= t.Q ? t.Q : 0));
   const int64_t bytes = counts[(int64_t)p * t.P + dest] * t.elem;
   const int64_t sloc = TUNA_LOC(TUNA_BUF_SEND, (sendbase[p] + sdispls[(int64_t)p * t.P + dest]) * t.elem);
-  sz[idx] = bytes;
-  loc[idx] = sloc;
+  if (sz) {
+    sz[idx] = bytes;
+    loc[idx] = sloc;
+  }
   // direct list entry (d = p as receiver, s = sigma as source index)
   if (dir_len) {
     const int d = p, s = sigma;
@@ -85,7 +105,8 @@ __global__ void tuna_init_tables_kernel(TunaTopo t, const int64_t *__restrict__ 
 // partner keeps it.  Non-moving slots keep their size.  Also accumulates the
 // per-round byte totals (round z = the slots whose digit equals z).  sz_next is
 // null in a plan's last phase: nothing reads the size table after it.
-__global__ void tuna_meta_exchange_kernel(TunaTopo t, PhaseDev ph, const int64_t *__restrict__ sz_cur,
+__global__ void tuna_meta_exchange_kernel(TunaTopo t, PhaseDev ph, TunaFirst first,
+                                          const int64_t *__restrict__ sz_cur,
                                           const int64_t *__restrict__ loc_cur, int64_t *sz_next,
                                           int64_t *keep_len, int64_t *keep_src, int64_t *del_len,
                                           int64_t *del_src, unsigned long long *round_bytes) {
@@ -105,7 +126,7 @@ __global__ void tuna_meta_exchange_kernel(TunaTopo t, PhaseDev ph, const int64_t
     const int v = ph.level == 0 ? jo : io;
     const int dig = (int)(((unsigned)v / (unsigned)ph.stride) % (unsigned)ph.radix);
     if (dig == 0) {
-      if (sz_next) sz_next[idx] = sz_cur[idx];
+      if (sz_next) sz_next[idx] = first.counts ? first_size(t, first, p, sigma) : sz_cur[idx];
     } else {
       const int dist = dig * (int)ph.stride;  // below Q (level 0) or N (level 1): a wrap is one addition
       int qs = q, ns = n;
@@ -118,8 +139,8 @@ __global__ void tuna_meta_exchange_kernel(TunaTopo t, PhaseDev ph, const int64_t
       }
       const int sender = ns * t.Q + qs;
       const int64_t c = row_position(t, ph, io, jo);
-      const int64_t size = sz_cur[(int64_t)sender * t.P + sigma];
-      const int64_t where = loc_cur[(int64_t)sender * t.P + sigma];
+      const int64_t size = first.counts ? first_size(t, first, sender, sigma) : sz_cur[(int64_t)sender * t.P + sigma];
+      const int64_t where = first.counts ? first_loc(t, first, sender, sigma) : loc_cur[(int64_t)sender * t.P + sigma];
       if (sz_next) sz_next[idx] = size;
       // sharded plans list a block only on the GPU that moves it: the receiver's in a
       // local phase (both ranks are there), the sender's in the global phase (a push)
@@ -168,7 +189,8 @@ __global__ void tuna_meta_exchange_kernel(TunaTopo t, PhaseDev ph, const int64_t
 // jo): it reads the tile along rows and writes it out by receiver, where each
 // receiver's slots are again consecutive; a round's bytes are summed per tile
 // column first.  Grid: (tiles of a Q x Q square, N, N), CTAs of 32 x 8 threads.
-__global__ void tuna_meta_exchange_diag_kernel(TunaTopo t, PhaseDev ph, const int64_t *__restrict__ sz_cur,
+__global__ void tuna_meta_exchange_diag_kernel(TunaTopo t, PhaseDev ph, TunaFirst first,
+                                               const int64_t *__restrict__ sz_cur,
                                                const int64_t *__restrict__ loc_cur, int64_t *sz_next,
                                                int64_t *keep_len, int64_t *keep_src, int64_t *del_len,
                                                int64_t *del_src, unsigned long long *round_bytes) {
@@ -183,8 +205,13 @@ __global__ void tuna_meta_exchange_diag_kernel(TunaTopo t, PhaseDev ph, const in
   for (int j = ty; j < 32; j += 8) {
     const int sd = s0 + j, g = g0 + tx;
     const bool in = sd < Q && g < Q;
-    s_sz[j][tx] = in ? sz_cur[(row0 + sd) * P + col0 + g] : 0;
-    s_loc[j][tx] = in ? loc_cur[(row0 + sd) * P + col0 + g] : 0;
+    if (first.counts) {
+      s_sz[j][tx] = in ? first_size(t, first, (int)row0 + sd, col0 + g) : 0;
+      s_loc[j][tx] = in ? first_loc(t, first, (int)row0 + sd, col0 + g) : 0;
+    } else {
+      s_sz[j][tx] = in ? sz_cur[(row0 + sd) * P + col0 + g] : 0;
+      s_loc[j][tx] = in ? loc_cur[(row0 + sd) * P + col0 + g] : 0;
+    }
   }
   __syncthreads();
   if (ty == 0 && g0 + tx >= 1 && g0 + tx < Q) {  // round z = jo: bytes sent by this tile's senders
@@ -454,7 +481,7 @@ __global__ void tuna_add_base_kernel(int64_t *pos, const int64_t *__restrict__ s
 // arrived: in direct-to-R mode it is in the DELIVER list and goes to its place in
 // the receive buffer; in classic mode every block stays in the workspace and a
 // rotation descriptor is recorded for the final reorder.
-__global__ void tuna_place_kernel(TunaTopo t, PhaseDev ph, const int64_t *__restrict__ loc_cur,
+__global__ void tuna_place_kernel(TunaTopo t, PhaseDev ph, TunaFirst first, const int64_t *__restrict__ loc_cur,
                                   int64_t *loc_next, int64_t *keep_pos,
                                   const int64_t *__restrict__ keep_base,
                                   const int64_t *__restrict__ keep_len, int64_t *del_pos,
@@ -471,7 +498,7 @@ __global__ void tuna_place_kernel(TunaTopo t, PhaseDev ph, const int64_t *__rest
   const int v = ph.level == 0 ? jo : io;
   const int dig = (int)(((unsigned)v / (unsigned)ph.stride) % (unsigned)ph.radix);
   if (dig == 0) {
-    if (loc_next) loc_next[idx] = loc_cur[idx];
+    if (loc_next) loc_next[idx] = first.counts ? first_loc(t, first, p, sigma) : loc_cur[idx];
     return;
   }
   const int64_t c = row_position(t, ph, io, jo);
